@@ -1,0 +1,357 @@
+// CPU oracle for the mixed-bit quantized AdamW step (STQuant, Algorithm 1 and Sec. 3.3-3.5).
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the hot path
+// computes.  It is used by the tests, by the smoke check and by the timed CPU-baseline leg of the
+// benchmark; the product path never calls it and shares no code, header or table with it.
+//
+// Everything is written element by element in the order the paper's Algorithm 1 states, with no
+// blocking, fusion or reordering.  fp32 operations are single IEEE round-to-nearest-even
+// operations (build with -ffp-contract=off, no fast-math); `fmaf` appears only where the
+// quantizer definition says "fused".  Rounding-to-integer steps are taken on the exact product,
+// which a double holds exactly for two fp32 factors.
+//
+// Parity status: the quantizer formulas are this build's reading of "linear symmetric" and
+// "logarithmic" block-wise quantization (Sec. 3.5 gives no formula); they are pinned by the
+// properties the tests check (half-step error bound, idempotence, monotone bound, exact block
+// maximum, agreement with library AdamW at 32 and 16 bits).  The claim that ~5 bits preserve
+// model quality needs the paper's training runs: parity unpinned for that claim.
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+
+namespace {
+
+inline uint32_t f2u(float f) { uint32_t u; std::memcpy(&u, &f, 4); return u; }
+inline float u2f(uint32_t u) { float f; std::memcpy(&f, &u, 4); return f; }
+
+// A block whose maximum is below this is stored as an all-zero block (scale 0).
+const float kTinyScale = 0x1p-100f;
+
+// ---- widths ---------------------------------------------------------------------------------
+inline bool width_ok(int b) { return b == 2 || b == 3 || b == 4 || b == 8 || b == 16 || b == 32; }
+inline int qmax_of(int b) { return (1 << (b - 1)) - 1; }   // linear: largest |q|
+inline int half_of(int b) { return 1 << (b - 1); }         // linear: offset of the stored code
+inline int K_of(int b) { return (1 << b) - 1; }            // log: largest code
+inline int R_of(int b) { int K = K_of(b); return K < 30 ? K : 30; }   // log: octaves covered
+
+// ---- bitstream (LSB-first, little-endian; element i occupies bits [i*b, (i+1)*b)) ------------
+inline uint32_t get_code(const uint8_t* s, uint64_t i, int b) {
+  uint64_t bit = i * (uint64_t)b;
+  uint32_t v = 0;
+  for (int k = 0; k < b; ++k, ++bit) v |= (uint32_t)((s[bit >> 3] >> (bit & 7)) & 1u) << k;
+  return v;
+}
+inline void put_code(uint8_t* s, uint64_t i, int b, uint32_t v) {
+  uint64_t bit = i * (uint64_t)b;
+  for (int k = 0; k < b; ++k, ++bit) {
+    uint8_t m = (uint8_t)(1u << (bit & 7));
+    if ((v >> k) & 1u) s[bit >> 3] |= m; else s[bit >> 3] &= (uint8_t)~m;
+  }
+}
+inline uint64_t codes_bytes(uint64_t n, int b) {
+  uint64_t by = (n * (uint64_t)b + 7) / 8;
+  return (by + 15) / 16 * 16;
+}
+
+// ---- lg: split base-2 logarithm of a non-negative float -------------------------------------
+// lg(x) = (E - 127) + P(t), E the biased exponent field, t = mantissa field * 2^-23 in [0,1),
+// P(t) = t*(c1 + t*(c2 + ... + t*c6)) ~ log2(1+t), Horner with fused steps, final multiply rounded.
+// (For zero/denormal inputs the fields are used literally; such values only occur in blocks that
+// the tiny-scale rule zeroes or far below the coding floor.)
+const float kP1 = 0x1.714b30p+0f, kP2 = -0x1.6fc360p-1f, kP3 = 0x1.d54a42p-2f,
+            kP4 = -0x1.1e4792p-2f, kP5 = 0x1.f9c008p-4f, kP6 = -0x1.b19412p-6f;
+inline int lg_E(float x) { return (int)(f2u(x) >> 23); }
+inline float lg_P(float x) {
+  float mant = u2f((f2u(x) & 0x007FFFFFu) | 0x3F800000u);
+  float t = mant - 1.0f;
+  float a = kP6;
+  a = fmaf(a, t, kP5);
+  a = fmaf(a, t, kP4);
+  a = fmaf(a, t, kP3);
+  a = fmaf(a, t, kP2);
+  a = fmaf(a, t, kP1);
+  return a * t;
+}
+
+// ---- ex: 2^e for e <= 0 -----------------------------------------------------------------------
+// i = round-half-even(e), f = e - i in [-1/2, 1/2], p = 1 + f*(e0 + f*(e1 + ... + f*e4)) fused,
+// ex = p * 2^i (exact scaling).  ex(0) == 1 exactly.
+const float kE0 = 0x1.62e42ap-1f, kE1 = 0x1.ebf9bcp-3f, kE2 = 0x1.c6b74cp-5f,
+            kE3 = 0x1.3cea84p-7f, kE4 = 0x1.5bbc6ap-10f;
+inline float ex2(float e) {
+  float i = nearbyintf(e);
+  float f = e - i;
+  float a = kE4;
+  a = fmaf(a, f, kE3);
+  a = fmaf(a, f, kE2);
+  a = fmaf(a, f, kE1);
+  a = fmaf(a, f, kE0);
+  float p = fmaf(a, f, 1.0f);
+  return ldexpf(p, (int)i);
+}
+
+// ---- linear symmetric block quantizer (first moment) ----------------------------------------
+// scale s = max|x|; q = clamp(round-half-even(x * fl(qmax/s)), -qmax, qmax); stored code q + 2^(b-1).
+void quant_lin_block(const float* x, uint64_t n, int b, uint32_t* code, float* scale) {
+  float s = 0.0f;
+  for (uint64_t i = 0; i < n; ++i) { float a = fabsf(x[i]); if (a > s) s = a; }
+  const int qmax = qmax_of(b), half = half_of(b);
+  if (s < kTinyScale) {
+    *scale = 0.0f;
+    for (uint64_t i = 0; i < n; ++i) code[i] = (uint32_t)half;
+    return;
+  }
+  *scale = s;
+  float inv = (float)qmax / s;
+  for (uint64_t i = 0; i < n; ++i) {
+    double r = nearbyint((double)x[i] * (double)inv);
+    if (r > qmax) r = qmax;
+    if (r < -qmax) r = -qmax;
+    code[i] = (uint32_t)((int)r + half);
+  }
+}
+inline float dequant_lin(uint32_t code, float s, int b) {
+  float invq = 1.0f / (float)qmax_of(b);
+  float q = (float)((int)code - half_of(b));
+  float y = q * invq;
+  return s * y;
+}
+
+// ---- logarithmic block quantizer (second moment, x >= 0) -------------------------------------
+// scale s = max x; code K is the block maximum, each code step is R/K octaves, code 0 is the floor
+// s*2^-R.  d = log-distance to the maximum in octaves, q = clamp(K + round-half-even(d*K/R), 0, K).
+void quant_log_block(const float* x, uint64_t n, int b, uint32_t* code, float* scale) {
+  float s = 0.0f;
+  for (uint64_t i = 0; i < n; ++i) if (x[i] > s) s = x[i];
+  if (s < kTinyScale) {
+    *scale = 0.0f;
+    for (uint64_t i = 0; i < n; ++i) code[i] = 0u;
+    return;
+  }
+  *scale = s;
+  const int K = K_of(b), R = R_of(b);
+  const float a_b = (float)K / (float)R;          // exact: 1, 1, 1, 8.5, 2184.5
+  const int Es = lg_E(s);
+  const float Ps = lg_P(s);
+  for (uint64_t i = 0; i < n; ++i) {
+    float de = (float)(lg_E(x[i]) - Es);
+    float dp = lg_P(x[i]) - Ps;
+    float d = de + dp;
+    double r = nearbyint((double)d * (double)a_b);
+    double q = (double)K + r;
+    if (q < 0) q = 0;
+    if (q > K) q = K;
+    code[i] = (uint32_t)q;
+  }
+}
+inline float dequant_log(uint32_t code, float s, int b) {
+  const int K = K_of(b), R = R_of(b);
+  const float c_b = (float)R / (float)K;
+  float rf = (float)((int)code - K);
+  float e = rf * c_b;
+  float y = ex2(e);
+  return s * y;
+}
+
+// ---- state (de)coding over a whole range ------------------------------------------------------
+// mode 0 = linear (m), 1 = log (v).  Width 32 stores raw fp32 and no scales.
+void decode_state(const uint8_t* codes, const float* scales, uint64_t n, int b, uint32_t block,
+                  int mode, float* out) {
+  if (b == 32) { std::memcpy(out, codes, n * 4); return; }
+  for (uint64_t i = 0; i < n; ++i) {
+    uint32_t c = get_code(codes, i, b);
+    float s = scales[i / block];
+    out[i] = mode == 0 ? dequant_lin(c, s, b) : dequant_log(c, s, b);
+  }
+}
+void encode_state(const float* x, uint64_t n, int b, uint32_t block, int mode, uint8_t* codes,
+                  float* scales) {
+  if (b == 32) { std::memcpy(codes, x, n * 4); return; }
+  std::memset(codes, 0, codes_bytes(n, b));
+  std::vector<uint32_t> tmp(block);
+  for (uint64_t j = 0, k = 0; j < n; j += block, ++k) {
+    uint64_t len = n - j < block ? n - j : block;
+    if (mode == 0) quant_lin_block(x + j, len, b, tmp.data(), scales + k);
+    else quant_log_block(x + j, len, b, tmp.data(), scales + k);
+    for (uint64_t i = 0; i < len; ++i) put_code(codes, j + i, b, tmp[i]);
+  }
+}
+
+inline float bf16_to_f32(uint16_t h) { return u2f((uint32_t)h << 16); }
+
+}  // namespace
+
+extern "C" {
+
+struct orc_hparams {
+  double lr, beta1, beta2, eps, weight_decay;
+  int64_t step;        // t >= 1, the step being taken
+  int decoupled_wd;    // 1 = AdamW (Algorithm 1); 0 = L2 term added to the gradient
+  int grad_dtype;      // 0 = fp32, 1 = bf16
+};
+
+uint64_t orc_codes_bytes(uint64_t n, int bits) { return bits == 32 ? n * 4 : codes_bytes(n, bits); }
+uint64_t orc_num_blocks(uint64_t n, uint32_t block) { return (n + block - 1) / block; }
+
+float orc_lg_P(float x) { return lg_P(x); }
+int orc_lg_E(float x) { return lg_E(x); }
+float orc_ex2(float e) { return ex2(e); }
+
+void orc_pack(const uint32_t* code, uint64_t n, int bits, uint8_t* out) {
+  std::memset(out, 0, codes_bytes(n, bits));
+  for (uint64_t i = 0; i < n; ++i) put_code(out, i, bits, code[i]);
+}
+void orc_unpack(const uint8_t* in, uint64_t n, int bits, uint32_t* code) {
+  for (uint64_t i = 0; i < n; ++i) code[i] = get_code(in, i, bits);
+}
+
+// Quantize / dequantize a whole tensor state.  mode 0 = linear (m), 1 = log (v).
+int orc_quantize(const float* x, uint64_t n, int bits, uint32_t block, int mode, uint8_t* codes,
+                 float* scales) {
+  if (!width_ok(bits) || block == 0) return -1;
+  encode_state(x, n, bits, block, mode, codes, scales);
+  return 0;
+}
+int orc_dequantize(const uint8_t* codes, const float* scales, uint64_t n, int bits, uint32_t block,
+                   int mode, float* out) {
+  if (!width_ok(bits) || block == 0) return -1;
+  decode_state(codes, scales, n, bits, block, mode, out);
+  return 0;
+}
+
+// Initial state (Algorithm 1, initialisation): m = v = 0 at the given widths.
+int orc_init_state(uint64_t n, uint32_t block, int bits_m, int bits_v, uint8_t* m_codes,
+                   float* m_scales, uint8_t* v_codes, float* v_scales) {
+  std::vector<float> z(n, 0.0f);
+  if (orc_quantize(z.data(), n, bits_m, block, 0, m_codes, m_scales)) return -1;
+  if (orc_quantize(z.data(), n, bits_v, block, 1, v_codes, v_scales)) return -1;
+  return 0;
+}
+
+// Per-layer gradient sums for the factor selection (Eq. 2, 3, 8): sum g, sum |g|, sum g^2, count.
+void orc_grad_stats(const void* grad, int grad_dtype, uint64_t n, double out[4]) {
+  double sg = 0, sa = 0, sq = 0;
+  for (uint64_t i = 0; i < n; ++i) {
+    float g = grad_dtype == 1 ? bf16_to_f32(((const uint16_t*)grad)[i]) : ((const float*)grad)[i];
+    double gd = (double)g;
+    sg += gd; sa += fabs(gd); sq += gd * gd;
+  }
+  out[0] = sg; out[1] = sa; out[2] = sq; out[3] = (double)n;
+}
+
+// One step of Algorithm 1's inner loop for one tensor (or any range that starts on a block
+// boundary).  Stored states come in at (bits_m_in, bits_v_in) and leave at (bits_m_out,
+// bits_v_out).  theta is updated in place.  stats, if non-null, receives the sums above.
+int orc_step(float* theta, const void* grad, uint64_t n, uint32_t block,
+             const uint8_t* m_codes_in, const float* m_scales_in, int bits_m_in,
+             const uint8_t* v_codes_in, const float* v_scales_in, int bits_v_in,
+             uint8_t* m_codes_out, float* m_scales_out, int bits_m_out,
+             uint8_t* v_codes_out, float* v_scales_out, int bits_v_out,
+             const orc_hparams* hp, double* stats) {
+  if (!width_ok(bits_m_in) || !width_ok(bits_v_in) || !width_ok(bits_m_out) || !width_ok(bits_v_out))
+    return -1;
+  if (block == 0 || hp->step < 1) return -1;
+  std::vector<float> m(n), v(n), g(n);
+
+  // stored m_{t-1}, v_{t-1}
+  decode_state(m_codes_in, m_scales_in, n, bits_m_in, block, 0, m.data());
+  decode_state(v_codes_in, v_scales_in, n, bits_v_in, block, 1, v.data());
+
+  // gradient as fp32 (bf16 widens exactly)
+  for (uint64_t i = 0; i < n; ++i)
+    g[i] = hp->grad_dtype == 1 ? bf16_to_f32(((const uint16_t*)grad)[i]) : ((const float*)grad)[i];
+  if (stats) orc_grad_stats(grad, hp->grad_dtype, n, stats);
+  if (!hp->decoupled_wd) {
+    const float wd = (float)hp->weight_decay;
+    for (uint64_t i = 0; i < n; ++i) { float l2 = wd * theta[i]; g[i] = g[i] + l2; }
+  }
+
+  // moments: m_t = b1*m + (1-b1)*g ; v_t = b2*v + (1-b2)*g^2, every operation rounded to fp32
+  // (the four coefficients are the fp32 roundings of beta and of 1-beta taken in double)
+  const float fb1 = (float)hp->beta1, fb2 = (float)hp->beta2;
+  const float omb1 = (float)(1.0 - hp->beta1), omb2 = (float)(1.0 - hp->beta2);
+  for (uint64_t i = 0; i < n; ++i) {
+    float a = fb1 * m[i];
+    float c = omb1 * g[i];
+    m[i] = a + c;
+    float p = fb2 * v[i];
+    float w = omb2 * g[i];
+    float w2 = w * g[i];
+    v[i] = p + w2;
+  }
+
+  // Quantize(m_t, linear), Quantize(v_t, log) at the widths assigned for this step
+  encode_state(m.data(), n, bits_m_out, block, 0, m_codes_out, m_scales_out);
+  encode_state(v.data(), n, bits_v_out, block, 1, v_codes_out, v_scales_out);
+
+  // the update consumes the quantized states
+  decode_state(m_codes_out, m_scales_out, n, bits_m_out, block, 0, m.data());
+  decode_state(v_codes_out, v_scales_out, n, bits_v_out, block, 1, v.data());
+
+  const double b1 = hp->beta1, b2 = hp->beta2, lr = hp->lr, eps = hp->eps;
+  const double bc1 = 1.0 - std::pow(b1, (double)hp->step);
+  const double bc2 = 1.0 - std::pow(b2, (double)hp->step);
+  const double decay = hp->decoupled_wd ? 1.0 - lr * (double)hp->weight_decay : 1.0;
+  for (uint64_t i = 0; i < n; ++i) {
+    double mt = (double)m[i] / bc1;
+    double vt = (double)v[i] / bc2;
+    double th = (double)theta[i] * decay - lr * mt / (std::sqrt(vt) + eps);
+    theta[i] = (float)th;
+  }
+  return 0;
+}
+
+// Width transition: codes' = Q_{b'}(D_b(codes)), block scales recomputed from the decoded values
+// (they come out unchanged whenever the source was itself quantized).
+int orc_repack(const uint8_t* codes_in, const float* scales_in, int bits_in, uint8_t* codes_out,
+               float* scales_out, int bits_out, uint64_t n, uint32_t block, int mode) {
+  if (!width_ok(bits_in) || !width_ok(bits_out) || block == 0) return -1;
+  std::vector<float> x(n);
+  decode_state(codes_in, scales_in, n, bits_in, block, mode, x.data());
+  encode_state(x.data(), n, bits_out, block, mode, codes_out, scales_out);
+  return 0;
+}
+
+// ---- transition decision (Algorithm 1, decision branch; Sec. 3.3-3.4) -------------------------
+struct orc_policy {
+  double n_ema, r_ema, v_ema;   // global running statistics, start at 0
+  double alpha, tau, eps_stat;
+  int cv_of_signed;             // 0: sigma(|g|)/mu(|g|) (Eq. 3); 1: sigma(g)/E|g| (Algorithm 1)
+};
+
+int orc_is_decision_step(int64_t t, int64_t U) { return (t % U == 0) || (t < 5); }
+
+// stats: L rows of {sum g, sum |g|, sum g^2, count}.  Writes bits[l] in {4,8,16,32} and, if
+// non-null, score[l].  Updates the three running averages first, as Algorithm 1 orders it.
+void orc_decide(orc_policy* p, const double* stats, int L, int64_t t, uint8_t* bits, double* score) {
+  std::vector<double> n(L), r(L), v(L);
+  double sn = 0, sr = 0, sv = 0;
+  for (int l = 0; l < L; ++l) {
+    const double* s = stats + 4 * l;
+    double N = s[3];
+    double mean_sq = s[2] / N;
+    double mean_abs = s[1] / N;
+    double mean = s[0] / N;
+    n[l] = std::sqrt(mean_sq);
+    v[l] = mean_sq;
+    double var = p->cv_of_signed ? mean_sq - mean * mean : mean_sq - mean_abs * mean_abs;
+    if (var < 0) var = 0;
+    r[l] = std::sqrt(var) / (mean_abs + p->eps_stat);
+    sn += n[l]; sr += r[l]; sv += v[l];
+  }
+  p->n_ema = p->alpha * (sn / L) + (1 - p->alpha) * p->n_ema;
+  p->r_ema = p->alpha * (sr / L) + (1 - p->alpha) * p->r_ema;
+  p->v_ema = p->alpha * (sv / L) + (1 - p->alpha) * p->v_ema;
+  const double S = 1.0 + 1.0 / std::cosh((double)t / p->tau);
+  for (int l = 0; l < L; ++l) {
+    double sc = 7.2 + std::log2(r[l] / (p->r_ema + p->eps_stat)) +
+                std::log2(n[l] / (p->n_ema + p->eps_stat)) + std::log2(S) +
+                std::log2(v[l] / (p->v_ema + p->eps_stat));
+    if (score) score[l] = sc;
+    bits[l] = sc < 6.8 ? 4 : sc < 12.0 ? 8 : sc < 24.0 ? 16 : 32;
+  }
+}
+
+}  // extern "C"
