@@ -1,0 +1,174 @@
+/*
+ * libstq — mixed-bit quantized AdamW step for NVIDIA B200 (sm_100a).
+ *
+ * The hot path of STQuant's training step (Algorithm 1, inner loop; Sec. 3.5): every parameter
+ * tensor keeps its first moment m (block-wise linear symmetric codes) and second moment v
+ * (block-wise logarithmic codes) at its own bit-width; one launch decodes m and v, applies the
+ * AdamW update with the re-quantized moments, and writes the new codes at the width assigned for
+ * this step.  On decision steps the per-layer gradient sums of Sec. 3.3 ride on the same pass and
+ * the host-side transition decision of Sec. 3.4 maps them to new widths.
+ *
+ * Conventions
+ *  - Every pointer in stq_tensor is a DEVICE pointer owned by the caller (host pointers only for
+ *    stq_step_host).  param, grad and code buffers must be 16-byte aligned, scale buffers 4-byte.
+ *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return without
+ *    synchronising, except stq_layer_stats and stq_step_host, which synchronise the stream.
+ *  - All arguments are validated on the host before anything is launched.  Return value: 0 on
+ *    success, a negative STQ_E_* code otherwise; nothing is launched when an error is returned.
+ *    The device code never traps, asserts or spins.
+ *  - A handle is bound to one device and is not thread-safe; use one handle per stream.
+ *
+ * Stored layout (per tensor, per state)
+ *  - widths b in {2,3,4,8,16}: codes are an LSB-first little-endian bitstream, element i in bits
+ *    [i*b, (i+1)*b); length stq_codes_bytes(numel, b) = ceil(numel*b/8) rounded up to 16 bytes,
+ *    padding bits zero.  Scales: one fp32 per block of `block` consecutive elements of the
+ *    flattened tensor (last block short), stq_scales_bytes(numel, block) bytes.
+ *  - width 32: the codes buffer holds the raw fp32 values (numel*4 rounded up to 16 bytes); the
+ *    scale pointers are ignored and may be NULL.
+ *  - first moment: code u = q + 2^(b-1), q in [-qmax, qmax], qmax = 2^(b-1)-1, value scale*q/qmax.
+ *  - second moment: code u in [0, 2^b-1]; value scale * 2^((u-K)*R/K), K = 2^b-1, R = min(K,30);
+ *    code 0 is a floor level, never zero.  A block whose scale is 0 decodes to all zeros.
+ */
+#ifndef STQ_H_
+#define STQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct stq_handle stq_handle;
+typedef struct stq_policy stq_policy;
+
+enum {
+  STQ_OK = 0,
+  STQ_E_NULL = -1,      /* a required pointer is NULL                                         */
+  STQ_E_BITS = -2,      /* a width outside {2,3,4,8,16,32}                                    */
+  STQ_E_BLOCK = -3,     /* block not in {128, 256, 512}                                       */
+  STQ_E_ALIGN = -4,     /* a buffer is not aligned as required                                */
+  STQ_E_ALIAS = -5,     /* in/out buffers overlap in a way the step cannot honour             */
+  STQ_E_NUMEL = -6,     /* numel == 0, or the table is empty or too large                     */
+  STQ_E_CUDA = -7,      /* a CUDA runtime call failed (see stq_last_cuda_error)               */
+  STQ_E_WORKSPACE = -8, /* the library could not grow its own workspace                       */
+  STQ_E_ARG = -9,       /* an invalid scalar argument (step < 1, unknown dtype or flag, ...)  */
+  STQ_E_STATE = -10     /* call order: no statistics pending for stq_layer_stats              */
+};
+
+enum { STQ_GRAD_F32 = 0, STQ_GRAD_BF16 = 1 };
+
+/* flags of stq_step */
+enum { STQ_WITH_STATS = 1u };
+
+/* One row per parameter tensor (a "layer" of the paper is one tensor). */
+typedef struct stq_tensor {
+  float* param;              /* fp32 master weights, numel elements, updated in place          */
+  const void* grad;          /* numel gradients, fp32 or bf16 (stq_hparams.grad_dtype)         */
+  const void* m_codes_in;    /* stored first moment: codes at width bits_m                     */
+  const float* m_scales_in;  /*                      block scales (ignored when bits_m == 32)  */
+  const void* v_codes_in;    /* stored second moment: codes at width bits_v                    */
+  const float* v_scales_in;
+  void* m_codes_out;         /* written at width bits_m_out; may be the same pointer as        */
+  float* m_scales_out;       /* m_codes_in only if bits_m_out == bits_m (no partial overlap);  */
+  void* v_codes_out;         /* scales_out may equal scales_in                                 */
+  float* v_scales_out;
+  uint64_t numel;
+  uint32_t block;            /* quantization block: 128, 256 or 512                            */
+  uint8_t bits_m, bits_v;          /* widths stored now                                        */
+  uint8_t bits_m_out, bits_v_out;  /* widths to write                                          */
+  float weight_decay;        /* per-tensor lambda                                              */
+  uint32_t reserved;         /* must be 0                                                      */
+} stq_tensor;
+
+typedef struct stq_hparams {
+  double lr, beta1, beta2, eps;
+  int64_t step;          /* t >= 1: the step being taken (bias correction 1 - beta^t)          */
+  int32_t decoupled_wd;  /* 1: AdamW as in Algorithm 1; 0: weight decay added to the gradient  */
+  int32_t grad_dtype;    /* STQ_GRAD_F32 or STQ_GRAD_BF16                                      */
+} stq_hparams;
+
+/* Handle: device copy of the tensor table, tile map and statistics workspace.
+ * stq_create makes `device` current for the call and allocates nothing large; workspaces grow on
+ * first use (cudaMalloc) and are freed by stq_destroy. */
+int stq_create(stq_handle** out, int device);
+int stq_destroy(stq_handle* h);
+
+/* Buffer sizes of the stored layout described above. */
+size_t stq_codes_bytes(uint64_t numel, int bits);
+size_t stq_scales_bytes(uint64_t numel, uint32_t block);
+
+/* Algorithm 1, initialisation: m = v = 0.  Writes the canonical zero state (first-moment codes
+ * 2^(b-1), second-moment codes 0, all scales 0) into the *_out buffers at bits_m_out/bits_v_out.
+ * param, grad and the *_in fields are ignored. */
+int stq_init_state(stq_handle* h, const stq_tensor* tensors, int L, void* stream);
+
+/* Algorithm 1, inner loop, for all L tensors in one pass:
+ *   m_t = beta1*m + (1-beta1)*g,  v_t = beta2*v + (1-beta2)*g^2      (states decoded from *_in)
+ *   codes/scales_out = Quantize(m_t, linear), Quantize(v_t, log)      (at bits_*_out)
+ *   param = param*(1 - lr*wd) - lr * (mq/(1-beta1^t)) / (sqrt(vq/(1-beta2^t)) + eps)
+ * where mq, vq are the values the new codes decode to.  With STQ_WITH_STATS the per-tensor sums
+ * sum g, sum |g|, sum g^2 (Eq. 2, 3, 8) are accumulated in the same pass; fetch them with
+ * stq_layer_stats. */
+int stq_step(stq_handle* h, const stq_tensor* tensors, int L, const stq_hparams* hp, unsigned flags,
+             void* stream);
+
+/* Gradient statistics alone (Algorithm 1 computes them before the update): reads only grad and
+ * numel of each row.  Fetch with stq_layer_stats. */
+int stq_grad_stats(stq_handle* h, const stq_tensor* tensors, int L, int grad_dtype, void* stream);
+
+/* Finishes the reduction started by the last stq_step(STQ_WITH_STATS) or stq_grad_stats on this
+ * handle and copies it to HOST memory: out[l] = {sum g, sum |g|, sum g^2, numel} for l < L.
+ * Synchronises `stream`.  The reduction order is fixed, so results are run-to-run identical. */
+int stq_layer_stats(stq_handle* h, double* out, int L, void* stream);
+
+/* Width transition without an optimizer step (implied by the per-step widths b_{l,t} of
+ * Sec. 3.1): codes_out = Quantize_{bits_out}(Decode_{bits}(codes_in)) for both states; block
+ * scales are recomputed and come out unchanged for quantized sources.  bits 32 on either side
+ * turns this into a plain quantize / decode of raw fp32 states.  param and grad are ignored. */
+int stq_repack(stq_handle* h, const stq_tensor* tensors, int L, void* stream);
+
+/* stq_step with every pointer in `tensors` a HOST pointer: the library stages the buffers through
+ * a device arena it owns (grown on demand), copies param/grad/codes/scales in, runs the step,
+ * copies param/codes/scales back and synchronises.  bytes_h2d / bytes_d2h (optional) receive
+ * the bytes copied. */
+int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hparams* hp,
+                  unsigned flags, uint64_t* bytes_h2d, uint64_t* bytes_d2h);
+
+/* Kernel launches issued through this handle so far. */
+uint64_t stq_launch_count(const stq_handle* h);
+/* Persistent grid the step kernel uses on this device (CTAs), and the device's SM count. */
+int stq_grid_size(const stq_handle* h);
+int stq_sm_count(const stq_handle* h);
+
+/* ---- transition decision (host only; Sec. 3.3-3.4, Algorithm 1 decision branch) -------------- */
+typedef struct stq_policy_cfg {
+  double alpha;         /* EMA factor of the three global running statistics                  */
+  double tau;           /* decay period of the annealing factor S_t = 1 + sech(t/tau) (Eq. 7) */
+  double eps_stat;      /* the small constant in r_l and in the score denominators            */
+  int64_t interval;     /* U: decide when t mod U == 0 or t < 5                               */
+  int32_t cv_of_signed; /* 0: sigma(|g|)/mu(|g|) (Eq. 3); 1: sigma(g)/E|g| (Algorithm 1 text)  */
+  int32_t reserved;
+} stq_policy_cfg;
+
+int stq_policy_create(stq_policy** out, const stq_policy_cfg* cfg);
+int stq_policy_destroy(stq_policy* p);
+/* 1 if Algorithm 1 takes the decision branch at step t. */
+int stq_policy_is_decision_step(const stq_policy* p, int64_t t);
+/* One decision, O(L): updates the running averages from stats[L][4] (as written by
+ * stq_layer_stats), then score_l = 7.2 + log2 ratios (Sec. 3.4) and bits_out[l] = Map(score_l)
+ * in {4, 8, 16, 32} with thresholds 6.8 / 12 / 24.  score_out may be NULL. */
+int stq_decide(stq_policy* p, const double* stats, int L, int64_t t, uint8_t* bits_out,
+               double* score_out);
+/* Running averages {n, r, v} for checkpointing. */
+int stq_policy_get_state(const stq_policy* p, double out[3]);
+int stq_policy_set_state(stq_policy* p, const double in[3]);
+
+const char* stq_strerror(int code);
+/* Text of the last CUDA error seen by this handle ("" if none). */
+const char* stq_last_cuda_error(const stq_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STQ_H_ */

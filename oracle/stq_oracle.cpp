@@ -192,7 +192,7 @@ struct orc_hparams {
   int grad_dtype;      // 0 = fp32, 1 = bf16
 };
 
-uint64_t orc_codes_bytes(uint64_t n, int bits) { return bits == 32 ? n * 4 : codes_bytes(n, bits); }
+uint64_t orc_codes_bytes(uint64_t n, int bits) { return codes_bytes(n, bits); }
 uint64_t orc_num_blocks(uint64_t n, uint32_t block) { return (n + block - 1) / block; }
 
 float orc_lg_P(float x) { return lg_P(x); }

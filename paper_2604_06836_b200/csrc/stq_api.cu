@@ -1,0 +1,527 @@
+// C-ABI host layer of libstq: argument validation, tensor-table and tile-map upload, launches.
+// No arithmetic of the method lives here; every step of the path runs in stq_kernels.cu.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/stq.h"
+#include "stq_internal.h"
+
+using stq::TensorDesc;
+
+struct stq_handle {
+  int device = 0;
+  int sm_count = 0;
+  int grid = 0;
+  uint64_t launches = 0;
+  std::string cuda_err;
+
+  // cached caller table (to skip re-uploads) and its device image
+  std::vector<stq_tensor> cached;
+  int cached_kind = -1;          // which entry point built the device table
+  std::vector<uint64_t> cached_sig;   // numel | wide<<63 per tensor: decides the tile map
+  TensorDesc* d_table = nullptr;
+  size_t d_table_cap = 0;
+  uint32_t* d_tile_map = nullptr;   // tile -> tensor index, narrow tiles first, then wide
+  size_t d_tile_cap = 0;
+  uint32_t* d_ntiles = nullptr;     // per tensor
+  size_t d_ntiles_cap = 0;
+  uint32_t n_tiles = 0, n_narrow = 0;
+
+  // pinned staging for uploads
+  void* h_stage = nullptr;
+  size_t h_stage_cap = 0;
+  cudaEvent_t stage_ev = nullptr;
+  bool stage_busy = false;
+
+  // statistics
+  double* d_partials = nullptr;
+  size_t d_partials_cap = 0;
+  double* d_stats = nullptr;
+  size_t d_stats_cap = 0;
+  double* h_stats = nullptr;
+  size_t h_stats_cap = 0;
+  int stats_L = 0;            // > 0: partials of a table with this many tensors are pending
+
+  // device arena of stq_step_host
+  uint8_t* d_arena = nullptr;
+  size_t d_arena_cap = 0;
+};
+
+namespace {
+
+enum Kind { kKindStep = 0, kKindRepack = 1, kKindInit = 2, kKindStats = 3 };
+
+bool width_ok(int b) { return b == 2 || b == 3 || b == 4 || b == 8 || b == 16 || b == 32; }
+bool block_ok(uint32_t b) { return b == 128 || b == 256 || b == 512; }
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int fail_cuda(stq_handle* h, cudaError_t e) {
+  h->cuda_err = cudaGetErrorString(e);
+  return STQ_E_CUDA;
+}
+#define STQ_CUDA(h, call)                                   \
+  do {                                                      \
+    cudaError_t e__ = (call);                               \
+    if (e__ != cudaSuccess) return fail_cuda((h), e__);     \
+  } while (0)
+
+template <class T>
+int grow(stq_handle* h, T*& p, size_t& cap, size_t need) {
+  if (need <= cap) return STQ_OK;
+  if (p) cudaFree(p);
+  p = nullptr;
+  cap = 0;
+  size_t want = need + need / 4 + 256;
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&p), want * sizeof(T));
+  if (e != cudaSuccess) { h->cuda_err = cudaGetErrorString(e); p = nullptr; return STQ_E_WORKSPACE; }
+  cap = want;
+  return STQ_OK;
+}
+
+int grow_stage(stq_handle* h, size_t bytes) {
+  if (bytes <= h->h_stage_cap) return STQ_OK;
+  if (h->stage_busy) { cudaEventSynchronize(h->stage_ev); h->stage_busy = false; }
+  if (h->h_stage) cudaFreeHost(h->h_stage);
+  h->h_stage = nullptr;
+  h->h_stage_cap = 0;
+  size_t want = bytes + bytes / 4 + 4096;
+  cudaError_t e = cudaMallocHost(&h->h_stage, want);
+  if (e != cudaSuccess) { h->cuda_err = cudaGetErrorString(e); h->h_stage = nullptr; return STQ_E_WORKSPACE; }
+  h->h_stage_cap = want;
+  return STQ_OK;
+}
+
+bool overlap(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+  return x < y + nb && y < x + na;
+}
+
+// Host-side validation of one row for the given entry point.
+int validate_row(const stq_tensor& t, int kind) {
+  if (t.numel == 0 || t.numel > (1ull << 40)) return STQ_E_NUMEL;
+  if (t.reserved != 0) return STQ_E_ARG;
+  if (kind == kKindStats) {
+    if (!t.grad) return STQ_E_NULL;
+    if (!aligned(t.grad, 16)) return STQ_E_ALIGN;
+    return STQ_OK;
+  }
+  if (!block_ok(t.block)) return STQ_E_BLOCK;
+  if (!width_ok(t.bits_m_out) || !width_ok(t.bits_v_out)) return STQ_E_BITS;
+  if (!t.m_codes_out || !t.v_codes_out) return STQ_E_NULL;
+  if (t.bits_m_out != 32 && !t.m_scales_out) return STQ_E_NULL;
+  if (t.bits_v_out != 32 && !t.v_scales_out) return STQ_E_NULL;
+  if (!aligned(t.m_codes_out, 16) || !aligned(t.v_codes_out, 16)) return STQ_E_ALIGN;
+  if (!aligned(t.m_scales_out, 4) || !aligned(t.v_scales_out, 4)) return STQ_E_ALIGN;
+  if (kind == kKindInit) return STQ_OK;
+
+  if (!width_ok(t.bits_m) || !width_ok(t.bits_v)) return STQ_E_BITS;
+  if (!t.m_codes_in || !t.v_codes_in) return STQ_E_NULL;
+  if (t.bits_m != 32 && !t.m_scales_in) return STQ_E_NULL;
+  if (t.bits_v != 32 && !t.v_scales_in) return STQ_E_NULL;
+  if (!aligned(t.m_codes_in, 16) || !aligned(t.v_codes_in, 16)) return STQ_E_ALIGN;
+  if (!aligned(t.m_scales_in, 4) || !aligned(t.v_scales_in, 4)) return STQ_E_ALIGN;
+  if (kind == kKindStep) {
+    if (!t.param || !t.grad) return STQ_E_NULL;
+    if (!aligned(t.param, 16) || !aligned(t.grad, 16)) return STQ_E_ALIGN;
+  }
+  // in-place is allowed only for identical pointer and identical width
+  const size_t mi = stq_codes_bytes(t.numel, t.bits_m), mo = stq_codes_bytes(t.numel, t.bits_m_out);
+  const size_t vi = stq_codes_bytes(t.numel, t.bits_v), vo = stq_codes_bytes(t.numel, t.bits_v_out);
+  if (overlap(t.m_codes_in, mi, t.m_codes_out, mo) &&
+      !(t.m_codes_in == t.m_codes_out && t.bits_m == t.bits_m_out))
+    return STQ_E_ALIAS;
+  if (overlap(t.v_codes_in, vi, t.v_codes_out, vo) &&
+      !(t.v_codes_in == t.v_codes_out && t.bits_v == t.bits_v_out))
+    return STQ_E_ALIAS;
+  if (overlap(t.m_codes_out, mo, t.v_codes_out, vo) || overlap(t.m_codes_in, mi, t.v_codes_out, vo) ||
+      overlap(t.v_codes_in, vi, t.m_codes_out, mo))
+    return STQ_E_ALIAS;
+  const size_t sb = stq_scales_bytes(t.numel, t.block);
+  if (t.bits_m != 32 && t.bits_m_out != 32 && t.m_scales_in != t.m_scales_out &&
+      overlap(t.m_scales_in, sb, t.m_scales_out, sb))
+    return STQ_E_ALIAS;
+  if (t.bits_v != 32 && t.bits_v_out != 32 && t.v_scales_in != t.v_scales_out &&
+      overlap(t.v_scales_in, sb, t.v_scales_out, sb))
+    return STQ_E_ALIAS;
+  return STQ_OK;
+}
+
+bool row_is_wide(const stq_tensor& t, int kind) {
+  if (kind == kKindStats) return false;
+  if (t.bits_m_out == 32 || t.bits_v_out == 32) return true;
+  if (kind != kKindInit && (t.bits_m == 32 || t.bits_v == 32)) return true;
+  return false;
+}
+
+// Builds (or reuses) the device table and tile map for `tensors`.
+int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStream_t stream) {
+  if (!h || !tensors) return STQ_E_NULL;
+  if (L <= 0 || L > (1 << 20)) return STQ_E_NUMEL;
+  for (int l = 0; l < L; ++l) {
+    int rc = validate_row(tensors[l], kind);
+    if (rc != STQ_OK) return rc;
+  }
+  STQ_CUDA(h, cudaSetDevice(h->device));
+  const bool same = h->cached_kind == kind && (int)h->cached.size() == L &&
+                    std::memcmp(h->cached.data(), tensors, sizeof(stq_tensor) * (size_t)L) == 0;
+  if (same) return STQ_OK;
+
+  // tile counts; narrow tensors first, wide (any 32-bit state) after
+  std::vector<uint32_t> ntiles(L), tile0(L);
+  std::vector<uint64_t> sig(L);
+  uint64_t total = 0, narrow = 0;
+  for (int l = 0; l < L; ++l) {
+    uint64_t nt = (tensors[l].numel + stq::kTile - 1) / stq::kTile;
+    ntiles[l] = (uint32_t)nt;
+    total += nt;
+    const bool wide = row_is_wide(tensors[l], kind);
+    if (!wide) narrow += nt;
+    sig[l] = tensors[l].numel | (wide ? 1ull << 63 : 0ull);
+  }
+  // the tile map depends only on sizes and on which tensors are wide: skip it when unchanged
+  const bool same_map = h->cached_kind >= 0 && sig == h->cached_sig && h->n_tiles == (uint32_t)total;
+  if (total > 0xFFFFFFF0ull) return STQ_E_NUMEL;
+
+  const size_t bytes_table = sizeof(TensorDesc) * (size_t)L;
+  const size_t bytes_map = sizeof(uint32_t) * (size_t)total;
+  const size_t bytes_nt = sizeof(uint32_t) * (size_t)L;
+  const size_t off_map = (bytes_table + 255) & ~size_t(255);
+  const size_t off_nt = (off_map + bytes_map + 255) & ~size_t(255);
+  int rc;
+  if ((rc = grow_stage(h, off_nt + bytes_nt)) != STQ_OK) return rc;
+  if ((rc = grow(h, h->d_table, h->d_table_cap, (size_t)L)) != STQ_OK) return rc;
+  if ((rc = grow(h, h->d_tile_map, h->d_tile_cap, (size_t)total)) != STQ_OK) return rc;
+  if ((rc = grow(h, h->d_ntiles, h->d_ntiles_cap, (size_t)L)) != STQ_OK) return rc;
+  if (h->stage_busy) { STQ_CUDA(h, cudaEventSynchronize(h->stage_ev)); h->stage_busy = false; }
+
+  uint8_t* st = static_cast<uint8_t*>(h->h_stage);
+  TensorDesc* ht = reinterpret_cast<TensorDesc*>(st);
+  uint32_t* hm = reinterpret_cast<uint32_t*>(st + off_map);
+  uint32_t* hn = reinterpret_cast<uint32_t*>(st + off_nt);
+  uint32_t next_narrow = 0, next_wide = (uint32_t)narrow;
+  for (int l = 0; l < L; ++l) {
+    const stq_tensor& t = tensors[l];
+    uint32_t& next = row_is_wide(t, kind) ? next_wide : next_narrow;
+    tile0[l] = next;
+    for (uint32_t i = 0; i < ntiles[l]; ++i) hm[next + i] = (uint32_t)l;
+    next += ntiles[l];
+    hn[l] = ntiles[l];
+    TensorDesc d;
+    std::memset(&d, 0, sizeof(d));
+    d.param = t.param;
+    d.grad = t.grad;
+    d.mc_in = static_cast<const uint8_t*>(t.m_codes_in);
+    d.ms_in = t.m_scales_in;
+    d.vc_in = static_cast<const uint8_t*>(t.v_codes_in);
+    d.vs_in = t.v_scales_in;
+    d.mc_out = static_cast<uint8_t*>(t.m_codes_out);
+    d.ms_out = t.m_scales_out;
+    d.vc_out = static_cast<uint8_t*>(t.v_codes_out);
+    d.vs_out = t.v_scales_out;
+    d.numel = t.numel;
+    d.tile0 = tile0[l];
+    d.block = kind == kKindStats ? 128u : t.block;
+    d.bm_in = t.bits_m; d.bv_in = t.bits_v; d.bm_out = t.bits_m_out; d.bv_out = t.bits_v_out;
+    d.wd = t.weight_decay;
+    ht[l] = d;
+  }
+  STQ_CUDA(h, cudaMemcpyAsync(h->d_table, ht, bytes_table, cudaMemcpyHostToDevice, stream));
+  if (!same_map) {
+    STQ_CUDA(h, cudaMemcpyAsync(h->d_tile_map, hm, bytes_map, cudaMemcpyHostToDevice, stream));
+    STQ_CUDA(h, cudaMemcpyAsync(h->d_ntiles, hn, bytes_nt, cudaMemcpyHostToDevice, stream));
+  }
+  STQ_CUDA(h, cudaEventRecord(h->stage_ev, stream));
+  h->stage_busy = true;
+  h->cached.assign(tensors, tensors + L);
+  h->cached_kind = kind;
+  h->cached_sig.swap(sig);
+  h->n_tiles = (uint32_t)total;
+  h->n_narrow = (uint32_t)narrow;
+  return STQ_OK;
+}
+
+int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::StepConsts& sc,
+        cudaStream_t stream) {
+  double* partials = nullptr;
+  if (stats) {
+    int rc = grow(h, h->d_partials, h->d_partials_cap, (size_t)h->n_tiles * 3);
+    if (rc != STQ_OK) return rc;
+    partials = h->d_partials;
+  }
+  if (h->n_narrow > 0) {
+    STQ_CUDA(h, stq::launch_tiles(mode, false, grad_dtype, stats, h->d_table, h->d_tile_map, 0, h->n_narrow,
+                                  sc, partials, h->grid, stream));
+    h->launches++;
+  }
+  if (h->n_tiles > h->n_narrow) {
+    STQ_CUDA(h, stq::launch_tiles(mode, true, grad_dtype, stats, h->d_table, h->d_tile_map, h->n_narrow,
+                                  h->n_tiles, sc, partials, h->grid, stream));
+    h->launches++;
+  }
+  return STQ_OK;
+}
+
+int check_hparams(const stq_hparams* hp, unsigned flags) {
+  if (!hp) return STQ_E_NULL;
+  if (hp->step < 1) return STQ_E_ARG;
+  if (hp->grad_dtype != STQ_GRAD_F32 && hp->grad_dtype != STQ_GRAD_BF16) return STQ_E_ARG;
+  if (flags & ~(unsigned)STQ_WITH_STATS) return STQ_E_ARG;
+  if (!(hp->beta1 >= 0.0 && hp->beta1 < 1.0 && hp->beta2 >= 0.0 && hp->beta2 < 1.0)) return STQ_E_ARG;
+  return STQ_OK;
+}
+
+stq::StepConsts make_consts(const stq_hparams* hp) {
+  stq::StepConsts sc;
+  sc.b1 = (float)hp->beta1;
+  sc.c1 = (float)(1.0 - hp->beta1);
+  sc.b2 = (float)hp->beta2;
+  sc.c2 = (float)(1.0 - hp->beta2);
+  const double bc1 = 1.0 - std::pow(hp->beta1, (double)hp->step);
+  const double bc2 = 1.0 - std::pow(hp->beta2, (double)hp->step);
+  sc.step_size = (float)(hp->lr / bc1);
+  sc.rsqrt_bc2 = (float)(1.0 / std::sqrt(bc2));
+  sc.eps = (float)hp->eps;
+  sc.l2_mode = hp->decoupled_wd ? 0 : 1;
+  sc.lr = hp->lr;
+  return sc;
+}
+
+}  // namespace
+
+extern "C" {
+
+int stq_create(stq_handle** out, int device) {
+  if (!out) return STQ_E_NULL;
+  *out = nullptr;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return STQ_E_CUDA;
+  if (cudaSetDevice(device) != cudaSuccess) return STQ_E_CUDA;
+  stq_handle* h = new (std::nothrow) stq_handle();
+  if (!h) return STQ_E_WORKSPACE;
+  h->device = device;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->stage_ev, cudaEventDisableTiming) != cudaSuccess) {
+    delete h;
+    return STQ_E_CUDA;
+  }
+  h->sm_count = prop.multiProcessorCount;
+  h->grid = h->sm_count * stq::step_ctas_per_sm();
+  *out = h;
+  return STQ_OK;
+}
+
+int stq_destroy(stq_handle* h) {
+  if (!h) return STQ_E_NULL;
+  cudaSetDevice(h->device);
+  if (h->stage_busy) cudaEventSynchronize(h->stage_ev);
+  cudaFree(h->d_table);
+  cudaFree(h->d_tile_map);
+  cudaFree(h->d_ntiles);
+  cudaFree(h->d_partials);
+  cudaFree(h->d_stats);
+  cudaFree(h->d_arena);
+  if (h->h_stage) cudaFreeHost(h->h_stage);
+  if (h->h_stats) cudaFreeHost(h->h_stats);
+  if (h->stage_ev) cudaEventDestroy(h->stage_ev);
+  delete h;
+  return STQ_OK;
+}
+
+size_t stq_codes_bytes(uint64_t numel, int bits) {
+  const uint64_t by = (numel * (uint64_t)bits + 7) / 8;
+  return (size_t)((by + 15) / 16 * 16);
+}
+
+size_t stq_scales_bytes(uint64_t numel, uint32_t block) {
+  if (block == 0) return 0;
+  return (size_t)((numel + block - 1) / block * 4);
+}
+
+int stq_init_state(stq_handle* h, const stq_tensor* tensors, int L, void* stream) {
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = prepare(h, tensors, L, kKindInit, s);
+  if (rc != STQ_OK) return rc;
+  stq::StepConsts sc;
+  std::memset(&sc, 0, sizeof(sc));
+  return run(h, stq::kInit, 0, false, sc, s);
+}
+
+int stq_step(stq_handle* h, const stq_tensor* tensors, int L, const stq_hparams* hp, unsigned flags,
+             void* stream) {
+  if (!h) return STQ_E_NULL;
+  int rc = check_hparams(hp, flags);
+  if (rc != STQ_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  rc = prepare(h, tensors, L, kKindStep, s);
+  if (rc != STQ_OK) return rc;
+  const bool stats = (flags & STQ_WITH_STATS) != 0;
+  rc = run(h, stq::kStep, hp->grad_dtype, stats, make_consts(hp), s);
+  if (rc == STQ_OK && stats) h->stats_L = L;
+  return rc;
+}
+
+int stq_grad_stats(stq_handle* h, const stq_tensor* tensors, int L, int grad_dtype, void* stream) {
+  if (!h) return STQ_E_NULL;
+  if (grad_dtype != STQ_GRAD_F32 && grad_dtype != STQ_GRAD_BF16) return STQ_E_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = prepare(h, tensors, L, kKindStats, s);
+  if (rc != STQ_OK) return rc;
+  stq::StepConsts sc;
+  std::memset(&sc, 0, sizeof(sc));
+  rc = run(h, stq::kStatsOnly, grad_dtype, true, sc, s);
+  if (rc == STQ_OK) h->stats_L = L;
+  return rc;
+}
+
+int stq_layer_stats(stq_handle* h, double* out, int L, void* stream) {
+  if (!h || !out) return STQ_E_NULL;
+  if (h->stats_L <= 0 || L != h->stats_L) return STQ_E_STATE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  STQ_CUDA(h, cudaSetDevice(h->device));
+  int rc = grow(h, h->d_stats, h->d_stats_cap, (size_t)L * 4);
+  if (rc != STQ_OK) return rc;
+  if ((size_t)L * 4 > h->h_stats_cap) {
+    if (h->h_stats) cudaFreeHost(h->h_stats);
+    h->h_stats = nullptr;
+    h->h_stats_cap = 0;
+    cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&h->h_stats), sizeof(double) * 4 * (size_t)L);
+    if (e != cudaSuccess) { h->cuda_err = cudaGetErrorString(e); return STQ_E_WORKSPACE; }
+    h->h_stats_cap = (size_t)L * 4;
+  }
+  STQ_CUDA(h, stq::launch_stats_finish(h->d_table, h->d_ntiles, L, h->d_partials, h->d_stats, s));
+  h->launches++;
+  STQ_CUDA(h, cudaMemcpyAsync(h->h_stats, h->d_stats, sizeof(double) * 4 * (size_t)L, cudaMemcpyDeviceToHost, s));
+  STQ_CUDA(h, cudaStreamSynchronize(s));
+  std::memcpy(out, h->h_stats, sizeof(double) * 4 * (size_t)L);
+  return STQ_OK;
+}
+
+int stq_repack(stq_handle* h, const stq_tensor* tensors, int L, void* stream) {
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = prepare(h, tensors, L, kKindRepack, s);
+  if (rc != STQ_OK) return rc;
+  stq::StepConsts sc;
+  std::memset(&sc, 0, sizeof(sc));
+  return run(h, stq::kRepack, 0, false, sc, s);
+}
+
+int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hparams* hp, unsigned flags,
+                  uint64_t* bytes_h2d, uint64_t* bytes_d2h) {
+  if (!h || !tensors) return STQ_E_NULL;
+  int rc = check_hparams(hp, flags);
+  if (rc != STQ_OK) return rc;
+  if (L <= 0 || L > (1 << 20)) return STQ_E_NUMEL;
+  STQ_CUDA(h, cudaSetDevice(h->device));
+  // validate with the host pointers (same rules: alignment, widths, aliasing)
+  for (int l = 0; l < L; ++l) {
+    rc = validate_row(tensors[l], kKindStep);
+    if (rc != STQ_OK) return rc;
+  }
+  // lay the device arena out: every buffer 256-byte aligned
+  auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
+  const size_t gsz = hp->grad_dtype == STQ_GRAD_BF16 ? 2 : 4;
+  size_t need = 0;
+  for (int l = 0; l < L; ++l) {
+    const stq_tensor& t = tensors[l];
+    const size_t sb = stq_scales_bytes(t.numel, t.block);
+    need += up(t.numel * 4) + up(t.numel * gsz);
+    need += up(stq_codes_bytes(t.numel, t.bits_m)) + up(stq_codes_bytes(t.numel, t.bits_v)) + 2 * up(sb);
+    if (t.bits_m_out != t.bits_m) need += up(stq_codes_bytes(t.numel, t.bits_m_out));
+    if (t.bits_v_out != t.bits_v) need += up(stq_codes_bytes(t.numel, t.bits_v_out));
+  }
+  rc = grow(h, h->d_arena, h->d_arena_cap, need);
+  if (rc != STQ_OK) return rc;
+
+  cudaStream_t s = nullptr;   // the legacy default stream: ordered with everything else
+  std::vector<stq_tensor> dev(tensors, tensors + L);
+  uint64_t h2d = 0, d2h = 0;
+  size_t off = 0;
+  auto place = [&](size_t bytes) { uint8_t* p = h->d_arena + off; off += up(bytes); return p; };
+  for (int l = 0; l < L; ++l) {
+    const stq_tensor& t = tensors[l];
+    stq_tensor& d = dev[l];
+    const size_t sb = stq_scales_bytes(t.numel, t.block);
+    const size_t mi = stq_codes_bytes(t.numel, t.bits_m), vi = stq_codes_bytes(t.numel, t.bits_v);
+    d.param = reinterpret_cast<float*>(place(t.numel * 4));
+    d.grad = place(t.numel * gsz);
+    d.m_codes_in = place(mi);
+    d.v_codes_in = place(vi);
+    d.m_scales_in = reinterpret_cast<float*>(place(sb));
+    d.v_scales_in = reinterpret_cast<float*>(place(sb));
+    d.m_codes_out = t.bits_m_out != t.bits_m ? place(stq_codes_bytes(t.numel, t.bits_m_out))
+                                             : const_cast<void*>(d.m_codes_in);
+    d.v_codes_out = t.bits_v_out != t.bits_v ? place(stq_codes_bytes(t.numel, t.bits_v_out))
+                                             : const_cast<void*>(d.v_codes_in);
+    d.m_scales_out = const_cast<float*>(d.m_scales_in);
+    d.v_scales_out = const_cast<float*>(d.v_scales_in);
+    STQ_CUDA(h, cudaMemcpyAsync(d.param, t.param, t.numel * 4, cudaMemcpyHostToDevice, s));
+    STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.grad), t.grad, t.numel * gsz, cudaMemcpyHostToDevice, s));
+    STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.m_codes_in), t.m_codes_in, mi, cudaMemcpyHostToDevice, s));
+    STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.v_codes_in), t.v_codes_in, vi, cudaMemcpyHostToDevice, s));
+    h2d += t.numel * 4 + t.numel * gsz + mi + vi;
+    if (t.bits_m != 32) {
+      STQ_CUDA(h, cudaMemcpyAsync(const_cast<float*>(d.m_scales_in), t.m_scales_in, sb, cudaMemcpyHostToDevice, s));
+      h2d += sb;
+    }
+    if (t.bits_v != 32) {
+      STQ_CUDA(h, cudaMemcpyAsync(const_cast<float*>(d.v_scales_in), t.v_scales_in, sb, cudaMemcpyHostToDevice, s));
+      h2d += sb;
+    }
+  }
+  rc = stq_step(h, dev.data(), L, hp, flags, s);
+  if (rc != STQ_OK) return rc;
+  for (int l = 0; l < L; ++l) {
+    const stq_tensor& t = tensors[l];
+    const stq_tensor& d = dev[l];
+    const size_t sb = stq_scales_bytes(t.numel, t.block);
+    const size_t mo = stq_codes_bytes(t.numel, t.bits_m_out), vo = stq_codes_bytes(t.numel, t.bits_v_out);
+    STQ_CUDA(h, cudaMemcpyAsync(t.param, d.param, t.numel * 4, cudaMemcpyDeviceToHost, s));
+    STQ_CUDA(h, cudaMemcpyAsync(t.m_codes_out, d.m_codes_out, mo, cudaMemcpyDeviceToHost, s));
+    STQ_CUDA(h, cudaMemcpyAsync(t.v_codes_out, d.v_codes_out, vo, cudaMemcpyDeviceToHost, s));
+    d2h += t.numel * 4 + mo + vo;
+    if (t.bits_m_out != 32) {
+      STQ_CUDA(h, cudaMemcpyAsync(t.m_scales_out, d.m_scales_out, sb, cudaMemcpyDeviceToHost, s));
+      d2h += sb;
+    }
+    if (t.bits_v_out != 32) {
+      STQ_CUDA(h, cudaMemcpyAsync(t.v_scales_out, d.v_scales_out, sb, cudaMemcpyDeviceToHost, s));
+      d2h += sb;
+    }
+  }
+  STQ_CUDA(h, cudaStreamSynchronize(s));
+  // the cached table now refers to arena addresses; drop it so a later device call re-uploads
+  h->cached_kind = -1;
+  if (bytes_h2d) *bytes_h2d = h2d;
+  if (bytes_d2h) *bytes_d2h = d2h;
+  return STQ_OK;
+}
+
+uint64_t stq_launch_count(const stq_handle* h) { return h ? h->launches : 0; }
+int stq_grid_size(const stq_handle* h) { return h ? h->grid : 0; }
+int stq_sm_count(const stq_handle* h) { return h ? h->sm_count : 0; }
+
+const char* stq_strerror(int code) {
+  switch (code) {
+    case STQ_OK: return "ok";
+    case STQ_E_NULL: return "a required pointer is NULL";
+    case STQ_E_BITS: return "bit-width not in {2,3,4,8,16,32}";
+    case STQ_E_BLOCK: return "block not in {128,256,512}";
+    case STQ_E_ALIGN: return "buffer not aligned (16 bytes for param/grad/codes, 4 for scales)";
+    case STQ_E_ALIAS: return "in/out buffers overlap (in-place needs the same pointer and width)";
+    case STQ_E_NUMEL: return "numel is 0, or the table is empty or too large";
+    case STQ_E_CUDA: return "CUDA runtime error";
+    case STQ_E_WORKSPACE: return "could not allocate library workspace";
+    case STQ_E_ARG: return "invalid scalar argument";
+    case STQ_E_STATE: return "no statistics pending for this table";
+    default: return "unknown error";
+  }
+}
+
+const char* stq_last_cuda_error(const stq_handle* h) { return h ? h->cuda_err.c_str() : ""; }
+
+}  // extern "C"

@@ -1,0 +1,58 @@
+// Internal interface between the C-ABI host layer (stq_api.cu) and the kernels (stq_kernels.cu).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace stq {
+
+constexpr int kTile = 4096;      // elements per tile; every tile lies inside one tensor
+constexpr int kThreads = 256;    // 8 warps; a warp owns 4 consecutive 128-element rows of the tile
+constexpr int kRowElems = 128;   // one row: lane l holds elements 4l .. 4l+3
+constexpr int kRowsPerWarp = 4;
+
+// Device-side row of the tensor table.
+struct TensorDesc {
+  float* param;
+  const void* grad;
+  const uint8_t* mc_in;
+  const float* ms_in;
+  const uint8_t* vc_in;
+  const float* vs_in;
+  uint8_t* mc_out;
+  float* ms_out;
+  uint8_t* vc_out;
+  float* vs_out;
+  unsigned long long numel;
+  unsigned int tile0;       // index of this tensor's first tile in the launch's tile order
+  unsigned int block;       // 128 / 256 / 512
+  unsigned char bm_in, bv_in, bm_out, bv_out;
+  float wd;                 // fp32(lambda)
+  unsigned int pad[2];
+};
+
+// Per-launch scalars of the AdamW update.
+struct StepConsts {
+  float b1, c1, b2, c2;     // fp32(beta), fp32(1-beta): the bit-exact moment recursion
+  float step_size;          // lr / (1 - beta1^t)
+  float rsqrt_bc2;          // 1 / sqrt(1 - beta2^t)
+  float eps;
+  int l2_mode;              // 1: g += wd*theta before the moments, no decoupled decay
+  double lr;                // decoupled decay factor is fp32(1 - lr*wd), formed per tile
+};
+
+enum Mode { kStep = 0, kRepack = 1, kInit = 2, kStatsOnly = 3 };
+
+// Launches the tile range [tile_begin, tile_end) of the table.  `wide` selects the variant that
+// can read/write 32-bit (raw fp32) states.  partials: 3 doubles per tile or nullptr.
+cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const TensorDesc* table,
+                         const uint32_t* tile_map, uint32_t tile_begin, uint32_t tile_end,
+                         const StepConsts& sc, double* partials, int grid, cudaStream_t stream);
+
+// out[l] = {sum over the tensor's tiles of partials (fixed order), numel}
+cudaError_t launch_stats_finish(const TensorDesc* table, const uint32_t* ntiles_of, int L,
+                                const double* partials, double* out, cudaStream_t stream);
+
+// Resident CTAs per SM of the step kernel (occupancy query), for sizing the persistent grid.
+int step_ctas_per_sm();
+
+}  // namespace stq

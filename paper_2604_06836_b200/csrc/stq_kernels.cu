@@ -1,0 +1,694 @@
+// Kernels of the mixed-bit quantized AdamW step for sm_100a.
+//
+// Work decomposition: the concatenated tensor list is cut into tiles of 4096 elements that never
+// cross a tensor; persistent CTAs of 8 warps stride over the tile list.  Inside a tile a warp owns
+// 4 consecutive rows of 128 elements and lane l of a row holds elements 4l..4l+3, so parameters
+// and fp32 gradients move as 128-bit accesses (512 contiguous bytes per warp), bf16 gradients as
+// 64-bit ones, and a lane's four codes are one 8/16/32/64-bit access at widths 2/4/8/16 (3-bit
+// rows are 48 bytes: 12 lanes move one word each and the 12-bit lane fields are exchanged with
+// shuffles).  A quantization block (128/256/512) is 1/2/4 whole rows of one warp, so the block
+// maximum is a lane-local max of 4 followed by one warp REDUX on the (non-negative) bit patterns.
+//
+// Arithmetic that decides codes is written with the *_rn intrinsics, which are never contracted,
+// and the file is compiled with -fmad=false; fused operations appear only where the quantizer is
+// defined with them.  Round-half-even to integer is done by adding 1.5*2^23 (one FFMA on the exact
+// product), and the integer sits in the low mantissa bits of the result, which is also how the
+// codes are packed: sum_k bits_k << (k*b) minus a per-width constant.
+#include "stq_internal.h"
+
+namespace stq {
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23: ulp 1, even
+constexpr uint32_t kMagicBits = 0x4B400000u;   // its bit pattern (low 22 bits clear)
+constexpr float kTwo23 = 8388608.0f;
+constexpr uint32_t kTwo23Bits = 0x4B000000u;
+constexpr float kTiny = 0x1p-100f;                //: smaller block maxima store a zero block
+constexpr int kZeroBlockExp = 1 << 20;            // exponent stand-in that floors every log code
+
+// P(t) ~ log2(1+t) = t*(c1 + t*(c2 + ... + t*c6)), t in [0,1)
+constexpr float kP1 = 0x1.714b30p+0f, kP2 = -0x1.6fc360p-1f, kP3 = 0x1.d54a42p-2f,
+                kP4 = -0x1.1e4792p-2f, kP5 = 0x1.f9c008p-4f, kP6 = -0x1.b19412p-6f;
+// 2^f ~ 1 + f*(e0 + f*(e1 + ... + f*e4)), |f| <= 1/2
+constexpr float kE0 = 0x1.62e42ap-1f, kE1 = 0x1.ebf9bcp-3f, kE2 = 0x1.c6b74cp-5f,
+                kE3 = 0x1.3cea84p-7f, kE4 = 0x1.5bbc6ap-10f;
+
+__device__ __forceinline__ float lg_poly(uint32_t bits) {
+  const float mant = __uint_as_float((bits & 0x007FFFFFu) | 0x3F800000u);
+  const float t = __fadd_rn(mant, -1.0f);
+  float a = kP6;
+  a = __fmaf_rn(a, t, kP5);
+  a = __fmaf_rn(a, t, kP4);
+  a = __fmaf_rn(a, t, kP3);
+  a = __fmaf_rn(a, t, kP2);
+  a = __fmaf_rn(a, t, kP1);
+  return __fmul_rn(a, t);
+}
+
+// 2^e for e <= 0 by nearest-integer range reduction; returns p * 2^i.
+__device__ __forceinline__ float ex2_poly(float e) {
+  const float ti = __fadd_rn(e, kMagic);          // low mantissa bits = round-half-even(e)
+  const float fi = __fadd_rn(ti, -kMagic);
+  const float f = __fadd_rn(e, -fi);
+  float a = kE4;
+  a = __fmaf_rn(a, f, kE3);
+  a = __fmaf_rn(a, f, kE2);
+  a = __fmaf_rn(a, f, kE1);
+  a = __fmaf_rn(a, f, kE0);
+  const float p = __fmaf_rn(a, f, 1.0f);
+  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(ti) << 23));
+}
+
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float y;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---- per-width constants (warp-uniform, set up once per tile) ---------------------------------
+struct LinW {
+  float invq;    // fl(1/qmax)
+  float qmaxf;
+  float halff;   // 2^(b-1), the code offset
+};
+struct LogW {
+  float a;       // K/R codes per octave (exact)
+  float c;       // fl(R/K) octaves per code
+  float negR;    // -R: lowest log-distance that still has a code
+  int K;
+};
+__device__ __forceinline__ LinW lin_width(int b) {
+  LinW w;
+  const int half = 1 << ((b > 16 ? 16 : b) - 1);
+  w.qmaxf = (float)(half - 1);
+  w.invq = __fdiv_rn(1.0f, w.qmaxf);
+  w.halff = (float)half;
+  return w;
+}
+__device__ __forceinline__ LogW log_width(int b) {
+  LogW w;
+  const int K = (1 << (b > 16 ? 16 : b)) - 1;
+  const int R = K < 30 ? K : 30;
+  w.K = K;
+  w.a = __fdiv_rn((float)K, (float)R);
+  w.c = __fdiv_rn((float)R, (float)K);
+  w.negR = -(float)R;
+  return w;
+}
+
+// ---- raw code words of one lane for one row ---------------------------------------------------
+template <bool WIDE>
+struct Raw {
+  uint32_t w[WIDE ? 4 : 2];
+};
+
+// Loads the lane's share of a row's codes.  row_e0 is a multiple of 128; `limit` is the padded
+// byte size of the code buffer, so tail rows never read past it.
+template <bool WIDE>
+__device__ __forceinline__ void load_codes(const uint8_t* base, unsigned long long row_e0, int b,
+                                           int lane, unsigned long long limit, Raw<WIDE>& r) {
+  r.w[0] = 0u;
+  r.w[1] = 0u;
+  const unsigned long long rb = (row_e0 >> 3) * (unsigned)b;
+  switch (b) {
+    case 2: {
+      const unsigned long long off = rb + lane;
+      if (off < limit) r.w[0] = *(base + off);
+    } break;
+    case 3: {
+      const unsigned long long off = rb + 4 * lane;
+      if (lane < 12 && off < limit) r.w[0] = *reinterpret_cast<const uint32_t*>(base + off);
+    } break;
+    case 4: {
+      const unsigned long long off = rb + 2 * lane;
+      if (off < limit) r.w[0] = *reinterpret_cast<const uint16_t*>(base + off);
+    } break;
+    case 8: {
+      const unsigned long long off = rb + 4 * lane;
+      if (off < limit) r.w[0] = *reinterpret_cast<const uint32_t*>(base + off);
+    } break;
+    case 16: {
+      const unsigned long long off = rb + 8 * lane;
+      if (off < limit) {
+        const uint2 v = *reinterpret_cast<const uint2*>(base + off);
+        r.w[0] = v.x;
+        r.w[1] = v.y;
+      }
+    } break;
+    default:
+      if constexpr (WIDE) {
+        r.w[2] = 0u;
+        r.w[3] = 0u;
+        const unsigned long long off = rb + 16 * lane;   // b == 32: rb = row_e0 * 4
+        if (off < limit) {
+          const uint4 v = *reinterpret_cast<const uint4*>(base + off);
+          r.w[0] = v.x; r.w[1] = v.y; r.w[2] = v.z; r.w[3] = v.w;
+        }
+      }
+      break;
+  }
+}
+
+// Splits the lane's raw words into its four codes.  Must be called by the whole warp (the 3-bit
+// case exchanges words between lanes).
+template <bool WIDE>
+__device__ __forceinline__ void split_codes(const Raw<WIDE>& r, int b, int lane, uint32_t (&c)[4]) {
+  switch (b) {
+    case 2:
+#pragma unroll
+      for (int k = 0; k < 4; ++k) c[k] = (r.w[0] >> (2 * k)) & 3u;
+      break;
+    case 3: {
+      const int bit = 12 * lane;
+      const uint32_t lo = __shfl_sync(kFull, r.w[0], bit >> 5);
+      const uint32_t hi = __shfl_sync(kFull, r.w[0], (bit >> 5) + 1);
+      const uint32_t f = __funnelshift_r(lo, hi, bit & 31);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) c[k] = (f >> (3 * k)) & 7u;
+    } break;
+    case 4:
+#pragma unroll
+      for (int k = 0; k < 4; ++k) c[k] = (r.w[0] >> (4 * k)) & 15u;
+      break;
+    case 8:
+#pragma unroll
+      for (int k = 0; k < 4; ++k) c[k] = (r.w[0] >> (8 * k)) & 255u;
+      break;
+    case 16:
+      c[0] = r.w[0] & 0xFFFFu; c[1] = r.w[0] >> 16;
+      c[2] = r.w[1] & 0xFFFFu; c[3] = r.w[1] >> 16;
+      break;
+    default:
+#pragma unroll
+      for (int k = 0; k < 4; ++k) c[k] = 0u;
+      break;
+  }
+}
+
+// Packs four values x_k = base + u_k (u_k < 2^b) into the lane's field and stores the row.
+// `keep` masks the bits of elements beyond the tensor's end (padding stays zero).
+__device__ __forceinline__ void store_codes(uint8_t* base, unsigned long long row_e0, int b, int lane,
+                                            unsigned long long limit, const uint32_t (&x)[4],
+                                            uint32_t sub, int nvl) {
+  const unsigned long long rb = (row_e0 >> 3) * (unsigned)b;
+  switch (b) {
+    case 2: {
+      uint32_t w = x[0] + (x[1] << 2) + (x[2] << 4) + (x[3] << 6) - sub * 85u;
+      w &= (1u << (2 * nvl)) - 1u;
+      const unsigned long long off = rb + lane;
+      if (off < limit) *(base + off) = (uint8_t)w;
+    } break;
+    case 3: {
+      uint32_t p = x[0] + (x[1] << 3) + (x[2] << 6) + (x[3] << 9) - sub * 585u;
+      p &= (1u << (3 * nvl)) - 1u;
+      // word j of the 48-byte row collects the 12-bit fields that overlap bits [32j, 32j+32)
+      const int j = lane;
+      const int first = (8 * j) / 3;
+      uint32_t w = 0u;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int src = first + i;
+        uint32_t v = __shfl_sync(kFull, p, src & 31);
+        const int sh = 12 * src - 32 * j;
+        if (sh >= 32) v = 0u;
+        else if (sh >= 0) v <<= sh;
+        else v >>= -sh;
+        w |= v;
+      }
+      const unsigned long long off = rb + 4 * lane;
+      if (lane < 12 && off < limit) *reinterpret_cast<uint32_t*>(base + off) = w;
+    } break;
+    case 4: {
+      uint32_t w = x[0] + (x[1] << 4) + (x[2] << 8) + (x[3] << 12) - sub * 4369u;
+      w &= (1u << (4 * nvl)) - 1u;
+      const unsigned long long off = rb + 2 * lane;
+      if (off < limit) *reinterpret_cast<uint16_t*>(base + off) = (uint16_t)w;
+    } break;
+    case 8: {
+      uint32_t w = x[0] + (x[1] << 8) + (x[2] << 16) + (x[3] << 24) - sub * 0x01010101u;
+      w &= nvl >= 4 ? 0xFFFFFFFFu : (1u << (8 * nvl)) - 1u;
+      const unsigned long long off = rb + 4 * lane;
+      if (off < limit) *reinterpret_cast<uint32_t*>(base + off) = w;
+    } break;
+    case 16: {
+      uint32_t w0 = x[0] + (x[1] << 16) - sub * 0x00010001u;
+      uint32_t w1 = x[2] + (x[3] << 16) - sub * 0x00010001u;
+      w0 &= nvl >= 2 ? 0xFFFFFFFFu : (nvl == 1 ? 0xFFFFu : 0u);
+      w1 &= nvl >= 4 ? 0xFFFFFFFFu : (nvl == 3 ? 0xFFFFu : 0u);
+      const unsigned long long off = rb + 8 * lane;
+      if (off < limit) *reinterpret_cast<uint2*>(base + off) = make_uint2(w0, w1);
+    } break;
+    default:
+      break;
+  }
+}
+
+__device__ __forceinline__ void store_raw32(uint8_t* base, unsigned long long row_e0, int lane,
+                                            unsigned long long limit, const float (&x)[4]) {
+  const unsigned long long off = row_e0 * 4 + 16 * lane;
+  if (off < limit) *reinterpret_cast<float4*>(base + off) = make_float4(x[0], x[1], x[2], x[3]);
+}
+
+__device__ __forceinline__ unsigned long long padded_code_bytes(unsigned long long numel, int b) {
+  const unsigned long long by = (numel * (unsigned)b + 7) >> 3;
+  return (by + 15) & ~15ull;
+}
+
+// ---- decode ------------------------------------------------------------------------------------
+__device__ __forceinline__ float decode_lin(uint32_t c, float s, const LinW& w) {
+  const float q = __fadd_rn(__uint_as_float(kTwo23Bits | c), -(kTwo23 + w.halff));
+  return __fmul_rn(s, __fmul_rn(q, w.invq));
+}
+__device__ __forceinline__ float decode_log(uint32_t c, float s, int b, const LogW& w) {
+  if (b <= 4) {   // one octave per code: 2^(c-K)
+    return __fmul_rn(s, __uint_as_float((c + (uint32_t)(127 - w.K)) << 23));
+  }
+  const float rf = __fadd_rn(__uint_as_float(kTwo23Bits | c), -(kTwo23 + (float)w.K));
+  return __fmul_rn(s, ex2_poly(__fmul_rn(rf, w.c)));
+}
+
+template <int GDT>
+struct GradRow;
+template <>
+struct GradRow<0> { float4 v; };
+template <>
+struct GradRow<1> { uint2 v; };
+
+template <int GDT>
+__device__ __forceinline__ void load_grad(const void* grad, unsigned long long e, int nvl, GradRow<GDT>& g) {
+  if constexpr (GDT == 0) {
+    const float* p = reinterpret_cast<const float*>(grad) + e;
+    if (nvl == 4) {
+      g.v = __ldg(reinterpret_cast<const float4*>(p));
+    } else {
+      g.v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (nvl > 0) g.v.x = __ldg(p);
+      if (nvl > 1) g.v.y = __ldg(p + 1);
+      if (nvl > 2) g.v.z = __ldg(p + 2);
+    }
+  } else {
+    const uint16_t* p = reinterpret_cast<const uint16_t*>(grad) + e;
+    if (nvl == 4) {
+      g.v = __ldg(reinterpret_cast<const uint2*>(p));
+    } else {
+      uint32_t a = 0, b = 0, c = 0;
+      if (nvl > 0) a = __ldg(p);
+      if (nvl > 1) b = __ldg(p + 1);
+      if (nvl > 2) c = __ldg(p + 2);
+      g.v = make_uint2(a | (b << 16), c);
+    }
+  }
+}
+template <int GDT>
+__device__ __forceinline__ void widen_grad(const GradRow<GDT>& g, float (&o)[4]) {
+  if constexpr (GDT == 0) {
+    o[0] = g.v.x; o[1] = g.v.y; o[2] = g.v.z; o[3] = g.v.w;
+  } else {
+    o[0] = __uint_as_float(g.v.x << 16);
+    o[1] = __uint_as_float(g.v.x & 0xFFFF0000u);
+    o[2] = __uint_as_float(g.v.y << 16);
+    o[3] = __uint_as_float(g.v.y & 0xFFFF0000u);
+  }
+}
+
+__device__ __forceinline__ float4 load_param(const float* p, int nvl) {
+  if (nvl == 4) return *reinterpret_cast<const float4*>(p);
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (nvl > 0) v.x = p[0];
+  if (nvl > 1) v.y = p[1];
+  if (nvl > 2) v.z = p[2];
+  return v;
+}
+__device__ __forceinline__ void store_param(float* p, int nvl, const float (&x)[4]) {
+  if (nvl == 4) {
+    *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
+  } else {
+    if (nvl > 0) p[0] = x[0];
+    if (nvl > 1) p[1] = x[1];
+    if (nvl > 2) p[2] = x[2];
+  }
+}
+
+// ---- the tile kernel ---------------------------------------------------------------------------
+template <int MODE, int GDT, bool STATS, bool WIDE>
+__global__ void __launch_bounds__(kThreads, 2)
+stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map,
+                uint32_t tile_begin, uint32_t tile_end, const StepConsts sc, double* __restrict__ partials) {
+  constexpr int R = kRowsPerWarp;
+  constexpr bool kHasGrad = (MODE == kStep || MODE == kStatsOnly);
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  __shared__ double s_part[kThreads / 32][3];
+
+  for (uint32_t tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
+    const TensorDesc* __restrict__ T = table + __ldg(tile_map + tile);
+    const unsigned long long numel = T->numel;
+    const unsigned long long e_warp =
+        (unsigned long long)(tile - T->tile0) * kTile + (unsigned)warp * (R * kRowElems);
+    float st_g = 0.f, st_a = 0.f, st_q = 0.f;
+
+    if (e_warp < numel) {
+      const uint32_t B = T->block;
+      const int lgB = 7 + (int)(B >> 8);   // 128 / 256 / 512
+      const int bm_in = T->bm_in, bv_in = T->bv_in, bm_out = T->bm_out, bv_out = T->bv_out;
+
+      int nvl[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const long long rem = (long long)numel - (long long)(e_warp + r * kRowElems) - 4 * lane;
+        nvl[r] = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
+      }
+
+      // ---- issue every load of the four rows before anything is consumed -------------------------
+      float4 th4[R];
+      GradRow<GDT> graw[R];
+      Raw<WIDE> rawm[R], rawv[R];
+      float s_m_in[R], s_v_in[R];
+      if constexpr (MODE == kStep) {
+        float* param = T->param;
+#pragma unroll
+        for (int r = 0; r < R; ++r) th4[r] = load_param(param + e_warp + r * kRowElems + 4 * lane, nvl[r]);
+      }
+      if constexpr (kHasGrad) {
+        const void* grad = T->grad;
+#pragma unroll
+        for (int r = 0; r < R; ++r) load_grad<GDT>(grad, e_warp + r * kRowElems + 4 * lane, nvl[r], graw[r]);
+      }
+      if constexpr (MODE == kStep || MODE == kRepack) {
+        const uint8_t* mc = T->mc_in;
+        const uint8_t* vc = T->vc_in;
+        const unsigned long long lim_m = padded_code_bytes(numel, bm_in);
+        const unsigned long long lim_v = padded_code_bytes(numel, bv_in);
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          load_codes<WIDE>(mc, e_warp + r * kRowElems, bm_in, lane, lim_m, rawm[r]);
+          load_codes<WIDE>(vc, e_warp + r * kRowElems, bv_in, lane, lim_v, rawv[r]);
+        }
+        const float* ms = T->ms_in;
+        const float* vs = T->vs_in;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const unsigned long long e_row = e_warp + r * kRowElems;
+          const bool live = e_row < numel;
+          s_m_in[r] = (live && bm_in != 32) ? ms[e_row >> lgB] : 0.f;
+          s_v_in[r] = (live && bv_in != 32) ? vs[e_row >> lgB] : 0.f;
+        }
+      }
+
+      if constexpr (MODE == kStatsOnly) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          float g[4];
+          widen_grad<GDT>(graw[r], g);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            st_g += g[k];
+            st_a += fabsf(g[k]);
+            st_q = __fmaf_rn(g[k], g[k], st_q);
+          }
+        }
+      } else {
+        // ---- decode stored states, form the new moments -----------------------------------------
+        float mt[R][4], vt[R][4], th[R][4];
+        if constexpr (MODE == kInit) {
+#pragma unroll
+          for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { mt[r][k] = 0.f; vt[r][k] = 0.f; }
+        } else {
+          const LinW lw_in = lin_width(bm_in);
+          const LogW gw_in = log_width(bv_in);
+          const float wd = T->wd;
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            float mh[4], vh[4];
+            if (WIDE && bm_in == 32) {
+              if constexpr (WIDE) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) mh[k] = __uint_as_float(rawm[r].w[k]);
+              }
+            } else {
+              uint32_t c[4];
+              split_codes<WIDE>(rawm[r], bm_in, lane, c);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) mh[k] = decode_lin(c[k], s_m_in[r], lw_in);
+            }
+            if (WIDE && bv_in == 32) {
+              if constexpr (WIDE) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) vh[k] = __uint_as_float(rawv[r].w[k]);
+              }
+            } else {
+              uint32_t c[4];
+              split_codes<WIDE>(rawv[r], bv_in, lane, c);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) vh[k] = decode_log(c[k], s_v_in[r], bv_in, gw_in);
+            }
+            if constexpr (MODE == kStep) {
+              th[r][0] = th4[r].x; th[r][1] = th4[r].y; th[r][2] = th4[r].z; th[r][3] = th4[r].w;
+              float g[4];
+              widen_grad<GDT>(graw[r], g);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                if constexpr (STATS) {
+                  st_g += g[k];
+                  st_a += fabsf(g[k]);
+                  st_q = __fmaf_rn(g[k], g[k], st_q);
+                }
+                float gk = g[k];
+                if (sc.l2_mode) gk = __fadd_rn(gk, __fmul_rn(wd, th[r][k]));
+                const float m = __fadd_rn(__fmul_rn(sc.b1, mh[k]), __fmul_rn(sc.c1, gk));
+                const float v = __fadd_rn(__fmul_rn(sc.b2, vh[k]), __fmul_rn(__fmul_rn(sc.c2, gk), gk));
+                // elements past the end of the tensor stay out of the block maximum
+                mt[r][k] = k < nvl[r] ? m : 0.f;
+                vt[r][k] = k < nvl[r] ? v : 0.f;
+              }
+            } else {   // kRepack: the stored values themselves are re-quantized
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                mt[r][k] = k < nvl[r] ? mh[k] : 0.f;
+                vt[r][k] = k < nvl[r] ? vh[k] : 0.f;
+              }
+            }
+          }
+        }
+
+        // ---- block maxima: lane max of 4, warp REDUX on the bit patterns, rows merged per block ----
+        uint32_t mxm[R], mxv[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const float am = fmaxf(fmaxf(fabsf(mt[r][0]), fabsf(mt[r][1])), fmaxf(fabsf(mt[r][2]), fabsf(mt[r][3])));
+          const float av = fmaxf(fmaxf(vt[r][0], vt[r][1]), fmaxf(vt[r][2], vt[r][3]));
+          mxm[r] = __reduce_max_sync(kFull, __float_as_uint(am));
+          mxv[r] = __reduce_max_sync(kFull, __float_as_uint(av));
+        }
+        if (B >= 256) {
+#pragma unroll
+          for (int r = 0; r < R; r += 2) {
+            mxm[r] = mxm[r + 1] = max(mxm[r], mxm[r + 1]);
+            mxv[r] = mxv[r + 1] = max(mxv[r], mxv[r + 1]);
+          }
+        }
+        if (B >= 512) {
+          const uint32_t a = max(mxm[0], mxm[2]), b = max(mxv[0], mxv[2]);
+#pragma unroll
+          for (int r = 0; r < R; ++r) { mxm[r] = a; mxv[r] = b; }
+        }
+
+        // ---- quantize, pack, store; decode the new codes; update the parameters -------------------
+        const LinW lw = lin_width(bm_out);
+        const LogW gw = log_width(bv_out);
+        const unsigned long long lim_mo = padded_code_bytes(numel, bm_out);
+        const unsigned long long lim_vo = padded_code_bytes(numel, bv_out);
+        uint8_t* mco = T->mc_out;
+        uint8_t* vco = T->vc_out;
+        float* mso = T->ms_out;
+        float* vso = T->vs_out;
+        float* param = T->param;
+        // decoupled decay as theta - (theta*lr*wd + update): the small term keeps its own precision
+        // (a factor 1 - lr*wd rounded to fp32 is off by ~1e-3 of the decay it applies)
+        const float lrwd = sc.l2_mode ? 0.0f : (float)(sc.lr * (double)T->wd);
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const unsigned long long e_row = e_warp + r * kRowElems;
+          if (e_row >= numel) break;
+          float mq[4], vq[4];
+
+          // first moment, linear symmetric
+          if (WIDE && bm_out == 32) {
+            if constexpr (WIDE) {
+              store_raw32(mco, e_row, lane, lim_mo, mt[r]);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) mq[k] = mt[r][k];
+            }
+          } else {
+            const float s_raw = __uint_as_float(mxm[r]);
+            const bool zero = s_raw < kTiny;
+            const float s = zero ? 0.f : s_raw;
+            const float inv = zero ? 0.f : __fdiv_rn(lw.qmaxf, s_raw);
+            const float mg = kMagic + lw.halff;
+            uint32_t x[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float t = __fmaf_rn(mt[r][k], inv, mg);    // low bits: q + 2^(b-1)
+              x[k] = __float_as_uint(t);
+              mq[k] = __fmul_rn(s, __fmul_rn(__fadd_rn(t, -mg), lw.invq));
+            }
+            store_codes(mco, e_row, bm_out, lane, lim_mo, x, kMagicBits, nvl[r]);
+            if (lane == 0 && (e_row & (B - 1)) == 0) mso[e_row >> lgB] = s;
+          }
+
+          // second moment, logarithmic
+          if (WIDE && bv_out == 32) {
+            if constexpr (WIDE) {
+              store_raw32(vco, e_row, lane, lim_vo, vt[r]);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) vq[k] = vt[r][k];
+            }
+          } else {
+            const float s_raw = __uint_as_float(mxv[r]);
+            const bool zero = s_raw < kTiny;
+            const float s = zero ? 0.f : s_raw;
+            const int Es = zero ? kZeroBlockExp : (int)(mxv[r] >> 23);
+            const float Ps = lg_poly(mxv[r]);
+            const uint32_t ebase = kMagicBits - (uint32_t)Es;
+            uint32_t x[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const uint32_t xb = __float_as_uint(vt[r][k]);
+              const float de = __fadd_rn(__uint_as_float(ebase + (xb >> 23)), -kMagic);   // float(E_x - E_s)
+              const float dp = __fadd_rn(lg_poly(xb), -Ps);
+              const float d = fmaxf(__fadd_rn(de, dp), gw.negR);
+              const float t = __fmaf_rn(d, gw.a, kMagic);       // low bits: code - K, in [-K, 0]
+              x[k] = __float_as_uint(t);
+              if constexpr (MODE == kStep) {
+                if (bv_out <= 4) {
+                  vq[k] = __fmul_rn(s, __uint_as_float((x[k] << 23) + 0x3F800000u));
+                } else {
+                  vq[k] = __fmul_rn(s, ex2_poly(__fmul_rn(__fadd_rn(t, -kMagic), gw.c)));
+                }
+              }
+            }
+            store_codes(vco, e_row, bv_out, lane, lim_vo, x, kMagicBits - (uint32_t)gw.K, nvl[r]);
+            if (lane == 0 && (e_row & (B - 1)) == 0) vso[e_row >> lgB] = s;
+          }
+
+          if constexpr (MODE == kStep) {
+            float out[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float den = __fmaf_rn(sqrt_approx(vq[k]), sc.rsqrt_bc2, sc.eps);
+              const float upd = __fdividef(__fmul_rn(mq[k], sc.step_size), den);
+              out[k] = __fadd_rn(th[r][k], -__fmaf_rn(th[r][k], lrwd, upd));
+            }
+            store_param(param + e_row + 4 * lane, nvl[r], out);
+          }
+        }
+      }
+    }
+
+    if constexpr (STATS || MODE == kStatsOnly) {
+      double dg = (double)st_g, da = (double)st_a, dq = (double)st_q;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        dg += __shfl_down_sync(kFull, dg, o);
+        da += __shfl_down_sync(kFull, da, o);
+        dq += __shfl_down_sync(kFull, dq, o);
+      }
+      if (lane == 0) { s_part[warp][0] = dg; s_part[warp][1] = da; s_part[warp][2] = dq; }
+      __syncthreads();
+      if (threadIdx.x < 3) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) s += s_part[w][threadIdx.x];
+        partials[(size_t)tile * 3 + threadIdx.x] = s;
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// One CTA per tensor: fixed-order sum of its tiles' partials.
+__global__ void __launch_bounds__(256)
+stq_stats_finish_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ ntiles_of, int L,
+                        const double* __restrict__ partials, double* __restrict__ out) {
+  const int l = blockIdx.x;
+  if (l >= L) return;
+  const uint32_t t0 = table[l].tile0, nt = ntiles_of[l];
+  double a[3] = {0.0, 0.0, 0.0};
+  for (uint32_t i = threadIdx.x; i < nt; i += blockDim.x) {
+#pragma unroll
+    for (int k = 0; k < 3; ++k) a[k] += partials[(size_t)(t0 + i) * 3 + k];
+  }
+  __shared__ double sh[256][3];
+#pragma unroll
+  for (int k = 0; k < 3; ++k) sh[threadIdx.x][k] = a[k];
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if ((int)threadIdx.x < s) {
+#pragma unroll
+      for (int k = 0; k < 3; ++k) sh[threadIdx.x][k] += sh[threadIdx.x + s][k];
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x < 3) out[(size_t)l * 4 + threadIdx.x] = sh[0][threadIdx.x];
+  if (threadIdx.x == 3) out[(size_t)l * 4 + 3] = (double)table[l].numel;
+}
+
+template <int MODE, int GDT, bool STATS, bool WIDE>
+cudaError_t launch_one(const TensorDesc* table, const uint32_t* tile_map, uint32_t tb, uint32_t te,
+                       const StepConsts& sc, double* partials, int grid, cudaStream_t stream) {
+  const uint32_t n = te - tb;
+  const int g = (int)(n < (uint32_t)grid ? n : (uint32_t)grid);
+  stq_tile_kernel<MODE, GDT, STATS, WIDE><<<g, kThreads, 0, stream>>>(table, tile_map, tb, te, sc, partials);
+  return cudaGetLastError();
+}
+
+template <int MODE, int GDT, bool STATS>
+cudaError_t launch_w(bool wide, const TensorDesc* table, const uint32_t* tile_map, uint32_t tb, uint32_t te,
+                     const StepConsts& sc, double* partials, int grid, cudaStream_t stream) {
+  return wide ? launch_one<MODE, GDT, STATS, true>(table, tile_map, tb, te, sc, partials, grid, stream)
+              : launch_one<MODE, GDT, STATS, false>(table, tile_map, tb, te, sc, partials, grid, stream);
+}
+
+}  // namespace
+
+cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const TensorDesc* table,
+                         const uint32_t* tile_map, uint32_t tile_begin, uint32_t tile_end,
+                         const StepConsts& sc, double* partials, int grid, cudaStream_t stream) {
+  if (tile_end <= tile_begin) return cudaSuccess;
+  switch (mode) {
+    case kStep:
+      if (grad_dtype == 0)
+        return stats ? launch_w<kStep, 0, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream)
+                     : launch_w<kStep, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+      return stats ? launch_w<kStep, 1, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream)
+                   : launch_w<kStep, 1, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+    case kRepack:
+      return launch_w<kRepack, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+    case kInit:
+      return launch_w<kInit, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+    case kStatsOnly:
+      return grad_dtype == 0
+                 ? launch_one<kStatsOnly, 0, true, false>(table, tile_map, tile_begin, tile_end, sc, partials, grid, stream)
+                 : launch_one<kStatsOnly, 1, true, false>(table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+  }
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_stats_finish(const TensorDesc* table, const uint32_t* ntiles_of, int L,
+                                const double* partials, double* out, cudaStream_t stream) {
+  stq_stats_finish_kernel<<<L, 256, 0, stream>>>(table, ntiles_of, L, partials, out);
+  return cudaGetLastError();
+}
+
+int step_ctas_per_sm() {
+  int n = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, stq_tile_kernel<kStep, 1, false, false>, kThreads, 0) !=
+      cudaSuccess)
+    return 1;
+  return n > 0 ? n : 1;
+}
+
+}  // namespace stq

@@ -1,0 +1,145 @@
+"""Device-side driver of a workload: allocates the tensors, builds the stq table, steps.
+
+Everything numerical happens inside libstq; this module only owns buffers (through torch) and
+keeps the per-tensor widths.  Used by the benchmark, the smoke check and the GPU tests.
+"""
+from __future__ import annotations
+
+from typing import Sequence
+
+import numpy as np
+import torch
+
+from . import stq
+from .workloads import Workload, draw_grad, draw_param, tensor_scales
+
+
+def _round_up(x: int, a: int) -> int:
+    return (x + a - 1) // a * a
+
+
+class Job:
+    """Parameters, gradients and quantized AdamW state of one workload on one device."""
+
+    def __init__(self, w: Workload, bits_m: Sequence[int], bits_v: Sequence[int], device="cuda",
+                 handle: stq.Handle | None = None, draw_params: bool = True):
+        self.w = w
+        self.device = torch.device(device)
+        self.handle = handle or stq.Handle(self.device.index if self.device.index is not None else torch.cuda.current_device())
+        self.numels = w.numels
+        self.L = len(self.numels)
+        self.block = w.block
+        self.grad_dtype = stq.GRAD_BF16 if w.grad_dtype == "bf16" else stq.GRAD_F32
+        self.gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
+        self.scales = tensor_scales(w)
+        # parameters and gradients live in two flat buffers; every tensor starts 256-byte aligned
+        offs, total = [], 0
+        for n in self.numels:
+            offs.append(total)
+            total += _round_up(n, 64)
+        self.offsets = offs
+        self.param_flat = torch.zeros(total, dtype=torch.float32, device=self.device)
+        self.grad_flat = torch.zeros(total, dtype=self.gdt, device=self.device)
+        self.params = [self.param_flat[o:o + n] for o, n in zip(offs, self.numels)]
+        self.grads = [self.grad_flat[o:o + n] for o, n in zip(offs, self.numels)]
+        if draw_params:
+            for i in range(self.L):
+                self.params[i].copy_(draw_param(w, i, self.device))
+        self.bits_m = np.asarray(bits_m, dtype=np.uint8).copy()
+        self.bits_v = np.asarray(bits_v, dtype=np.uint8).copy()
+        self.states = [stq.alloc_state(n, self.block, int(bm), int(bv), self.device)
+                       for n, bm, bv in zip(self.numels, self.bits_m, self.bits_v)]
+        self.wd = [w.weight_decay] * self.L
+        self._tbl = None
+        self.t = 0
+        self.handle.init_state(self._make_table(self.states, self.states, with_inputs=False))
+        self._tbl = None
+
+    # ---- tables ----------------------------------------------------------------------------------
+    def _make_table(self, st_in, st_out, with_inputs=True):
+        rows = [stq.make_row(n, self.block, si if with_inputs else None, so,
+                             self.params[i] if with_inputs else None,
+                             self.grads[i] if with_inputs else None, self.wd[i])
+                for i, (n, si, so) in enumerate(zip(self.numels, st_in, st_out))]
+        return stq.table(rows)
+
+    def table(self):
+        """In-place table at the current widths (cached until the widths change)."""
+        if self._tbl is None:
+            self._tbl = self._make_table(self.states, self.states)
+        return self._tbl
+
+    # ---- inputs ----------------------------------------------------------------------------------
+    def draw_grads(self, step: int):
+        for i in range(self.L):
+            self.grads[i].copy_(draw_grad(self.w, i, step, self.device, scale=float(self.scales[i])))
+
+    # ---- the path --------------------------------------------------------------------------------
+    def hp(self, t: int) -> dict:
+        w = self.w
+        return dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, t=t, grad_dtype=self.grad_dtype)
+
+    def step(self, t: int | None = None, stats: bool = False, new_bits=None, stream=None):
+        """One optimizer step.  new_bits = (bits_m, bits_v) arrays switches widths inside the step."""
+        self.t = self.t + 1 if t is None else t
+        flags = stq.WITH_STATS if stats else 0
+        if new_bits is None:
+            self.handle.step(self.table(), flags=flags, stream=stream, **self.hp(self.t))
+            return
+        bm, bv = (np.asarray(a, dtype=np.uint8) for a in new_bits)
+        new_states = []
+        for i, n in enumerate(self.numels):
+            if bm[i] == self.bits_m[i] and bv[i] == self.bits_v[i]:
+                new_states.append(self.states[i])
+            else:
+                new_states.append(self._fresh_state(i, int(bm[i]), int(bv[i])))
+        self.handle.step(self._make_table(self.states, new_states), flags=flags, stream=stream, **self.hp(self.t))
+        self._adopt(new_states, bm, bv)
+
+    def repack(self, new_bits, stream=None):
+        """Width transition between steps."""
+        bm, bv = (np.asarray(a, dtype=np.uint8) for a in new_bits)
+        idx = [i for i in range(self.L) if bm[i] != self.bits_m[i] or bv[i] != self.bits_v[i]]
+        if not idx:
+            return
+        new_states = list(self.states)
+        rows = []
+        for i in idx:
+            new_states[i] = self._fresh_state(i, int(bm[i]), int(bv[i]))
+            rows.append(stq.make_row(self.numels[i], self.block, self.states[i], new_states[i]))
+        self.handle.repack(stq.table(rows), stream=stream)
+        self._adopt(new_states, bm, bv)
+
+    def layer_stats(self, stream=None) -> np.ndarray:
+        return self.handle.layer_stats(self.L, stream=stream)
+
+    def _fresh_state(self, i: int, bm: int, bv: int) -> stq.QState:
+        """New buffers for the states whose width changes; unchanged states keep their buffers."""
+        old = self.states[i]
+        n = self.numels[i]
+        mc, ms = (old.m_codes, old.m_scales) if bm == old.bits_m else (
+            stq.alloc_codes(n, bm, self.device), stq.alloc_scales(n, bm, self.block, self.device))
+        vc, vs = (old.v_codes, old.v_scales) if bv == old.bits_v else (
+            stq.alloc_codes(n, bv, self.device), stq.alloc_scales(n, bv, self.block, self.device))
+        return stq.QState(mc, ms, bm, vc, vs, bv)
+
+    def _adopt(self, new_states, bm, bv):
+        torch.cuda.current_stream().synchronize()   # old buffers are released below
+        self.states = new_states
+        self.bits_m, self.bits_v = bm.copy(), bv.copy()
+        self._tbl = None
+
+    # ---- accounting ------------------------------------------------------------------------------
+    def algorithmic_bytes(self) -> int:
+        """Bytes one step must move: theta r+w, grad, codes r+w, scales r+w."""
+        gb = 2 if self.w.grad_dtype == "bf16" else 4
+        total = 0
+        for n, bm, bv in zip(self.numels, self.bits_m, self.bits_v):
+            nb = (n + self.block - 1) // self.block
+            total += n * (8 + gb) + 2 * ((n * int(bm) + 7) // 8 + (n * int(bv) + 7) // 8)
+            total += 4 * nb * ((bm != 32) + (bv != 32)) * 2
+        return int(total)
+
+    def state_bytes(self) -> int:
+        return int(sum(s.m_codes.numel() + s.v_codes.numel() + 4 * (s.m_scales.numel() + s.v_scales.numel())
+                       for s in self.states))

@@ -1,0 +1,285 @@
+"""Thin ctypes binding over libstq (the C-ABI declared in ``include/stq.h``).
+
+Argument marshalling only: torch tensors supply device memory and streams, every step of the path
+runs in the library's CUDA kernels.  There is no fallback: if the library is missing or a call
+fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libstq.so")
+
+GRAD_F32, GRAD_BF16 = 0, 1
+WITH_STATS = 1
+WIDTHS = (2, 3, 4, 8, 16, 32)
+
+
+class StqError(RuntimeError):
+    def __init__(self, code: int, what: str, detail: str = ""):
+        super().__init__(f"{what}: error {code} ({_strerror(code)}){' - ' + detail if detail else ''}")
+        self.code = code
+
+
+class CTensor(C.Structure):
+    """struct stq_tensor"""
+    _fields_ = [
+        ("param", C.c_void_p), ("grad", C.c_void_p),
+        ("m_codes_in", C.c_void_p), ("m_scales_in", C.c_void_p),
+        ("v_codes_in", C.c_void_p), ("v_scales_in", C.c_void_p),
+        ("m_codes_out", C.c_void_p), ("m_scales_out", C.c_void_p),
+        ("v_codes_out", C.c_void_p), ("v_scales_out", C.c_void_p),
+        ("numel", C.c_uint64), ("block", C.c_uint32),
+        ("bits_m", C.c_uint8), ("bits_v", C.c_uint8), ("bits_m_out", C.c_uint8), ("bits_v_out", C.c_uint8),
+        ("weight_decay", C.c_float), ("reserved", C.c_uint32),
+    ]
+
+
+class CHParams(C.Structure):
+    """struct stq_hparams"""
+    _fields_ = [("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
+                ("step", C.c_int64), ("decoupled_wd", C.c_int32), ("grad_dtype", C.c_int32)]
+
+
+class CPolicyCfg(C.Structure):
+    """struct stq_policy_cfg"""
+    _fields_ = [("alpha", C.c_double), ("tau", C.c_double), ("eps_stat", C.c_double),
+                ("interval", C.c_int64), ("cv_of_signed", C.c_int32), ("reserved", C.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libstq.so; raises if it has not been built (``python -m paper_2604_06836_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2604_06836_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        vp, PT = C.c_void_p, C.POINTER(CTensor)
+        L.stq_create.argtypes = [C.POINTER(vp), C.c_int]
+        L.stq_destroy.argtypes = [vp]
+        L.stq_codes_bytes.argtypes = [C.c_uint64, C.c_int]
+        L.stq_codes_bytes.restype = C.c_size_t
+        L.stq_scales_bytes.argtypes = [C.c_uint64, C.c_uint32]
+        L.stq_scales_bytes.restype = C.c_size_t
+        L.stq_init_state.argtypes = [vp, PT, C.c_int, vp]
+        L.stq_step.argtypes = [vp, PT, C.c_int, C.POINTER(CHParams), C.c_uint, vp]
+        L.stq_grad_stats.argtypes = [vp, PT, C.c_int, C.c_int, vp]
+        L.stq_layer_stats.argtypes = [vp, vp, C.c_int, vp]
+        L.stq_repack.argtypes = [vp, PT, C.c_int, vp]
+        L.stq_step_host.argtypes = [vp, PT, C.c_int, C.POINTER(CHParams), C.c_uint,
+                                    C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+        L.stq_launch_count.argtypes = [vp]
+        L.stq_launch_count.restype = C.c_uint64
+        L.stq_grid_size.argtypes = [vp]
+        L.stq_sm_count.argtypes = [vp]
+        L.stq_policy_create.argtypes = [C.POINTER(vp), C.POINTER(CPolicyCfg)]
+        L.stq_policy_destroy.argtypes = [vp]
+        L.stq_policy_is_decision_step.argtypes = [vp, C.c_int64]
+        L.stq_decide.argtypes = [vp, vp, C.c_int, C.c_int64, vp, vp]
+        L.stq_policy_get_state.argtypes = [vp, vp]
+        L.stq_policy_set_state.argtypes = [vp, vp]
+        L.stq_strerror.argtypes = [C.c_int]
+        L.stq_strerror.restype = C.c_char_p
+        L.stq_last_cuda_error.argtypes = [vp]
+        L.stq_last_cuda_error.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def _strerror(code: int) -> str:
+    try:
+        return lib().stq_strerror(code).decode()
+    except Exception:   # pragma: no cover
+        return "?"
+
+
+def codes_bytes(numel: int, bits: int) -> int:
+    return int(lib().stq_codes_bytes(numel, bits))
+
+
+def scales_bytes(numel: int, block: int) -> int:
+    return int(lib().stq_scales_bytes(numel, block))
+
+
+# ------------------------------------------------------------------------------------------------
+# per-tensor buffers (torch owns the memory)
+# ------------------------------------------------------------------------------------------------
+@dataclass
+class QState:
+    """Stored optimizer state of one tensor: packed codes + block scales for m and v."""
+    m_codes: torch.Tensor   # uint8[codes_bytes]
+    m_scales: torch.Tensor  # float32[nblocks] (empty at width 32)
+    bits_m: int
+    v_codes: torch.Tensor
+    v_scales: torch.Tensor
+    bits_v: int
+
+
+def alloc_codes(numel: int, bits: int, device) -> torch.Tensor:
+    return torch.zeros(codes_bytes(numel, bits), dtype=torch.uint8, device=device)
+
+
+def alloc_scales(numel: int, bits: int, block: int, device) -> torch.Tensor:
+    n = scales_bytes(numel, block) // 4
+    return torch.zeros(n, dtype=torch.float32, device=device)
+
+
+def alloc_state(numel: int, block: int, bits_m: int, bits_v: int, device) -> QState:
+    return QState(alloc_codes(numel, bits_m, device), alloc_scales(numel, bits_m, block, device), bits_m,
+                  alloc_codes(numel, bits_v, device), alloc_scales(numel, bits_v, block, device), bits_v)
+
+
+def _ptr(t: torch.Tensor | None) -> int | None:
+    return None if t is None or t.numel() == 0 else t.data_ptr()
+
+
+def make_row(numel: int, block: int, st_in: QState | None, st_out: QState, param: torch.Tensor | None = None,
+             grad: torch.Tensor | None = None, weight_decay: float = 0.0) -> CTensor:
+    """One table row.  st_out may be st_in (in-place) when the widths are unchanged."""
+    r = CTensor()
+    r.param = _ptr(param)
+    r.grad = _ptr(grad)
+    if st_in is not None:
+        r.m_codes_in, r.m_scales_in = _ptr(st_in.m_codes), _ptr(st_in.m_scales)
+        r.v_codes_in, r.v_scales_in = _ptr(st_in.v_codes), _ptr(st_in.v_scales)
+        r.bits_m, r.bits_v = st_in.bits_m, st_in.bits_v
+    else:
+        r.bits_m, r.bits_v = st_out.bits_m, st_out.bits_v
+    r.m_codes_out, r.m_scales_out = _ptr(st_out.m_codes), _ptr(st_out.m_scales)
+    r.v_codes_out, r.v_scales_out = _ptr(st_out.v_codes), _ptr(st_out.v_scales)
+    r.bits_m_out, r.bits_v_out = st_out.bits_m, st_out.bits_v
+    r.numel, r.block, r.weight_decay, r.reserved = numel, block, weight_decay, 0
+    return r
+
+
+def table(rows: Sequence[CTensor]):
+    return (CTensor * len(rows))(*rows)
+
+
+def _stream_ptr(stream) -> int | None:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream or None
+
+
+class Handle:
+    """Owns one stq_handle (device table, tile map, statistics workspace)."""
+
+    def __init__(self, device: int | None = None):
+        if device is None:
+            device = torch.cuda.current_device()
+        self.device = int(device)
+        self._h = C.c_void_p()
+        rc = lib().stq_create(C.byref(self._h), self.device)
+        if rc != 0:
+            raise StqError(rc, "stq_create")
+
+    def close(self):
+        if getattr(self, "_h", None) and self._h.value:
+            lib().stq_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):   # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int, what: str):
+        if rc != 0:
+            raise StqError(rc, what, lib().stq_last_cuda_error(self._h).decode())
+
+    def init_state(self, tbl, stream=None):
+        self._check(lib().stq_init_state(self._h, tbl, len(tbl), _stream_ptr(stream)), "stq_init_state")
+
+    def step(self, tbl, *, lr, beta1, beta2, eps, t, grad_dtype=GRAD_F32, decoupled_wd=True, flags=0, stream=None):
+        hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype)
+        self._check(lib().stq_step(self._h, tbl, len(tbl), C.byref(hp), flags, _stream_ptr(stream)), "stq_step")
+
+    def grad_stats(self, tbl, grad_dtype=GRAD_F32, stream=None):
+        self._check(lib().stq_grad_stats(self._h, tbl, len(tbl), grad_dtype, _stream_ptr(stream)), "stq_grad_stats")
+
+    def layer_stats(self, L: int, stream=None) -> np.ndarray:
+        out = np.zeros((L, 4), dtype=np.float64)
+        self._check(lib().stq_layer_stats(self._h, out.ctypes.data_as(C.c_void_p), L, _stream_ptr(stream)),
+                    "stq_layer_stats")
+        return out
+
+    def repack(self, tbl, stream=None):
+        self._check(lib().stq_repack(self._h, tbl, len(tbl), _stream_ptr(stream)), "stq_repack")
+
+    def step_host(self, tbl, *, lr, beta1, beta2, eps, t, grad_dtype=GRAD_F32, decoupled_wd=True, flags=0):
+        hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype)
+        h2d, d2h = C.c_uint64(0), C.c_uint64(0)
+        self._check(lib().stq_step_host(self._h, tbl, len(tbl), C.byref(hp), flags, C.byref(h2d), C.byref(d2h)),
+                    "stq_step_host")
+        return int(h2d.value), int(d2h.value)
+
+    @property
+    def launch_count(self) -> int:
+        return int(lib().stq_launch_count(self._h))
+
+    @property
+    def grid_size(self) -> int:
+        return int(lib().stq_grid_size(self._h))
+
+    @property
+    def sm_count(self) -> int:
+        return int(lib().stq_sm_count(self._h))
+
+
+class Policy:
+    """Host-side transition decision (stq_policy)."""
+
+    def __init__(self, alpha=0.1, tau=100.0, eps_stat=1e-8, interval=10, cv_of_signed=False):
+        cfg = CPolicyCfg(alpha, tau, eps_stat, interval, 1 if cv_of_signed else 0, 0)
+        self._p = C.c_void_p()
+        rc = lib().stq_policy_create(C.byref(self._p), C.byref(cfg))
+        if rc != 0:
+            raise StqError(rc, "stq_policy_create")
+
+    def close(self):
+        if getattr(self, "_p", None) and self._p.value:
+            lib().stq_policy_destroy(self._p)
+            self._p = C.c_void_p()
+
+    def __del__(self):   # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def is_decision_step(self, t: int) -> bool:
+        return bool(lib().stq_policy_is_decision_step(self._p, t))
+
+    def decide(self, stats: np.ndarray, t: int):
+        stats = np.ascontiguousarray(stats, dtype=np.float64)
+        L = stats.shape[0]
+        bits = np.zeros(L, dtype=np.uint8)
+        score = np.zeros(L, dtype=np.float64)
+        rc = lib().stq_decide(self._p, stats.ctypes.data_as(C.c_void_p), L, t,
+                              bits.ctypes.data_as(C.c_void_p), score.ctypes.data_as(C.c_void_p))
+        if rc != 0:
+            raise StqError(rc, "stq_decide")
+        return bits, score
+
+    @property
+    def state(self) -> np.ndarray:
+        out = np.zeros(3, dtype=np.float64)
+        lib().stq_policy_get_state(self._p, out.ctypes.data_as(C.c_void_p))
+        return out
+
+    @state.setter
+    def state(self, v):
+        v = np.ascontiguousarray(v, dtype=np.float64)
+        lib().stq_policy_set_state(self._p, v.ctypes.data_as(C.c_void_p))

@@ -1,0 +1,122 @@
+"""Test-side glue: runs the CPU oracle next to the CUDA path on the same inputs and compares.
+
+Only the tests (and the smoke check) import this; it is the one place where the oracle and the
+product meet, and it contains no arithmetic of the method beyond the comparison itself.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle as O
+from paper_2604_06836_b200 import stq
+from paper_2604_06836_b200.runner import Job
+
+
+def to_np(t: torch.Tensor) -> np.ndarray:
+    """Device tensor -> numpy; bf16 comes back as its uint16 bit patterns."""
+    t = t.detach().cpu().contiguous()
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).numpy().view(np.uint16).copy()
+    return t.numpy().copy()
+
+
+class OracleJob:
+    """The oracle's copy of a Job: same parameters, same widths, zero initial state."""
+
+    def __init__(self, job: Job):
+        self.w = job.w
+        self.block = job.block
+        self.numels = list(job.numels)
+        self.theta = [to_np(p) for p in job.params]
+        # largest magnitude each element (or one of its single-step changes) has had so far: rounding
+        # differences are relative to the operands of the update, which may exceed the current value
+        self.upd_mag = [np.abs(th) for th in self.theta]
+        self.bits_m = job.bits_m.copy()
+        self.bits_v = job.bits_v.copy()
+        self.states = [O.new_state(n, self.block, int(bm), int(bv))
+                       for n, bm, bv in zip(self.numels, self.bits_m, self.bits_v)]
+        self.wd = list(job.wd)
+
+    def step(self, grads, t: int, want_stats=False, new_bits=None, decoupled_wd=True):
+        w = self.w
+        stats = np.zeros((len(self.numels), 4))
+        bm, bv = (self.bits_m, self.bits_v) if new_bits is None else (np.asarray(a, np.uint8) for a in new_bits)
+        for i, g in enumerate(grads):
+            before = self.theta[i].copy()
+            self.states[i], s = O.step(self.theta[i], g, self.states[i], self.block, lr=w.lr, beta1=w.beta1,
+                                       beta2=w.beta2, eps=w.eps, weight_decay=self.wd[i], t=t,
+                                       bits_m_out=int(bm[i]), bits_v_out=int(bv[i]),
+                                       decoupled_wd=decoupled_wd, want_stats=want_stats)
+            self.upd_mag[i] = np.maximum(self.upd_mag[i], np.maximum(np.abs(self.theta[i] - before), np.abs(self.theta[i])))
+            if want_stats:
+                stats[i] = s
+        self.bits_m, self.bits_v = np.array(bm, np.uint8), np.array(bv, np.uint8)
+        return stats
+
+    def repack(self, new_bits):
+        bm, bv = (np.asarray(a, np.uint8) for a in new_bits)
+        for i, n in enumerate(self.numels):
+            st = self.states[i]
+            if bm[i] != st.bits_m:
+                st.m_codes, st.m_scales = O.repack(st.m_codes, st.m_scales, st.bits_m, int(bm[i]), n, self.block, O.LINEAR)
+                st.bits_m = int(bm[i])
+            if bv[i] != st.bits_v:
+                st.v_codes, st.v_scales = O.repack(st.v_codes, st.v_scales, st.bits_v, int(bv[i]), n, self.block, O.LOG)
+                st.bits_v = int(bv[i])
+        self.bits_m, self.bits_v = bm.copy(), bv.copy()
+
+
+def assert_states_equal(gs: stq.QState, os_: O.State, tag=""):
+    """Packed codes and scales must agree byte for byte."""
+    assert gs.bits_m == os_.bits_m and gs.bits_v == os_.bits_v, tag
+    for name, g, o, bits in (("m", gs.m_codes, os_.m_codes, gs.bits_m), ("v", gs.v_codes, os_.v_codes, gs.bits_v)):
+        g = to_np(g)
+        assert g.size == o.size, (tag, name, g.size, o.size)
+        if not (g == o).all():
+            bad = np.flatnonzero(g != o)
+            raise AssertionError(f"{tag}: {name} codes differ at {bad.size} bytes, first {bad[:8]} "
+                                 f"gpu {g[bad[:8]]} oracle {o[bad[:8]]} (bits {bits})")
+    for name, g, o, bits in (("m", gs.m_scales, os_.m_scales, gs.bits_m), ("v", gs.v_scales, os_.v_scales, gs.bits_v)):
+        if bits == 32:
+            continue
+        g = to_np(g)
+        if not (g.view(np.uint32) == o.view(np.uint32)).all():
+            bad = np.flatnonzero(g.view(np.uint32) != o.view(np.uint32))
+            raise AssertionError(f"{tag}: {name} scales differ at blocks {bad[:8]}: gpu {g[bad[:8]]} oracle {o[bad[:8]]}")
+
+
+def assert_theta_close(g: torch.Tensor, o: np.ndarray, rel: float, tag="", upd: np.ndarray | None = None):
+    """|a-b| <= rel * max(|b|, upd, 1e-3 * absmax(b)) element-wise, upd = largest magnitude the
+    element or one of its single-step changes has had.
+
+    The parameter is a difference of two fp32 terms (parameter, decay + update); where they nearly
+    cancel, the error is relative to the terms, not to the small result, hence the upd leg."""
+    g = to_np(g).astype(np.float64)
+    o = o.astype(np.float64)
+    floor = 1e-3 * np.abs(o).max() if o.size else 0.0
+    mag = np.maximum(np.abs(o), floor)
+    if upd is not None:
+        mag = np.maximum(mag, upd.astype(np.float64))
+    lim = rel * mag
+    err = np.abs(g - o)
+    if not (err <= lim).all():
+        k = int(np.argmax(err / np.maximum(lim, 1e-300)))
+        raise AssertionError(f"{tag}: theta differs: idx {k} gpu {g[k]!r} oracle {o[k]!r} err {err[k]:.3e} lim {lim[k]:.3e}")
+
+
+def assert_stats_close(g: np.ndarray, o: np.ndarray, tag=""):
+    assert g.shape == o.shape
+    # sum g cancels, so it is held to the scale of sum |g|
+    assert (np.abs(g[:, 0] - o[:, 0]) <= 2e-6 * np.maximum(o[:, 1], 1e-300)).all(), (tag, g[:, 0], o[:, 0])
+    np.testing.assert_allclose(g[:, 1], o[:, 1], rtol=2e-6, err_msg=tag)
+    np.testing.assert_allclose(g[:, 2], o[:, 2], rtol=2e-6, err_msg=tag)
+    assert (g[:, 3] == o[:, 3]).all()
+
+
+def compare_job(job: Job, oj: OracleJob, rel: float, tag=""):
+    torch.cuda.synchronize()
+    for i in range(job.L):
+        assert_states_equal(job.states[i], oj.states[i], f"{tag} tensor {i} ({job.w.shapes[i][0]})")
+        assert_theta_close(job.params[i], oj.theta[i], rel, f"{tag} tensor {i} ({job.w.shapes[i][0]})",
+                           upd=oj.upd_mag[i])

@@ -1,0 +1,193 @@
+"""Parity of the CUDA path with the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from paper_2604_06836_b200 import stq, workloads as W   # noqa: E402
+from paper_2604_06836_b200.runner import Job             # noqa: E402
+
+REL_1STEP = 1e-6     # parameters after one step
+REL_100 = 1e-4       # parameters after 100 steps
+
+
+@pytest.fixture(scope="module")
+def H():
+    import harness
+    return harness
+
+
+def _single(n, block, gdt, seed=0):
+    return W.Workload(f"single-{n}", (("w", (n,)),), block, gdt, "student_t", nu=4,
+                      scale_log10=(-3.0, -3.0), bits_kind="fixed", seed=seed)
+
+
+@pytest.mark.parametrize("gdt", ["fp32", "bf16"])
+@pytest.mark.parametrize("block", [128, 256, 512])
+@pytest.mark.parametrize("bm", [2, 3, 4, 8, 16])
+@pytest.mark.parametrize("bv", [2, 3, 4, 8, 16])
+def test_every_width_pair_three_steps(H, O, bm, bv, block, gdt):
+    n = 4096 * 3 + 128 * 5 + 52          # several tiles, a partial tile, a ragged last block
+    w = _single(n, block, gdt, seed=bm * 100 + bv)
+    job = Job(w, [bm], [bv])
+    oj = H.OracleJob(job)
+    H.compare_job(job, oj, 0.0, "init")
+    for t in (1, 2, 3):
+        job.draw_grads(t)
+        oj.step([H.to_np(g) for g in job.grads], t)
+        job.step(t)
+        H.compare_job(job, oj, REL_1STEP * t, f"t={t}")
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 127, 128, 129, 255, 257, 1000, 4095, 4096, 4097, 8191, 12289])
+@pytest.mark.parametrize("bits", [(3, 3), (8, 4), (16, 2), (2, 16)])
+def test_ragged_sizes(H, O, n, bits):
+    for block, gdt in ((128, "fp32"), (256, "bf16")):
+        w = _single(n, block, gdt, seed=n)
+        job = Job(w, [bits[0]], [bits[1]])
+        oj = H.OracleJob(job)
+        for t in (1, 2):
+            job.draw_grads(t)
+            st = oj.step([H.to_np(g) for g in job.grads], t, want_stats=True)
+            job.step(t, stats=True)
+            H.compare_job(job, oj, REL_1STEP * t, f"n={n} t={t}")
+            H.assert_stats_close(job.layer_stats(), st, f"n={n}")
+
+
+def test_states_at_32_bits_and_mixed(H, O):
+    """Raw fp32 states (the paper's 32-bit candidate) and tables mixing 32-bit and packed tensors."""
+    shapes = [("a", (5000,)), ("b", (4096,)), ("c", (777,)), ("d", (9000,))]
+    w = W.Workload("mixed32", tuple(shapes), 128, "fp32", "student_t", nu=4, scale_log10=(-4.0, -2.0), seed=11)
+    job = Job(w, [32, 8, 32, 4], [32, 32, 3, 4])
+    oj = H.OracleJob(job)
+    for t in range(1, 6):
+        job.draw_grads(t)
+        oj.step([H.to_np(g) for g in job.grads], t)
+        job.step(t)
+        H.compare_job(job, oj, REL_1STEP * t, f"t={t}")
+
+
+def test_cfg1_single_tensor_warmup_then_m8_v4(H, O):
+    """1,048,576 parameters: ten warm-up steps with fp32 states, quantize to m8/v4, measured step 11 with stats."""
+    w = W.config("cfg1")
+    job = Job(w, [32], [32])
+    oj = H.OracleJob(job)
+    for t in range(1, w.warmup_fp32_steps + 1):
+        job.draw_grads(t)
+        oj.step([H.to_np(g) for g in job.grads], t)
+        job.step(t)
+    H.compare_job(job, oj, REL_1STEP * 10, "warm-up")   # fp32 moments are bit-exact, theta has rounded 10 times
+    job.repack(([8], [4]))
+    oj.repack(([8], [4]))
+    H.compare_job(job, oj, REL_1STEP * 10, "quantized")
+    t = w.warmup_fp32_steps + 1
+    job.draw_grads(0)
+    before = [th.copy() for th in oj.theta]
+    st = oj.step([H.to_np(g) for g in job.grads], t, want_stats=True)
+    # measured step alone: start the GPU from the oracle's parameters so only one step's rounding shows
+    job.params[0].copy_(torch.from_numpy(before[0]).cuda())
+    job.step(t, stats=True)
+    H.compare_job(job, oj, REL_1STEP, "measured step")
+    H.assert_stats_close(job.layer_stats(), st, "cfg1")
+
+
+def _run_config(H, w, steps, churn_in_step=True):
+    bm, bv, _ = W.draw_bits(w)
+    job = Job(w, bm, bv)
+    oj = H.OracleJob(job)
+    pol_g = stq.Policy(alpha=0.1, tau=100.0, eps_stat=1e-8, interval=w.decision_interval)
+    import oracle
+    pol_o = oracle.new_policy(0.1, 100.0, 1e-8)
+    decision = 0
+    for t in range(1, steps + 1):
+        job.draw_grads(t)
+        grads = [H.to_np(g) for g in job.grads]
+        dec = pol_g.is_decision_step(t)
+        assert dec == oracle.is_decision_step(t, w.decision_interval)
+        new_bits = None
+        if dec and w.churn > 0 and t >= 5:
+            nbm, nbv, _ = W.churn_bits(w, job.bits_m, job.bits_v, decision)
+            decision += 1
+            if churn_in_step and decision % 2 == 0:
+                new_bits = (nbm, nbv)          # width change fused into the step
+            else:
+                job.repack((nbm, nbv))         # width change between steps
+                oj.repack((nbm, nbv))
+        st_o = oj.step(grads, t, want_stats=dec, new_bits=new_bits)
+        job.step(t, stats=dec, new_bits=new_bits)
+        rel = REL_1STEP * max(1, t) if t <= 10 else REL_100
+        H.compare_job(job, oj, rel, f"{w.name} t={t}")
+        if dec:
+            st_g = job.layer_stats()
+            H.assert_stats_close(st_g, st_o, f"{w.name} t={t}")
+            # the paper's policy runs in shadow on both sides, on the GPU's statistics
+            bg, sg = pol_g.decide(st_g, t)
+            bo, so = oracle.decide(pol_o, st_g, t)
+            assert (bg == bo).all()
+            np.testing.assert_allclose(sg, so, rtol=1e-12, atol=1e-12)
+    return job, oj
+
+
+def test_small_gpt2_100_steps_k10(H, O):
+    w = W.scaled(W.config("cfg2"), W.small_gpt2(), steps=100)
+    _run_config(H, w, 100)
+
+
+def test_small_vit_100_steps_k20_with_width_churn(H, O):
+    w = W.scaled(W.config("cfg3"), W.small_vit(), steps=100)
+    _run_config(H, w, 100)
+
+
+def test_small_gpt2_bf16_m48_v348(H, O):
+    w = W.scaled(W.config("cfg4"), W.small_gpt2(d=136, n_layer=3), steps=50)
+    _run_config(H, w, 50)
+
+
+def test_small_gpt2_xl_recipe(H, O):
+    w = W.scaled(W.config("cfg5"), W.small_gpt2(d=100, n_layer=4, vocab=523), steps=20)
+    _run_config(H, w, 20)
+
+
+def test_l2_mode_and_per_tensor_weight_decay(H, O):
+    shapes = [("a", (3000,)), ("b", (513,))]
+    w = W.Workload("l2", tuple(shapes), 128, "fp32", "normal", scale_log10=(-3.0, -3.0), seed=5)
+    job = Job(w, [8, 4], [4, 8])
+    job.wd = [0.1, 0.0]
+    job._tbl = None
+    oj = H.OracleJob(job)
+    for t in (1, 2, 3):
+        job.draw_grads(t)
+        oj.step([H.to_np(g) for g in job.grads], t, decoupled_wd=False)
+        job.handle.step(job.table(), decoupled_wd=False, **job.hp(t))
+        H.compare_job(job, oj, REL_1STEP * t, f"l2 t={t}")
+
+
+def test_grad_stats_only_pass(H, O):
+    import oracle
+    w = W.scaled(W.config("cfg4"), W.small_gpt2(d=136, n_layer=1), steps=1)
+    bm, bv, _ = W.draw_bits(w)
+    job = Job(w, bm, bv)
+    job.draw_grads(1)
+    job.handle.grad_stats(job.table(), job.grad_dtype)
+    got = job.layer_stats()
+    want = np.stack([oracle.grad_stats(H.to_np(g)) for g in job.grads])
+    H.assert_stats_close(got, want, "stats-only")
+    job._tbl = None
+    job.step(1)     # the step table is rebuilt after a stats-only table
+
+
+def test_run_to_run_identical(H, O):
+    w = W.scaled(W.config("cfg2"), W.small_gpt2(), steps=3)
+    outs = []
+    for _ in range(2):
+        bm, bv, _ = W.draw_bits(w)
+        job = Job(w, bm, bv)
+        for t in (1, 2, 3):
+            job.draw_grads(t)
+            job.step(t, stats=True)
+        st = job.layer_stats()
+        outs.append((torch.cat([p.clone() for p in job.params]).cpu(), st,
+                     torch.cat([s.m_codes for s in job.states] + [s.v_codes for s in job.states]).cpu()))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][2], outs[1][2])
+    assert (outs[0][1] == outs[1][1]).all()
