@@ -1,0 +1,354 @@
+#!/usr/bin/env python
+"""Benchmark of the mixed-bit quantized AdamW step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg5] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path over the workload: the fused step kernel over every
+tensor, and on decision steps (every K_dec steps of the workload) the fused statistics, their
+fetch, and the host transition decision.  Each rank runs an independent replica (the path does not
+shard); the line reports the aggregate over ranks.  Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2604_06836_b200 import workloads as W  # noqa: E402
+
+METRIC = "quantized_adamw_step_params_per_s"
+UNIT = "params/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per parameter of the step kernel from the ncu capture
+# summarised in profiles/ (None until a capture exists); scaled by the parameters per launch.
+NCU_TRAFFIC_BYTES_PER_PARAM = None
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int, period=0.02):
+        super().__init__(daemon=True)
+        self.period, self.index = period, index
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            uuid = torch.cuda.get_device_properties(index).uuid
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        return {"sm_mhz": (float(np.median(self.samples)) if self.samples else None),
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------------
+# the oracle arm (CPU baseline / --impl reference)
+# ------------------------------------------------------------------------------------------------
+def oracle_sample_run(w: W.Workload, bits_m, bits_v, budget_s: float, repeats: int = 1):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: block-aligned chunks
+    taken round-robin from the tensor list, one chunk per task, tasks spread over the host cores."""
+    import oracle as O
+    from concurrent.futures import ThreadPoolExecutor
+
+    cores = os.cpu_count() or 1
+    chunk = 1 << 18
+    # calibrate the single-thread rate on one chunk
+    rng = np.random.default_rng(0)
+    th = rng.normal(0, 0.02, chunk).astype(np.float32)
+    g32 = (rng.standard_t(3, chunk) * 1e-3).astype(np.float32)
+    g = torch.from_numpy(g32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16).copy() \
+        if w.grad_dtype == "bf16" else g32
+    st = O.new_state(chunk, w.block, 4, 4)
+    kw = dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, weight_decay=w.weight_decay)
+    t0 = time.perf_counter()
+    st, _ = O.step(th, g, st, w.block, t=1, **kw)
+    rate1 = chunk / (time.perf_counter() - t0)
+    want = int(min(w.total_params, 1 << 27, max(chunk, rate1 * cores * budget_s)))
+    # build the sample: chunks of the real tensors' sizes and widths
+    tasks, taken = [], 0
+    numels = w.numels
+    order = np.argsort(numels)[::-1]
+    i = 0
+    while taken < want and i < 100000:
+        l = int(order[i % len(order)])
+        n = int(min(chunk, numels[l], want - taken))
+        if n <= 0:
+            break
+        n = max(w.block, n // w.block * w.block) if n >= w.block else n
+        th = rng.normal(0, 0.02, n).astype(np.float32)
+        g32 = (rng.standard_t(3, n) * 1e-3).astype(np.float32)
+        g = torch.from_numpy(g32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16).copy() \
+            if w.grad_dtype == "bf16" else g32
+        tasks.append([th, g, O.new_state(n, w.block, int(bits_m[l]), int(bits_v[l]))])
+        taken += n
+        i += 1
+
+    def one(task, t):
+        task[2], _ = O.step(task[0], task[1], task[2], w.block, t=t, **kw)
+
+    times = []
+    with ThreadPoolExecutor(max_workers=cores) as ex:
+        list(ex.map(lambda tk: one(tk, 1), tasks))          # populate the states (untimed)
+        for r in range(repeats):
+            t0 = time.perf_counter()
+            list(ex.map(lambda tk: one(tk, 2 + r), tasks))
+            times.append(time.perf_counter() - t0)
+    return {"params": taken, "seconds": times, "cores": min(cores, len(tasks)),
+            "sample": f"{taken} params in {len(tasks)} block-aligned chunks of <= {chunk} drawn from the "
+                      f"largest tensors of the workload at their widths, one oracle step each, "
+                      f"{min(cores, len(tasks))} threads"}
+
+
+def run_reference(args, w, bits_m, bits_v):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    res = oracle_sample_run(w, bits_m, bits_v, budget_s=max(2.0, 60.0 / max(1, args.steps + args.warmup)),
+                            repeats=args.steps + args.warmup)
+    timed = res["seconds"][args.warmup:]
+    sec = float(np.mean(timed))
+    value = res["params"] / sec
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "params": w.total_params, "block": w.block, "grad_dtype": w.grad_dtype,
+                   "mean_bits": W.mean_bits(w, bits_m, bits_v), "step_is": "one oracle step over the sample"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": res["cores"], "kind": "oracle", "sample": res["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args, w, bits_m, bits_v):
+    from paper_2604_06836_b200 import stq
+    from paper_2604_06836_b200.runner import Job
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if use_dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    job = Job(w, bits_m, bits_v, device=dev)
+    job.draw_grads(1)
+    pol = stq.Policy(alpha=0.1, tau=100.0, eps_stat=1e-8, interval=w.decision_interval)
+    stream = torch.cuda.current_stream()
+
+    def one_step(t):
+        dec = t % w.decision_interval == 0          # the t < 5 clause belongs to the start of training
+        job.step(t, stats=dec)
+        if dec:
+            st = job.layer_stats()
+            pol.decide(st, t)                        # the paper's policy in shadow: widths stay the seeded ones
+        return dec
+
+    t = 0
+    for _ in range(args.warmup):
+        t += 1
+        one_step(t)
+    barrier()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    is_dec = []
+    launches0 = job.handle.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        t += 1
+        dec = t % w.decision_interval == 0
+        ev[i][0].record(stream)
+        job.step(t, stats=dec)
+        ev[i][1].record(stream)
+        if dec:
+            pol.decide(job.layer_stats(), t)
+        is_dec.append(dec)
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    launches = job.handle.launch_count - launches0
+    total_ms = e0.elapsed_time(e1)
+    kern_ms = np.array([a.elapsed_time(b) for a, b in ev])
+    is_dec = np.array(is_dec)
+
+    # ---- end to end through the host-buffer entry point ----------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(job, w, args)
+
+    if use_dist:
+        tt = torch.tensor([total_ms, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(tt[0]), float(tt[1])
+    else:
+        e2e_ms = e2e["ms"] if e2e else 0.0
+
+    params = w.total_params
+    value = world * params * args.steps / (total_ms * 1e-3)
+    alg_bytes = job.algorithmic_bytes()
+    k_ms = float(kern_ms.mean())
+    achieved = alg_bytes / (k_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "params": params, "tensors": len(w.shapes), "block": w.block,
+                   "grad_dtype": w.grad_dtype, "mean_bits": round(W.mean_bits(w, bits_m, bits_v), 3),
+                   "decision_interval": w.decision_interval, "decision_steps_timed": int(is_dec.sum()),
+                   "l2": "inputs larger than L2 (%.1f GB touched per step)" % (alg_bytes / 1e9),
+                   "parallelism": "replicas" if world > 1 else "single", "grid": job.handle.grid_size,
+                   "state_bytes": job.state_bytes(), "fp32_state_bytes": 8 * params},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": (NCU_TRAFFIC_BYTES_PER_PARAM * params if NCU_TRAFFIC_BYTES_PER_PARAM else None),
+                     "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": alg_bytes,
+                     "bytes_per_param": alg_bytes / params, "kernel_ms_mean": k_ms,
+                     "kernel_ms_plain": float(kern_ms[~is_dec].mean()) if (~is_dec).any() else None,
+                     "kernel_ms_with_stats": float(kern_ms[is_dec].mean()) if is_dec.any() else None,
+                     "frac_of_nominal_8000": achieved / 8000.0},
+        "clocks": clocks,
+        "gpu_launches": int(launches),
+        "gpu_params_per_s_per_gpu": params * args.steps / (total_ms * 1e-3),
+    }
+    if e2e:
+        line["e2e"] = {"value": world * params * e2e["steps"] / (e2e_ms * 1e-3), "unit": UNIT,
+                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"],
+                       "ms_per_step": e2e_ms / e2e["steps"]}
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        res = oracle_sample_run(w, bits_m, bits_v, budget_s=8.0, repeats=1)
+        line["cpu_baseline"] = {"value": res["params"] / res["seconds"][0], "unit": UNIT, "cores": res["cores"],
+                                "kind": "oracle", "sample": res["sample"]}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if use_dist:
+        dist.destroy_process_group()
+
+
+def run_e2e(job, w, args):
+    """The same step through stq_step_host: pinned host buffers in, host buffers out, copies timed."""
+    from paper_2604_06836_b200 import stq
+    steps = max(1, min(args.e2e_steps, args.steps))
+    torch.cuda.synchronize()
+    host_p = job.param_flat.cpu().pin_memory()
+    host_g = job.grad_flat.cpu().pin_memory()
+    rows = []
+    host_states = []
+    for i, n in enumerate(job.numels):
+        s = job.states[i]
+        hs = stq.QState(s.m_codes.cpu().pin_memory(), s.m_scales.cpu().pin_memory(), s.bits_m,
+                        s.v_codes.cpu().pin_memory(), s.v_scales.cpu().pin_memory(), s.bits_v)
+        host_states.append(hs)
+        o = job.offsets[i]
+        rows.append(stq.make_row(n, job.block, hs, hs, host_p[o:o + n], host_g[o:o + n], job.wd[i]))
+    tbl = stq.table(rows)
+    hp = job.hp(job.t + 1)
+    job.handle.step_host(tbl, **hp)          # warm-up: grows the device arena
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    h2d = d2h = 0
+    for k in range(steps):
+        hp = job.hp(job.t + 2 + k)
+        h2d, d2h = job.handle.step_host(tbl, **hp)
+    torch.cuda.synchronize()
+    ms = (time.perf_counter() - t0) * 1e3
+    job._tbl = None
+    return {"ms": ms, "steps": steps, "h2d": h2d, "d2h": d2h}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="cfg5", help="cfg1..cfg5 (default: the 1.5B bandwidth run)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = W.config(args.config)
+    bits_m, bits_v, _ = W.draw_bits(w)
+    if args.impl == "reference":
+        run_reference(args, w, bits_m, bits_v)
+    else:
+        run_ours(args, w, bits_m, bits_v)
+
+
+if __name__ == "__main__":
+    main()

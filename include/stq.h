@@ -15,7 +15,7 @@
  *    synchronising, except stq_layer_stats and stq_step_host, which synchronise the stream.
  *  - All arguments are validated on the host before anything is launched.  Return value: 0 on
  *    success, a negative STQ_E_* code otherwise; nothing is launched when an error is returned.
- *    The device code never traps, asserts or spins.
+ *    The device code never traps or asserts, and every wait in it is bounded (stq_device_status).
  *  - A handle is bound to one device and is not thread-safe; use one handle per stream.
  *
  * Stored layout (per tensor, per state)
@@ -46,14 +46,15 @@ enum {
   STQ_OK = 0,
   STQ_E_NULL = -1,      /* a required pointer is NULL                                         */
   STQ_E_BITS = -2,      /* a width outside {2,3,4,8,16,32}                                    */
-  STQ_E_BLOCK = -3,     /* block not in {128, 256, 512}                                       */
+  STQ_E_BLOCK = -3,     /* block not in {128, 256}                                            */
   STQ_E_ALIGN = -4,     /* a buffer is not aligned as required                                */
   STQ_E_ALIAS = -5,     /* in/out buffers overlap in a way the step cannot honour             */
   STQ_E_NUMEL = -6,     /* numel == 0, or the table is empty or too large                     */
   STQ_E_CUDA = -7,      /* a CUDA runtime call failed (see stq_last_cuda_error)               */
   STQ_E_WORKSPACE = -8, /* the library could not grow its own workspace                       */
   STQ_E_ARG = -9,       /* an invalid scalar argument (step < 1, unknown dtype or flag, ...)  */
-  STQ_E_STATE = -10     /* call order: no statistics pending for stq_layer_stats              */
+  STQ_E_STATE = -10,    /* call order: no statistics pending for stq_layer_stats              */
+  STQ_E_TIMEOUT = -11   /* a bounded wait inside a kernel ran out (stq_device_status)         */
 };
 
 enum { STQ_GRAD_F32 = 0, STQ_GRAD_BF16 = 1 };
@@ -74,7 +75,7 @@ typedef struct stq_tensor {
   void* v_codes_out;         /* scales_out may equal scales_in                                 */
   float* v_scales_out;
   uint64_t numel;
-  uint32_t block;            /* quantization block: 128, 256 or 512                            */
+  uint32_t block;            /* quantization block: 128 or 256                                 */
   uint8_t bits_m, bits_v;          /* widths stored now                                        */
   uint8_t bits_m_out, bits_v_out;  /* widths to write                                          */
   float weight_decay;        /* per-tensor lambda                                              */
@@ -134,6 +135,12 @@ int stq_repack(stq_handle* h, const stq_tensor* tensors, int L, void* stream);
  * the bytes copied. */
 int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hparams* hp,
                   unsigned flags, uint64_t* bytes_h2d, uint64_t* bytes_d2h);
+
+/* Synchronises `stream` and reports whether any kernel launched through this handle gave up on a
+ * bounded wait (its asynchronous copies did not complete in ~2 s): STQ_E_TIMEOUT, else STQ_OK.
+ * The device never spins without a limit; after a time-out the outputs of that launch are
+ * undefined and the handle should be destroyed. */
+int stq_device_status(stq_handle* h, void* stream);
 
 /* Kernel launches issued through this handle so far. */
 uint64_t stq_launch_count(const stq_handle* h);

@@ -121,7 +121,13 @@ inline float dequant_lin(uint32_t code, float s, int b) {
 
 // ---- logarithmic block quantizer (second moment, x >= 0) -------------------------------------
 // scale s = max x; code K is the block maximum, each code step is R/K octaves, code 0 is the floor
-// s*2^-R.  d = log-distance to the maximum in octaves, q = clamp(K + round-half-even(d*K/R), 0, K).
+// s*2^-R.
+//  * b <= 4 (R = K, one octave per code): the code is the nearest octave below the maximum,
+//    q = clamp(K + floor(log2(x/s) + 1/2), 0, K), taken as the exponent of y = fl(x * c) with
+//    c = fl(fl(1/s) * sqrt2): floor(log2(x*sqrt2/s)) is that exponent.
+//  * b = 8, 16: d = log-distance to the maximum in octaves from the split logarithm,
+//    q = clamp(K + round-half-even(d*K/R), 0, K).
+const float kSqrt2 = 0x1.6a09e6p+0f;
 void quant_log_block(const float* x, uint64_t n, int b, uint32_t* code, float* scale) {
   float s = 0.0f;
   for (uint64_t i = 0; i < n; ++i) if (x[i] > s) s = x[i];
@@ -132,7 +138,19 @@ void quant_log_block(const float* x, uint64_t n, int b, uint32_t* code, float* s
   }
   *scale = s;
   const int K = K_of(b), R = R_of(b);
-  const float a_b = (float)K / (float)R;          // exact: 1, 1, 1, 8.5, 2184.5
+  if (b <= 4) {
+    const float rs = 1.0f / s;
+    const float c = rs * kSqrt2;
+    for (uint64_t i = 0; i < n; ++i) {
+      float y = x[i] * c;
+      int q = K + (lg_E(y) - 127);
+      if (q < 0) q = 0;
+      if (q > K) q = K;
+      code[i] = (uint32_t)q;
+    }
+    return;
+  }
+  const float a_b = (float)K / (float)R;          // exact: 8.5, 2184.5
   const int Es = lg_E(s);
   const float Ps = lg_P(s);
   for (uint64_t i = 0; i < n; ++i) {

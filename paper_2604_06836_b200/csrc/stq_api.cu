@@ -25,11 +25,12 @@ struct stq_handle {
   std::vector<uint64_t> cached_sig;   // numel | wide<<63 per tensor: decides the tile map
   TensorDesc* d_table = nullptr;
   size_t d_table_cap = 0;
-  uint32_t* d_tile_map = nullptr;   // tile -> tensor index, narrow tiles first, then wide
+  // tile -> tensor index; order: fast tiles, then the remaining narrow tiles, then wide ones
+  uint32_t* d_tile_map = nullptr;
   size_t d_tile_cap = 0;
-  uint32_t* d_ntiles = nullptr;     // per tensor
-  size_t d_ntiles_cap = 0;
-  uint32_t n_tiles = 0, n_narrow = 0;
+  uint32_t n_tiles = 0, n_fast = 0, n_narrow = 0;   // n_narrow counts fast + remaining narrow
+  int fast_grid = 0;
+  int* d_err = nullptr;             // raised by a kernel whose bounded wait ran out
 
   // pinned staging for uploads
   void* h_stage = nullptr;
@@ -56,7 +57,7 @@ namespace {
 enum Kind { kKindStep = 0, kKindRepack = 1, kKindInit = 2, kKindStats = 3 };
 
 bool width_ok(int b) { return b == 2 || b == 3 || b == 4 || b == 8 || b == 16 || b == 32; }
-bool block_ok(uint32_t b) { return b == 128 || b == 256 || b == 512; }
+bool block_ok(uint32_t b) { return b >= 128 && b <= (uint32_t)stq::kMaxBlock && (b & (b - 1)) == 0; }
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 int fail_cuda(stq_handle* h, cudaError_t e) {
@@ -170,48 +171,58 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
                     std::memcmp(h->cached.data(), tensors, sizeof(stq_tensor) * (size_t)L) == 0;
   if (same) return STQ_OK;
 
-  // tile counts; narrow tensors first, wide (any 32-bit state) after
-  std::vector<uint32_t> ntiles(L), tile0(L);
+  // Tile classes.  "Fast": full tiles of a step whose widths do not change (2..16 bits); they go to
+  // the main kernel.  The rest (ragged last tile, width change, 32-bit state, other entry points)
+  // goes to the generic kernel: narrow tiles first, wide (any 32-bit state) after.
+  std::vector<uint32_t> nfast(L), nslow(L);
   std::vector<uint64_t> sig(L);
-  uint64_t total = 0, narrow = 0;
+  uint64_t total = 0, fast = 0, slow_narrow = 0;
   for (int l = 0; l < L; ++l) {
-    uint64_t nt = (tensors[l].numel + stq::kTile - 1) / stq::kTile;
-    ntiles[l] = (uint32_t)nt;
+    const stq_tensor& t = tensors[l];
+    const uint64_t nt = (t.numel + stq::kTile - 1) / stq::kTile;
+    const bool wide = row_is_wide(t, kind);
+    const bool fast_ok = kind == kKindStep && !wide && t.bits_m == t.bits_m_out && t.bits_v == t.bits_v_out &&
+                         t.numel < (1ull << 32);
+    const uint64_t nf = fast_ok ? t.numel / stq::kTile : 0;
+    nfast[l] = (uint32_t)nf;
+    nslow[l] = (uint32_t)(nt - nf);
     total += nt;
-    const bool wide = row_is_wide(tensors[l], kind);
-    if (!wide) narrow += nt;
-    sig[l] = tensors[l].numel | (wide ? 1ull << 63 : 0ull);
+    fast += nf;
+    if (!wide) slow_narrow += nt - nf;
+    sig[l] = t.numel | (wide ? 1ull << 63 : 0ull) | (fast_ok ? 1ull << 62 : 0ull);
   }
-  // the tile map depends only on sizes and on which tensors are wide: skip it when unchanged
-  const bool same_map = h->cached_kind >= 0 && sig == h->cached_sig && h->n_tiles == (uint32_t)total;
   if (total > 0xFFFFFFF0ull) return STQ_E_NUMEL;
+  // the tile map depends only on sizes and classes: skip it when unchanged
+  const bool same_map = h->cached_kind >= 0 && sig == h->cached_sig && h->n_tiles == (uint32_t)total;
 
   const size_t bytes_table = sizeof(TensorDesc) * (size_t)L;
   const size_t bytes_map = sizeof(uint32_t) * (size_t)total;
-  const size_t bytes_nt = sizeof(uint32_t) * (size_t)L;
   const size_t off_map = (bytes_table + 255) & ~size_t(255);
-  const size_t off_nt = (off_map + bytes_map + 255) & ~size_t(255);
   int rc;
-  if ((rc = grow_stage(h, off_nt + bytes_nt)) != STQ_OK) return rc;
+  if ((rc = grow_stage(h, off_map + bytes_map)) != STQ_OK) return rc;
   if ((rc = grow(h, h->d_table, h->d_table_cap, (size_t)L)) != STQ_OK) return rc;
   if ((rc = grow(h, h->d_tile_map, h->d_tile_cap, (size_t)total)) != STQ_OK) return rc;
-  if ((rc = grow(h, h->d_ntiles, h->d_ntiles_cap, (size_t)L)) != STQ_OK) return rc;
   if (h->stage_busy) { STQ_CUDA(h, cudaEventSynchronize(h->stage_ev)); h->stage_busy = false; }
 
   uint8_t* st = static_cast<uint8_t*>(h->h_stage);
   TensorDesc* ht = reinterpret_cast<TensorDesc*>(st);
   uint32_t* hm = reinterpret_cast<uint32_t*>(st + off_map);
-  uint32_t* hn = reinterpret_cast<uint32_t*>(st + off_nt);
-  uint32_t next_narrow = 0, next_wide = (uint32_t)narrow;
+  uint32_t next_fast = 0, next_narrow = (uint32_t)fast, next_wide = (uint32_t)(fast + slow_narrow);
   for (int l = 0; l < L; ++l) {
     const stq_tensor& t = tensors[l];
-    uint32_t& next = row_is_wide(t, kind) ? next_wide : next_narrow;
-    tile0[l] = next;
-    for (uint32_t i = 0; i < ntiles[l]; ++i) hm[next + i] = (uint32_t)l;
-    next += ntiles[l];
-    hn[l] = ntiles[l];
     TensorDesc d;
     std::memset(&d, 0, sizeof(d));
+    d.tile0 = next_fast;
+    d.nfast = nfast[l];
+    if (!same_map)
+      for (uint32_t i = 0; i < nfast[l]; ++i) hm[next_fast + i] = (uint32_t)l;
+    next_fast += nfast[l];
+    uint32_t& next = row_is_wide(t, kind) ? next_wide : next_narrow;
+    d.tile0s = next;
+    d.nslow = nslow[l];
+    if (!same_map)
+      for (uint32_t i = 0; i < nslow[l]; ++i) hm[next + i] = (uint32_t)l;
+    next += nslow[l];
     d.param = t.param;
     d.grad = t.grad;
     d.mc_in = static_cast<const uint8_t*>(t.m_codes_in);
@@ -223,24 +234,22 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     d.vc_out = static_cast<uint8_t*>(t.v_codes_out);
     d.vs_out = t.v_scales_out;
     d.numel = t.numel;
-    d.tile0 = tile0[l];
     d.block = kind == kKindStats ? 128u : t.block;
     d.bm_in = t.bits_m; d.bv_in = t.bits_v; d.bm_out = t.bits_m_out; d.bv_out = t.bits_v_out;
     d.wd = t.weight_decay;
     ht[l] = d;
   }
   STQ_CUDA(h, cudaMemcpyAsync(h->d_table, ht, bytes_table, cudaMemcpyHostToDevice, stream));
-  if (!same_map) {
+  if (!same_map)
     STQ_CUDA(h, cudaMemcpyAsync(h->d_tile_map, hm, bytes_map, cudaMemcpyHostToDevice, stream));
-    STQ_CUDA(h, cudaMemcpyAsync(h->d_ntiles, hn, bytes_nt, cudaMemcpyHostToDevice, stream));
-  }
   STQ_CUDA(h, cudaEventRecord(h->stage_ev, stream));
   h->stage_busy = true;
   h->cached.assign(tensors, tensors + L);
   h->cached_kind = kind;
   h->cached_sig.swap(sig);
   h->n_tiles = (uint32_t)total;
-  h->n_narrow = (uint32_t)narrow;
+  h->n_fast = (uint32_t)fast;
+  h->n_narrow = (uint32_t)(fast + slow_narrow);
   return STQ_OK;
 }
 
@@ -252,9 +261,14 @@ int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::St
     if (rc != STQ_OK) return rc;
     partials = h->d_partials;
   }
-  if (h->n_narrow > 0) {
-    STQ_CUDA(h, stq::launch_tiles(mode, false, grad_dtype, stats, h->d_table, h->d_tile_map, 0, h->n_narrow,
-                                  sc, partials, h->grid, stream));
+  if (h->n_fast > 0) {   // only a step table has fast tiles
+    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, h->d_table, h->d_tile_map, h->n_fast, sc, partials,
+                                      h->d_err, h->fast_grid, stream));
+    h->launches++;
+  }
+  if (h->n_narrow > h->n_fast) {
+    STQ_CUDA(h, stq::launch_tiles(mode, false, grad_dtype, stats, h->d_table, h->d_tile_map, h->n_fast,
+                                  h->n_narrow, sc, partials, h->grid, stream));
     h->launches++;
   }
   if (h->n_tiles > h->n_narrow) {
@@ -311,6 +325,13 @@ int stq_create(stq_handle** out, int device) {
   }
   h->sm_count = prop.multiProcessorCount;
   h->grid = h->sm_count * stq::step_ctas_per_sm();
+  h->fast_grid = h->sm_count * stq::fast_ctas_per_sm();
+  if (cudaMalloc(reinterpret_cast<void**>(&h->d_err), sizeof(int)) != cudaSuccess ||
+      cudaMemset(h->d_err, 0, sizeof(int)) != cudaSuccess) {
+    cudaEventDestroy(h->stage_ev);
+    delete h;
+    return STQ_E_WORKSPACE;
+  }
   *out = h;
   return STQ_OK;
 }
@@ -321,7 +342,7 @@ int stq_destroy(stq_handle* h) {
   if (h->stage_busy) cudaEventSynchronize(h->stage_ev);
   cudaFree(h->d_table);
   cudaFree(h->d_tile_map);
-  cudaFree(h->d_ntiles);
+  cudaFree(h->d_err);
   cudaFree(h->d_partials);
   cudaFree(h->d_stats);
   cudaFree(h->d_arena);
@@ -393,12 +414,22 @@ int stq_layer_stats(stq_handle* h, double* out, int L, void* stream) {
     if (e != cudaSuccess) { h->cuda_err = cudaGetErrorString(e); return STQ_E_WORKSPACE; }
     h->h_stats_cap = (size_t)L * 4;
   }
-  STQ_CUDA(h, stq::launch_stats_finish(h->d_table, h->d_ntiles, L, h->d_partials, h->d_stats, s));
+  STQ_CUDA(h, stq::launch_stats_finish(h->d_table, L, h->d_partials, h->d_stats, s));
   h->launches++;
   STQ_CUDA(h, cudaMemcpyAsync(h->h_stats, h->d_stats, sizeof(double) * 4 * (size_t)L, cudaMemcpyDeviceToHost, s));
   STQ_CUDA(h, cudaStreamSynchronize(s));
   std::memcpy(out, h->h_stats, sizeof(double) * 4 * (size_t)L);
   return STQ_OK;
+}
+
+int stq_device_status(stq_handle* h, void* stream) {
+  if (!h) return STQ_E_NULL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  STQ_CUDA(h, cudaSetDevice(h->device));
+  int flag = 0;
+  STQ_CUDA(h, cudaMemcpyAsync(&flag, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, s));
+  STQ_CUDA(h, cudaStreamSynchronize(s));
+  return flag ? STQ_E_TIMEOUT : STQ_OK;
 }
 
 int stq_repack(stq_handle* h, const stq_tensor* tensors, int L, void* stream) {
@@ -502,7 +533,7 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
 }
 
 uint64_t stq_launch_count(const stq_handle* h) { return h ? h->launches : 0; }
-int stq_grid_size(const stq_handle* h) { return h ? h->grid : 0; }
+int stq_grid_size(const stq_handle* h) { return h ? h->fast_grid : 0; }
 int stq_sm_count(const stq_handle* h) { return h ? h->sm_count : 0; }
 
 const char* stq_strerror(int code) {
@@ -510,7 +541,7 @@ const char* stq_strerror(int code) {
     case STQ_OK: return "ok";
     case STQ_E_NULL: return "a required pointer is NULL";
     case STQ_E_BITS: return "bit-width not in {2,3,4,8,16,32}";
-    case STQ_E_BLOCK: return "block not in {128,256,512}";
+    case STQ_E_BLOCK: return "block not in {128,256}";
     case STQ_E_ALIGN: return "buffer not aligned (16 bytes for param/grad/codes, 4 for scales)";
     case STQ_E_ALIAS: return "in/out buffers overlap (in-place needs the same pointer and width)";
     case STQ_E_NUMEL: return "numel is 0, or the table is empty or too large";
@@ -518,6 +549,7 @@ const char* stq_strerror(int code) {
     case STQ_E_WORKSPACE: return "could not allocate library workspace";
     case STQ_E_ARG: return "invalid scalar argument";
     case STQ_E_STATE: return "no statistics pending for this table";
+    case STQ_E_TIMEOUT: return "a bounded wait inside a kernel ran out (results of that launch are invalid)";
     default: return "unknown error";
   }
 }

@@ -5,10 +5,12 @@
 
 namespace stq {
 
-constexpr int kTile = 4096;      // elements per tile; every tile lies inside one tensor
-constexpr int kThreads = 256;    // 8 warps; a warp owns 4 consecutive 128-element rows of the tile
+constexpr int kThreads = 256;    // 8 warps per CTA
 constexpr int kRowElems = 128;   // one row: lane l holds elements 4l .. 4l+3
-constexpr int kRowsPerWarp = 4;
+constexpr int kRowsPerWarp = 2;  // a warp owns this many consecutive rows of a tile
+constexpr int kTile = (kThreads / 32) * kRowsPerWarp * kRowElems;   // elements per tile; a tile lies inside one tensor
+constexpr int kMaxBlock = kRowsPerWarp * kRowElems;                 // a quantization block never leaves its warp
+constexpr int kFastCtasPerSm = 4;
 
 // Device-side row of the tensor table.
 struct TensorDesc {
@@ -23,11 +25,13 @@ struct TensorDesc {
   uint8_t* vc_out;
   float* vs_out;
   unsigned long long numel;
-  unsigned int tile0;       // index of this tensor's first tile in the launch's tile order
-  unsigned int block;       // 128 / 256 / 512
+  unsigned int tile0;       // first "fast" tile (full tile, same width in and out) of this tensor
+  unsigned int nfast;       // number of fast tiles; they cover elements [0, nfast * kTile)
+  unsigned int tile0s;      // first tile of the rest (ragged tail, or the whole tensor if it is not fast)
+  unsigned int nslow;
+  unsigned int block;       // 128 / 256
   unsigned char bm_in, bv_in, bm_out, bv_out;
   float wd;                 // fp32(lambda)
-  unsigned int pad[2];
 };
 
 // Per-launch scalars of the AdamW update.
@@ -48,9 +52,16 @@ cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const
                          const uint32_t* tile_map, uint32_t tile_begin, uint32_t tile_end,
                          const StepConsts& sc, double* partials, int grid, cudaStream_t stream);
 
+// The main step kernel over the fast tiles [0, n_fast) (stq_step_fast.cu).  err_flag is set to 1 if
+// a bounded wait inside the kernel ran out.
+cudaError_t launch_step_fast(int grad_dtype, bool stats, const TensorDesc* table, const uint32_t* tile_map,
+                             uint32_t n_fast, const StepConsts& sc, double* partials, int* err_flag, int grid,
+                             cudaStream_t stream);
+int fast_ctas_per_sm();
+
 // out[l] = {sum over the tensor's tiles of partials (fixed order), numel}
-cudaError_t launch_stats_finish(const TensorDesc* table, const uint32_t* ntiles_of, int L,
-                                const double* partials, double* out, cudaStream_t stream);
+cudaError_t launch_stats_finish(const TensorDesc* table, int L, const double* partials, double* out,
+                                cudaStream_t stream);
 
 // Resident CTAs per SM of the step kernel (occupancy query), for sizing the persistent grid.
 int step_ctas_per_sm();

@@ -1,12 +1,15 @@
 // Kernels of the mixed-bit quantized AdamW step for sm_100a.
 //
-// Work decomposition: the concatenated tensor list is cut into tiles of 4096 elements that never
+// Generic path (ragged tails, 32-bit states, width changes, init, repack, statistics alone); the
+// main step kernel is in stq_step_fast.cu.
+//
+// Work decomposition: the concatenated tensor list is cut into tiles of kTile elements that never
 // cross a tensor; persistent CTAs of 8 warps stride over the tile list.  Inside a tile a warp owns
-// 4 consecutive rows of 128 elements and lane l of a row holds elements 4l..4l+3, so parameters
+// kRowsPerWarp consecutive rows of 128 elements and lane l of a row holds elements 4l..4l+3, so parameters
 // and fp32 gradients move as 128-bit accesses (512 contiguous bytes per warp), bf16 gradients as
 // 64-bit ones, and a lane's four codes are one 8/16/32/64-bit access at widths 2/4/8/16 (3-bit
 // rows are 48 bytes: 12 lanes move one word each and the 12-bit lane fields are exchanged with
-// shuffles).  A quantization block (128/256/512) is 1/2/4 whole rows of one warp, so the block
+// shuffles).  A quantization block (128/256) is 1/2 whole rows of one warp, so the block
 // maximum is a lane-local max of 4 followed by one warp REDUX on the (non-negative) bit patterns.
 //
 // Arithmetic that decides codes is written with the *_rn intrinsics, which are never contracted,
@@ -26,6 +29,7 @@ constexpr float kTwo23 = 8388608.0f;
 constexpr uint32_t kTwo23Bits = 0x4B000000u;
 constexpr float kTiny = 0x1p-100f;                //: smaller block maxima store a zero block
 constexpr int kZeroBlockExp = 1 << 20;            // exponent stand-in that floors every log code
+constexpr float kSqrt2 = 0x1.6a09e6p+0f;
 
 // P(t) ~ log2(1+t) = t*(c1 + t*(c2 + ... + t*c6)), t in [0,1)
 constexpr float kP1 = 0x1.714b30p+0f, kP2 = -0x1.6fc360p-1f, kP3 = 0x1.d54a42p-2f,
@@ -345,12 +349,12 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
     const TensorDesc* __restrict__ T = table + __ldg(tile_map + tile);
     const unsigned long long numel = T->numel;
     const unsigned long long e_warp =
-        (unsigned long long)(tile - T->tile0) * kTile + (unsigned)warp * (R * kRowElems);
+        (unsigned long long)(T->nfast + (tile - T->tile0s)) * kTile + (unsigned)warp * (R * kRowElems);
     float st_g = 0.f, st_a = 0.f, st_q = 0.f;
 
     if (e_warp < numel) {
       const uint32_t B = T->block;
-      const int lgB = 7 + (int)(B >> 8);   // 128 / 256 / 512
+      const int lgB = 7 + (int)(B >> 8);   // 128 / 256
       const int bm_in = T->bm_in, bv_in = T->bv_in, bm_out = T->bm_out, bv_out = T->bv_out;
 
       int nvl[R];
@@ -490,11 +494,6 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
             mxv[r] = mxv[r + 1] = max(mxv[r], mxv[r + 1]);
           }
         }
-        if (B >= 512) {
-          const uint32_t a = max(mxm[0], mxm[2]), b = max(mxv[0], mxv[2]);
-#pragma unroll
-          for (int r = 0; r < R; ++r) { mxm[r] = a; mxv[r] = b; }
-        }
 
         // ---- quantize, pack, store; decode the new codes; update the parameters -------------------
         const LinW lw = lin_width(bm_out);
@@ -550,27 +549,37 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
             const float s_raw = __uint_as_float(mxv[r]);
             const bool zero = s_raw < kTiny;
             const float s = zero ? 0.f : s_raw;
-            const int Es = zero ? kZeroBlockExp : (int)(mxv[r] >> 23);
-            const float Ps = lg_poly(mxv[r]);
-            const uint32_t ebase = kMagicBits - (uint32_t)Es;
             uint32_t x[4];
+            uint32_t sub;
+            if (bv_out <= 4) {
+              // one octave per code: the code is the exponent of x*sqrt2/s, floored at -K
+              const float c = zero ? 0.f : __fmul_rn(__frcp_rn(s_raw), kSqrt2);
+              const float ymin = __uint_as_float((uint32_t)(127 - gw.K) << 23);
+              sub = (uint32_t)(127 - gw.K);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const uint32_t xb = __float_as_uint(vt[r][k]);
-              const float de = __fadd_rn(__uint_as_float(ebase + (xb >> 23)), -kMagic);   // float(E_x - E_s)
-              const float dp = __fadd_rn(lg_poly(xb), -Ps);
-              const float d = fmaxf(__fadd_rn(de, dp), gw.negR);
-              const float t = __fmaf_rn(d, gw.a, kMagic);       // low bits: code - K, in [-K, 0]
-              x[k] = __float_as_uint(t);
-              if constexpr (MODE == kStep) {
-                if (bv_out <= 4) {
-                  vq[k] = __fmul_rn(s, __uint_as_float((x[k] << 23) + 0x3F800000u));
-                } else {
+              for (int k = 0; k < 4; ++k) {
+                const uint32_t yb = __float_as_uint(fmaxf(__fmul_rn(vt[r][k], c), ymin));
+                x[k] = yb >> 23;
+                if constexpr (MODE == kStep) vq[k] = __fmul_rn(s, __uint_as_float(yb & 0x7F800000u));
+              }
+            } else {
+              const int Es = zero ? kZeroBlockExp : (int)(mxv[r] >> 23);
+              const float Ps = lg_poly(mxv[r]);
+              const uint32_t ebase = kMagicBits - (uint32_t)Es;
+              sub = kMagicBits - (uint32_t)gw.K;
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const uint32_t xb = __float_as_uint(vt[r][k]);
+                const float de = __fadd_rn(__uint_as_float(ebase + (xb >> 23)), -kMagic);   // float(E_x - E_s)
+                const float dp = __fadd_rn(lg_poly(xb), -Ps);
+                const float d = fmaxf(__fadd_rn(de, dp), gw.negR);
+                const float t = __fmaf_rn(d, gw.a, kMagic);       // low bits: code - K, in [-K, 0]
+                x[k] = __float_as_uint(t);
+                if constexpr (MODE == kStep)
                   vq[k] = __fmul_rn(s, ex2_poly(__fmul_rn(__fadd_rn(t, -kMagic), gw.c)));
-                }
               }
             }
-            store_codes(vco, e_row, bv_out, lane, lim_vo, x, kMagicBits - (uint32_t)gw.K, nvl[r]);
+            store_codes(vco, e_row, bv_out, lane, lim_vo, x, sub, nvl[r]);
             if (lane == 0 && (e_row & (B - 1)) == 0) vso[e_row >> lgB] = s;
           }
 
@@ -609,17 +618,18 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
   }
 }
 
-// One CTA per tensor: fixed-order sum of its tiles' partials.
+// One CTA per tensor: fixed-order sum of its tiles' partials (fast range, then the rest).
 __global__ void __launch_bounds__(256)
-stq_stats_finish_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ ntiles_of, int L,
-                        const double* __restrict__ partials, double* __restrict__ out) {
+stq_stats_finish_kernel(const TensorDesc* __restrict__ table, int L, const double* __restrict__ partials,
+                        double* __restrict__ out) {
   const int l = blockIdx.x;
   if (l >= L) return;
-  const uint32_t t0 = table[l].tile0, nt = ntiles_of[l];
+  const uint32_t t0 = table[l].tile0, nf = table[l].nfast, t0s = table[l].tile0s, ns = table[l].nslow;
   double a[3] = {0.0, 0.0, 0.0};
-  for (uint32_t i = threadIdx.x; i < nt; i += blockDim.x) {
+  for (uint32_t i = threadIdx.x; i < nf + ns; i += blockDim.x) {
+    const size_t t = i < nf ? (size_t)t0 + i : (size_t)t0s + (i - nf);
 #pragma unroll
-    for (int k = 0; k < 3; ++k) a[k] += partials[(size_t)(t0 + i) * 3 + k];
+    for (int k = 0; k < 3; ++k) a[k] += partials[t * 3 + k];
   }
   __shared__ double sh[256][3];
 #pragma unroll
@@ -677,9 +687,9 @@ cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const
   return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_stats_finish(const TensorDesc* table, const uint32_t* ntiles_of, int L,
-                                const double* partials, double* out, cudaStream_t stream) {
-  stq_stats_finish_kernel<<<L, 256, 0, stream>>>(table, ntiles_of, L, partials, out);
+cudaError_t launch_stats_finish(const TensorDesc* table, int L, const double* partials, double* out,
+                                cudaStream_t stream) {
+  stq_stats_finish_kernel<<<L, 256, 0, stream>>>(table, L, partials, out);
   return cudaGetLastError();
 }
 

@@ -78,6 +78,7 @@ def lib() -> C.CDLL:
         L.stq_repack.argtypes = [vp, PT, C.c_int, vp]
         L.stq_step_host.argtypes = [vp, PT, C.c_int, C.POINTER(CHParams), C.c_uint,
                                     C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+        L.stq_device_status.argtypes = [vp, vp]
         L.stq_launch_count.argtypes = [vp]
         L.stq_launch_count.restype = C.c_uint64
         L.stq_grid_size.argtypes = [vp]
@@ -224,6 +225,10 @@ class Handle:
         self._check(lib().stq_step_host(self._h, tbl, len(tbl), C.byref(hp), flags, C.byref(h2d), C.byref(d2h)),
                     "stq_step_host")
         return int(h2d.value), int(d2h.value)
+
+    def device_status(self, stream=None):
+        """Synchronises the stream; raises if a kernel gave up on a bounded wait."""
+        self._check(lib().stq_device_status(self._h, _stream_ptr(stream)), "stq_device_status")
 
     @property
     def launch_count(self) -> int:

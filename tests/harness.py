@@ -115,7 +115,7 @@ def assert_stats_close(g: np.ndarray, o: np.ndarray, tag=""):
 
 
 def compare_job(job: Job, oj: OracleJob, rel: float, tag=""):
-    torch.cuda.synchronize()
+    job.handle.device_status()      # synchronises; raises if a kernel gave up on a bounded wait
     for i in range(job.L):
         assert_states_equal(job.states[i], oj.states[i], f"{tag} tensor {i} ({job.w.shapes[i][0]})")
         assert_theta_close(job.params[i], oj.theta[i], rel, f"{tag} tensor {i} ({job.w.shapes[i][0]})",

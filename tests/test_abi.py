@@ -37,14 +37,14 @@ def test_buffer_sizes(stq_lib, O, bits):
     for n in (1, 7, 128, 129, 1000, 4096, 50257 * 1600):
         want = ((n * bits + 7) // 8 + 15) // 16 * 16
         assert stq.codes_bytes(n, bits) == want == O.codes_bytes(n, bits)
-        for block in (128, 256, 512):
+        for block in (128, 256):
             assert stq.scales_bytes(n, block) == 4 * ((n + block - 1) // block) == 4 * O.num_blocks(n, block)
 
 
 def test_errors_without_a_device_or_with_bad_arguments(stq_lib):
     from paper_2604_06836_b200 import stq
     assert stq_lib.stq_strerror(0) == b"ok"
-    for code in range(-10, 0):
+    for code in range(-11, 0):
         assert stq_lib.stq_strerror(code) not in (b"ok", b"unknown error")
     h = C.c_void_p()
     assert stq_lib.stq_create(None, 0) == -1
