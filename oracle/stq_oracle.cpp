@@ -93,7 +93,8 @@ inline float ex2(float e) {
 }
 
 // ---- linear symmetric block quantizer (first moment) ----------------------------------------
-// scale s = max|x|; q = clamp(round-half-even(x * fl(qmax/s)), -qmax, qmax); stored code q + 2^(b-1).
+// scale s = max|x|; inv = fl(qmax * fl(1/s)); q = clamp(round-half-even(x * inv), -qmax, qmax);
+// stored code q + 2^(b-1).
 void quant_lin_block(const float* x, uint64_t n, int b, uint32_t* code, float* scale) {
   float s = 0.0f;
   for (uint64_t i = 0; i < n; ++i) { float a = fabsf(x[i]); if (a > s) s = a; }
@@ -104,7 +105,8 @@ void quant_lin_block(const float* x, uint64_t n, int b, uint32_t* code, float* s
     return;
   }
   *scale = s;
-  float inv = (float)qmax / s;
+  float rs = 1.0f / s;
+  float inv = (float)qmax * rs;
   for (uint64_t i = 0; i < n; ++i) {
     double r = nearbyint((double)x[i] * (double)inv);
     if (r > qmax) r = qmax;
@@ -286,18 +288,17 @@ int orc_step(float* theta, const void* grad, uint64_t n, uint32_t block,
     for (uint64_t i = 0; i < n; ++i) { float l2 = wd * theta[i]; g[i] = g[i] + l2; }
   }
 
-  // moments: m_t = b1*m + (1-b1)*g ; v_t = b2*v + (1-b2)*g^2, every operation rounded to fp32
+  // moments: m_t = fma(b1, m, fl(c1*g)) ; v_t = fma(b2, v, fl(fl(c2*g)*g)) in fp32: the new term is
+  // rounded, the decayed state is added with one fused rounding
   // (the four coefficients are the fp32 roundings of beta and of 1-beta taken in double)
   const float fb1 = (float)hp->beta1, fb2 = (float)hp->beta2;
   const float omb1 = (float)(1.0 - hp->beta1), omb2 = (float)(1.0 - hp->beta2);
   for (uint64_t i = 0; i < n; ++i) {
-    float a = fb1 * m[i];
     float c = omb1 * g[i];
-    m[i] = a + c;
-    float p = fb2 * v[i];
+    m[i] = fmaf(fb1, m[i], c);
     float w = omb2 * g[i];
     float w2 = w * g[i];
-    v[i] = p + w2;
+    v[i] = fmaf(fb2, v[i], w2);
   }
 
   // Quantize(m_t, linear), Quantize(v_t, log) at the widths assigned for this step

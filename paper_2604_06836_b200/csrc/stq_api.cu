@@ -1,5 +1,6 @@
 // C-ABI host layer of libstq: argument validation, tensor-table and tile-map upload, launches.
 // No arithmetic of the method lives here; every step of the path runs in stq_kernels.cu.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -181,15 +182,17 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     const stq_tensor& t = tensors[l];
     const uint64_t nt = (t.numel + stq::kTile - 1) / stq::kTile;
     const bool wide = row_is_wide(t, kind);
+    // (the main kernel moves the scales with 16-byte bulk copies as well)
     const bool fast_ok = kind == kKindStep && !wide && t.bits_m == t.bits_m_out && t.bits_v == t.bits_v_out &&
-                         t.numel < (1ull << 32);
+                         t.numel < (1ull << 32) && aligned(t.m_scales_in, 16) && aligned(t.v_scales_in, 16);
     const uint64_t nf = fast_ok ? t.numel / stq::kTile : 0;
     nfast[l] = (uint32_t)nf;
     nslow[l] = (uint32_t)(nt - nf);
     total += nt;
     fast += nf;
     if (!wide) slow_narrow += nt - nf;
-    sig[l] = t.numel | (wide ? 1ull << 63 : 0ull) | (fast_ok ? 1ull << 62 : 0ull);
+    sig[l] = t.numel | (wide ? 1ull << 63 : 0ull) | (fast_ok ? 1ull << 62 : 0ull) |
+             ((uint64_t)t.bits_m << 56) | ((uint64_t)t.bits_v << 48);   // numel <= 2^40
   }
   if (total > 0xFFFFFFF0ull) return STQ_E_NUMEL;
   // the tile map depends only on sizes and classes: skip it when unchanged
@@ -207,16 +210,34 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   uint8_t* st = static_cast<uint8_t*>(h->h_stage);
   TensorDesc* ht = reinterpret_cast<TensorDesc*>(st);
   uint32_t* hm = reinterpret_cast<uint32_t*>(st + off_map);
-  uint32_t next_fast = 0, next_narrow = (uint32_t)fast, next_wide = (uint32_t)(fast + slow_narrow);
+  // Fast tiles are laid out grouped by width pair: the main kernel runs a body specialised on the
+  // pair, and a change of body costs an instruction-cache refill on every SM, so tensors that share
+  // a pair are made neighbours in the tile order (at most 25 changes per launch).  The order of the
+  // table itself is untouched.
+  std::vector<int> order(L);
+  for (int l = 0; l < L; ++l) order[l] = l;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+    const int ka = tensors[a].bits_v * 64 + tensors[a].bits_m, kb = tensors[b].bits_v * 64 + tensors[b].bits_m;
+    return ka < kb;
+  });
+  std::vector<uint32_t> fast0(L);
+  {
+    uint32_t next_fast = 0;
+    for (int i = 0; i < L; ++i) {
+      const int l = order[i];
+      fast0[l] = next_fast;
+      if (!same_map)
+        for (uint32_t k = 0; k < nfast[l]; ++k) hm[next_fast + k] = (uint32_t)l;
+      next_fast += nfast[l];
+    }
+  }
+  uint32_t next_narrow = (uint32_t)fast, next_wide = (uint32_t)(fast + slow_narrow);
   for (int l = 0; l < L; ++l) {
     const stq_tensor& t = tensors[l];
     TensorDesc d;
     std::memset(&d, 0, sizeof(d));
-    d.tile0 = next_fast;
+    d.tile0 = fast0[l];
     d.nfast = nfast[l];
-    if (!same_map)
-      for (uint32_t i = 0; i < nfast[l]; ++i) hm[next_fast + i] = (uint32_t)l;
-    next_fast += nfast[l];
     uint32_t& next = row_is_wide(t, kind) ? next_wide : next_narrow;
     d.tile0s = next;
     d.nslow = nslow[l];
@@ -257,7 +278,7 @@ int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::St
         cudaStream_t stream) {
   double* partials = nullptr;
   if (stats) {
-    int rc = grow(h, h->d_partials, h->d_partials_cap, (size_t)h->n_tiles * 3);
+    int rc = grow(h, h->d_partials, h->d_partials_cap, (size_t)h->n_tiles * 3 * (stq::kThreads / 32));
     if (rc != STQ_OK) return rc;
     partials = h->d_partials;
   }

@@ -10,7 +10,8 @@ constexpr int kRowElems = 128;   // one row: lane l holds elements 4l .. 4l+3
 constexpr int kRowsPerWarp = 2;  // a warp owns this many consecutive rows of a tile
 constexpr int kTile = (kThreads / 32) * kRowsPerWarp * kRowElems;   // elements per tile; a tile lies inside one tensor
 constexpr int kMaxBlock = kRowsPerWarp * kRowElems;                 // a quantization block never leaves its warp
-constexpr int kFastCtasPerSm = 4;
+constexpr int kFastCtasPerSm = 3;   // resident CTAs per SM of the main step kernel
+constexpr int kFastStages = 3;      // depth of its shared-memory ring
 
 // Device-side row of the tensor table.
 struct TensorDesc {
@@ -47,7 +48,7 @@ struct StepConsts {
 enum Mode { kStep = 0, kRepack = 1, kInit = 2, kStatsOnly = 3 };
 
 // Launches the tile range [tile_begin, tile_end) of the table.  `wide` selects the variant that
-// can read/write 32-bit (raw fp32) states.  partials: 3 doubles per tile or nullptr.
+// can read/write 32-bit (raw fp32) states.  partials: 3 doubles per warp and tile, or nullptr.
 cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const TensorDesc* table,
                          const uint32_t* tile_map, uint32_t tile_begin, uint32_t tile_end,
                          const StepConsts& sc, double* partials, int grid, cudaStream_t stream);

@@ -343,7 +343,6 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
   constexpr bool kHasGrad = (MODE == kStep || MODE == kStatsOnly);
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
-  __shared__ double s_part[kThreads / 32][3];
 
   for (uint32_t tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
     const TensorDesc* __restrict__ T = table + __ldg(tile_map + tile);
@@ -462,8 +461,8 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
                 }
                 float gk = g[k];
                 if (sc.l2_mode) gk = __fadd_rn(gk, __fmul_rn(wd, th[r][k]));
-                const float m = __fadd_rn(__fmul_rn(sc.b1, mh[k]), __fmul_rn(sc.c1, gk));
-                const float v = __fadd_rn(__fmul_rn(sc.b2, vh[k]), __fmul_rn(__fmul_rn(sc.c2, gk), gk));
+                const float m = __fmaf_rn(sc.b1, mh[k], __fmul_rn(sc.c1, gk));
+                const float v = __fmaf_rn(sc.b2, vh[k], __fmul_rn(__fmul_rn(sc.c2, gk), gk));
                 // elements past the end of the tensor stay out of the block maximum
                 mt[r][k] = k < nvl[r] ? m : 0.f;
                 vt[r][k] = k < nvl[r] ? v : 0.f;
@@ -525,7 +524,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
             const float s_raw = __uint_as_float(mxm[r]);
             const bool zero = s_raw < kTiny;
             const float s = zero ? 0.f : s_raw;
-            const float inv = zero ? 0.f : __fdiv_rn(lw.qmaxf, s_raw);
+            const float inv = zero ? 0.f : __fmul_rn(lw.qmaxf, __frcp_rn(s_raw));
             const float mg = kMagic + lw.halff;
             uint32_t x[4];
 #pragma unroll
@@ -598,6 +597,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
     }
 
     if constexpr (STATS || MODE == kStatsOnly) {
+      // one partial per warp and tile; the finishing kernel adds them in a fixed order
       double dg = (double)st_g, da = (double)st_a, dq = (double)st_q;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
@@ -605,15 +605,10 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
         da += __shfl_down_sync(kFull, da, o);
         dq += __shfl_down_sync(kFull, dq, o);
       }
-      if (lane == 0) { s_part[warp][0] = dg; s_part[warp][1] = da; s_part[warp][2] = dq; }
-      __syncthreads();
-      if (threadIdx.x < 3) {
-        double s = 0.0;
-#pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) s += s_part[w][threadIdx.x];
-        partials[(size_t)tile * 3 + threadIdx.x] = s;
+      if (lane == 0) {
+        double* p = partials + ((size_t)tile * (kThreads / 32) + warp) * 3;
+        p[0] = dg; p[1] = da; p[2] = dq;
       }
-      __syncthreads();
     }
   }
 }
@@ -625,11 +620,13 @@ stq_stats_finish_kernel(const TensorDesc* __restrict__ table, int L, const doubl
   const int l = blockIdx.x;
   if (l >= L) return;
   const uint32_t t0 = table[l].tile0, nf = table[l].nfast, t0s = table[l].tile0s, ns = table[l].nslow;
+  constexpr uint32_t W = kThreads / 32;   // partials per tile
   double a[3] = {0.0, 0.0, 0.0};
-  for (uint32_t i = threadIdx.x; i < nf + ns; i += blockDim.x) {
-    const size_t t = i < nf ? (size_t)t0 + i : (size_t)t0s + (i - nf);
+  for (uint32_t i = threadIdx.x; i < (nf + ns) * W; i += blockDim.x) {
+    const uint32_t ti = i / W;
+    const size_t t = ti < nf ? (size_t)t0 + ti : (size_t)t0s + (ti - nf);
 #pragma unroll
-    for (int k = 0; k < 3; ++k) a[k] += partials[t * 3 + k];
+    for (int k = 0; k < 3; ++k) a[k] += partials[(t * W + (i % W)) * 3 + k];
   }
   __shared__ double sh[256][3];
 #pragma unroll

@@ -2,18 +2,20 @@
 // this step (2..16 bits).  Everything else (ragged last tiles, 32-bit states, width changes inside
 // the step, init, repack) goes through the generic kernel in stq_kernels.cu.
 //
-// Data movement: a persistent CTA walks its tiles through a two-stage shared-memory ring.  One
-// elected thread issues, per tile, four bulk asynchronous copies (parameters, gradients, m codes,
-// v codes: each a contiguous, 16-byte aligned range because a tile starts at a multiple of 1024
-// elements) that complete on an mbarrier; the eight warps wait on the barrier, pull their rows into
-// registers with conflict-free 128/64/32-bit shared loads, and release the stage right away, so the
-// copies of the tile after next are in flight while this tile is computed.  Results go straight
-// from registers to global memory with 128-bit (parameters) and 8..64-bit (codes) stores.  Every
-// wait on a barrier is bounded; on expiry the kernel raises an error flag and returns.
+// Data movement: a persistent CTA walks its tiles through a shared-memory ring.  A producer warp
+// (one elected lane) runs ahead: per tile it writes a small descriptor and issues six bulk
+// asynchronous copies (parameters, gradients, m codes, v codes, m scales, v scales: each a contiguous,
+// 16-byte aligned range because a tile starts at a multiple of 2048 elements) that complete on the
+// stage's "full" mbarrier.  The eight consumer warps never synchronise with each other: each waits
+// on "full", pulls its rows into registers with conflict-free 128/64/32-bit shared loads, arrives on
+// the stage's "empty" mbarrier (which lets the producer refill it) and computes.  Results go
+// straight from registers to global memory with 128-bit (parameters) and 8..64-bit (codes) stores.
+// Every wait on a barrier is bounded; on expiry the kernel raises an error flag and returns.
 //
-// Arithmetic: identical to the generic kernel (same roundings, see there), specialised per width
-// so that shifts and masks are immediates, with the per-block constants (one division, one
-// reciprocal or logarithm of the block maximum) computed by one lane per row and broadcast.
+// Arithmetic: identical to the generic kernel (same roundings, see there).  The whole tile body is
+// specialised on the pair of widths (one dispatch per tile), so shifts and masks are immediates;
+// the per-block constants (a reciprocal or a logarithm of the block maximum) are computed by one
+// lane per row and broadcast.
 #include "stq_internal.h"
 
 namespace stq {
@@ -34,13 +36,35 @@ constexpr float kE0 = 0x1.62e42ap-1f, kE1 = 0x1.ebf9bcp-3f, kE2 = 0x1.c6b74cp-5f
                 kE3 = 0x1.3cea84p-7f, kE4 = 0x1.5bbc6ap-10f;
 
 constexpr int R = kRowsPerWarp;
-constexpr int kStages = 2;
+constexpr int kStages = kFastStages;
+constexpr int kConsumerWarps = kThreads / 32;
+constexpr int kFastThreads = kThreads + 32;      // + the producer warp
 constexpr int kOffTheta = 0;
 constexpr int kOffGrad = 4 * kTile;
 constexpr int kOffMc = 8 * kTile;
 constexpr int kOffVc = 10 * kTile;
-constexpr int kStageBytes = 12 * kTile;
-constexpr int kSmemBytes = kStages * kStageBytes + 64;
+constexpr int kOffMs = 12 * kTile;               // block scales of the tile (at most kTile/128 floats)
+constexpr int kOffVs = kOffMs + 64;
+constexpr int kStageBytes = 12 * kTile + 128;
+
+// What the consumers need to know about a staged tile; written by the producer.
+struct __align__(16) TileInfo {
+  float* param;        // all pointers are already advanced to the tile's first element / block
+  uint8_t* mco;
+  uint8_t* vco;
+  float* mso;
+  float* vso;
+  uint32_t wim, wiv;   // width indices (0..4 for 2,3,4,8,16 bits)
+  uint32_t lgB;
+  float wdx;           // fp32(lr*wd) (AdamW) or fp32(wd) (L2 mode)
+  uint32_t pad[2];
+};
+static_assert(sizeof(TileInfo) == 64, "TileInfo is read with four 128-bit loads");
+
+constexpr int kOffInfo = kStages * kStageBytes;
+constexpr int kOffBars = kOffInfo + kStages * 64;        // full[kStages], empty[kStages]
+constexpr int kOffLut = kOffBars + 16 * kStages;         // 256 floats: decode table of the 8-bit log code
+constexpr int kSmemBytes = kOffLut + 1024;
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: far beyond any copy; then give up
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -50,6 +74,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -121,6 +148,7 @@ struct Wd {
   static constexpr int K = (1 << B) - 1;
   static constexpr int Roct = K < 30 ? K : 30;
   static constexpr uint32_t mask = (uint32_t)K;
+  static constexpr uint32_t emin = (uint32_t)(127 - K);   // exponent field of the octave floor level
   // sum_k 2^(k*B) over the elements packed into one 32-bit word
   static constexpr uint32_t fieldsum = B == 2 ? 85u : B == 3 ? 585u : B == 4 ? 4369u : B == 8 ? 0x01010101u : 0x00010001u;
 };
@@ -171,12 +199,16 @@ __device__ __forceinline__ void decode_lin_row(const uint32_t (&w)[2], float s, 
 }
 
 template <int B>
-__device__ __forceinline__ void decode_log_row(const uint32_t (&w)[2], float s, float (&out)[4]) {
-  if constexpr (B <= 4) {
+__device__ __forceinline__ void decode_log_row(const uint32_t (&w)[2], float s, const float* lut8, float (&out)[4]) {
+  if constexpr (B == 8) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) out[k] = __fmul_rn(s, lut8[(w[0] >> (8 * k)) & 255u]);
+  } else if constexpr (B <= 4) {
+    // 2^(code - K): the code drops into the low bits of the exponent field (127 - K has them clear)
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const uint32_t c = (w[0] >> (B * k)) & Wd<B>::mask;
-      out[k] = __fmul_rn(s, __uint_as_float((c + (uint32_t)(127 - Wd<B>::K)) << 23));
+      const uint32_t e = ((w[0] << (23 - B * k)) & (Wd<B>::mask << 23)) | (Wd<B>::emin << 23);
+      out[k] = __fmul_rn(s, __uint_as_float(e));
     }
   } else {
     constexpr float cb = (float)Wd<B>::Roct / (float)Wd<B>::K;
@@ -189,44 +221,43 @@ __device__ __forceinline__ void decode_log_row(const uint32_t (&w)[2], float s, 
   }
 }
 
-// Packs x_k = base + u_k into the lane's field(s) and stores them.  row_ptr: the row's codes in
-// global memory.
+// Stores the lane's packed field(s) of one row.  f: the 4*B-bit field (two words at 16 bits).
 template <int B>
-__device__ __forceinline__ void pack_store_row(uint8_t* row_ptr, int lane, const uint32_t (&x)[4], uint32_t base) {
+__device__ __forceinline__ void store_fields(uint8_t* row_ptr, int lane, uint32_t f0, uint32_t f1) {
   if constexpr (B == 2) {
-    const uint32_t w = x[0] + (x[1] << 2) + (x[2] << 4) + (x[3] << 6) - base * Wd<2>::fieldsum;
-    *(row_ptr + lane) = (uint8_t)w;
+    *(row_ptr + lane) = (uint8_t)f0;
   } else if constexpr (B == 3) {
-    const uint32_t p = (x[0] + (x[1] << 3) + (x[2] << 6) + (x[3] << 9) - base * Wd<3>::fieldsum) & 0xFFFu;
-    const int first = (8 * lane) / 3;
-    uint32_t w = 0u;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int src = first + i;
-      uint32_t v = __shfl_sync(kFull, p, src & 31);
-      const int sh = 12 * src - 32 * lane;
-      if (sh >= 32) v = 0u;
-      else if (sh >= 0) v <<= sh;
-      else v >>= -sh;
-      w |= v;
-    }
-    if (lane < 12) *reinterpret_cast<uint32_t*>(row_ptr + 4 * lane) = w;
+    // a lane pair shares three bytes: even lane owns bits 0..11, odd lane bits 12..23
+    const uint32_t p = f0 & 0xFFFu;
+    const uint32_t other = __shfl_xor_sync(kFull, p, 1);
+    uint8_t* base = row_ptr + 3 * (lane >> 1);
+    const bool odd = lane & 1;
+    *(base + (odd ? 2 : 0)) = (uint8_t)(odd ? (p >> 4) : p);
+    if (!odd) *(base + 1) = (uint8_t)((p >> 8) | (other << 4));
   } else if constexpr (B == 4) {
-    const uint32_t w = x[0] + (x[1] << 4) + (x[2] << 8) + (x[3] << 12) - base * Wd<4>::fieldsum;
-    *reinterpret_cast<uint16_t*>(row_ptr + 2 * lane) = (uint16_t)w;
+    *reinterpret_cast<uint16_t*>(row_ptr + 2 * lane) = (uint16_t)f0;
   } else if constexpr (B == 8) {
-    const uint32_t w = x[0] + (x[1] << 8) + (x[2] << 16) + (x[3] << 24) - base * Wd<8>::fieldsum;
-    *reinterpret_cast<uint32_t*>(row_ptr + 4 * lane) = w;
+    *reinterpret_cast<uint32_t*>(row_ptr + 4 * lane) = f0;
   } else {
-    const uint32_t w0 = x[0] + (x[1] << 16) - base * Wd<16>::fieldsum;
-    const uint32_t w1 = x[2] + (x[3] << 16) - base * Wd<16>::fieldsum;
-    *reinterpret_cast<uint2*>(row_ptr + 8 * lane) = make_uint2(w0, w1);
+    *reinterpret_cast<uint2*>(row_ptr + 8 * lane) = make_uint2(f0, f1);
   }
 }
 
-// Quantize one row of new first moments, store the codes, return the decoded values.
+// Packs x_k = base + u_k (u_k < 2^B) and stores the row's codes.
 template <int B>
-__device__ __forceinline__ void encode_lin_row(uint8_t* row_ptr, int lane, const float (&m)[4], float s, float inv,
+__device__ __forceinline__ void pack_store_row(uint8_t* row_ptr, int lane, const uint32_t (&x)[4], uint32_t base) {
+  if constexpr (B == 16) {
+    store_fields<B>(row_ptr, lane, x[0] + (x[1] << 16) - base * Wd<16>::fieldsum,
+                    x[2] + (x[3] << 16) - base * Wd<16>::fieldsum);
+  } else {
+    store_fields<B>(row_ptr, lane, x[0] + (x[1] << B) + (x[2] << (2 * B)) + (x[3] << (3 * B)) - base * Wd<B>::fieldsum, 0u);
+  }
+}
+
+// Quantize one row of new first moments, store the codes, return the decoded values times `gain`
+// (s_dec = stored scale * gain).
+template <int B>
+__device__ __forceinline__ void encode_lin_row(uint8_t* row_ptr, int lane, const float (&m)[4], float s_dec, float inv,
                                                float (&mq)[4]) {
   constexpr float invq = 1.0f / (float)Wd<B>::qmax;
   constexpr float mg = kMagic + (float)Wd<B>::half;
@@ -235,46 +266,42 @@ __device__ __forceinline__ void encode_lin_row(uint8_t* row_ptr, int lane, const
   for (int k = 0; k < 4; ++k) {
     const float t = __fmaf_rn(m[k], inv, mg);
     x[k] = __float_as_uint(t);
-    mq[k] = __fmul_rn(s, __fmul_rn(__fadd_rn(t, -mg), invq));
+    mq[k] = __fmul_rn(s_dec, __fmul_rn(__fadd_rn(t, -mg), invq));
   }
   pack_store_row<B>(row_ptr, lane, x, kMagicBits);
 }
 
-// Per-block constants of the log quantizer: octave widths need c = sqrt2/s, the others E_s and P(s).
-struct LogBlock {
-  float s;      // stored scale (0 for a zero block)
-  float c;      // octave widths: fl(fl(1/s)*sqrt2), 0 for a zero block
-  float Ps;     // 8/16 bit: P(s)
-  uint32_t ebase;   // 8/16 bit: kMagicBits - E_s
-};
-
+// Quantize one row of new second moments.  lgc: sqrt2/s (octave widths) or P(s) (8, 16 bits);
+// ebase: kMagicBits - E_s (8, 16 bits).
 template <int B>
-__device__ __forceinline__ void encode_log_row(uint8_t* row_ptr, int lane, const float (&v)[4], const LogBlock& lb,
-                                               float (&vq)[4]) {
-  uint32_t x[4];
+__device__ __forceinline__ void encode_log_row(uint8_t* row_ptr, int lane, const float (&v)[4], float s, float lgc,
+                                               uint32_t ebase, const float* lut8, float (&vq)[4]) {
   if constexpr (B <= 4) {
-    constexpr uint32_t emin = (uint32_t)(127 - Wd<B>::K);
-    const float ymin = __uint_as_float(emin << 23);
+    const float ymin = __uint_as_float(Wd<B>::emin << 23);
+    uint32_t f = 0u;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const uint32_t yb = __float_as_uint(fmaxf(__fmul_rn(v[k], lb.c), ymin));
-      x[k] = yb >> 23;
-      vq[k] = __fmul_rn(lb.s, __uint_as_float(yb & 0x7F800000u));
+      // exponent of x*sqrt2/s, floored at -K: its low B bits are the code
+      const uint32_t yb = __float_as_uint(fmaxf(__fmul_rn(v[k], lgc), ymin));
+      f |= (yb >> (23 - B * k)) & (Wd<B>::mask << (B * k));
+      vq[k] = __fmul_rn(s, __uint_as_float(yb & 0x7F800000u));
     }
-    pack_store_row<B>(row_ptr, lane, x, emin);
+    store_fields<B>(row_ptr, lane, f, 0u);
   } else {
     constexpr float a = (float)Wd<B>::K / (float)Wd<B>::Roct;
     constexpr float cb = (float)Wd<B>::Roct / (float)Wd<B>::K;
     constexpr float negR = -(float)Wd<B>::Roct;
+    uint32_t x[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const uint32_t xb = __float_as_uint(v[k]);
-      const float de = __fadd_rn(__uint_as_float(lb.ebase + (xb >> 23)), -kMagic);
-      const float dp = __fadd_rn(lg_poly(xb), -lb.Ps);
+      const float de = __fadd_rn(__uint_as_float(ebase + (xb >> 23)), -kMagic);
+      const float dp = __fadd_rn(lg_poly(xb), -lgc);
       const float d = fmaxf(__fadd_rn(de, dp), negR);
       const float t = __fmaf_rn(d, a, kMagic);
       x[k] = __float_as_uint(t);
-      vq[k] = __fmul_rn(lb.s, ex2_poly(__fmul_rn(__fadd_rn(t, -kMagic), cb)));
+      if constexpr (B == 8) vq[k] = __fmul_rn(s, lut8[(x[k] + 255u) & 255u]);   // low bits are code - 255
+      else vq[k] = __fmul_rn(s, ex2_poly(__fmul_rn(__fadd_rn(t, -kMagic), cb)));
     }
     pack_store_row<B>(row_ptr, lane, x, kMagicBits - (uint32_t)Wd<B>::K);
   }
@@ -294,23 +321,173 @@ __device__ __forceinline__ void lds_grad(const uint8_t* stage, int elem, float (
   }
 }
 
-#define STQ_WIDTH_SWITCH(bits, CALL)           \
-  switch (bits) {                              \
-    case 2: { CALL(2); } break;                \
-    case 3: { CALL(3); } break;                \
-    case 4: { CALL(4); } break;                \
-    case 8: { CALL(8); } break;                \
-    default: { CALL(16); } break;              \
+// One staged tile, one warp: R rows of 128 elements.  Specialised on both widths.
+template <int BM, int BV, int GDT>
+__device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, const TileInfo& ti, const StepConsts& sc,
+                                          const float* __restrict__ lut8, int lane, int warp, uint32_t empty_bar,
+                                          double* __restrict__ part) {
+  const int lgB = (int)ti.lgB;
+  const int row0 = warp * R;
+
+  // ---- staged tile -> registers, decode ---------------------------------------------------------------
+  float th[R][4], g[R][4], mt[R][4], vt[R][4];
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const int elem = (row0 + r) * kRowElems + 4 * lane;
+    const float4 t4 = *reinterpret_cast<const float4*>(stage + kOffTheta + 4 * elem);
+    th[r][0] = t4.x; th[r][1] = t4.y; th[r][2] = t4.z; th[r][3] = t4.w;
+    lds_grad<GDT>(stage, elem, g[r]);
+    const int blk = ((row0 + r) * kRowElems) >> lgB;
+    const float sm = *reinterpret_cast<const float*>(stage + kOffMs + 4 * blk);
+    const float sv = *reinterpret_cast<const float*>(stage + kOffVs + 4 * blk);
+    uint32_t w[2];
+    lds_codes<BM>(stage + kOffMc + (row0 + r) * (16 * BM), lane, w);
+    decode_lin_row<BM>(w, sm, mt[r]);
+    lds_codes<BV>(stage + kOffVc + (row0 + r) * (16 * BV), lane, w);
+    decode_log_row<BV>(w, sv, lut8, vt[r]);
+  }
+  // this warp is done with the stage
+  __syncwarp();
+  if (lane == 0) mbar_arrive(empty_bar);
+
+  // ---- statistics over the raw gradient (decision steps) -------------------------------------------------
+  if (part != nullptr) {
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f;
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        a0 += g[r][k];
+        a1 += fabsf(g[r][k]);
+        a2 = __fmaf_rn(g[r][k], g[r][k], a2);
+      }
+    // Pairwise fp32 butterfly that spreads the three sums over the lanes on the way down:
+    // after xor 16 the low half carries (sum0, sum1) and the high half (sum2, -); after xor 8
+    // lanes 0-7 / 8-15 / 16-23 carry sum0 / sum1 / sum2; three more steps finish each group.
+    const bool hi = lane & 16;
+    float x = (hi ? a2 : a0) + __shfl_xor_sync(kFull, hi ? a0 : a2, 16);
+    float y = (hi ? 0.f : a1) + __shfl_xor_sync(kFull, hi ? a1 : 0.f, 16);
+    const bool q = lane & 8;
+    float z = (q ? y : x) + __shfl_xor_sync(kFull, q ? x : y, 8);
+    z += __shfl_xor_sync(kFull, z, 4);
+    z += __shfl_xor_sync(kFull, z, 2);
+    z += __shfl_xor_sync(kFull, z, 1);
+    if ((lane & 7) == 0 && lane < 24) part[lane >> 3] = (double)z;
   }
 
-template <int GDT, bool STATS>
-__global__ void __launch_bounds__(kThreads, kFastCtasPerSm)
+  // ---- moments ------------------------------------------------------------------------------------------
+  if (sc.l2_mode) {
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) g[r][k] = __fadd_rn(g[r][k], __fmul_rn(ti.wdx, th[r][k]));
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float gk = g[r][k];
+      mt[r][k] = __fmaf_rn(sc.b1, mt[r][k], __fmul_rn(sc.c1, gk));
+      vt[r][k] = __fmaf_rn(sc.b2, vt[r][k], __fmul_rn(__fmul_rn(sc.c2, gk), gk));
+    }
+  }
+
+  // ---- block maxima ----------------------------------------------------------------------------------
+  uint32_t mxm[R], mxv[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const float am = fmaxf(fmaxf(fabsf(mt[r][0]), fabsf(mt[r][1])), fmaxf(fabsf(mt[r][2]), fabsf(mt[r][3])));
+    const float av = fmaxf(fmaxf(vt[r][0], vt[r][1]), fmaxf(vt[r][2], vt[r][3]));
+    mxm[r] = __reduce_max_sync(kFull, __float_as_uint(am));
+    mxv[r] = __reduce_max_sync(kFull, __float_as_uint(av));
+  }
+  if (lgB >= 8) {
+#pragma unroll
+    for (int r = 0; r < R; r += 2) {
+      mxm[r] = mxm[r + 1] = max(mxm[r], mxm[r + 1]);
+      mxv[r] = mxv[r + 1] = max(mxv[r], mxv[r + 1]);
+    }
+  }
+  if (R >= 4 && lgB >= 9) {
+    const uint32_t a = max(mxm[0], mxm[R - 2]), b = max(mxv[0], mxv[R - 2]);
+#pragma unroll
+    for (int r = 0; r < R; ++r) { mxm[r] = a; mxv[r] = b; }
+  }
+
+  // ---- per-block constants: one lane per (row, state) works them out, then they are broadcast ----------
+  // lanes 0..R-1: inv = fl(qmax * fl(1/s_m));  lanes R..2R-1 (octave widths): c = fl(sqrt2 * fl(1/s_v))
+  float inv_m[R], lgc[R];
+  {
+    uint32_t mine = mxm[0];
+#pragma unroll
+    for (int r = 1; r < R; ++r)
+      if ((lane & (R - 1)) == r) mine = mxm[r];
+    if constexpr (BV <= 4) {
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+        if ((lane & (2 * R - 1)) == R + r) mine = mxv[r];
+    }
+    const float x = __uint_as_float(mine);
+    const float mul = (BV <= 4 && (lane & R)) ? kSqrt2 : (float)Wd<BM>::qmax;
+    const float val = x < kTiny ? 0.f : __fmul_rn(mul, __frcp_rn(x));
+#pragma unroll
+    for (int r = 0; r < R; ++r) inv_m[r] = __shfl_sync(kFull, val, r);
+    if constexpr (BV <= 4) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) lgc[r] = __shfl_sync(kFull, val, R + r);
+    } else {
+      uint32_t mv = mxv[0];
+#pragma unroll
+      for (int r = 1; r < R; ++r)
+        if ((lane & (R - 1)) == r) mv = mxv[r];
+      const float ps = lg_poly(mv);
+#pragma unroll
+      for (int r = 0; r < R; ++r) lgc[r] = __shfl_sync(kFull, ps, r);
+    }
+  }
+
+  // ---- quantize, pack, store; decode the new codes; update the parameters ----------------------------
+  const float lrwd = sc.l2_mode ? 0.0f : ti.wdx;
+  float* param = ti.param + row0 * kRowElems + 4 * lane;
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const float sm_raw = __uint_as_float(mxm[r]);
+    const float s_m = sm_raw < kTiny ? 0.f : sm_raw;
+    const float sv_raw = __uint_as_float(mxv[r]);
+    const bool vzero = sv_raw < kTiny;
+    const float s_v = vzero ? 0.f : sv_raw;
+    const uint32_t ebase = kMagicBits - (vzero ? (uint32_t)kZeroBlockExp : (mxv[r] >> 23));
+    float mq[4], vq[4];
+    // mq comes out multiplied by lr/(1-beta1^t): the decode scale carries the factor
+    encode_lin_row<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], __fmul_rn(s_m, sc.step_size), inv_m[r], mq);
+    encode_log_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], s_v, lgc[r], ebase, lut8, vq);
+    const int e_row = (row0 + r) * kRowElems;
+    if (lane == 0 && (e_row & ((1 << lgB) - 1)) == 0) {
+      ti.mso[e_row >> lgB] = s_m;
+      ti.vso[e_row >> lgB] = s_v;
+    }
+    float out[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float den = __fmaf_rn(sqrt_fast(vq[k]), sc.rsqrt_bc2, sc.eps);
+      const float upd = __fmul_rn(mq[k], rcp_fast(den));
+      out[k] = __fadd_rn(th[r][k], -__fmaf_rn(th[r][k], lrwd, upd));
+    }
+    *reinterpret_cast<float4*>(param + r * kRowElems) = make_float4(out[0], out[1], out[2], out[3]);
+  }
+}
+
+__device__ __forceinline__ uint32_t width_index(uint32_t b) { return b == 2 ? 0u : b == 3 ? 1u : b == 4 ? 2u : b == 8 ? 3u : 4u; }
+
+template <int GDT>
+__global__ void __launch_bounds__(kFastThreads, kFastCtasPerSm)
 stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map, uint32_t n_fast,
                      const StepConsts sc, double* __restrict__ partials, int* __restrict__ err_flag) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ double s_part[kThreads / 32][3];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t bar0 = smem_u32(smem + kStages * kStageBytes);
+  const uint32_t full0 = smem_u32(smem + kOffBars);
+  const uint32_t empty0 = full0 + 8 * kStages;
+  float* lut8 = reinterpret_cast<float*>(smem + kOffLut);
   const uint32_t first = blockIdx.x, stride = gridDim.x;
   if (first >= n_fast) return;
   const uint32_t n_my = (n_fast - first + stride - 1) / stride;
@@ -318,244 +495,113 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
 
   if (tid == 0) {
 #pragma unroll
-    for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, kConsumerWarps);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if (tid < 256) {   // decode table of the 8-bit log code: ex((q - 255) * fl(30/255))
+    constexpr float cb = (float)Wd<8>::Roct / (float)Wd<8>::K;
+    lut8[tid] = ex2_poly(__fmul_rn((float)(tid - 255), cb));
+  }
   __syncthreads();
 
-  // thread 0: start the copies of one tile into stage s
-  auto issue = [&](uint32_t it, int s) {
-    const uint32_t tile = first + it * stride;
-    const TensorDesc* T = table + __ldg(tile_map + tile);
-    const unsigned long long e0 = (unsigned long long)(tile - T->tile0) * kTile;
-    const uint32_t bm = T->bm_in, bv = T->bv_in;
-    const uint32_t nb_m = (kTile / 8) * bm, nb_v = (kTile / 8) * bv;
-    const uint32_t bar = bar0 + 8 * s;
-    const uint32_t dst = smem_u32(smem + s * kStageBytes);
-    mbar_expect_tx(bar, kTile * 4 + kTile * gsz + nb_m + nb_v);
-    bulk_g2s(dst + kOffTheta, T->param + e0, kTile * 4, bar);
-    bulk_g2s(dst + kOffGrad, reinterpret_cast<const uint8_t*>(T->grad) + e0 * gsz, kTile * gsz, bar);
-    bulk_g2s(dst + kOffMc, T->mc_in + (e0 >> 3) * bm, nb_m, bar);
-    bulk_g2s(dst + kOffVc, T->vc_in + (e0 >> 3) * bv, nb_v, bar);
-  };
-  if (tid == 0) {
-#pragma unroll
-    for (int s = 0; s < kStages; ++s)
-      if ((uint32_t)s < n_my) issue(s, s);
+  if (warp == kConsumerWarps) {
+    // ================================ producer ========================================================
+    if (lane != 0) return;
+    uint32_t it = 0;
+    int s = 0;
+    uint32_t phase = 0;       // parity of the use of stage s that is being filled
+    bool ok = true;
+    for (; it < n_my; ++it) {
+      if (it >= (uint32_t)kStages && !mbar_wait(empty0 + 8 * s, phase ^ 1u)) { ok = false; break; }
+      const uint32_t tile = first + it * stride;
+      const TensorDesc* T = table + __ldg(tile_map + tile);
+      const unsigned long long e0 = (unsigned long long)(tile - T->tile0) * kTile;
+      const uint32_t bm = T->bm_in, bv = T->bv_in;
+      const uint32_t lgB = 7u + (T->block >> 8);
+      const uint32_t nb_m = (kTile / 8) * bm, nb_v = (kTile / 8) * bv, nb_s = (uint32_t)(kTile * 4) >> lgB;
+      TileInfo ti;
+      ti.param = T->param + e0;
+      ti.mco = T->mc_out + (e0 >> 3) * bm;
+      ti.vco = T->vc_out + (e0 >> 3) * bv;
+      ti.mso = T->ms_out + (e0 >> lgB);
+      ti.vso = T->vs_out + (e0 >> lgB);
+      ti.wim = width_index(bm);
+      ti.wiv = width_index(bv);
+      ti.lgB = lgB;
+      ti.wdx = sc.l2_mode ? T->wd : (float)(sc.lr * (double)T->wd);
+      ti.pad[0] = ti.pad[1] = 0u;
+      *reinterpret_cast<TileInfo*>(smem + kOffInfo + 64 * s) = ti;
+      const uint32_t bar = full0 + 8 * s;
+      const uint32_t dst = smem_u32(smem + s * kStageBytes);
+      mbar_expect_tx(bar, kTile * 4 + kTile * gsz + nb_m + nb_v + 2 * nb_s);
+      bulk_g2s(dst + kOffTheta, T->param + e0, kTile * 4, bar);
+      bulk_g2s(dst + kOffGrad, reinterpret_cast<const uint8_t*>(T->grad) + e0 * gsz, kTile * gsz, bar);
+      bulk_g2s(dst + kOffMc, T->mc_in + (e0 >> 3) * bm, nb_m, bar);
+      bulk_g2s(dst + kOffVc, T->vc_in + (e0 >> 3) * bv, nb_v, bar);
+      bulk_g2s(dst + kOffMs, T->ms_in + (e0 >> lgB), nb_s, bar);
+      bulk_g2s(dst + kOffVs, T->vs_in + (e0 >> lgB), nb_s, bar);
+      if (++s == kStages) { s = 0; phase ^= 1u; }
+    }
+    // Before this CTA's shared memory is given up, every copy issued must have landed: wait until
+    // the consumers have drained the last stages (normal path), or, after a time-out, give the
+    // outstanding copies one more bounded wait.
+    const uint32_t issued = it;
+    const uint32_t from = issued > (uint32_t)kStages ? issued - kStages : 0u;
+    for (uint32_t j = from; j < issued; ++j) {
+      const int sj = j % kStages;
+      const uint32_t pj = (j / kStages) & 1u;
+      if (ok) ok = mbar_wait(empty0 + 8 * sj, pj);
+      else mbar_wait(full0 + 8 * sj, pj);
+    }
+    if (!ok) atomicExch(err_flag, 1);
+    return;
   }
 
-  uint32_t failed_at = 0xFFFFFFFFu;
+  // ================================== consumers =========================================================
+  int s = 0;
+  uint32_t phase = 0;
   for (uint32_t it = 0; it < n_my; ++it) {
-    const int s = it % kStages;
-    const uint32_t parity = (it / kStages) & 1u;
-    const uint32_t tile = first + it * stride;
-    const TensorDesc* __restrict__ T = table + __ldg(tile_map + tile);
-    const uint32_t e_warp = (tile - T->tile0) * (uint32_t)kTile + (uint32_t)warp * (R * kRowElems);   // fits: checked on the host
-    const int bm = T->bm_in, bv = T->bv_in;
-    const int lgB = 7 + (int)(T->block >> 8);
-    const float* ms_in = T->ms_in;
-    const float* vs_in = T->vs_in;
-    float s_m_in[R], s_v_in[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const uint32_t blk = (e_warp + r * kRowElems) >> lgB;
-      s_m_in[r] = __ldg(ms_in + blk);
-      s_v_in[r] = __ldg(vs_in + blk);
-    }
-
-    // a thread whose wait ran out still reaches the barrier below, so the CTA gives up as one
-    const bool landed = mbar_wait(bar0 + 8 * s, parity);
-
-    // ---- staged tile -> registers ---------------------------------------------------------------------
-    const uint8_t* stage = smem + s * kStageBytes;
-    float th[R][4], g[R][4];
-    uint32_t wm[R][2], wv[R][2];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const int row = warp * R + r;
-      const int elem = row * kRowElems + 4 * lane;
-      const float4 t4 = *reinterpret_cast<const float4*>(stage + kOffTheta + 4 * elem);
-      th[r][0] = t4.x; th[r][1] = t4.y; th[r][2] = t4.z; th[r][3] = t4.w;
-      lds_grad<GDT>(stage, elem, g[r]);
-    }
-#define STQ_LDS_M(BW)                                                                   \
-  _Pragma("unroll") for (int r = 0; r < R; ++r)                                         \
-      lds_codes<BW>(stage + kOffMc + (warp * R + r) * (16 * BW), lane, wm[r]);
-#define STQ_LDS_V(BW)                                                                   \
-  _Pragma("unroll") for (int r = 0; r < R; ++r)                                         \
-      lds_codes<BW>(stage + kOffVc + (warp * R + r) * (16 * BW), lane, wv[r]);
-    STQ_WIDTH_SWITCH(bm, STQ_LDS_M)
-    STQ_WIDTH_SWITCH(bv, STQ_LDS_V)
-
-    // the stage is free again: everyone has its data in registers
-    if (__syncthreads_or(!landed)) {
-      failed_at = it;
+    if (!mbar_wait(full0 + 8 * s, phase)) {
+      if (lane == 0) atomicExch(err_flag, 1);
       break;
     }
-    if (tid == 0 && it + kStages < n_my) issue(it + kStages, s);
+    const uint8_t* stage = smem + s * kStageBytes;
+    const TileInfo ti = *reinterpret_cast<const TileInfo*>(smem + kOffInfo + 64 * s);
+    const uint32_t ebar = empty0 + 8 * s;
+    double* part = partials ? partials + ((size_t)(first + it * stride) * kConsumerWarps + warp) * 3 : nullptr;
 
-    // ---- decode, moments -------------------------------------------------------------------------------
-    float mt[R][4], vt[R][4];
-#define STQ_DEC_M(BW) \
-  _Pragma("unroll") for (int r = 0; r < R; ++r) decode_lin_row<BW>(wm[r], s_m_in[r], mt[r]);
-#define STQ_DEC_V(BW) \
-  _Pragma("unroll") for (int r = 0; r < R; ++r) decode_log_row<BW>(wv[r], s_v_in[r], vt[r]);
-    STQ_WIDTH_SWITCH(bm, STQ_DEC_M)
-    STQ_WIDTH_SWITCH(bv, STQ_DEC_V)
-
-    float st_g = 0.f, st_a = 0.f, st_q = 0.f;
-    const float wd = T->wd;
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        float gk = g[r][k];
-        if constexpr (STATS) {
-          st_g += gk;
-          st_a += fabsf(gk);
-          st_q = __fmaf_rn(gk, gk, st_q);
-        }
-        if (sc.l2_mode) gk = __fadd_rn(gk, __fmul_rn(wd, th[r][k]));
-        mt[r][k] = __fadd_rn(__fmul_rn(sc.b1, mt[r][k]), __fmul_rn(sc.c1, gk));
-        vt[r][k] = __fadd_rn(__fmul_rn(sc.b2, vt[r][k]), __fmul_rn(__fmul_rn(sc.c2, gk), gk));
-      }
+#define STQ_CASE(IM, IV, BM, BV) \
+  case IM * 5 + IV: tile_body<BM, BV, GDT>(stage, ti, sc, lut8, lane, warp, ebar, part); break;
+#define STQ_CASES_M(IM, BM) \
+  STQ_CASE(IM, 0, BM, 2) STQ_CASE(IM, 1, BM, 3) STQ_CASE(IM, 2, BM, 4) STQ_CASE(IM, 3, BM, 8) STQ_CASE(IM, 4, BM, 16)
+    switch (ti.wim * 5 + ti.wiv) {
+      STQ_CASES_M(0, 2)
+      STQ_CASES_M(1, 3)
+      STQ_CASES_M(2, 4)
+      STQ_CASES_M(3, 8)
+      STQ_CASES_M(4, 16)
+      default: break;
     }
-
-    // ---- block maxima ----------------------------------------------------------------------------------
-    uint32_t mxm[R], mxv[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const float am = fmaxf(fmaxf(fabsf(mt[r][0]), fabsf(mt[r][1])), fmaxf(fabsf(mt[r][2]), fabsf(mt[r][3])));
-      const float av = fmaxf(fmaxf(vt[r][0], vt[r][1]), fmaxf(vt[r][2], vt[r][3]));
-      mxm[r] = __reduce_max_sync(kFull, __float_as_uint(am));
-      mxv[r] = __reduce_max_sync(kFull, __float_as_uint(av));
-    }
-    if (lgB >= 8) {
-#pragma unroll
-      for (int r = 0; r < R; r += 2) {
-        mxm[r] = mxm[r + 1] = max(mxm[r], mxm[r + 1]);
-        mxv[r] = mxv[r + 1] = max(mxv[r], mxv[r + 1]);
-      }
-    }
-    if (R >= 4 && lgB >= 9) {
-      const uint32_t a = max(mxm[0], mxm[R - 2]), b = max(mxv[0], mxv[R - 2]);
-#pragma unroll
-      for (int r = 0; r < R; ++r) { mxm[r] = a; mxv[r] = b; }
-    }
-
-    // ---- per-block constants: lane r works out row r's, then they are broadcast ------------------------
-    uint32_t my_m = mxm[0], my_v = mxv[0];
-#pragma unroll
-    for (int r = 1; r < R; ++r) {
-      if ((lane & (R - 1)) == r) { my_m = mxm[r]; my_v = mxv[r]; }
-    }
-    float my_inv, my_lg;   // my_lg: sqrt2/s for the octave widths, P(s) for 8 and 16 bits
-    {
-      const float sm = __uint_as_float(my_m);
-      const float qmaxf = (float)((1 << (bm - 1)) - 1);
-      my_inv = sm < kTiny ? 0.f : __fdiv_rn(qmaxf, sm);
-      const float sv = __uint_as_float(my_v);
-      if (bv <= 4) my_lg = sv < kTiny ? 0.f : __fmul_rn(__frcp_rn(sv), kSqrt2);
-      else my_lg = lg_poly(my_v);
-    }
-    float s_m[R], inv_m[R];
-    LogBlock lb[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const float sm = __uint_as_float(mxm[r]);
-      s_m[r] = sm < kTiny ? 0.f : sm;
-      inv_m[r] = __shfl_sync(kFull, my_inv, r);
-      const float sv = __uint_as_float(mxv[r]);
-      const bool zero = sv < kTiny;
-      lb[r].s = zero ? 0.f : sv;
-      lb[r].c = lb[r].Ps = __shfl_sync(kFull, my_lg, r);
-      lb[r].ebase = kMagicBits - (uint32_t)(zero ? kZeroBlockExp : (int)(mxv[r] >> 23));
-    }
-
-    // ---- quantize, pack, store; decode the new codes ---------------------------------------------------
-    uint8_t* mco = T->mc_out;
-    uint8_t* vco = T->vc_out;
-    float mq[R][4], vq[R][4];
-#define STQ_ENC_M(BW)                                                                                   \
-  _Pragma("unroll") for (int r = 0; r < R; ++r)                                                         \
-      encode_lin_row<BW>(mco + (size_t)((e_warp + r * kRowElems) >> 3) * BW, lane, mt[r], s_m[r], inv_m[r], mq[r]);
-#define STQ_ENC_V(BW)                                                                                   \
-  _Pragma("unroll") for (int r = 0; r < R; ++r)                                                         \
-      encode_log_row<BW>(vco + (size_t)((e_warp + r * kRowElems) >> 3) * BW, lane, vt[r], lb[r], vq[r]);
-    STQ_WIDTH_SWITCH(bm, STQ_ENC_M)
-    STQ_WIDTH_SWITCH(bv, STQ_ENC_V)
-    if (lane == 0) {
-      float* mso = T->ms_out;
-      float* vso = T->vs_out;
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-        const uint32_t e_row = e_warp + r * kRowElems;
-        if ((e_row & ((1u << lgB) - 1u)) == 0) {
-          mso[e_row >> lgB] = s_m[r];
-          vso[e_row >> lgB] = lb[r].s;
-        }
-      }
-    }
-
-    // ---- parameter update ------------------------------------------------------------------------------
-    const float lrwd = sc.l2_mode ? 0.0f : (float)(sc.lr * (double)wd);
-    float* param = T->param + e_warp + 4 * lane;
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      float out[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const float den = __fmaf_rn(sqrt_fast(vq[r][k]), sc.rsqrt_bc2, sc.eps);
-        const float upd = __fmul_rn(__fmul_rn(mq[r][k], sc.step_size), rcp_fast(den));
-        out[k] = __fadd_rn(th[r][k], -__fmaf_rn(th[r][k], lrwd, upd));
-      }
-      *reinterpret_cast<float4*>(param + r * kRowElems) = make_float4(out[0], out[1], out[2], out[3]);
-    }
-
-    if constexpr (STATS) {
-      double dg = (double)st_g, da = (double)st_a, dq = (double)st_q;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        dg += __shfl_down_sync(kFull, dg, o);
-        da += __shfl_down_sync(kFull, da, o);
-        dq += __shfl_down_sync(kFull, dq, o);
-      }
-      if (lane == 0) { s_part[warp][0] = dg; s_part[warp][1] = da; s_part[warp][2] = dq; }
-      __syncthreads();
-      if (tid < 3) {
-        double a = 0.0;
-#pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) a += s_part[w][tid];
-        partials[(size_t)tile * 3 + tid] = a;
-      }
-    }
-  }
-
-  // A CTA that gave up raises the flag and waits (bounded again) for the copies it still has in
-  // flight, so none lands in shared memory that no longer belongs to it.
-  if (failed_at != 0xFFFFFFFFu) {
-    if (tid == 0) {
-      atomicExch(err_flag, 1);
-      for (uint32_t j = failed_at; j < n_my && j < failed_at + kStages; ++j)
-        mbar_wait(bar0 + 8 * (j % kStages), (j / kStages) & 1u);
-    }
-    __syncthreads();
+    if (++s == kStages) { s = 0; phase ^= 1u; }
   }
 }
 
-template <int GDT, bool STATS>
+template <int GDT>
 cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, uint32_t n_fast, const StepConsts& sc,
                           double* partials, int* err_flag, int grid, cudaStream_t stream) {
   static bool attr_set = false;
-  auto kern = stq_step_fast_kernel<GDT, STATS>;
+  auto kern = stq_step_fast_kernel<GDT>;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   const int g = (int)(n_fast < (uint32_t)grid ? n_fast : (uint32_t)grid);
-  kern<<<g, kThreads, kSmemBytes, stream>>>(table, tile_map, n_fast, sc, partials, err_flag);
+  kern<<<g, kFastThreads, kSmemBytes, stream>>>(table, tile_map, n_fast, sc, partials, err_flag);
   return cudaGetLastError();
 }
 
@@ -565,18 +611,16 @@ cudaError_t launch_step_fast(int grad_dtype, bool stats, const TensorDesc* table
                              uint32_t n_fast, const StepConsts& sc, double* partials, int* err_flag, int grid,
                              cudaStream_t stream) {
   if (n_fast == 0) return cudaSuccess;
-  if (grad_dtype == 0)
-    return stats ? launch_fast_t<0, true>(table, tile_map, n_fast, sc, partials, err_flag, grid, stream)
-                 : launch_fast_t<0, false>(table, tile_map, n_fast, sc, partials, err_flag, grid, stream);
-  return stats ? launch_fast_t<1, true>(table, tile_map, n_fast, sc, partials, err_flag, grid, stream)
-               : launch_fast_t<1, false>(table, tile_map, n_fast, sc, partials, err_flag, grid, stream);
+  double* p = stats ? partials : nullptr;
+  return grad_dtype == 0 ? launch_fast_t<0>(table, tile_map, n_fast, sc, p, err_flag, grid, stream)
+                         : launch_fast_t<1>(table, tile_map, n_fast, sc, p, err_flag, grid, stream);
 }
 
 int fast_ctas_per_sm() {
   int n = 0;
-  auto kern = stq_step_fast_kernel<1, false>;
+  auto kern = stq_step_fast_kernel<1>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return 1;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kThreads, kSmemBytes) != cudaSuccess) return 1;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kFastThreads, kSmemBytes) != cudaSuccess) return 1;
   return n > 0 ? n : 1;
 }
 

@@ -67,22 +67,45 @@ def test_32bit_state_l2_mode_matches_torch_adam(O):
     assert np.abs(th - ref).max() <= 2e-6 * np.abs(ref).max()
 
 
+def _fma32(a, b, c):
+    """Correctly rounded fp32 fma of python floats holding fp32 values, by exact rational arithmetic."""
+    from fractions import Fraction
+    x = Fraction(a) * Fraction(b) + Fraction(c)
+    if x == 0:
+        return np.float32(0.0)
+    sign = -1 if x < 0 else 1
+    x = abs(x)
+    e = x.numerator.bit_length() - x.denominator.bit_length()      # 2^(e-1) < x < 2^(e+1)
+    if Fraction(2) ** e > x:
+        e -= 1
+    e = max(e, -126)                                               # subnormal results share the smallest exponent
+    scaled = x / Fraction(2) ** (e - 23)                           # significand with 24 bits before the point
+    q, r = divmod(scaled.numerator, scaled.denominator)
+    twice = 2 * r
+    if twice > scaled.denominator or (twice == scaled.denominator and q % 2 == 1):
+        q += 1
+    return np.float32(sign * float(Fraction(q) * Fraction(2) ** (e - 23)))
+
+
 def test_32bit_moments_are_the_fp32_recursion_bit_for_bit(O):
-    """m_t = fl(fl(b1*m) + fl(c1*g)), v_t = fl(fl(b2*v) + fl(fl(c2*g)*g)) in fp32, with
-    b = fp32(beta) and c = fp32(1 - beta) (the subtraction taken in double)."""
+    """m_t = fma(b1, m, fl(c1*g)), v_t = fma(b2, v, fl(fl(c2*g)*g)) in fp32, with b = fp32(beta) and
+    c = fp32(1 - beta) (the subtraction taken in double)."""
     rng = np.random.default_rng(2)
-    n = 300
+    n = 200
     th = rng.normal(0, 0.02, n).astype(np.float32)
     st = O.new_state(n, 128, 32, 32)
     m = np.zeros(n, np.float32)
     v = np.zeros(n, np.float32)
     b1, b2 = np.float32(0.9), np.float32(0.999)
-    for t in range(1, 6):
+    c1, c2 = np.float32(1 - 0.9), np.float32(1 - 0.999)
+    for t in range(1, 5):
         g = rng.normal(0, 1e-3, n).astype(np.float32)
         st, _ = O.step(th, g, st, 128, t=t, **HP)
-        m = b1 * m + np.float32(1 - 0.9) * g
-        v = b2 * v + (np.float32(1 - 0.999) * g) * g
-        assert m.dtype == np.float32 and v.dtype == np.float32
+        new_m = c1 * g
+        new_v = (c2 * g) * g
+        assert new_m.dtype == np.float32 and new_v.dtype == np.float32
+        m = np.array([_fma32(float(b1), float(a), float(c)) for a, c in zip(m, new_m)], np.float32)
+        v = np.array([_fma32(float(b2), float(a), float(c)) for a, c in zip(v, new_v)], np.float32)
         assert (st.m_codes.view(np.float32)[:n] == m).all()
         assert (st.v_codes.view(np.float32)[:n] == v).all()
 
@@ -151,8 +174,9 @@ def test_width_change_inside_a_step_equals_step_at_new_width(O):
     mh = O.dequantize(st.m_codes, st.m_scales, n, 8, 128, O.LINEAR)
     vh = O.dequantize(st.v_codes, st.v_scales, n, 4, 128, O.LOG)
     b1, b2 = np.float32(0.9), np.float32(0.999)
-    m = b1 * mh + np.float32(1 - 0.9) * g2
-    v = b2 * vh + (np.float32(1 - 0.999) * g2) * g2
+    m = np.array([_fma32(float(b1), float(a), float(c)) for a, c in zip(mh, np.float32(1 - 0.9) * g2)], np.float32)
+    v = np.array([_fma32(float(b2), float(a), float(c))
+                  for a, c in zip(vh, (np.float32(1 - 0.999) * g2) * g2)], np.float32)
     cm, sm = O.quantize(m, 4, 128, O.LINEAR)
     cv, sv = O.quantize(v, 8, 128, O.LOG)
     assert (cm == st_a.m_codes).all() and (sm == st_a.m_scales).all()
