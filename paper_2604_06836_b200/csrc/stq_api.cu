@@ -6,6 +6,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "../../include/stq.h"
@@ -32,6 +33,7 @@ struct stq_handle {
   uint32_t n_tiles = 0, n_fast = 0, n_narrow = 0;   // n_narrow counts fast + remaining narrow
   int fast_grid = 0;
   int* d_err = nullptr;             // raised by a kernel whose bounded wait ran out
+  stq::FastSched* d_sched = nullptr;   // work list of the main step kernel
 
   // pinned staging for uploads
   void* h_stage = nullptr;
@@ -201,8 +203,9 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   const size_t bytes_table = sizeof(TensorDesc) * (size_t)L;
   const size_t bytes_map = sizeof(uint32_t) * (size_t)total;
   const size_t off_map = (bytes_table + 255) & ~size_t(255);
+  const size_t off_sched = (off_map + bytes_map + 255) & ~size_t(255);
   int rc;
-  if ((rc = grow_stage(h, off_map + bytes_map)) != STQ_OK) return rc;
+  if ((rc = grow_stage(h, off_sched + sizeof(stq::FastSched))) != STQ_OK) return rc;
   if ((rc = grow(h, h->d_table, h->d_table_cap, (size_t)L)) != STQ_OK) return rc;
   if ((rc = grow(h, h->d_tile_map, h->d_tile_cap, (size_t)total)) != STQ_OK) return rc;
   if (h->stage_busy) { STQ_CUDA(h, cudaEventSynchronize(h->stage_ev)); h->stage_busy = false; }
@@ -221,15 +224,55 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     return ka < kb;
   });
   std::vector<uint32_t> fast0(L);
+  stq::FastSched* hs = reinterpret_cast<stq::FastSched*>(st + off_sched);
+  std::memset(hs, 0, sizeof(*hs));
   {
+    // groups of equal width pair, and an estimate of their cost for the initial spread of the CTAs
+    // (relative cost per tile from measurement: 8- and 16-bit log codes and 3-bit packing cost more;
+    // the estimate only decides where CTAs start, the balance itself is dynamic)
+    double cost[stq::kFastMaxGroups] = {0.0};
     uint32_t next_fast = 0;
+    int last_key = -1;
     for (int i = 0; i < L; ++i) {
       const int l = order[i];
       fast0[l] = next_fast;
+      if (nfast[l] == 0) continue;
+      const stq_tensor& t = tensors[l];
+      const int key = t.bits_v * 64 + t.bits_m;
+      if (key != last_key && hs->ng < (uint32_t)stq::kFastMaxGroups) {
+        hs->grp_begin[hs->ng++] = next_fast;
+        last_key = key;
+      }
+      double w = t.bits_v == 16 ? 1.45 : t.bits_v == 8 ? 1.2 : 1.0;
+      if (t.bits_v == 3 || t.bits_m == 3) w += 0.06;
+      if (t.bits_m == 16) w += 0.08;
+      cost[hs->ng - 1] += w * nfast[l];
       if (!same_map)
         for (uint32_t k = 0; k < nfast[l]; ++k) hm[next_fast + k] = (uint32_t)l;
       next_fast += nfast[l];
     }
+    hs->grp_begin[hs->ng] = next_fast;
+    // CTAs per group in proportion to cost (largest remainders), at least one each
+    const int G = h->fast_grid;
+    double total_cost = 0.0;
+    for (uint32_t g = 0; g < hs->ng; ++g) total_cost += cost[g];
+    std::vector<int> share(hs->ng, 0);
+    std::vector<std::pair<double, int>> rem;
+    int given = 0;
+    for (uint32_t g = 0; g < hs->ng; ++g) {
+      const double exact = total_cost > 0 ? cost[g] / total_cost * G : 0.0;
+      share[g] = std::max(1, (int)exact);
+      given += share[g];
+      rem.push_back({exact - (int)exact, (int)g});
+    }
+    std::sort(rem.begin(), rem.end(), [](const std::pair<double, int>& a, const std::pair<double, int>& b) {
+      return a.first > b.first;
+    });
+    for (size_t k = 0; given < G && !rem.empty(); ++k, ++given) share[rem[k % rem.size()].second]++;
+    int c = 0;
+    for (uint32_t g = 0; g < hs->ng; ++g)
+      for (int k = 0; k < share[g] && c < G; ++k) hs->cta_group[c++] = (uint16_t)g;
+    for (; c < G; ++c) hs->cta_group[c] = (uint16_t)(hs->ng ? c % hs->ng : 0);
   }
   uint32_t next_narrow = (uint32_t)fast, next_wide = (uint32_t)(fast + slow_narrow);
   for (int l = 0; l < L; ++l) {
@@ -263,6 +306,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   STQ_CUDA(h, cudaMemcpyAsync(h->d_table, ht, bytes_table, cudaMemcpyHostToDevice, stream));
   if (!same_map)
     STQ_CUDA(h, cudaMemcpyAsync(h->d_tile_map, hm, bytes_map, cudaMemcpyHostToDevice, stream));
+  STQ_CUDA(h, cudaMemcpyAsync(h->d_sched, hs, sizeof(stq::FastSched), cudaMemcpyHostToDevice, stream));
   STQ_CUDA(h, cudaEventRecord(h->stage_ev, stream));
   h->stage_busy = true;
   h->cached.assign(tensors, tensors + L);
@@ -283,7 +327,7 @@ int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::St
     partials = h->d_partials;
   }
   if (h->n_fast > 0) {   // only a step table has fast tiles
-    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, h->d_table, h->d_tile_map, h->n_fast, sc, partials,
+    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, h->d_table, h->d_tile_map, h->d_sched, sc, partials,
                                       h->d_err, h->fast_grid, stream));
     h->launches++;
   }
@@ -347,8 +391,10 @@ int stq_create(stq_handle** out, int device) {
   h->sm_count = prop.multiProcessorCount;
   h->grid = h->sm_count * stq::step_ctas_per_sm();
   h->fast_grid = h->sm_count * stq::fast_ctas_per_sm();
+  if (h->fast_grid > stq::kFastMaxGrid) h->fast_grid = stq::kFastMaxGrid;
   if (cudaMalloc(reinterpret_cast<void**>(&h->d_err), sizeof(int)) != cudaSuccess ||
-      cudaMemset(h->d_err, 0, sizeof(int)) != cudaSuccess) {
+      cudaMemset(h->d_err, 0, sizeof(int)) != cudaSuccess ||
+      cudaMalloc(reinterpret_cast<void**>(&h->d_sched), sizeof(stq::FastSched)) != cudaSuccess) {
     cudaEventDestroy(h->stage_ev);
     delete h;
     return STQ_E_WORKSPACE;
@@ -364,6 +410,7 @@ int stq_destroy(stq_handle* h) {
   cudaFree(h->d_table);
   cudaFree(h->d_tile_map);
   cudaFree(h->d_err);
+  cudaFree(h->d_sched);
   cudaFree(h->d_partials);
   cudaFree(h->d_stats);
   cudaFree(h->d_arena);

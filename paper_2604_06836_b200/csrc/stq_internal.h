@@ -7,11 +7,11 @@ namespace stq {
 
 constexpr int kThreads = 256;    // 8 warps per CTA
 constexpr int kRowElems = 128;   // one row: lane l holds elements 4l .. 4l+3
-constexpr int kRowsPerWarp = 2;  // a warp owns this many consecutive rows of a tile
+constexpr int kRowsPerWarp = 4;  // a warp owns this many consecutive rows of a tile
 constexpr int kTile = (kThreads / 32) * kRowsPerWarp * kRowElems;   // elements per tile; a tile lies inside one tensor
 constexpr int kMaxBlock = kRowsPerWarp * kRowElems;                 // a quantization block never leaves its warp
-constexpr int kFastCtasPerSm = 3;   // resident CTAs per SM of the main step kernel
-constexpr int kFastStages = 3;      // depth of its shared-memory ring
+constexpr int kFastCtasPerSm = 2;   // resident CTAs per SM of the main step kernel
+constexpr int kFastStages = 2;      // depth of its shared-memory ring
 
 // Device-side row of the tensor table.
 struct TensorDesc {
@@ -53,10 +53,22 @@ cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const
                          const uint32_t* tile_map, uint32_t tile_begin, uint32_t tile_end,
                          const StepConsts& sc, double* partials, int grid, cudaStream_t stream);
 
-// The main step kernel over the fast tiles [0, n_fast) (stq_step_fast.cu).  err_flag is set to 1 if
-// a bounded wait inside the kernel ran out.
+// Work list of the main step kernel: the fast tiles [0, n_fast) of the tile order, cut into groups
+// of equal width pair.  Lives in device memory; the counters are zeroed before every launch.
+constexpr int kFastMaxGroups = 32;     // 25 width pairs exist
+constexpr int kFastMaxGrid = 4096;
+constexpr uint32_t kFastChunk = 16;    // tiles handed out per counter increment
+struct FastSched {
+  uint32_t ctr[kFastMaxGroups];            // chunks handed out so far, per group
+  uint32_t ng;                             // number of groups
+  uint32_t grp_begin[kFastMaxGroups + 1];  // tile range of group g: [grp_begin[g], grp_begin[g+1])
+  uint16_t cta_group[kFastMaxGrid];        // group a CTA starts in
+};
+
+// The main step kernel (stq_step_fast.cu) with `grid` CTAs.  err_flag is set to 1 if a bounded wait
+// inside the kernel ran out.
 cudaError_t launch_step_fast(int grad_dtype, bool stats, const TensorDesc* table, const uint32_t* tile_map,
-                             uint32_t n_fast, const StepConsts& sc, double* partials, int* err_flag, int grid,
+                             FastSched* sched, const StepConsts& sc, double* partials, int* err_flag, int grid,
                              cudaStream_t stream);
 int fast_ctas_per_sm();
 

@@ -353,7 +353,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
 
     if (e_warp < numel) {
       const uint32_t B = T->block;
-      const int lgB = 7 + (int)(B >> 8);   // 128 / 256
+      const int lgB = B == 128 ? 7 : B == 256 ? 8 : 9;
       const int bm_in = T->bm_in, bv_in = T->bv_in, bm_out = T->bm_out, bv_out = T->bv_out;
 
       int nvl[R];
@@ -492,6 +492,11 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
             mxm[r] = mxm[r + 1] = max(mxm[r], mxm[r + 1]);
             mxv[r] = mxv[r + 1] = max(mxv[r], mxv[r + 1]);
           }
+        }
+        if (R >= 4 && B >= 512) {
+          const uint32_t a = max(mxm[0], mxm[R - 2]), b = max(mxv[0], mxv[R - 2]);
+#pragma unroll
+          for (int r = 0; r < R; ++r) { mxm[r] = a; mxv[r] = b; }
         }
 
         // ---- quantize, pack, store; decode the new codes; update the parameters -------------------

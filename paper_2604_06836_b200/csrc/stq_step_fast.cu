@@ -43,9 +43,11 @@ constexpr int kOffTheta = 0;
 constexpr int kOffGrad = 4 * kTile;
 constexpr int kOffMc = 8 * kTile;
 constexpr int kOffVc = 10 * kTile;
-constexpr int kOffMs = 12 * kTile;               // block scales of the tile (at most kTile/128 floats)
-constexpr int kOffVs = kOffMs + 64;
-constexpr int kStageBytes = 12 * kTile + 128;
+constexpr int kScaleBytes = (kTile / 128) * 4;   // block scales of one state of the tile, at most
+constexpr int kOffMs = 12 * kTile;
+constexpr int kOffVs = kOffMs + kScaleBytes;
+constexpr int kStageBytes = 12 * kTile + 2 * kScaleBytes;
+static_assert(kScaleBytes % 16 == 0 && kStageBytes % 128 == 0, "bulk copies need 16-byte aligned destinations");
 
 // What the consumers need to know about a staged tile; written by the producer.
 struct __align__(16) TileInfo {
@@ -57,7 +59,8 @@ struct __align__(16) TileInfo {
   uint32_t wim, wiv;   // width indices (0..4 for 2,3,4,8,16 bits)
   uint32_t lgB;
   float wdx;           // fp32(lr*wd) (AdamW) or fp32(wd) (L2 mode)
-  uint32_t pad[2];
+  uint32_t tile;       // index of the tile in the launch's tile order; 0xFFFFFFFF closes the stream
+  uint32_t pad;
 };
 static_assert(sizeof(TileInfo) == 64, "TileInfo is read with four 128-bit loads");
 
@@ -477,20 +480,24 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
   }
 }
 
+// Scheduling: the fast tiles are grouped by width pair (one body each).  A CTA starts in the group
+// the host assigned to it and takes chunks of kFastChunk consecutive tiles from that group's
+// counter; when its group runs dry it moves on to the next one that still has work.  So a CTA runs
+// few different bodies (a change of body is an instruction-cache refill), the tiles of a group are
+// streamed together, and the balance is dynamic.
 __device__ __forceinline__ uint32_t width_index(uint32_t b) { return b == 2 ? 0u : b == 3 ? 1u : b == 4 ? 2u : b == 8 ? 3u : 4u; }
 
 template <int GDT>
 __global__ void __launch_bounds__(kFastThreads, kFastCtasPerSm)
-stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map, uint32_t n_fast,
-                     const StepConsts sc, double* __restrict__ partials, int* __restrict__ err_flag) {
+stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map,
+                     FastSched* __restrict__ sched, const StepConsts sc, double* __restrict__ partials,
+                     int* __restrict__ err_flag) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t full0 = smem_u32(smem + kOffBars);
   const uint32_t empty0 = full0 + 8 * kStages;
   float* lut8 = reinterpret_cast<float*>(smem + kOffLut);
-  const uint32_t first = blockIdx.x, stride = gridDim.x;
-  if (first >= n_fast) return;
-  const uint32_t n_my = (n_fast - first + stride - 1) / stride;
+  constexpr uint32_t kEnd = 0xFFFFFFFFu;   // TileInfo.tile of the closing stage
   constexpr uint32_t gsz = GDT == 0 ? 4u : 2u;
 
   if (tid == 0) {
@@ -511,68 +518,93 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
   if (warp == kConsumerWarps) {
     // ================================ producer ========================================================
     if (lane != 0) return;
-    uint32_t it = 0;
+    const uint32_t ng = sched->ng;
+    uint32_t grp = sched->cta_group[blockIdx.x];
+    uint32_t dry = 0;          // consecutive groups found empty
+    uint32_t issued = 0;
     int s = 0;
-    uint32_t phase = 0;       // parity of the use of stage s that is being filled
+    uint32_t phase = 0;        // parity of the use of stage s that is being filled
+    uint32_t last_use[kStages];   // parity of the latest fill of each stage (2: never filled)
+#pragma unroll
+    for (int k = 0; k < kStages; ++k) last_use[k] = 2u;
     bool ok = true;
-    for (; it < n_my; ++it) {
-      if (it >= (uint32_t)kStages && !mbar_wait(empty0 + 8 * s, phase ^ 1u)) { ok = false; break; }
-      const uint32_t tile = first + it * stride;
-      const TensorDesc* T = table + __ldg(tile_map + tile);
-      const unsigned long long e0 = (unsigned long long)(tile - T->tile0) * kTile;
-      const uint32_t bm = T->bm_in, bv = T->bv_in;
-      const uint32_t lgB = 7u + (T->block >> 8);
-      const uint32_t nb_m = (kTile / 8) * bm, nb_v = (kTile / 8) * bv, nb_s = (uint32_t)(kTile * 4) >> lgB;
-      TileInfo ti;
-      ti.param = T->param + e0;
-      ti.mco = T->mc_out + (e0 >> 3) * bm;
-      ti.vco = T->vc_out + (e0 >> 3) * bv;
-      ti.mso = T->ms_out + (e0 >> lgB);
-      ti.vso = T->vs_out + (e0 >> lgB);
-      ti.wim = width_index(bm);
-      ti.wiv = width_index(bv);
-      ti.lgB = lgB;
-      ti.wdx = sc.l2_mode ? T->wd : (float)(sc.lr * (double)T->wd);
-      ti.pad[0] = ti.pad[1] = 0u;
-      *reinterpret_cast<TileInfo*>(smem + kOffInfo + 64 * s) = ti;
-      const uint32_t bar = full0 + 8 * s;
-      const uint32_t dst = smem_u32(smem + s * kStageBytes);
-      mbar_expect_tx(bar, kTile * 4 + kTile * gsz + nb_m + nb_v + 2 * nb_s);
-      bulk_g2s(dst + kOffTheta, T->param + e0, kTile * 4, bar);
-      bulk_g2s(dst + kOffGrad, reinterpret_cast<const uint8_t*>(T->grad) + e0 * gsz, kTile * gsz, bar);
-      bulk_g2s(dst + kOffMc, T->mc_in + (e0 >> 3) * bm, nb_m, bar);
-      bulk_g2s(dst + kOffVc, T->vc_in + (e0 >> 3) * bv, nb_v, bar);
-      bulk_g2s(dst + kOffMs, T->ms_in + (e0 >> lgB), nb_s, bar);
-      bulk_g2s(dst + kOffVs, T->vs_in + (e0 >> lgB), nb_s, bar);
-      if (++s == kStages) { s = 0; phase ^= 1u; }
+    while (ok && dry < ng) {
+      const uint32_t gbeg = sched->grp_begin[grp], gend = sched->grp_begin[grp + 1];
+      const uint32_t c = atomicAdd(&sched->ctr[grp], 1u);
+      const unsigned long long t0 = (unsigned long long)gbeg + (unsigned long long)c * kFastChunk;
+      if (t0 >= gend) {        // this group has been handed out completely
+        ++dry;
+        grp = grp + 1 == ng ? 0u : grp + 1;
+        continue;
+      }
+      dry = 0;
+      const uint32_t t1 = (uint32_t)(t0 + kFastChunk < gend ? t0 + kFastChunk : gend);
+      for (uint32_t tile = (uint32_t)t0; tile < t1; ++tile) {
+        if (issued >= (uint32_t)kStages && !mbar_wait(empty0 + 8 * s, phase ^ 1u)) { ok = false; break; }
+        const TensorDesc* T = table + __ldg(tile_map + tile);
+        const unsigned long long e0 = (unsigned long long)(tile - T->tile0) * kTile;
+        const uint32_t bm = T->bm_in, bv = T->bv_in;
+        const uint32_t lgB = T->block == 128 ? 7u : T->block == 256 ? 8u : 9u;
+        const uint32_t nb_m = (kTile / 8) * bm, nb_v = (kTile / 8) * bv, nb_s = (uint32_t)(kTile * 4) >> lgB;
+        TileInfo ti;
+        ti.param = T->param + e0;
+        ti.mco = T->mc_out + (e0 >> 3) * bm;
+        ti.vco = T->vc_out + (e0 >> 3) * bv;
+        ti.mso = T->ms_out + (e0 >> lgB);
+        ti.vso = T->vs_out + (e0 >> lgB);
+        ti.wim = width_index(bm);
+        ti.wiv = width_index(bv);
+        ti.lgB = lgB;
+        ti.wdx = sc.l2_mode ? T->wd : (float)(sc.lr * (double)T->wd);
+        ti.tile = tile;
+        ti.pad = 0u;
+        *reinterpret_cast<TileInfo*>(smem + kOffInfo + 64 * s) = ti;
+        const uint32_t bar = full0 + 8 * s;
+        const uint32_t dst = smem_u32(smem + s * kStageBytes);
+        mbar_expect_tx(bar, kTile * 4 + kTile * gsz + nb_m + nb_v + 2 * nb_s);
+        bulk_g2s(dst + kOffTheta, T->param + e0, kTile * 4, bar);
+        bulk_g2s(dst + kOffGrad, reinterpret_cast<const uint8_t*>(T->grad) + e0 * gsz, kTile * gsz, bar);
+        bulk_g2s(dst + kOffMc, T->mc_in + (e0 >> 3) * bm, nb_m, bar);
+        bulk_g2s(dst + kOffVc, T->vc_in + (e0 >> 3) * bv, nb_v, bar);
+        bulk_g2s(dst + kOffMs, T->ms_in + (e0 >> lgB), nb_s, bar);
+        bulk_g2s(dst + kOffVs, T->vs_in + (e0 >> lgB), nb_s, bar);
+        ++issued;
+#pragma unroll
+        for (int k = 0; k < kStages; ++k)
+          if (k == s) last_use[k] = phase;
+        if (++s == kStages) { s = 0; phase ^= 1u; }
+      }
     }
-    // Before this CTA's shared memory is given up, every copy issued must have landed: wait until
-    // the consumers have drained the last stages (normal path), or, after a time-out, give the
-    // outstanding copies one more bounded wait.
-    const uint32_t issued = it;
-    const uint32_t from = issued > (uint32_t)kStages ? issued - kStages : 0u;
-    for (uint32_t j = from; j < issued; ++j) {
-      const int sj = j % kStages;
-      const uint32_t pj = (j / kStages) & 1u;
-      if (ok) ok = mbar_wait(empty0 + 8 * sj, pj);
-      else mbar_wait(full0 + 8 * sj, pj);
+    // Closing stage: tells the consumers that no tile follows.  Its turn comes only after the
+    // consumers have released the stage, i.e. after every copy issued into it has landed and been
+    // read.  After a time-out the copies still in flight get one more bounded wait instead, so that
+    // none lands in shared memory that no longer belongs to this CTA.
+    if (ok && issued >= (uint32_t)kStages) ok = mbar_wait(empty0 + 8 * s, phase ^ 1u);
+    if (ok) {
+      reinterpret_cast<TileInfo*>(smem + kOffInfo + 64 * s)->tile = kEnd;
+      mbar_arrive(full0 + 8 * s);
+    } else {
+      atomicExch(err_flag, 1);
+#pragma unroll
+      for (int k = 0; k < kStages; ++k)
+        if (last_use[k] != 2u) mbar_wait(full0 + 8 * k, last_use[k]);
     }
-    if (!ok) atomicExch(err_flag, 1);
     return;
   }
 
   // ================================== consumers =========================================================
   int s = 0;
   uint32_t phase = 0;
-  for (uint32_t it = 0; it < n_my; ++it) {
+  while (true) {
     if (!mbar_wait(full0 + 8 * s, phase)) {
       if (lane == 0) atomicExch(err_flag, 1);
       break;
     }
     const uint8_t* stage = smem + s * kStageBytes;
     const TileInfo ti = *reinterpret_cast<const TileInfo*>(smem + kOffInfo + 64 * s);
+    if (ti.tile == kEnd) break;
     const uint32_t ebar = empty0 + 8 * s;
-    double* part = partials ? partials + ((size_t)(first + it * stride) * kConsumerWarps + warp) * 3 : nullptr;
+    double* part = partials ? partials + ((size_t)ti.tile * kConsumerWarps + warp) * 3 : nullptr;
 
 #define STQ_CASE(IM, IV, BM, BV) \
   case IM * 5 + IV: tile_body<BM, BV, GDT>(stage, ti, sc, lut8, lane, warp, ebar, part); break;
@@ -591,7 +623,7 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
 }
 
 template <int GDT>
-cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, uint32_t n_fast, const StepConsts& sc,
+cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, FastSched* sched, const StepConsts& sc,
                           double* partials, int* err_flag, int grid, cudaStream_t stream) {
   static bool attr_set = false;
   auto kern = stq_step_fast_kernel<GDT>;
@@ -600,20 +632,21 @@ cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, uin
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  const int g = (int)(n_fast < (uint32_t)grid ? n_fast : (uint32_t)grid);
-  kern<<<g, kFastThreads, kSmemBytes, stream>>>(table, tile_map, n_fast, sc, partials, err_flag);
+  // the group counters start every launch at zero
+  cudaError_t e = cudaMemsetAsync(sched, 0, sizeof(uint32_t) * kFastMaxGroups, stream);
+  if (e != cudaSuccess) return e;
+  kern<<<grid, kFastThreads, kSmemBytes, stream>>>(table, tile_map, sched, sc, partials, err_flag);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_step_fast(int grad_dtype, bool stats, const TensorDesc* table, const uint32_t* tile_map,
-                             uint32_t n_fast, const StepConsts& sc, double* partials, int* err_flag, int grid,
+                             FastSched* sched, const StepConsts& sc, double* partials, int* err_flag, int grid,
                              cudaStream_t stream) {
-  if (n_fast == 0) return cudaSuccess;
   double* p = stats ? partials : nullptr;
-  return grad_dtype == 0 ? launch_fast_t<0>(table, tile_map, n_fast, sc, p, err_flag, grid, stream)
-                         : launch_fast_t<1>(table, tile_map, n_fast, sc, p, err_flag, grid, stream);
+  return grad_dtype == 0 ? launch_fast_t<0>(table, tile_map, sched, sc, p, err_flag, grid, stream)
+                         : launch_fast_t<1>(table, tile_map, sched, sc, p, err_flag, grid, stream);
 }
 
 int fast_ctas_per_sm() {
