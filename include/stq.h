@@ -54,7 +54,9 @@ enum {
   STQ_E_WORKSPACE = -8, /* the library could not grow its own workspace                       */
   STQ_E_ARG = -9,       /* an invalid scalar argument (step < 1, unknown dtype or flag, ...)  */
   STQ_E_STATE = -10,    /* call order: no statistics pending for stq_layer_stats              */
-  STQ_E_TIMEOUT = -11   /* a bounded wait inside a kernel ran out (stq_device_status)         */
+  STQ_E_TIMEOUT = -11,  /* a bounded wait inside a kernel ran out (stq_device_status)         */
+  STQ_E_TOO_LARGE = -12 /* the tensor exceeds the fixed capacity of an entry point that does  */
+                        /* not allocate (stq_grad_stats_static)                               */
 };
 
 enum { STQ_GRAD_F32 = 0, STQ_GRAD_BF16 = 1 };
@@ -122,6 +124,26 @@ int stq_grad_stats(stq_handle* h, const stq_tensor* tensors, int L, int grad_dty
  * handle and copies it to HOST memory: out[l] = {sum g, sum |g|, sum g^2, numel} for l < L.
  * Synchronises `stream`.  The reduction order is fixed, so results are run-to-run identical. */
 int stq_layer_stats(stq_handle* h, double* out, int L, void* stream);
+
+/* The same sums as stq_grad_stats + stq_layer_stats for ONE gradient tensor, for callers that must
+ * not trigger a device allocation (the paper has no counterpart: this is plumbing).  Typical
+ * cases: the training process has already given all free device memory to its own caching
+ * allocator, so a cudaMalloc from a library can fail or stall the device in mid-step; or the
+ * caller runs under a fixed memory budget.  This call needs no handle, calls no allocating routine
+ * and keeps its scratch (one partial sum per 4096 elements) in a static device array inside the
+ * library: 393,472 bytes that every GPU loading the library holds until the process exits.
+ *   - numel may be at most STQ_STATIC_STATS_MAX_NUMEL; larger tensors are rejected with
+ *     STQ_E_TOO_LARGE and nothing is launched (split the tensor and add the sums).
+ *   - grad: device pointer, 16-byte aligned, fp32 or bf16.  out: DEVICE pointer to 4 doubles
+ *     {sum g, sum |g|, sum g^2, numel}, written on `stream`; the call does not synchronise.
+ *   - `device` is made current.  The first call on a device also looks up the device address of
+ *     the scratch array; make that first call before any stream capture begins.
+ *   - All calls on a device share the scratch array, which keeps the previous call's contents;
+ *     the one word that must start at zero is cleared on `stream` by every call.  Calls that
+ *     overlap on the GPU (different streams without ordering between them) race on the scratch:
+ *     keep them ordered. */
+#define STQ_STATIC_STATS_MAX_NUMEL (64ull * 1024 * 1024)
+int stq_grad_stats_static(int device, const void* grad, uint64_t numel, int grad_dtype, double* out, void* stream);
 
 /* Width transition without an optimizer step (implied by the per-step widths b_{l,t} of
  * Sec. 3.1): codes_out = Quantize_{bits_out}(Decode_{bits}(codes_in)) for both states; block

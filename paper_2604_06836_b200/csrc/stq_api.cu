@@ -618,6 +618,7 @@ const char* stq_strerror(int code) {
     case STQ_E_ARG: return "invalid scalar argument";
     case STQ_E_STATE: return "no statistics pending for this table";
     case STQ_E_TIMEOUT: return "a bounded wait inside a kernel ran out (results of that launch are invalid)";
+    case STQ_E_TOO_LARGE: return "tensor larger than the fixed capacity of this non-allocating entry point";
     default: return "unknown error";
   }
 }

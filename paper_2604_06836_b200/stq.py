@@ -79,6 +79,7 @@ def lib() -> C.CDLL:
         L.stq_step_host.argtypes = [vp, PT, C.c_int, C.POINTER(CHParams), C.c_uint,
                                     C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
         L.stq_device_status.argtypes = [vp, vp]
+        L.stq_grad_stats_static.argtypes = [C.c_int, vp, C.c_uint64, C.c_int, vp, vp]
         L.stq_launch_count.argtypes = [vp]
         L.stq_launch_count.restype = C.c_uint64
         L.stq_grid_size.argtypes = [vp]
@@ -171,6 +172,23 @@ def _stream_ptr(stream) -> int | None:
     if stream is None:
         stream = torch.cuda.current_stream()
     return stream.cuda_stream or None
+
+
+STATIC_STATS_MAX_NUMEL = 64 * 1024 * 1024
+
+
+def grad_stats_static(grad: torch.Tensor, out: torch.Tensor, stream=None) -> int:
+    """Gradient sums of one tensor through the entry point that allocates nothing.
+
+    For callers that cannot let a library allocate device memory (all free memory already belongs
+    to the framework's caching allocator, or a fixed budget is in force): the scratch space is a
+    static array inside libstq.  ``out`` is a caller-owned float64[4] tensor on the same device; the
+    call is asynchronous on the stream.  Returns the C status code (0 = ok) instead of raising, so
+    that callers can test for STQ_E_TOO_LARGE (-12) and fall back to splitting the tensor."""
+    assert out.dtype == torch.float64 and out.numel() >= 4 and out.is_cuda and grad.is_cuda
+    dt = GRAD_BF16 if grad.dtype == torch.bfloat16 else GRAD_F32
+    return int(lib().stq_grad_stats_static(grad.device.index or 0, grad.data_ptr(), grad.numel(), dt,
+                                           out.data_ptr(), _stream_ptr(stream)))
 
 
 class Handle:

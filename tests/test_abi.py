@@ -44,7 +44,7 @@ def test_buffer_sizes(stq_lib, O, bits):
 def test_errors_without_a_device_or_with_bad_arguments(stq_lib):
     from paper_2604_06836_b200 import stq
     assert stq_lib.stq_strerror(0) == b"ok"
-    for code in range(-11, 0):
+    for code in range(-12, 0):
         assert stq_lib.stq_strerror(code) not in (b"ok", b"unknown error")
     h = C.c_void_p()
     assert stq_lib.stq_create(None, 0) == -1
