@@ -29,9 +29,9 @@ METRIC = "quantized_adamw_step_params_per_s"
 UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per parameter of the step kernel from the ncu capture
-# summarised in profiles/ (None until a capture exists); scaled by the parameters per launch.
-NCU_TRAFFIC_BYTES_PER_PARAM = None
+# dram__bytes_read.sum + dram__bytes_write.sum per parameter of the step kernel from the ncu captures
+# summarised in profiles/ (cfg5s is the cfg5 recipe on 6 layers), scaled by the parameters per launch.
+NCU_TRAFFIC_BYTES_PER_PARAM = {"cfg5": 12.377, "cfg5s": 12.377, "cfg2": 14.268}
 
 
 def dist_env():
@@ -276,7 +276,8 @@ def run_ours(args, w, bits_m, bits_v):
                    "parallelism": "replicas" if world > 1 else "single", "grid": job.handle.grid_size,
                    "state_bytes": job.state_bytes(), "fp32_state_bytes": 8 * params},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": (NCU_TRAFFIC_BYTES_PER_PARAM * params if NCU_TRAFFIC_BYTES_PER_PARAM else None),
+                     "traffic": (NCU_TRAFFIC_BYTES_PER_PARAM[args.config] * params
+                                 if args.config in NCU_TRAFFIC_BYTES_PER_PARAM else None),
                      "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": alg_bytes,
                      "bytes_per_param": alg_bytes / params, "kernel_ms_mean": k_ms,
                      "kernel_ms_plain": float(kern_ms[~is_dec].mean()) if (~is_dec).any() else None,

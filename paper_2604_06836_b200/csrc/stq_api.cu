@@ -46,6 +46,11 @@ struct stq_handle {
   size_t d_partials_cap = 0;
   double* d_stats = nullptr;
   size_t d_stats_cap = 0;
+  uint32_t* d_seg_map = nullptr;   // statistics segment -> tensor
+  size_t d_seg_map_cap = 0;
+  double* d_seg_sums = nullptr;
+  size_t d_seg_sums_cap = 0;
+  uint32_t n_seg = 0;
   double* h_stats = nullptr;
   size_t h_stats_cap = 0;
   int stats_L = 0;            // > 0: partials of a table with this many tensors are pending
@@ -204,8 +209,12 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   const size_t bytes_map = sizeof(uint32_t) * (size_t)total;
   const size_t off_map = (bytes_table + 255) & ~size_t(255);
   const size_t off_sched = (off_map + bytes_map + 255) & ~size_t(255);
+  uint64_t n_seg = 0;
+  for (int l = 0; l < L; ++l) n_seg += ((uint64_t)nfast[l] + nslow[l] + stq::kStatSegTiles - 1) / stq::kStatSegTiles;
+  const size_t off_seg = (off_sched + sizeof(stq::FastSched) + 255) & ~size_t(255);
   int rc;
-  if ((rc = grow_stage(h, off_sched + sizeof(stq::FastSched))) != STQ_OK) return rc;
+  if ((rc = grow_stage(h, off_seg + sizeof(uint32_t) * (size_t)n_seg)) != STQ_OK) return rc;
+  if ((rc = grow(h, h->d_seg_map, h->d_seg_map_cap, (size_t)n_seg)) != STQ_OK) return rc;
   if ((rc = grow(h, h->d_table, h->d_table_cap, (size_t)L)) != STQ_OK) return rc;
   if ((rc = grow(h, h->d_tile_map, h->d_tile_cap, (size_t)total)) != STQ_OK) return rc;
   if (h->stage_busy) { STQ_CUDA(h, cudaEventSynchronize(h->stage_ev)); h->stage_busy = false; }
@@ -275,10 +284,15 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     for (; c < G; ++c) hs->cta_group[c] = (uint16_t)(hs->ng ? c % hs->ng : 0);
   }
   uint32_t next_narrow = (uint32_t)fast, next_wide = (uint32_t)(fast + slow_narrow);
+  uint32_t* hseg = reinterpret_cast<uint32_t*>(st + off_seg);
+  uint32_t next_seg = 0;
   for (int l = 0; l < L; ++l) {
     const stq_tensor& t = tensors[l];
     TensorDesc d;
     std::memset(&d, 0, sizeof(d));
+    d.seg0 = next_seg;
+    for (uint32_t k = 0; k < (nfast[l] + nslow[l] + stq::kStatSegTiles - 1) / stq::kStatSegTiles; ++k)
+      hseg[next_seg++] = (uint32_t)l;
     d.tile0 = fast0[l];
     d.nfast = nfast[l];
     uint32_t& next = row_is_wide(t, kind) ? next_wide : next_narrow;
@@ -307,6 +321,9 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   if (!same_map)
     STQ_CUDA(h, cudaMemcpyAsync(h->d_tile_map, hm, bytes_map, cudaMemcpyHostToDevice, stream));
   STQ_CUDA(h, cudaMemcpyAsync(h->d_sched, hs, sizeof(stq::FastSched), cudaMemcpyHostToDevice, stream));
+  if (!same_map)
+    STQ_CUDA(h, cudaMemcpyAsync(h->d_seg_map, hseg, sizeof(uint32_t) * (size_t)n_seg, cudaMemcpyHostToDevice, stream));
+  h->n_seg = (uint32_t)n_seg;
   STQ_CUDA(h, cudaEventRecord(h->stage_ev, stream));
   h->stage_busy = true;
   h->cached.assign(tensors, tensors + L);
@@ -413,6 +430,8 @@ int stq_destroy(stq_handle* h) {
   cudaFree(h->d_sched);
   cudaFree(h->d_partials);
   cudaFree(h->d_stats);
+  cudaFree(h->d_seg_map);
+  cudaFree(h->d_seg_sums);
   cudaFree(h->d_arena);
   if (h->h_stage) cudaFreeHost(h->h_stage);
   if (h->h_stats) cudaFreeHost(h->h_stats);
@@ -482,8 +501,11 @@ int stq_layer_stats(stq_handle* h, double* out, int L, void* stream) {
     if (e != cudaSuccess) { h->cuda_err = cudaGetErrorString(e); return STQ_E_WORKSPACE; }
     h->h_stats_cap = (size_t)L * 4;
   }
-  STQ_CUDA(h, stq::launch_stats_finish(h->d_table, L, h->d_partials, h->d_stats, s));
-  h->launches++;
+  rc = grow(h, h->d_seg_sums, h->d_seg_sums_cap, (size_t)h->n_seg * 3);
+  if (rc != STQ_OK) return rc;
+  STQ_CUDA(h, stq::launch_stats_finish(h->d_table, L, h->d_seg_map, h->n_seg, h->d_partials, h->d_seg_sums,
+                                       h->d_stats, s));
+  h->launches += 2;
   STQ_CUDA(h, cudaMemcpyAsync(h->h_stats, h->d_stats, sizeof(double) * 4 * (size_t)L, cudaMemcpyDeviceToHost, s));
   STQ_CUDA(h, cudaStreamSynchronize(s));
   std::memcpy(out, h->h_stats, sizeof(double) * 4 * (size_t)L);
@@ -609,7 +631,7 @@ const char* stq_strerror(int code) {
     case STQ_OK: return "ok";
     case STQ_E_NULL: return "a required pointer is NULL";
     case STQ_E_BITS: return "bit-width not in {2,3,4,8,16,32}";
-    case STQ_E_BLOCK: return "block not in {128,256}";
+    case STQ_E_BLOCK: return "block not in {128,256,512}";
     case STQ_E_ALIGN: return "buffer not aligned (16 bytes for param/grad/codes, 4 for scales)";
     case STQ_E_ALIAS: return "in/out buffers overlap (in-place needs the same pointer and width)";
     case STQ_E_NUMEL: return "numel is 0, or the table is empty or too large";

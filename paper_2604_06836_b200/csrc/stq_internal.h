@@ -30,7 +30,8 @@ struct TensorDesc {
   unsigned int nfast;       // number of fast tiles; they cover elements [0, nfast * kTile)
   unsigned int tile0s;      // first tile of the rest (ragged tail, or the whole tensor if it is not fast)
   unsigned int nslow;
-  unsigned int block;       // 128 / 256
+  unsigned int seg0;        // first statistics segment (kStatSegTiles tiles each) of this tensor
+  unsigned int block;       // 128 / 256 / 512
   unsigned char bm_in, bv_in, bm_out, bv_out;
   float wd;                 // fp32(lambda)
 };
@@ -72,9 +73,13 @@ cudaError_t launch_step_fast(int grad_dtype, bool stats, const TensorDesc* table
                              cudaStream_t stream);
 int fast_ctas_per_sm();
 
-// out[l] = {sum over the tensor's tiles of partials (fixed order), numel}
-cudaError_t launch_stats_finish(const TensorDesc* table, int L, const double* partials, double* out,
-                                cudaStream_t stream);
+// Second stage of the statistics.  A tensor's tiles (fast range, then the rest) are cut into
+// segments of kStatSegTiles tiles; seg_map[s] is the tensor of segment s.  First every segment is
+// summed (seg_sums: 3 doubles per segment), then every tensor adds its segments:
+// out[l] = {sum g, sum |g|, sum g^2, numel}.  All orders are fixed, so results are reproducible.
+constexpr int kStatSegTiles = 32;
+cudaError_t launch_stats_finish(const TensorDesc* table, int L, const uint32_t* seg_map, uint32_t n_seg,
+                                const double* partials, double* seg_sums, double* out, cudaStream_t stream);
 
 // Resident CTAs per SM of the step kernel (occupancy query), for sizing the persistent grid.
 int step_ctas_per_sm();

@@ -618,20 +618,51 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
   }
 }
 
-// One CTA per tensor: fixed-order sum of its tiles' partials (fast range, then the rest).
+// Statistics, second stage, step 1: one CTA per segment of kStatSegTiles tiles of one tensor.
 __global__ void __launch_bounds__(256)
-stq_stats_finish_kernel(const TensorDesc* __restrict__ table, int L, const double* __restrict__ partials,
+stq_stats_segment_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ seg_map, uint32_t n_seg,
+                         const double* __restrict__ partials, double* __restrict__ seg_sums) {
+  constexpr uint32_t W = kThreads / 32;   // partials per tile
+  const uint32_t sidx = blockIdx.x;
+  if (sidx >= n_seg) return;
+  const TensorDesc* T = table + seg_map[sidx];
+  const uint32_t j = sidx - T->seg0;                       // segment number inside the tensor
+  const uint32_t nt = T->nfast + T->nslow;
+  const uint32_t first = j * kStatSegTiles;
+  const uint32_t count = min((uint32_t)kStatSegTiles, nt - first) * W;
+  double a[3] = {0.0, 0.0, 0.0};
+  for (uint32_t i = threadIdx.x; i < count; i += blockDim.x) {
+    const uint32_t ti = first + i / W;
+    const size_t t = ti < T->nfast ? (size_t)T->tile0 + ti : (size_t)T->tile0s + (ti - T->nfast);
+#pragma unroll
+    for (int k = 0; k < 3; ++k) a[k] += partials[(t * W + (i % W)) * 3 + k];
+  }
+  __shared__ double sh[256][3];
+#pragma unroll
+  for (int k = 0; k < 3; ++k) sh[threadIdx.x][k] = a[k];
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if ((int)threadIdx.x < s) {
+#pragma unroll
+      for (int k = 0; k < 3; ++k) sh[threadIdx.x][k] += sh[threadIdx.x + s][k];
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x < 3) seg_sums[(size_t)sidx * 3 + threadIdx.x] = sh[0][threadIdx.x];
+}
+
+// Step 2: one CTA per tensor adds its segments.
+__global__ void __launch_bounds__(256)
+stq_stats_finish_kernel(const TensorDesc* __restrict__ table, int L, const double* __restrict__ seg_sums,
                         double* __restrict__ out) {
   const int l = blockIdx.x;
   if (l >= L) return;
-  const uint32_t t0 = table[l].tile0, nf = table[l].nfast, t0s = table[l].tile0s, ns = table[l].nslow;
-  constexpr uint32_t W = kThreads / 32;   // partials per tile
+  const uint32_t nt = table[l].nfast + table[l].nslow;
+  const uint32_t ns = (nt + kStatSegTiles - 1) / kStatSegTiles, s0 = table[l].seg0;
   double a[3] = {0.0, 0.0, 0.0};
-  for (uint32_t i = threadIdx.x; i < (nf + ns) * W; i += blockDim.x) {
-    const uint32_t ti = i / W;
-    const size_t t = ti < nf ? (size_t)t0 + ti : (size_t)t0s + (ti - nf);
+  for (uint32_t i = threadIdx.x; i < ns; i += blockDim.x) {
 #pragma unroll
-    for (int k = 0; k < 3; ++k) a[k] += partials[(t * W + (i % W)) * 3 + k];
+    for (int k = 0; k < 3; ++k) a[k] += seg_sums[(size_t)(s0 + i) * 3 + k];
   }
   __shared__ double sh[256][3];
 #pragma unroll
@@ -689,9 +720,12 @@ cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const
   return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_stats_finish(const TensorDesc* table, int L, const double* partials, double* out,
-                                cudaStream_t stream) {
-  stq_stats_finish_kernel<<<L, 256, 0, stream>>>(table, L, partials, out);
+cudaError_t launch_stats_finish(const TensorDesc* table, int L, const uint32_t* seg_map, uint32_t n_seg,
+                                const double* partials, double* seg_sums, double* out, cudaStream_t stream) {
+  stq_stats_segment_kernel<<<n_seg, 256, 0, stream>>>(table, seg_map, n_seg, partials, seg_sums);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  stq_stats_finish_kernel<<<L, 256, 0, stream>>>(table, L, seg_sums, out);
   return cudaGetLastError();
 }
 

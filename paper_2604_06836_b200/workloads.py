@@ -107,6 +107,10 @@ def config(name: str) -> Workload:
         return Workload("cfg5-gpt2-xl-1.5B", tuple(gpt2_shapes(48, 1600)), 128, "bf16", "student_t",
                         nu=3, scale_log10=(-5.0, -2.0), bits_mean=(4.9, 5.1), steps=20,
                         decision_interval=5, seed=5)
+    if name == "cfg5s":   # the cfg5 recipe on 6 of the 48 layers: small enough for a full profiler capture
+        return Workload("cfg5s-gpt2-xl-6-layers", tuple(gpt2_shapes(6, 1600)), 128, "bf16", "student_t",
+                        nu=3, scale_log10=(-5.0, -2.0), bits_mean=(4.9, 5.1), steps=20,
+                        decision_interval=5, seed=5)
     raise KeyError(name)
 
 

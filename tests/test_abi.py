@@ -37,7 +37,7 @@ def test_buffer_sizes(stq_lib, O, bits):
     for n in (1, 7, 128, 129, 1000, 4096, 50257 * 1600):
         want = ((n * bits + 7) // 8 + 15) // 16 * 16
         assert stq.codes_bytes(n, bits) == want == O.codes_bytes(n, bits)
-        for block in (128, 256):
+        for block in (128, 256, 512):
             assert stq.scales_bytes(n, block) == 4 * ((n + block - 1) // block) == 4 * O.num_blocks(n, block)
 
 

@@ -24,7 +24,7 @@ def _single(n, block, gdt, seed=0):
 
 
 @pytest.mark.parametrize("gdt", ["fp32", "bf16"])
-@pytest.mark.parametrize("block", [128, 256])
+@pytest.mark.parametrize("block", [128, 256, 512])
 @pytest.mark.parametrize("bm", [2, 3, 4, 8, 16])
 @pytest.mark.parametrize("bv", [2, 3, 4, 8, 16])
 def test_every_width_pair_three_steps(H, O, bm, bv, block, gdt):
