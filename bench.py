@@ -252,14 +252,9 @@ def run_ours(args, w, bits_m, bits_v):
     if not args.no_e2e:
         e2e = run_e2e(job, w, args)
 
-    if use_dist:
-        tt = torch.tensor([total_ms, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(tt[0]), float(tt[1])
-    else:
-        e2e_ms = e2e["ms"] if e2e else 0.0
-
+    from paper_2604_06836_b200 import multi
     params = w.total_params
+    total_ms, e2e_ms = multi.max_over_ranks([total_ms, e2e["ms"] if e2e else 0.0], dev)   # slowest rank
     value = world * params * args.steps / (total_ms * 1e-3)
     alg_bytes = job.algorithmic_bytes()
     k_ms = float(kern_ms.mean())

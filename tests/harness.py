@@ -120,3 +120,90 @@ def compare_job(job: Job, oj: OracleJob, rel: float, tag=""):
         assert_states_equal(job.states[i], oj.states[i], f"{tag} tensor {i} ({job.w.shapes[i][0]})")
         assert_theta_close(job.params[i], oj.theta[i], rel, f"{tag} tensor {i} ({job.w.shapes[i][0]})",
                            upd=oj.upd_mag[i])
+
+
+class SampledOracle:
+    """Oracle on a sample of quantization blocks of a full-size Job.
+
+    Blocks are independent given (theta, grad, stored state), so a few blocks per tensor, gathered
+    into a small tensor (the ragged last block, if any, goes last), can be stepped by the oracle one
+    by one and compared with the same blocks of the GPU buffers."""
+
+    def __init__(self, job: Job, per_tensor: int = 6, seed: int = 0):
+        self.job = job
+        self.block = job.block
+        rng = np.random.RandomState(seed)
+        self.sel, self.n_mini = [], []
+        for n in job.numels:
+            nb_full = n // self.block
+            tail = n - nb_full * self.block
+            pick = set()
+            if nb_full:
+                pick.update([0, nb_full - 1])
+                # blocks on either side of tile boundaries (4096 elements) and random ones
+                for b in (4096 // self.block - 1, 4096 // self.block):
+                    if b < nb_full:
+                        pick.add(b)
+                pick.update(rng.randint(0, nb_full, size=per_tensor).tolist())
+            blocks = sorted(pick)
+            self.sel.append((np.array(blocks, dtype=np.int64), tail, nb_full))
+            self.n_mini.append(len(blocks) * self.block + tail)
+        self.theta = [self._gather_elems(p, i) for i, p in enumerate(job.params)]
+        self.states = [O.new_state(self.n_mini[i], self.block, int(job.bits_m[i]), int(job.bits_v[i]))
+                       for i in range(job.L)]
+        self.mag = [np.abs(t) for t in self.theta]
+
+    def _elem_index(self, i: int) -> torch.Tensor:
+        blocks, tail, nb_full = self.sel[i]
+        idx = (blocks[:, None] * self.block + np.arange(self.block)[None, :]).ravel()
+        if tail:
+            idx = np.concatenate([idx, nb_full * self.block + np.arange(tail)])
+        return torch.from_numpy(idx).to(self.job.device)
+
+    def _gather_elems(self, t: torch.Tensor, i: int) -> np.ndarray:
+        return to_np(t[self._elem_index(i)])
+
+    def _gather_codes(self, codes: torch.Tensor, bits: int, i: int) -> np.ndarray:
+        blocks, tail, nb_full = self.sel[i]
+        bb = self.block * bits // 8
+        idx = (blocks[:, None] * bb + np.arange(bb)[None, :]).ravel()
+        if tail:
+            idx = np.concatenate([idx, nb_full * bb + np.arange((tail * bits + 7) // 8)])
+        got = to_np(codes[torch.from_numpy(idx).to(codes.device)])
+        out = np.zeros(O.codes_bytes(self.n_mini[i], bits), dtype=np.uint8)
+        out[:got.size] = got
+        return out
+
+    def _gather_scales(self, scales: torch.Tensor, i: int) -> np.ndarray:
+        blocks, tail, nb_full = self.sel[i]
+        idx = np.concatenate([blocks, [nb_full]]) if tail else blocks
+        return to_np(scales[torch.from_numpy(idx).to(scales.device)])
+
+    def step(self, t: int):
+        """Oracle step on the sample, with the gradients currently held by the job."""
+        w = self.job.w
+        for i in range(self.job.L):
+            if self.n_mini[i] == 0:
+                continue
+            g = self._gather_elems(self.job.grads[i], i)
+            before = self.theta[i].copy()
+            self.states[i], _ = O.step(self.theta[i], g, self.states[i], self.block, lr=w.lr, beta1=w.beta1,
+                                       beta2=w.beta2, eps=w.eps, weight_decay=self.job.wd[i], t=t)
+            self.mag[i] = np.maximum(self.mag[i], np.maximum(np.abs(self.theta[i]), np.abs(self.theta[i] - before)))
+
+    def compare(self, rel: float, tag=""):
+        job = self.job
+        job.handle.device_status()
+        for i in range(job.L):
+            if self.n_mini[i] == 0:
+                continue
+            gs, os_ = job.states[i], self.states[i]
+            name = f"{tag} tensor {i} ({job.w.shapes[i][0]}, bits {gs.bits_m}/{gs.bits_v})"
+            assert (self._gather_codes(gs.m_codes, gs.bits_m, i) == os_.m_codes).all(), name + " m codes"
+            assert (self._gather_codes(gs.v_codes, gs.bits_v, i) == os_.v_codes).all(), name + " v codes"
+            assert (self._gather_scales(gs.m_scales, i).view(np.uint32) == os_.m_scales.view(np.uint32)).all(), name
+            assert (self._gather_scales(gs.v_scales, i).view(np.uint32) == os_.v_scales.view(np.uint32)).all(), name
+            g = self._gather_elems(job.params[i], i).astype(np.float64)
+            o = self.theta[i].astype(np.float64)
+            lim = rel * np.maximum(self.mag[i].astype(np.float64), 1e-3 * np.abs(o).max())
+            assert (np.abs(g - o) <= lim).all(), name + f" theta: max err {np.abs(g - o).max():.3e}"
