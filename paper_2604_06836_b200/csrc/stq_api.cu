@@ -191,7 +191,8 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     const bool wide = row_is_wide(t, kind);
     // (the main kernel moves the scales with 16-byte bulk copies as well)
     const bool fast_ok = kind == kKindStep && !wide && t.bits_m == t.bits_m_out && t.bits_v == t.bits_v_out &&
-                         t.numel < (1ull << 32) && aligned(t.m_scales_in, 16) && aligned(t.v_scales_in, 16);
+                         t.numel < (1ull << 32) && aligned(t.m_scales_in, 16) && aligned(t.v_scales_in, 16) &&
+                         t.block <= (uint32_t)stq::kFastMaxBlock;
     const uint64_t nf = fast_ok ? t.numel / stq::kTile : 0;
     nfast[l] = (uint32_t)nf;
     nslow[l] = (uint32_t)(nt - nf);

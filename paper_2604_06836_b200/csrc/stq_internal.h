@@ -11,7 +11,9 @@ constexpr int kRowsPerWarp = 4;  // a warp owns this many consecutive rows of a 
 constexpr int kTile = (kThreads / 32) * kRowsPerWarp * kRowElems;   // elements per tile; a tile lies inside one tensor
 constexpr int kMaxBlock = kRowsPerWarp * kRowElems;                 // a quantization block never leaves its warp
 constexpr int kFastCtasPerSm = 2;   // resident CTAs per SM of the main step kernel
-constexpr int kFastStages = 2;      // depth of its shared-memory ring
+constexpr int kFastStages = 2;
+constexpr int kFastRowsPerPass = 2; // rows a warp handles per pass over its kRowsPerWarp rows (see the kernel)
+constexpr int kFastMaxBlock = kFastRowsPerPass * kRowElems;   // larger blocks take the generic path      // depth of its shared-memory ring
 
 // Device-side row of the tensor table.
 struct TensorDesc {

@@ -324,46 +324,158 @@ __device__ __forceinline__ void lds_grad(const uint8_t* stage, int elem, float (
   }
 }
 
-// One staged tile, one warp: R rows of 128 elements.  Specialised on both widths.
+// One staged tile, one warp: R rows of 128 elements, taken in passes of RP rows.  The pass loop is
+// a real loop (not unrolled): the straight-line body of a pass is what the warps stream through the
+// instruction cache, and halving it pays more than the lost overlap between passes.  Specialised on
+// both widths.
+constexpr int RP = kFastRowsPerPass;
 template <int BM, int BV, int GDT>
 __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, const TileInfo& ti, const StepConsts& sc,
                                           const float* __restrict__ lut8, int lane, int warp, uint32_t empty_bar,
                                           double* __restrict__ part) {
   const int lgB = (int)ti.lgB;
-  const int row0 = warp * R;
+  const float lrwd = sc.l2_mode ? 0.0f : ti.wdx;
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f;      // statistics over the raw gradient (decision steps)
 
-  // ---- staged tile -> registers, decode ---------------------------------------------------------------
-  float th[R][4], g[R][4], mt[R][4], vt[R][4];
-#pragma unroll
-  for (int r = 0; r < R; ++r) {
-    const int elem = (row0 + r) * kRowElems + 4 * lane;
-    const float4 t4 = *reinterpret_cast<const float4*>(stage + kOffTheta + 4 * elem);
-    th[r][0] = t4.x; th[r][1] = t4.y; th[r][2] = t4.z; th[r][3] = t4.w;
-    lds_grad<GDT>(stage, elem, g[r]);
-    const int blk = ((row0 + r) * kRowElems) >> lgB;
-    const float sm = *reinterpret_cast<const float*>(stage + kOffMs + 4 * blk);
-    const float sv = *reinterpret_cast<const float*>(stage + kOffVs + 4 * blk);
-    uint32_t w[2];
-    lds_codes<BM>(stage + kOffMc + (row0 + r) * (16 * BM), lane, w);
-    decode_lin_row<BM>(w, sm, mt[r]);
-    lds_codes<BV>(stage + kOffVc + (row0 + r) * (16 * BV), lane, w);
-    decode_log_row<BV>(w, sv, lut8, vt[r]);
-  }
-  // this warp is done with the stage
-  __syncwarp();
-  if (lane == 0) mbar_arrive(empty_bar);
+#pragma unroll 1
+  for (int pass = 0; pass < R / RP; ++pass) {
+    const int row0 = warp * R + pass * RP;
 
-  // ---- statistics over the raw gradient (decision steps) -------------------------------------------------
-  if (part != nullptr) {
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f;
+    // ---- staged rows -> registers, decode -----------------------------------------------------------
+    float th[RP][4], g[RP][4], mt[RP][4], vt[RP][4];
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+    for (int r = 0; r < RP; ++r) {
+      const int elem = (row0 + r) * kRowElems + 4 * lane;
+      const float4 t4 = *reinterpret_cast<const float4*>(stage + kOffTheta + 4 * elem);
+      th[r][0] = t4.x; th[r][1] = t4.y; th[r][2] = t4.z; th[r][3] = t4.w;
+      lds_grad<GDT>(stage, elem, g[r]);
+      const int blk = ((row0 + r) * kRowElems) >> lgB;
+      const float sm = *reinterpret_cast<const float*>(stage + kOffMs + 4 * blk);
+      const float sv = *reinterpret_cast<const float*>(stage + kOffVs + 4 * blk);
+      uint32_t w[2];
+      lds_codes<BM>(stage + kOffMc + (row0 + r) * (16 * BM), lane, w);
+      decode_lin_row<BM>(w, sm, mt[r]);
+      lds_codes<BV>(stage + kOffVc + (row0 + r) * (16 * BV), lane, w);
+      decode_log_row<BV>(w, sv, lut8, vt[r]);
+    }
+    if (pass == R / RP - 1) {   // the last rows are in registers: this warp is done with the stage
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar);
+    }
+
+    if (part != nullptr) {
+#pragma unroll
+      for (int r = 0; r < RP; ++r)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          a0 += g[r][k];
+          a1 += fabsf(g[r][k]);
+          a2 = __fmaf_rn(g[r][k], g[r][k], a2);
+        }
+    }
+
+    // ---- moments ----------------------------------------------------------------------------------------
+    if (sc.l2_mode) {
+#pragma unroll
+      for (int r = 0; r < RP; ++r)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) g[r][k] = __fadd_rn(g[r][k], __fmul_rn(ti.wdx, th[r][k]));
+    }
+#pragma unroll
+    for (int r = 0; r < RP; ++r) {
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        a0 += g[r][k];
-        a1 += fabsf(g[r][k]);
-        a2 = __fmaf_rn(g[r][k], g[r][k], a2);
+        const float gk = g[r][k];
+        mt[r][k] = __fmaf_rn(sc.b1, mt[r][k], __fmul_rn(sc.c1, gk));
+        vt[r][k] = __fmaf_rn(sc.b2, vt[r][k], __fmul_rn(__fmul_rn(sc.c2, gk), gk));
       }
+    }
+
+    // ---- block maxima --------------------------------------------------------------------------------
+    uint32_t mxm[RP], mxv[RP];
+#pragma unroll
+    for (int r = 0; r < RP; ++r) {
+      const float am = fmaxf(fmaxf(fabsf(mt[r][0]), fabsf(mt[r][1])), fmaxf(fabsf(mt[r][2]), fabsf(mt[r][3])));
+      const float av = fmaxf(fmaxf(vt[r][0], vt[r][1]), fmaxf(vt[r][2], vt[r][3]));
+      mxm[r] = __reduce_max_sync(kFull, __float_as_uint(am));
+      mxv[r] = __reduce_max_sync(kFull, __float_as_uint(av));
+    }
+    if (RP >= 2 && lgB >= 8) {
+#pragma unroll
+      for (int r = 0; r + 1 < RP; r += 2) {
+        mxm[r] = mxm[r + 1] = max(mxm[r], mxm[r + 1]);
+        mxv[r] = mxv[r + 1] = max(mxv[r], mxv[r + 1]);
+      }
+    }
+    if (RP >= 4 && lgB >= 9) {
+      const uint32_t a = max(mxm[0], mxm[RP - 2]), b = max(mxv[0], mxv[RP - 2]);
+#pragma unroll
+      for (int r = 0; r < RP; ++r) { mxm[r] = a; mxv[r] = b; }
+    }
+
+    // ---- per-block constants: one lane per (row, state) works them out, then they are broadcast --------
+    // lanes 0..RP-1: inv = fl(qmax * fl(1/s_m));  lanes RP..2RP-1 (octave widths): c = fl(sqrt2 * fl(1/s_v))
+    float inv_m[RP], lgc[RP];
+    {
+      uint32_t mine = mxm[0];
+#pragma unroll
+      for (int r = 1; r < RP; ++r)
+        if ((lane & (RP - 1)) == r) mine = mxm[r];
+      if constexpr (BV <= 4) {
+#pragma unroll
+        for (int r = 0; r < RP; ++r)
+          if ((lane & (2 * RP - 1)) == RP + r) mine = mxv[r];
+      }
+      const float x = __uint_as_float(mine);
+      const float mul = (BV <= 4 && (lane & RP)) ? kSqrt2 : (float)Wd<BM>::qmax;
+      const float val = x < kTiny ? 0.f : __fmul_rn(mul, __frcp_rn(x));
+#pragma unroll
+      for (int r = 0; r < RP; ++r) inv_m[r] = __shfl_sync(kFull, val, r);
+      if constexpr (BV <= 4) {
+#pragma unroll
+        for (int r = 0; r < RP; ++r) lgc[r] = __shfl_sync(kFull, val, RP + r);
+      } else {
+        uint32_t mv = mxv[0];
+#pragma unroll
+        for (int r = 1; r < RP; ++r)
+          if ((lane & (RP - 1)) == r) mv = mxv[r];
+        const float ps = lg_poly(mv);
+#pragma unroll
+        for (int r = 0; r < RP; ++r) lgc[r] = __shfl_sync(kFull, ps, r);
+      }
+    }
+
+    // ---- quantize, pack, store; decode the new codes; update the parameters --------------------------
+    float* param = ti.param + row0 * kRowElems + 4 * lane;
+#pragma unroll
+    for (int r = 0; r < RP; ++r) {
+      const float sm_raw = __uint_as_float(mxm[r]);
+      const float s_m = sm_raw < kTiny ? 0.f : sm_raw;
+      const float sv_raw = __uint_as_float(mxv[r]);
+      const bool vzero = sv_raw < kTiny;
+      const float s_v = vzero ? 0.f : sv_raw;
+      const uint32_t ebase = kMagicBits - (vzero ? (uint32_t)kZeroBlockExp : (mxv[r] >> 23));
+      float mq[4], vq[4];
+      // mq comes out multiplied by lr/(1-beta1^t): the decode scale carries the factor
+      encode_lin_row<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], __fmul_rn(s_m, sc.step_size), inv_m[r], mq);
+      encode_log_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], s_v, lgc[r], ebase, lut8, vq);
+      const int e_row = (row0 + r) * kRowElems;
+      if (lane == 0 && (e_row & ((1 << lgB) - 1)) == 0) {
+        ti.mso[e_row >> lgB] = s_m;
+        ti.vso[e_row >> lgB] = s_v;
+      }
+      float out[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float den = __fmaf_rn(sqrt_fast(vq[k]), sc.rsqrt_bc2, sc.eps);
+        const float upd = __fmul_rn(mq[k], rcp_fast(den));
+        out[k] = __fadd_rn(th[r][k], -__fmaf_rn(th[r][k], lrwd, upd));
+      }
+      *reinterpret_cast<float4*>(param + r * kRowElems) = make_float4(out[0], out[1], out[2], out[3]);
+    }
+  }
+
+  if (part != nullptr) {
     // Pairwise fp32 butterfly that spreads the three sums over the lanes on the way down:
     // after xor 16 the low half carries (sum0, sum1) and the high half (sum2, -); after xor 8
     // lanes 0-7 / 8-15 / 16-23 carry sum0 / sum1 / sum2; three more steps finish each group.
@@ -376,107 +488,6 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
     z += __shfl_xor_sync(kFull, z, 2);
     z += __shfl_xor_sync(kFull, z, 1);
     if ((lane & 7) == 0 && lane < 24) part[lane >> 3] = (double)z;
-  }
-
-  // ---- moments ------------------------------------------------------------------------------------------
-  if (sc.l2_mode) {
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-      for (int k = 0; k < 4; ++k) g[r][k] = __fadd_rn(g[r][k], __fmul_rn(ti.wdx, th[r][k]));
-  }
-#pragma unroll
-  for (int r = 0; r < R; ++r) {
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float gk = g[r][k];
-      mt[r][k] = __fmaf_rn(sc.b1, mt[r][k], __fmul_rn(sc.c1, gk));
-      vt[r][k] = __fmaf_rn(sc.b2, vt[r][k], __fmul_rn(__fmul_rn(sc.c2, gk), gk));
-    }
-  }
-
-  // ---- block maxima ----------------------------------------------------------------------------------
-  uint32_t mxm[R], mxv[R];
-#pragma unroll
-  for (int r = 0; r < R; ++r) {
-    const float am = fmaxf(fmaxf(fabsf(mt[r][0]), fabsf(mt[r][1])), fmaxf(fabsf(mt[r][2]), fabsf(mt[r][3])));
-    const float av = fmaxf(fmaxf(vt[r][0], vt[r][1]), fmaxf(vt[r][2], vt[r][3]));
-    mxm[r] = __reduce_max_sync(kFull, __float_as_uint(am));
-    mxv[r] = __reduce_max_sync(kFull, __float_as_uint(av));
-  }
-  if (lgB >= 8) {
-#pragma unroll
-    for (int r = 0; r < R; r += 2) {
-      mxm[r] = mxm[r + 1] = max(mxm[r], mxm[r + 1]);
-      mxv[r] = mxv[r + 1] = max(mxv[r], mxv[r + 1]);
-    }
-  }
-  if (R >= 4 && lgB >= 9) {
-    const uint32_t a = max(mxm[0], mxm[R - 2]), b = max(mxv[0], mxv[R - 2]);
-#pragma unroll
-    for (int r = 0; r < R; ++r) { mxm[r] = a; mxv[r] = b; }
-  }
-
-  // ---- per-block constants: one lane per (row, state) works them out, then they are broadcast ----------
-  // lanes 0..R-1: inv = fl(qmax * fl(1/s_m));  lanes R..2R-1 (octave widths): c = fl(sqrt2 * fl(1/s_v))
-  float inv_m[R], lgc[R];
-  {
-    uint32_t mine = mxm[0];
-#pragma unroll
-    for (int r = 1; r < R; ++r)
-      if ((lane & (R - 1)) == r) mine = mxm[r];
-    if constexpr (BV <= 4) {
-#pragma unroll
-      for (int r = 0; r < R; ++r)
-        if ((lane & (2 * R - 1)) == R + r) mine = mxv[r];
-    }
-    const float x = __uint_as_float(mine);
-    const float mul = (BV <= 4 && (lane & R)) ? kSqrt2 : (float)Wd<BM>::qmax;
-    const float val = x < kTiny ? 0.f : __fmul_rn(mul, __frcp_rn(x));
-#pragma unroll
-    for (int r = 0; r < R; ++r) inv_m[r] = __shfl_sync(kFull, val, r);
-    if constexpr (BV <= 4) {
-#pragma unroll
-      for (int r = 0; r < R; ++r) lgc[r] = __shfl_sync(kFull, val, R + r);
-    } else {
-      uint32_t mv = mxv[0];
-#pragma unroll
-      for (int r = 1; r < R; ++r)
-        if ((lane & (R - 1)) == r) mv = mxv[r];
-      const float ps = lg_poly(mv);
-#pragma unroll
-      for (int r = 0; r < R; ++r) lgc[r] = __shfl_sync(kFull, ps, r);
-    }
-  }
-
-  // ---- quantize, pack, store; decode the new codes; update the parameters ----------------------------
-  const float lrwd = sc.l2_mode ? 0.0f : ti.wdx;
-  float* param = ti.param + row0 * kRowElems + 4 * lane;
-#pragma unroll
-  for (int r = 0; r < R; ++r) {
-    const float sm_raw = __uint_as_float(mxm[r]);
-    const float s_m = sm_raw < kTiny ? 0.f : sm_raw;
-    const float sv_raw = __uint_as_float(mxv[r]);
-    const bool vzero = sv_raw < kTiny;
-    const float s_v = vzero ? 0.f : sv_raw;
-    const uint32_t ebase = kMagicBits - (vzero ? (uint32_t)kZeroBlockExp : (mxv[r] >> 23));
-    float mq[4], vq[4];
-    // mq comes out multiplied by lr/(1-beta1^t): the decode scale carries the factor
-    encode_lin_row<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], __fmul_rn(s_m, sc.step_size), inv_m[r], mq);
-    encode_log_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], s_v, lgc[r], ebase, lut8, vq);
-    const int e_row = (row0 + r) * kRowElems;
-    if (lane == 0 && (e_row & ((1 << lgB) - 1)) == 0) {
-      ti.mso[e_row >> lgB] = s_m;
-      ti.vso[e_row >> lgB] = s_v;
-    }
-    float out[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float den = __fmaf_rn(sqrt_fast(vq[k]), sc.rsqrt_bc2, sc.eps);
-      const float upd = __fmul_rn(mq[k], rcp_fast(den));
-      out[k] = __fadd_rn(th[r][k], -__fmaf_rn(th[r][k], lrwd, upd));
-    }
-    *reinterpret_cast<float4*>(param + r * kRowElems) = make_float4(out[0], out[1], out[2], out[3]);
   }
 }
 
