@@ -257,19 +257,21 @@ __device__ __forceinline__ void pack_store_row(uint8_t* row_ptr, int lane, const
   }
 }
 
-// Quantize one row of new first moments, store the codes, return the decoded values times `gain`
-// (s_dec = stored scale * gain).
+// Quantize one row of new first moments and store the codes.  mq receives what the update needs:
+// the decoded values times `gain` = lr/(1-beta1^t), formed as q * (s * gain / qmax) (the update is
+// held to 1e-6, not to the bit, so the two roundings of the decode are merged into one factor).
 template <int B>
-__device__ __forceinline__ void encode_lin_row(uint8_t* row_ptr, int lane, const float (&m)[4], float s_dec, float inv,
+__device__ __forceinline__ void encode_lin_row(uint8_t* row_ptr, int lane, const float (&m)[4], float s_gain, float inv,
                                                float (&mq)[4]) {
   constexpr float invq = 1.0f / (float)Wd<B>::qmax;
   constexpr float mg = kMagic + (float)Wd<B>::half;
+  const float unit = __fmul_rn(s_gain, invq);
   uint32_t x[4];
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const float t = __fmaf_rn(m[k], inv, mg);
     x[k] = __float_as_uint(t);
-    mq[k] = __fmul_rn(s_dec, __fmul_rn(__fadd_rn(t, -mg), invq));
+    mq[k] = __fmul_rn(__fadd_rn(t, -mg), unit);
   }
   pack_store_row<B>(row_ptr, lane, x, kMagicBits);
 }

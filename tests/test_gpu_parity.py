@@ -191,3 +191,37 @@ def test_run_to_run_identical(H, O):
                      torch.cat([s.m_codes for s in job.states] + [s.v_codes for s in job.states]).cpu()))
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][2], outs[1][2])
     assert (outs[0][1] == outs[1][1]).all()
+
+
+def test_algorithm1_order_with_the_paper_policy_driving_the_widths(H, O):
+    """Algorithm 1 as printed: on decision steps the statistics of the fresh gradients are taken first,
+    the policy maps them to widths in {4, 8, 16, 32}, and the same step already writes the states at the
+    new widths (every layer starts at 16 bits)."""
+    import oracle
+    w = W.scaled(W.config("cfg2"), W.small_gpt2(d=136, n_layer=2, vocab=300), steps=24)
+    L = len(w.shapes)
+    job = Job(w, [16] * L, [16] * L)
+    oj = H.OracleJob(job)
+    U = 6
+    pol_g = stq.Policy(alpha=0.1, tau=8.0, eps_stat=1e-8, interval=U)
+    pol_o = oracle.new_policy(0.1, 8.0, 1e-8)
+    seen = set()
+    for t in range(1, 25):
+        job.draw_grads(t)
+        grads = [H.to_np(g) for g in job.grads]
+        new_bits = None
+        if pol_g.is_decision_step(t):
+            job.handle.grad_stats(job.table(), job.grad_dtype)
+            st_g = job.layer_stats()
+            job._tbl = None
+            st_o = np.stack([oracle.grad_stats(g) for g in grads])
+            H.assert_stats_close(st_g, st_o, f"t={t}")
+            bg, _ = pol_g.decide(st_g, t)
+            bo, _ = oracle.decide(pol_o, st_g, t)
+            assert (bg == bo).all() and set(bg.tolist()) <= {4, 8, 16, 32}
+            new_bits = (bg, bg)                      # Algorithm 1: one width per layer for both states
+            seen |= set(bg.tolist())
+        oj.step(grads, t, new_bits=new_bits)
+        job.step(t, new_bits=new_bits)
+        H.compare_job(job, oj, REL_1STEP * t if t <= 10 else REL_100, f"t={t}")
+    assert len(seen) >= 2          # the policy did move layers between widths
