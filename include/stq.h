@@ -153,8 +153,10 @@ int stq_repack(stq_handle* h, const stq_tensor* tensors, int L, void* stream);
 
 /* stq_step with every pointer in `tensors` a HOST pointer: the library stages the buffers through
  * a device arena it owns (grown on demand), copies param/grad/codes/scales in, runs the step,
- * copies param/codes/scales back and synchronises.  bytes_h2d / bytes_d2h (optional) receive
- * the bytes copied. */
+ * copies param/codes/scales back and synchronises the device.  Chunks of consecutive tensors
+ * (~256 MB) are pipelined over three internal streams, so with pinned host buffers the copies in,
+ * the kernels and the copies out overlap (a step with STQ_WITH_STATS runs as one chunk).
+ * bytes_h2d / bytes_d2h (optional) receive the bytes copied. */
 int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hparams* hp,
                   unsigned flags, uint64_t* bytes_h2d, uint64_t* bytes_d2h);
 

@@ -55,9 +55,11 @@ struct stq_handle {
   size_t h_stats_cap = 0;
   int stats_L = 0;            // > 0: partials of a table with this many tensors are pending
 
-  // device arena of stq_step_host
+  // device arena, streams and events of stq_step_host
   uint8_t* d_arena = nullptr;
   size_t d_arena_cap = 0;
+  cudaStream_t host_streams[3] = {nullptr, nullptr, nullptr};
+  std::vector<cudaEvent_t> host_events;
 };
 
 namespace {
@@ -279,10 +281,16 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
       return a.first > b.first;
     });
     for (size_t k = 0; given < G && !rem.empty(); ++k, ++given) share[rem[k % rem.size()].second]++;
-    int c = 0;
+    // Groups are ordered by v width, i.e. from memory-bound bodies to instruction-bound ones.  CTA c
+    // and CTA c + (number of SMs) tend to share an SM, so the second wave is handed out in reverse:
+    // an SM then hosts one CTA from either end, and the issue slots the memory-bound one leaves idle
+    // serve the other.
+    std::vector<uint16_t> glist;
     for (uint32_t g = 0; g < hs->ng; ++g)
-      for (int k = 0; k < share[g] && c < G; ++k) hs->cta_group[c++] = (uint16_t)g;
-    for (; c < G; ++c) hs->cta_group[c] = (uint16_t)(hs->ng ? c % hs->ng : 0);
+      for (int k = 0; k < share[g] && (int)glist.size() < G; ++k) glist.push_back((uint16_t)g);
+    while ((int)glist.size() < G) glist.push_back((uint16_t)(hs->ng ? glist.size() % hs->ng : 0));
+    const int wave = std::min(G, h->sm_count);
+    for (int c = 0; c < G; ++c) hs->cta_group[c] = c < wave ? glist[c] : glist[G - 1 - (c - wave)];
   }
   uint32_t next_narrow = (uint32_t)fast, next_wide = (uint32_t)(fast + slow_narrow);
   uint32_t* hseg = reinterpret_cast<uint32_t*>(st + off_seg);
@@ -434,6 +442,9 @@ int stq_destroy(stq_handle* h) {
   cudaFree(h->d_seg_map);
   cudaFree(h->d_seg_sums);
   cudaFree(h->d_arena);
+  for (cudaStream_t st : h->host_streams)
+    if (st) cudaStreamDestroy(st);
+  for (cudaEvent_t e : h->host_events) cudaEventDestroy(e);
   if (h->h_stage) cudaFreeHost(h->h_stage);
   if (h->h_stats) cudaFreeHost(h->h_stats);
   if (h->stage_ev) cudaEventDestroy(h->stage_ev);
@@ -559,63 +570,101 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
   rc = grow(h, h->d_arena, h->d_arena_cap, need);
   if (rc != STQ_OK) return rc;
 
-  cudaStream_t s = nullptr;   // the legacy default stream: ordered with everything else
+  // Chunks of consecutive tensors are pipelined over three streams: copies in, the step, copies out.
+  // With pinned host buffers the two copy directions and the kernels overlap; pageable buffers make
+  // the copies synchronous but stay correct.  A step with statistics needs one table, hence one chunk.
+  if (!h->host_streams[0]) {
+    for (int k = 0; k < 3; ++k) STQ_CUDA(h, cudaStreamCreateWithFlags(&h->host_streams[k], cudaStreamNonBlocking));
+  }
+  cudaStream_t s_in = h->host_streams[0], s_run = h->host_streams[1], s_out = h->host_streams[2];
+  STQ_CUDA(h, cudaDeviceSynchronize());   // earlier work on other streams may still use the arena or the buffers
   std::vector<stq_tensor> dev(tensors, tensors + L);
   uint64_t h2d = 0, d2h = 0;
   size_t off = 0;
   auto place = [&](size_t bytes) { uint8_t* p = h->d_arena + off; off += up(bytes); return p; };
-  for (int l = 0; l < L; ++l) {
-    const stq_tensor& t = tensors[l];
-    stq_tensor& d = dev[l];
-    const size_t sb = stq_scales_bytes(t.numel, t.block);
-    const size_t mi = stq_codes_bytes(t.numel, t.bits_m), vi = stq_codes_bytes(t.numel, t.bits_v);
-    d.param = reinterpret_cast<float*>(place(t.numel * 4));
-    d.grad = place(t.numel * gsz);
-    d.m_codes_in = place(mi);
-    d.v_codes_in = place(vi);
-    d.m_scales_in = reinterpret_cast<float*>(place(sb));
-    d.v_scales_in = reinterpret_cast<float*>(place(sb));
-    d.m_codes_out = t.bits_m_out != t.bits_m ? place(stq_codes_bytes(t.numel, t.bits_m_out))
-                                             : const_cast<void*>(d.m_codes_in);
-    d.v_codes_out = t.bits_v_out != t.bits_v ? place(stq_codes_bytes(t.numel, t.bits_v_out))
-                                             : const_cast<void*>(d.v_codes_in);
-    d.m_scales_out = const_cast<float*>(d.m_scales_in);
-    d.v_scales_out = const_cast<float*>(d.v_scales_in);
-    STQ_CUDA(h, cudaMemcpyAsync(d.param, t.param, t.numel * 4, cudaMemcpyHostToDevice, s));
-    STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.grad), t.grad, t.numel * gsz, cudaMemcpyHostToDevice, s));
-    STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.m_codes_in), t.m_codes_in, mi, cudaMemcpyHostToDevice, s));
-    STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.v_codes_in), t.v_codes_in, vi, cudaMemcpyHostToDevice, s));
-    h2d += t.numel * 4 + t.numel * gsz + mi + vi;
-    if (t.bits_m != 32) {
-      STQ_CUDA(h, cudaMemcpyAsync(const_cast<float*>(d.m_scales_in), t.m_scales_in, sb, cudaMemcpyHostToDevice, s));
-      h2d += sb;
+  const size_t chunk_bytes = (flags & STQ_WITH_STATS) ? ~size_t(0) : (size_t(256) << 20);
+  size_t n_events = 0;
+  auto next_event = [&](cudaEvent_t* ev) -> cudaError_t {
+    if (n_events == h->host_events.size()) {
+      cudaEvent_t e;
+      cudaError_t rc2 = cudaEventCreateWithFlags(&e, cudaEventDisableTiming);
+      if (rc2 != cudaSuccess) return rc2;
+      h->host_events.push_back(e);
     }
-    if (t.bits_v != 32) {
-      STQ_CUDA(h, cudaMemcpyAsync(const_cast<float*>(d.v_scales_in), t.v_scales_in, sb, cudaMemcpyHostToDevice, s));
-      h2d += sb;
+    *ev = h->host_events[n_events++];
+    return cudaSuccess;
+  };
+  int a = 0;
+  while (a < L) {
+    // ---- copies in (stream s_in) ----
+    size_t moved = 0;
+    int b = a;
+    for (; b < L && (b == a || moved < chunk_bytes); ++b) {
+      const stq_tensor& t = tensors[b];
+      stq_tensor& d = dev[b];
+      const size_t sb = stq_scales_bytes(t.numel, t.block);
+      const size_t mi = stq_codes_bytes(t.numel, t.bits_m), vi = stq_codes_bytes(t.numel, t.bits_v);
+      d.param = reinterpret_cast<float*>(place(t.numel * 4));
+      d.grad = place(t.numel * gsz);
+      d.m_codes_in = place(mi);
+      d.v_codes_in = place(vi);
+      d.m_scales_in = reinterpret_cast<float*>(place(sb));
+      d.v_scales_in = reinterpret_cast<float*>(place(sb));
+      d.m_codes_out = t.bits_m_out != t.bits_m ? place(stq_codes_bytes(t.numel, t.bits_m_out))
+                                               : const_cast<void*>(d.m_codes_in);
+      d.v_codes_out = t.bits_v_out != t.bits_v ? place(stq_codes_bytes(t.numel, t.bits_v_out))
+                                               : const_cast<void*>(d.v_codes_in);
+      d.m_scales_out = const_cast<float*>(d.m_scales_in);
+      d.v_scales_out = const_cast<float*>(d.v_scales_in);
+      STQ_CUDA(h, cudaMemcpyAsync(d.param, t.param, t.numel * 4, cudaMemcpyHostToDevice, s_in));
+      STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.grad), t.grad, t.numel * gsz, cudaMemcpyHostToDevice, s_in));
+      STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.m_codes_in), t.m_codes_in, mi, cudaMemcpyHostToDevice, s_in));
+      STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.v_codes_in), t.v_codes_in, vi, cudaMemcpyHostToDevice, s_in));
+      size_t bytes = t.numel * 4 + t.numel * gsz + mi + vi;
+      if (t.bits_m != 32) {
+        STQ_CUDA(h, cudaMemcpyAsync(const_cast<float*>(d.m_scales_in), t.m_scales_in, sb, cudaMemcpyHostToDevice, s_in));
+        bytes += sb;
+      }
+      if (t.bits_v != 32) {
+        STQ_CUDA(h, cudaMemcpyAsync(const_cast<float*>(d.v_scales_in), t.v_scales_in, sb, cudaMemcpyHostToDevice, s_in));
+        bytes += sb;
+      }
+      h2d += bytes;
+      moved += bytes;
     }
+    cudaEvent_t ev_in, ev_run;
+    STQ_CUDA(h, next_event(&ev_in));
+    STQ_CUDA(h, next_event(&ev_run));
+    STQ_CUDA(h, cudaEventRecord(ev_in, s_in));
+    // ---- the step on this chunk (stream s_run) ----
+    STQ_CUDA(h, cudaStreamWaitEvent(s_run, ev_in, 0));
+    rc = stq_step(h, dev.data() + a, b - a, hp, flags, s_run);
+    if (rc != STQ_OK) { cudaDeviceSynchronize(); return rc; }
+    STQ_CUDA(h, cudaEventRecord(ev_run, s_run));
+    // ---- copies out (stream s_out) ----
+    STQ_CUDA(h, cudaStreamWaitEvent(s_out, ev_run, 0));
+    for (int l = a; l < b; ++l) {
+      const stq_tensor& t = tensors[l];
+      const stq_tensor& d = dev[l];
+      const size_t sb = stq_scales_bytes(t.numel, t.block);
+      const size_t mo = stq_codes_bytes(t.numel, t.bits_m_out), vo = stq_codes_bytes(t.numel, t.bits_v_out);
+      STQ_CUDA(h, cudaMemcpyAsync(t.param, d.param, t.numel * 4, cudaMemcpyDeviceToHost, s_out));
+      STQ_CUDA(h, cudaMemcpyAsync(t.m_codes_out, d.m_codes_out, mo, cudaMemcpyDeviceToHost, s_out));
+      STQ_CUDA(h, cudaMemcpyAsync(t.v_codes_out, d.v_codes_out, vo, cudaMemcpyDeviceToHost, s_out));
+      d2h += t.numel * 4 + mo + vo;
+      if (t.bits_m_out != 32) {
+        STQ_CUDA(h, cudaMemcpyAsync(t.m_scales_out, d.m_scales_out, sb, cudaMemcpyDeviceToHost, s_out));
+        d2h += sb;
+      }
+      if (t.bits_v_out != 32) {
+        STQ_CUDA(h, cudaMemcpyAsync(t.v_scales_out, d.v_scales_out, sb, cudaMemcpyDeviceToHost, s_out));
+        d2h += sb;
+      }
+    }
+    a = b;
   }
-  rc = stq_step(h, dev.data(), L, hp, flags, s);
-  if (rc != STQ_OK) return rc;
-  for (int l = 0; l < L; ++l) {
-    const stq_tensor& t = tensors[l];
-    const stq_tensor& d = dev[l];
-    const size_t sb = stq_scales_bytes(t.numel, t.block);
-    const size_t mo = stq_codes_bytes(t.numel, t.bits_m_out), vo = stq_codes_bytes(t.numel, t.bits_v_out);
-    STQ_CUDA(h, cudaMemcpyAsync(t.param, d.param, t.numel * 4, cudaMemcpyDeviceToHost, s));
-    STQ_CUDA(h, cudaMemcpyAsync(t.m_codes_out, d.m_codes_out, mo, cudaMemcpyDeviceToHost, s));
-    STQ_CUDA(h, cudaMemcpyAsync(t.v_codes_out, d.v_codes_out, vo, cudaMemcpyDeviceToHost, s));
-    d2h += t.numel * 4 + mo + vo;
-    if (t.bits_m_out != 32) {
-      STQ_CUDA(h, cudaMemcpyAsync(t.m_scales_out, d.m_scales_out, sb, cudaMemcpyDeviceToHost, s));
-      d2h += sb;
-    }
-    if (t.bits_v_out != 32) {
-      STQ_CUDA(h, cudaMemcpyAsync(t.v_scales_out, d.v_scales_out, sb, cudaMemcpyDeviceToHost, s));
-      d2h += sb;
-    }
-  }
-  STQ_CUDA(h, cudaStreamSynchronize(s));
+  STQ_CUDA(h, cudaStreamSynchronize(s_out));
+  STQ_CUDA(h, cudaStreamSynchronize(s_run));
   // the cached table now refers to arena addresses; drop it so a later device call re-uploads
   h->cached_kind = -1;
   if (bytes_h2d) *bytes_h2d = h2d;

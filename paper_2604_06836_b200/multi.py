@@ -32,3 +32,18 @@ def aggregate_throughput(units_this_rank: float, ms_this_rank: float, device="cp
     (ms,) = max_over_ranks([ms_this_rank], device)
     (units,) = sum_over_ranks([units_this_rank], device)
     return units / (ms * 1e-3), ms
+
+
+def sync_layer_stats(stats, device="cpu"):
+    """Cross-rank aggregate of the per-layer gradient sums (the paper's "distributed engine" step).
+
+    stats: [L, 4] float64 rows {sum g, sum |g|, sum g^2, count} of this rank's local gradients, as
+    returned by ``stq_layer_stats``.  All four columns are sums over elements, so the job-wide
+    statistics are their sums over ranks; every rank then takes the same O(L) decision.  One
+    all-reduce of 4L doubles on decision steps only; identity without a process group."""
+    import numpy as np
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return np.asarray(stats, dtype=np.float64)
+    t = torch.as_tensor(np.ascontiguousarray(stats, dtype=np.float64), device=device).clone()
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return t.cpu().numpy()
