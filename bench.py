@@ -256,6 +256,29 @@ def run_ours(args, w, bits_m, bits_v):
     kern_ms = np.array([a.elapsed_time(b) for a, b in ev])
     is_dec = np.array(is_dec)
 
+    # ---- cost of the decision step in the paper's order (statistics before the update) ------------------
+    # Outside the timed region: the gradient-only pass, the fetch of the per-layer sums and the host
+    # decision, i.e. what Algorithm 1 adds every U steps (its O(N/K) overhead); the timed steps use the
+    # fused order, whose extra cost is kernel_ms_with_stats - kernel_ms_plain plus the same fetch.
+    tbl = job.table()
+    job.handle.grad_stats(tbl, job.grad_dtype)
+    job.layer_stats()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record(stream)
+    for _ in range(5):
+        job.handle.grad_stats(tbl, job.grad_dtype)
+    g1.record(stream)
+    torch.cuda.synchronize()
+    grad_stats_ms = g0.elapsed_time(g1) / 5
+    h0 = time.perf_counter()
+    st_ = job.layer_stats()
+    h1 = time.perf_counter()
+    pol.decide(st_, t + 1)
+    h2 = time.perf_counter()
+    job._tbl = None
+    decision = {"grad_stats_pass_ms": grad_stats_ms, "stats_fetch_ms": (h1 - h0) * 1e3,
+                "host_decide_ms": (h2 - h1) * 1e3, "tensors": job.L}
+
     # ---- end to end through the host-buffer entry point ----------------------------------------------
     e2e = None
     if not args.no_e2e:
@@ -288,6 +311,7 @@ def run_ours(args, w, bits_m, bits_v):
                      "kernel_ms_with_stats": float(kern_ms[is_dec].mean()) if is_dec.any() else None,
                      "frac_of_nominal_8000": achieved / 8000.0},
         "clocks": clocks,
+        "decision_step": decision,
         "gpu_launches": int(launches),
         "gpu_params_per_s_per_gpu": params * args.steps / (total_ms * 1e-3),
     }

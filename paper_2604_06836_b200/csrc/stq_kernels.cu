@@ -618,6 +618,70 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
   }
 }
 
+// Statistics alone (Algorithm 1 takes them before the update): a streaming reduction over the
+// gradients.  Same tile order and the same per-(tile, warp) partials as the fused path, so the
+// second stage is shared.  A warp owns 512 consecutive elements of the tile; a lane reads them as
+// 128-bit loads at a 512-byte warp stride.
+template <int GDT>
+__global__ void __launch_bounds__(kThreads)
+stq_grad_stats_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map,
+                      uint32_t tile_begin, uint32_t tile_end, double* __restrict__ partials) {
+  constexpr int kPerLoad = GDT == 0 ? 4 : 8;                 // elements per 128-bit load
+  constexpr int kLoads = (kTile / (kThreads / 32)) / (32 * kPerLoad);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (uint32_t tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
+    const TensorDesc* __restrict__ T = table + __ldg(tile_map + tile);
+    const unsigned long long numel = T->numel;
+    const unsigned long long e_warp = (unsigned long long)(T->nfast + (tile - T->tile0s)) * kTile +
+                                      (unsigned)warp * (kTile / (kThreads / 32));
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f;
+    uint4 raw[kLoads];
+    bool whole[kLoads];
+#pragma unroll
+    for (int j = 0; j < kLoads; ++j) {
+      const unsigned long long e = e_warp + (unsigned long long)(j * 32 + lane) * kPerLoad;
+      whole[j] = e + kPerLoad <= numel;
+      raw[j] = make_uint4(0u, 0u, 0u, 0u);
+      if (whole[j]) {
+        raw[j] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(T->grad) + e * (GDT == 0 ? 4 : 2)));
+      } else if (e < numel) {     // ragged end of the tensor: element by element
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        for (int k = 0; k < kPerLoad && e + k < numel; ++k) {
+          if constexpr (GDT == 0) w[k] = __float_as_uint(__ldg(reinterpret_cast<const float*>(T->grad) + e + k));
+          else w[k >> 1] |= (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(T->grad) + e + k) << (16 * (k & 1));
+        }
+        raw[j] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kLoads; ++j) {
+      const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if constexpr (GDT == 0) {
+          const float g = __uint_as_float(w[k]);
+          a0 += g; a1 += fabsf(g); a2 = __fmaf_rn(g, g, a2);
+        } else {
+          const float g0 = __uint_as_float(w[k] << 16), g1 = __uint_as_float(w[k] & 0xFFFF0000u);
+          a0 += g0; a1 += fabsf(g0); a2 = __fmaf_rn(g0, g0, a2);
+          a0 += g1; a1 += fabsf(g1); a2 = __fmaf_rn(g1, g1, a2);
+        }
+      }
+    }
+    // pairwise butterfly that spreads the three sums over the lanes on the way down
+    const bool hi = lane & 16;
+    float x = (hi ? a2 : a0) + __shfl_xor_sync(kFull, hi ? a0 : a2, 16);
+    float y = (hi ? 0.f : a1) + __shfl_xor_sync(kFull, hi ? a1 : 0.f, 16);
+    const bool q = lane & 8;
+    float z = (q ? y : x) + __shfl_xor_sync(kFull, q ? x : y, 8);
+    z += __shfl_xor_sync(kFull, z, 4);
+    z += __shfl_xor_sync(kFull, z, 2);
+    z += __shfl_xor_sync(kFull, z, 1);
+    if ((lane & 7) == 0 && lane < 24)
+      partials[((size_t)tile * (kThreads / 32) + warp) * 3 + (lane >> 3)] = (double)z;
+  }
+}
+
 // Statistics, second stage, step 1: one CTA per segment of kStatSegTiles tiles of one tensor.
 __global__ void __launch_bounds__(256)
 stq_stats_segment_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ seg_map, uint32_t n_seg,
@@ -712,10 +776,16 @@ cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const
       return launch_w<kRepack, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
     case kInit:
       return launch_w<kInit, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
-    case kStatsOnly:
-      return grad_dtype == 0
-                 ? launch_one<kStatsOnly, 0, true, false>(table, tile_map, tile_begin, tile_end, sc, partials, grid, stream)
-                 : launch_one<kStatsOnly, 1, true, false>(table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+    case kStatsOnly: {
+      const uint32_t n = tile_end - tile_begin;
+      const uint32_t want = (uint32_t)grid * 4u;   // small CTAs, 32 registers: many fit per SM
+      const int g = (int)(n < want ? n : want);
+      if (grad_dtype == 0)
+        stq_grad_stats_kernel<0><<<g, kThreads, 0, stream>>>(table, tile_map, tile_begin, tile_end, partials);
+      else
+        stq_grad_stats_kernel<1><<<g, kThreads, 0, stream>>>(table, tile_map, tile_begin, tile_end, partials);
+      return cudaGetLastError();
+    }
   }
   return cudaErrorInvalidValue;
 }
