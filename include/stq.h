@@ -166,6 +166,12 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
  * undefined and the handle should be destroyed. */
 int stq_device_status(stq_handle* h, void* stream);
 
+/* Exercises the time-out path without stalling anything: launches a one-warp kernel that waits, with
+ * a ~0.1 ms limit, on a barrier nothing completes, and raises the handle's error flag exactly as a
+ * stalled copy in the step kernel would.  Afterwards stq_device_status returns STQ_E_TIMEOUT for this
+ * handle (the flag is sticky); the CUDA context stays usable.  For tests of the failure reporting. */
+int stq_selftest_wait_timeout(stq_handle* h, void* stream);
+
 /* Kernel launches issued through this handle so far. */
 uint64_t stq_launch_count(const stq_handle* h);
 /* Persistent grid the step kernel uses on this device (CTAs), and the device's SM count. */

@@ -672,6 +672,15 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
   return STQ_OK;
 }
 
+int stq_selftest_wait_timeout(stq_handle* h, void* stream) {
+  if (!h) return STQ_E_NULL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  STQ_CUDA(h, cudaSetDevice(h->device));
+  STQ_CUDA(h, stq::launch_wait_timeout_selftest(h->d_err, s));
+  h->launches++;
+  return STQ_OK;
+}
+
 uint64_t stq_launch_count(const stq_handle* h) { return h ? h->launches : 0; }
 int stq_grid_size(const stq_handle* h) { return h ? h->fast_grid : 0; }
 int stq_sm_count(const stq_handle* h) { return h ? h->sm_count : 0; }

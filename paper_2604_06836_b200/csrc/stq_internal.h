@@ -74,6 +74,8 @@ cudaError_t launch_step_fast(int grad_dtype, bool stats, const TensorDesc* table
                              FastSched* sched, const StepConsts& sc, double* partials, int* err_flag, int grid,
                              cudaStream_t stream);
 int fast_ctas_per_sm();
+// Launches the time-out self-test (see stq_step_fast.cu): sets *err_flag after a ~0.1 ms bounded wait.
+cudaError_t launch_wait_timeout_selftest(int* err_flag, cudaStream_t stream);
 
 // Second stage of the statistics.  A tensor's tiles (fast range, then the rest) are cut into
 // segments of kStatSegTiles tiles; seg_map[s] is the tensor of segment s.  First every segment is

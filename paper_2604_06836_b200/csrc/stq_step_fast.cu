@@ -92,12 +92,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: returns false if the phase did not complete within kWaitCycles.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait: returns false if the phase did not complete within `limit` cycles.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitCycles) return false;
+    if (clock64() - t0 > limit) return false;
   }
   return true;
 }
@@ -635,6 +635,21 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
   }
 }
 
+// Self-test of the time-out path: one warp waits, with a short limit, on a barrier phase that nothing
+// will ever complete, finds the limit, raises the flag and returns.  The same code path a stalled
+// copy would take in the step kernel, without stalling anything.
+__global__ void stq_wait_timeout_selftest_kernel(int* __restrict__ err_flag, long long limit_cycles) {
+  __shared__ __align__(8) unsigned long long bar;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    mbar_init(b, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool done = mbar_wait(b, 0u, limit_cycles);
+  if (!done && threadIdx.x == 0) atomicExch(err_flag, 1);
+}
+
 template <int GDT>
 cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, FastSched* sched, const StepConsts& sc,
                           double* partials, int* err_flag, int grid, cudaStream_t stream) {
@@ -660,6 +675,11 @@ cudaError_t launch_step_fast(int grad_dtype, bool stats, const TensorDesc* table
   double* p = stats ? partials : nullptr;
   return grad_dtype == 0 ? launch_fast_t<0>(table, tile_map, sched, sc, p, err_flag, grid, stream)
                          : launch_fast_t<1>(table, tile_map, sched, sc, p, err_flag, grid, stream);
+}
+
+cudaError_t launch_wait_timeout_selftest(int* err_flag, cudaStream_t stream) {
+  stq_wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(err_flag, 200000ll);   // ~0.1 ms
+  return cudaGetLastError();
 }
 
 int fast_ctas_per_sm() {

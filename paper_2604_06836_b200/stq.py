@@ -79,6 +79,7 @@ def lib() -> C.CDLL:
         L.stq_step_host.argtypes = [vp, PT, C.c_int, C.POINTER(CHParams), C.c_uint,
                                     C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
         L.stq_device_status.argtypes = [vp, vp]
+        L.stq_selftest_wait_timeout.argtypes = [vp, vp]
         L.stq_grad_stats_static.argtypes = [C.c_int, vp, C.c_uint64, C.c_int, vp, vp]
         L.stq_launch_count.argtypes = [vp]
         L.stq_launch_count.restype = C.c_uint64
@@ -247,6 +248,10 @@ class Handle:
     def device_status(self, stream=None):
         """Synchronises the stream; raises if a kernel gave up on a bounded wait."""
         self._check(lib().stq_device_status(self._h, _stream_ptr(stream)), "stq_device_status")
+
+    def selftest_wait_timeout(self, stream=None):
+        """Runs the bounded-wait self-test; afterwards device_status() raises with code -11."""
+        self._check(lib().stq_selftest_wait_timeout(self._h, _stream_ptr(stream)), "stq_selftest_wait_timeout")
 
     @property
     def launch_count(self) -> int:

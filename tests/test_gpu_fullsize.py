@@ -145,3 +145,67 @@ def test_host_buffer_step_matches_device_step():
     for hs, s in zip(hstates, job.states):
         assert torch.equal(hs.m_codes, s.m_codes.cpu()) and torch.equal(hs.v_codes, s.v_codes.cpu())
         assert torch.equal(hs.m_scales, s.m_scales.cpu()) and torch.equal(hs.v_scales, s.v_scales.cpu())
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives():
+    """Every wait in the kernels is bounded; when one runs out the kernel raises a flag and returns.
+    The self-test takes that path with a 0.1 ms limit on a barrier nothing completes."""
+    from paper_2604_06836_b200 import stq
+    h = stq.Handle()
+    h.device_status()                                   # clean
+    h.selftest_wait_timeout()
+    with pytest.raises(stq.StqError) as ei:
+        h.device_status()
+    assert ei.value.code == -11
+    h.close()
+    # the context is alive and a fresh handle works
+    w = W.scaled(W.config("cfg2"), W.small_gpt2(d=72, n_layer=1, vocab=200), steps=1)
+    bm, bv, _ = W.draw_bits(w)
+    job = Job(w, bm, bv)
+    job.draw_grads(1)
+    job.step(1)
+    job.handle.device_status()
+    assert torch.isfinite(job.param_flat).all()
+
+
+def test_nothing_is_written_outside_the_callers_buffers():
+    """Every buffer sits between guard regions filled with a pattern; after init, steps with and
+    without a width change, and a re-pack, the guards are intact (ragged sizes, all widths)."""
+    from paper_2604_06836_b200 import stq
+    dev = "cuda"
+    G = 256   # guard bytes on each side
+    h = stq.Handle()
+
+    def guarded(nbytes):
+        buf = torch.full((nbytes + 2 * G,), 0xA5, dtype=torch.uint8, device=dev)
+        return buf, buf[G:G + nbytes]
+
+    def intact(buf, nbytes):
+        return bool((buf[:G] == 0xA5).all() and (buf[G + nbytes:] == 0xA5).all())
+
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
+    for n in (1, 129, 1000, 4097, 12289 + 77):
+        for (bm, bv, bm2, bv2) in [(3, 3, 3, 3), (2, 16, 8, 4), (8, 4, 32, 3), (16, 2, 2, 32)]:
+            bufs = {}
+            def mk(name, nbytes):
+                bufs[name] = guarded(nbytes) + (nbytes,)
+                return bufs[name][1]
+            p = mk("p", _r16(4 * n)).view(torch.float32)[:n]
+            g = mk("g", _r16(4 * n)).view(torch.float32)[:n]
+            p.normal_(0, 0.02); g.normal_(0, 1e-3)
+            sb = stq.scales_bytes(n, 128)
+            def state(tag, a, b):
+                return stq.QState(mk(tag + "mc", stq.codes_bytes(n, a)), mk(tag + "ms", _r16(sb)).view(torch.float32)[:sb // 4], a,
+                                  mk(tag + "vc", stq.codes_bytes(n, b)), mk(tag + "vs", _r16(sb)).view(torch.float32)[:sb // 4], b)
+            s1, s2, s3 = state("a", bm, bv), state("b", bm2, bv2), state("c", bm, bv)
+            h.init_state(stq.table([stq.make_row(n, 128, None, s1)]))
+            h.step(stq.table([stq.make_row(n, 128, s1, s1, p, g, 0.01)]), t=1, **hp)            # in place
+            h.step(stq.table([stq.make_row(n, 128, s1, s2, p, g, 0.01)]), t=2, **hp)            # width change in the step
+            h.repack(stq.table([stq.make_row(n, 128, s2, s3)]))                                  # and back by re-pack
+            h.device_status()
+            for name, (buf, _, nbytes) in bufs.items():
+                assert intact(buf, nbytes), (n, bm, bv, bm2, bv2, name)
+
+
+def _r16(x):
+    return (x + 15) // 16 * 16
