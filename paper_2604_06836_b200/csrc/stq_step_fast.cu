@@ -653,15 +653,12 @@ __global__ void stq_wait_timeout_selftest_kernel(int* __restrict__ err_flag, lon
 template <int GDT>
 cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, FastSched* sched, const StepConsts& sc,
                           double* partials, int* err_flag, int grid, cudaStream_t stream) {
-  static bool attr_set = false;
   auto kern = stq_step_fast_kernel<GDT>;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  // per device and cheap, so simply repeated: the kernel needs more than the default 48 KB
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e != cudaSuccess) return e;
   // the group counters start every launch at zero
-  cudaError_t e = cudaMemsetAsync(sched, 0, sizeof(uint32_t) * kFastMaxGroups, stream);
+  e = cudaMemsetAsync(sched, 0, sizeof(uint32_t) * kFastMaxGroups, stream);
   if (e != cudaSuccess) return e;
   kern<<<grid, kFastThreads, kSmemBytes, stream>>>(table, tile_map, sched, sc, partials, err_flag);
   return cudaGetLastError();
