@@ -179,17 +179,35 @@ class SampledOracle:
         idx = np.concatenate([blocks, [nb_full]]) if tail else blocks
         return to_np(scales[torch.from_numpy(idx).to(scales.device)])
 
-    def step(self, t: int):
-        """Oracle step on the sample, with the gradients currently held by the job."""
+    def step(self, t: int, new_bits=None):
+        """Oracle step on the sample, with the gradients currently held by the job.  new_bits =
+        (bits_m, bits_v) arrays switches widths inside the step."""
         w = self.job.w
         for i in range(self.job.L):
             if self.n_mini[i] == 0:
                 continue
             g = self._gather_elems(self.job.grads[i], i)
             before = self.theta[i].copy()
+            bm = None if new_bits is None else int(new_bits[0][i])
+            bv = None if new_bits is None else int(new_bits[1][i])
             self.states[i], _ = O.step(self.theta[i], g, self.states[i], self.block, lr=w.lr, beta1=w.beta1,
-                                       beta2=w.beta2, eps=w.eps, weight_decay=self.job.wd[i], t=t)
+                                       beta2=w.beta2, eps=w.eps, weight_decay=self.job.wd[i], t=t,
+                                       bits_m_out=bm, bits_v_out=bv)
             self.mag[i] = np.maximum(self.mag[i], np.maximum(np.abs(self.theta[i]), np.abs(self.theta[i] - before)))
+
+    def repack(self, new_bits):
+        """Width transition between steps on the sampled blocks."""
+        for i in range(self.job.L):
+            st, n = self.states[i], self.n_mini[i]
+            if n == 0:
+                continue
+            bm, bv = int(new_bits[0][i]), int(new_bits[1][i])
+            if bm != st.bits_m:
+                st.m_codes, st.m_scales = O.repack(st.m_codes, st.m_scales, st.bits_m, bm, n, self.block, O.LINEAR)
+                st.bits_m = bm
+            if bv != st.bits_v:
+                st.v_codes, st.v_scales = O.repack(st.v_codes, st.v_scales, st.bits_v, bv, n, self.block, O.LOG)
+                st.bits_v = bv
 
     def compare(self, rel: float, tag=""):
         job = self.job
