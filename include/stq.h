@@ -25,6 +25,7 @@
  *    flattened tensor (last block short), stq_scales_bytes(numel, block) bytes.
  *  - width 32: the codes buffer holds the raw fp32 values (numel*4 rounded up to 16 bytes); the
  *    scale pointers are ignored and may be NULL.
+ *  - gradients: fp32, bf16 or fp16, one type per call.
  *  - first moment: code u = q + 2^(b-1), q in [-qmax, qmax], qmax = 2^(b-1)-1, value scale*q/qmax.
  *  - second moment: code u in [0, 2^b-1]; value scale * 2^((u-K)*R/K), K = 2^b-1, R = min(K,30);
  *    code 0 is a floor level, never zero.  A block whose scale is 0 decodes to all zeros.
@@ -59,7 +60,10 @@ enum {
                         /* not allocate (stq_grad_stats_static)                               */
 };
 
-enum { STQ_GRAD_F32 = 0, STQ_GRAD_BF16 = 1 };
+enum { STQ_GRAD_F32 = 0, STQ_GRAD_BF16 = 1, STQ_GRAD_F16 = 2 };
+
+/* type of the optional low-precision copy of the updated parameters (stq_tensor.param_lp) */
+enum { STQ_LP_NONE = 0, STQ_LP_BF16 = 1, STQ_LP_F16 = 2 };
 
 /* flags of stq_step */
 enum { STQ_WITH_STATS = 1u };
@@ -81,14 +85,23 @@ typedef struct stq_tensor {
   uint8_t bits_m, bits_v;          /* widths stored now                                        */
   uint8_t bits_m_out, bits_v_out;  /* widths to write                                          */
   float weight_decay;        /* per-tensor lambda                                              */
-  uint32_t reserved;         /* must be 0                                                      */
+  uint32_t lp_dtype;         /* STQ_LP_*: type of param_lp (STQ_LP_NONE: no copy)              */
+  void* param_lp;            /* optional: numel elements that receive the updated parameters   */
+                             /* rounded (nearest-even) to lp_dtype, the model's working copy   */
+                             /* in mixed-precision training; 8-byte aligned; written by         */
+                             /* stq_step only                                                  */
 } stq_tensor;
 
 typedef struct stq_hparams {
   double lr, beta1, beta2, eps;
   int64_t step;          /* t >= 1: the step being taken (bias correction 1 - beta^t)          */
   int32_t decoupled_wd;  /* 1: AdamW as in Algorithm 1; 0: weight decay added to the gradient  */
-  int32_t grad_dtype;    /* STQ_GRAD_F32 or STQ_GRAD_BF16                                      */
+  int32_t grad_dtype;    /* STQ_GRAD_F32, STQ_GRAD_BF16 or STQ_GRAD_F16                        */
+  /* Loss-scaled training (the paper trains in FP16): both are DEVICE pointers to one float, or NULL. */
+  const float* inv_grad_scale; /* every gradient is multiplied by *inv_grad_scale (1 / loss scale)   */
+                               /* before anything else (statistics included)                         */
+  const float* found_inf;      /* if *found_inf != 0 the step is skipped: no buffer is touched, and   */
+                               /* statistics requested with the step are not produced                */
 } stq_hparams;
 
 /* Handle: device copy of the tensor table, tile map and statistics workspace.

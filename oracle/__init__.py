@@ -33,7 +33,7 @@ def build(force: bool = False) -> str:
 class HParams(C.Structure):
     _fields_ = [("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
                 ("weight_decay", C.c_double), ("step", C.c_int64), ("decoupled_wd", C.c_int),
-                ("grad_dtype", C.c_int)]
+                ("grad_dtype", C.c_int), ("inv_grad_scale", C.c_float), ("found_inf", C.c_int)]
 
 
 class Policy(C.Structure):
@@ -72,6 +72,10 @@ def lib():
                                vp, vp, C.c_int, vp, vp, C.c_int,
                                C.POINTER(HParams), vp]
         L.orc_repack.argtypes = [vp, vp, C.c_int, vp, vp, C.c_int, C.c_uint64, C.c_uint32, C.c_int]
+        L.orc_round_lp.argtypes = [vp, C.c_uint64, C.c_int, vp]
+        L.orc_round_lp.restype = None
+        L.orc_widen_f16.argtypes = [vp, C.c_uint64, vp]
+        L.orc_widen_f16.restype = None
         L.orc_is_decision_step.argtypes = [C.c_int64, C.c_int64]
         L.orc_decide.argtypes = [C.POINTER(Policy), vp, C.c_int, C.c_int64, vp, vp]
         L.orc_decide.restype = None
@@ -157,11 +161,16 @@ def init_state(n: int, block: int, bits_m: int, bits_v: int):
     return mc, ms, vc, vs
 
 
-def grad_stats(grad: np.ndarray) -> np.ndarray:
-    """grad: float32, or uint16 holding bf16 bit patterns."""
-    dt = 1 if grad.dtype == np.uint16 else 0
-    if dt == 0:
-        _chk(grad, np.float32)
+def _grad_dtype(grad: np.ndarray, fp16: bool) -> int:
+    if grad.dtype == np.uint16:
+        return 2 if fp16 else 1
+    _chk(grad, np.float32)
+    return 0
+
+
+def grad_stats(grad: np.ndarray, fp16: bool = False) -> np.ndarray:
+    """grad: float32, or uint16 holding bf16 (default) or fp16 (fp16=True) bit patterns."""
+    dt = _grad_dtype(grad, fp16)
     out = np.zeros(4, dtype=np.float64)
     lib().orc_grad_stats(_p(grad), dt, grad.size, _p(out))
     return out
@@ -185,19 +194,21 @@ def new_state(n: int, block: int, bits_m: int, bits_v: int) -> State:
 
 def step(theta: np.ndarray, grad: np.ndarray, st: State, block: int, *, lr, beta1, beta2, eps,
          weight_decay, t: int, bits_m_out: int | None = None, bits_v_out: int | None = None,
-         decoupled_wd: bool = True, want_stats: bool = False):
-    """One Algorithm-1 step on one tensor.  theta is updated in place; returns (new State, stats)."""
+         decoupled_wd: bool = True, want_stats: bool = False, fp16_grad: bool = False,
+         inv_grad_scale: float = 1.0, found_inf: bool = False):
+    """One Algorithm-1 step on one tensor.  theta is updated in place; returns (new State, stats).
+    A uint16 grad holds bf16 bit patterns, or fp16 ones with fp16_grad=True."""
     _chk(theta, np.float32)
     n = theta.size
-    dt = 1 if grad.dtype == np.uint16 else 0
-    if dt == 0:
-        _chk(grad, np.float32)
+    dt = _grad_dtype(grad, fp16_grad)
     assert grad.size == n
+    if found_inf:
+        return st, (np.zeros(4) if want_stats else None)
     bm = st.bits_m if bits_m_out is None else bits_m_out
     bv = st.bits_v if bits_v_out is None else bits_v_out
     mc, ms = alloc_state(n, bm, block)
     vc, vs = alloc_state(n, bv, block)
-    hp = HParams(lr, beta1, beta2, eps, weight_decay, t, 1 if decoupled_wd else 0, dt)
+    hp = HParams(lr, beta1, beta2, eps, weight_decay, t, 1 if decoupled_wd else 0, dt, inv_grad_scale, 0)
     stats = np.zeros(4, dtype=np.float64) if want_stats else None
     rc = lib().orc_step(_p(theta), _p(grad), n, block,
                         _p(st.m_codes), _p(st.m_scales), st.bits_m,
@@ -205,6 +216,21 @@ def step(theta: np.ndarray, grad: np.ndarray, st: State, block: int, *, lr, beta
                         _p(mc), _p(ms), bm, _p(vc), _p(vs), bv, C.byref(hp), _p(stats))
     assert rc == 0
     return State(mc, ms, bm, vc, vs, bv), stats
+
+
+def round_lp(x: np.ndarray, lp: str) -> np.ndarray:
+    """Nearest-even rounding of fp32 values to "bf16" or "fp16"; returns the uint16 bit patterns."""
+    x = _chk(np.ascontiguousarray(x), np.float32)
+    out = np.zeros(x.size, dtype=np.uint16)
+    lib().orc_round_lp(_p(x), x.size, 1 if lp == "bf16" else 2, _p(out))
+    return out
+
+
+def widen_f16(bits: np.ndarray) -> np.ndarray:
+    _chk(bits, np.uint16)
+    out = np.zeros(bits.size, dtype=np.float32)
+    lib().orc_widen_f16(_p(bits), bits.size, _p(out))
+    return out
 
 
 def repack(codes: np.ndarray, scales: np.ndarray, bits_in: int, bits_out: int, n: int, block: int,

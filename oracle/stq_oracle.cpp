@@ -201,6 +201,44 @@ void encode_state(const float* x, uint64_t n, int b, uint32_t block, int mode, u
 
 inline float bf16_to_f32(uint16_t h) { return u2f((uint32_t)h << 16); }
 
+// IEEE binary16 -> binary32 (exact).
+inline float f16_to_f32(uint16_t h) {
+  const uint32_t sign = (uint32_t)(h & 0x8000u) << 16;
+  const int e = (h >> 10) & 0x1F;
+  const uint32_t m = h & 0x3FFu;
+  if (e == 0) {                       // zero or subnormal: m * 2^-24
+    const float v = (float)m * 0x1p-24f;
+    return u2f(f2u(v) | sign);
+  }
+  if (e == 31) return u2f(sign | 0x7F800000u | (m << 13));
+  return u2f(sign | ((uint32_t)(e + 112) << 23) | (m << 13));
+}
+
+// binary32 -> bfloat16 / binary16, round to nearest even (finite inputs).
+inline uint16_t f32_to_bf16(float x) {
+  const uint32_t u = f2u(x);
+  return (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+}
+inline uint16_t f32_to_f16(float x) {
+  const uint32_t u = f2u(x);
+  const uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+  const float a = std::fabs(x);
+  if (a >= 65520.0f) return sign | 0x7C00u;                 // rounds to infinity
+  if (a < 0x1p-14f) {                                        // subnormal half: multiples of 2^-24
+    const double q = std::nearbyint((double)a * 0x1p24);     // exact scaling, ties to even
+    return sign | (uint16_t)q;                               // 1024 is the smallest normal: carries over correctly
+  }
+  const uint32_t au = f2u(a);
+  const uint32_t rounded = au + 0xFFFu + ((au >> 13) & 1u);  // 13 mantissa bits dropped
+  return sign | (uint16_t)(((rounded >> 13) - (112u << 10)) & 0x7FFFu);
+}
+
+inline float grad_to_f32(const void* grad, int dtype, uint64_t i) {
+  if (dtype == 1) return bf16_to_f32(((const uint16_t*)grad)[i]);
+  if (dtype == 2) return f16_to_f32(((const uint16_t*)grad)[i]);
+  return ((const float*)grad)[i];
+}
+
 }  // namespace
 
 extern "C" {
@@ -209,7 +247,9 @@ struct orc_hparams {
   double lr, beta1, beta2, eps, weight_decay;
   int64_t step;        // t >= 1, the step being taken
   int decoupled_wd;    // 1 = AdamW (Algorithm 1); 0 = L2 term added to the gradient
-  int grad_dtype;      // 0 = fp32, 1 = bf16
+  int grad_dtype;      // 0 = fp32, 1 = bf16, 2 = fp16
+  float inv_grad_scale;  // loss-scaled training: every gradient is multiplied by this first (1 = off)
+  int found_inf;         // non-zero: a non-finite gradient was found, the step is skipped
 };
 
 uint64_t orc_codes_bytes(uint64_t n, int bits) { return codes_bytes(n, bits); }
@@ -254,7 +294,7 @@ int orc_init_state(uint64_t n, uint32_t block, int bits_m, int bits_v, uint8_t* 
 void orc_grad_stats(const void* grad, int grad_dtype, uint64_t n, double out[4]) {
   double sg = 0, sa = 0, sq = 0;
   for (uint64_t i = 0; i < n; ++i) {
-    float g = grad_dtype == 1 ? bf16_to_f32(((const uint16_t*)grad)[i]) : ((const float*)grad)[i];
+    float g = grad_to_f32(grad, grad_dtype, i);
     double gd = (double)g;
     sg += gd; sa += fabs(gd); sq += gd * gd;
   }
@@ -273,16 +313,16 @@ int orc_step(float* theta, const void* grad, uint64_t n, uint32_t block,
   if (!width_ok(bits_m_in) || !width_ok(bits_v_in) || !width_ok(bits_m_out) || !width_ok(bits_v_out))
     return -1;
   if (block == 0 || hp->step < 1) return -1;
+  if (hp->found_inf) return 0;          // skipped step: nothing is touched
   std::vector<float> m(n), v(n), g(n);
 
   // stored m_{t-1}, v_{t-1}
   decode_state(m_codes_in, m_scales_in, n, bits_m_in, block, 0, m.data());
   decode_state(v_codes_in, v_scales_in, n, bits_v_in, block, 1, v.data());
 
-  // gradient as fp32 (bf16 widens exactly)
-  for (uint64_t i = 0; i < n; ++i)
-    g[i] = hp->grad_dtype == 1 ? bf16_to_f32(((const uint16_t*)grad)[i]) : ((const float*)grad)[i];
-  if (stats) orc_grad_stats(grad, hp->grad_dtype, n, stats);
+  // gradient as fp32 (bf16 and fp16 widen exactly), brought back from the loss scale
+  for (uint64_t i = 0; i < n; ++i) g[i] = grad_to_f32(grad, hp->grad_dtype, i) * hp->inv_grad_scale;
+  if (stats) orc_grad_stats(g.data(), 0, n, stats);
   if (!hp->decoupled_wd) {
     const float wd = (float)hp->weight_decay;
     for (uint64_t i = 0; i < n; ++i) { float l2 = wd * theta[i]; g[i] = g[i] + l2; }
@@ -320,6 +360,14 @@ int orc_step(float* theta, const void* grad, uint64_t n, uint32_t block,
     theta[i] = (float)th;
   }
   return 0;
+}
+
+// Low-precision working copy of the parameters: nearest-even rounding to bf16 (1) or fp16 (2).
+void orc_round_lp(const float* x, uint64_t n, int lp_dtype, uint16_t* out) {
+  for (uint64_t i = 0; i < n; ++i) out[i] = lp_dtype == 1 ? f32_to_bf16(x[i]) : f32_to_f16(x[i]);
+}
+void orc_widen_f16(const uint16_t* x, uint64_t n, float* out) {
+  for (uint64_t i = 0; i < n; ++i) out[i] = f16_to_f32(x[i]);
 }
 
 // Width transition: codes' = Q_{b'}(D_b(codes)), block scales recomputed from the decoded values

@@ -32,6 +32,7 @@ struct stq_handle {
   size_t d_tile_cap = 0;
   uint32_t n_tiles = 0, n_fast = 0, n_narrow = 0;   // n_narrow counts fast + remaining narrow
   int fast_grid = 0;
+  bool any_lp = false;              // some tensor of the current table wants a low-precision copy
   int* d_err = nullptr;             // raised by a kernel whose bounded wait ran out
   stq::FastSched* d_sched = nullptr;   // work list of the main step kernel
 
@@ -114,7 +115,11 @@ bool overlap(const void* a, size_t na, const void* b, size_t nb) {
 // Host-side validation of one row for the given entry point.
 int validate_row(const stq_tensor& t, int kind) {
   if (t.numel == 0 || t.numel > (1ull << 40)) return STQ_E_NUMEL;
-  if (t.reserved != 0) return STQ_E_ARG;
+  if (t.lp_dtype > STQ_LP_F16) return STQ_E_ARG;
+  if (kind == kKindStep && t.lp_dtype != STQ_LP_NONE) {
+    if (!t.param_lp) return STQ_E_NULL;
+    if (!aligned(t.param_lp, 8)) return STQ_E_ALIGN;
+  }
   if (kind == kKindStats) {
     if (!t.grad) return STQ_E_NULL;
     if (!aligned(t.grad, 16)) return STQ_E_ALIGN;
@@ -324,6 +329,8 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     d.block = kind == kKindStats ? 128u : t.block;
     d.bm_in = t.bits_m; d.bv_in = t.bits_v; d.bm_out = t.bits_m_out; d.bv_out = t.bits_v_out;
     d.wd = t.weight_decay;
+    d.lp_dtype = kind == kKindStep ? t.lp_dtype : 0u;
+    d.param_lp = kind == kKindStep && t.lp_dtype != STQ_LP_NONE ? t.param_lp : nullptr;
     ht[l] = d;
   }
   STQ_CUDA(h, cudaMemcpyAsync(h->d_table, ht, bytes_table, cudaMemcpyHostToDevice, stream));
@@ -338,6 +345,8 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   h->cached.assign(tensors, tensors + L);
   h->cached_kind = kind;
   h->cached_sig.swap(sig);
+  h->any_lp = false;
+  for (int l = 0; l < L; ++l) h->any_lp = h->any_lp || (kind == kKindStep && tensors[l].lp_dtype != STQ_LP_NONE);
   h->n_tiles = (uint32_t)total;
   h->n_fast = (uint32_t)fast;
   h->n_narrow = (uint32_t)(fast + slow_narrow);
@@ -353,7 +362,8 @@ int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::St
     partials = h->d_partials;
   }
   if (h->n_fast > 0) {   // only a step table has fast tiles
-    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, h->d_table, h->d_tile_map, h->d_sched, sc, partials,
+    const bool amp = h->any_lp || sc.inv_scale != nullptr;
+    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, amp, h->d_table, h->d_tile_map, h->d_sched, sc, partials,
                                       h->d_err, h->fast_grid, stream));
     h->launches++;
   }
@@ -373,8 +383,9 @@ int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::St
 int check_hparams(const stq_hparams* hp, unsigned flags) {
   if (!hp) return STQ_E_NULL;
   if (hp->step < 1) return STQ_E_ARG;
-  if (hp->grad_dtype != STQ_GRAD_F32 && hp->grad_dtype != STQ_GRAD_BF16) return STQ_E_ARG;
+  if (hp->grad_dtype < STQ_GRAD_F32 || hp->grad_dtype > STQ_GRAD_F16) return STQ_E_ARG;
   if (flags & ~(unsigned)STQ_WITH_STATS) return STQ_E_ARG;
+  if (!aligned(hp->inv_grad_scale, 4) || !aligned(hp->found_inf, 4)) return STQ_E_ALIGN;
   if (!(hp->beta1 >= 0.0 && hp->beta1 < 1.0 && hp->beta2 >= 0.0 && hp->beta2 < 1.0)) return STQ_E_ARG;
   return STQ_OK;
 }
@@ -392,6 +403,8 @@ stq::StepConsts make_consts(const stq_hparams* hp) {
   sc.eps = (float)hp->eps;
   sc.l2_mode = hp->decoupled_wd ? 0 : 1;
   sc.lr = hp->lr;
+  sc.inv_scale = hp->inv_grad_scale;
+  sc.found_inf = hp->found_inf;
   return sc;
 }
 
@@ -487,7 +500,7 @@ int stq_step(stq_handle* h, const stq_tensor* tensors, int L, const stq_hparams*
 
 int stq_grad_stats(stq_handle* h, const stq_tensor* tensors, int L, int grad_dtype, void* stream) {
   if (!h) return STQ_E_NULL;
-  if (grad_dtype != STQ_GRAD_F32 && grad_dtype != STQ_GRAD_BF16) return STQ_E_ARG;
+  if (grad_dtype < STQ_GRAD_F32 || grad_dtype > STQ_GRAD_F16) return STQ_E_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int rc = prepare(h, tensors, L, kKindStats, s);
   if (rc != STQ_OK) return rc;
@@ -557,7 +570,7 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
   }
   // lay the device arena out: every buffer 256-byte aligned
   auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
-  const size_t gsz = hp->grad_dtype == STQ_GRAD_BF16 ? 2 : 4;
+  const size_t gsz = hp->grad_dtype == STQ_GRAD_F32 ? 4 : 2;
   size_t need = 0;
   for (int l = 0; l < L; ++l) {
     const stq_tensor& t = tensors[l];
@@ -566,7 +579,9 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
     need += up(stq_codes_bytes(t.numel, t.bits_m)) + up(stq_codes_bytes(t.numel, t.bits_v)) + 2 * up(sb);
     if (t.bits_m_out != t.bits_m) need += up(stq_codes_bytes(t.numel, t.bits_m_out));
     if (t.bits_v_out != t.bits_v) need += up(stq_codes_bytes(t.numel, t.bits_v_out));
+    if (t.lp_dtype != STQ_LP_NONE) need += up(t.numel * 2);
   }
+  if (hp->inv_grad_scale || hp->found_inf) return STQ_E_ARG;   // device pointers have no place in the host-buffer call
   rc = grow(h, h->d_arena, h->d_arena_cap, need);
   if (rc != STQ_OK) return rc;
 
@@ -616,6 +631,7 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
                                                : const_cast<void*>(d.v_codes_in);
       d.m_scales_out = const_cast<float*>(d.m_scales_in);
       d.v_scales_out = const_cast<float*>(d.v_scales_in);
+      if (t.lp_dtype != STQ_LP_NONE) d.param_lp = place(t.numel * 2);
       STQ_CUDA(h, cudaMemcpyAsync(d.param, t.param, t.numel * 4, cudaMemcpyHostToDevice, s_in));
       STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.grad), t.grad, t.numel * gsz, cudaMemcpyHostToDevice, s_in));
       STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.m_codes_in), t.m_codes_in, mi, cudaMemcpyHostToDevice, s_in));
@@ -652,6 +668,10 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
       STQ_CUDA(h, cudaMemcpyAsync(t.m_codes_out, d.m_codes_out, mo, cudaMemcpyDeviceToHost, s_out));
       STQ_CUDA(h, cudaMemcpyAsync(t.v_codes_out, d.v_codes_out, vo, cudaMemcpyDeviceToHost, s_out));
       d2h += t.numel * 4 + mo + vo;
+      if (t.lp_dtype != STQ_LP_NONE) {
+        STQ_CUDA(h, cudaMemcpyAsync(t.param_lp, d.param_lp, t.numel * 2, cudaMemcpyDeviceToHost, s_out));
+        d2h += t.numel * 2;
+      }
       if (t.bits_m_out != 32) {
         STQ_CUDA(h, cudaMemcpyAsync(t.m_scales_out, d.m_scales_out, sb, cudaMemcpyDeviceToHost, s_out));
         d2h += sb;

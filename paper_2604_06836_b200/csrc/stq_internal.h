@@ -36,6 +36,8 @@ struct TensorDesc {
   unsigned int block;       // 128 / 256 / 512
   unsigned char bm_in, bv_in, bm_out, bv_out;
   float wd;                 // fp32(lambda)
+  unsigned int lp_dtype;    // 0: none, 1: bf16, 2: fp16
+  void* param_lp;           // low-precision copy of the updated parameters, or nullptr
 };
 
 // Per-launch scalars of the AdamW update.
@@ -46,6 +48,8 @@ struct StepConsts {
   float eps;
   int l2_mode;              // 1: g += wd*theta before the moments, no decoupled decay
   double lr;                // decoupled decay factor is fp32(1 - lr*wd), formed per tile
+  const float* inv_scale;   // device: gradients are multiplied by *inv_scale first (nullptr: no)
+  const float* found_inf;   // device: a non-zero value skips the whole step (nullptr: never)
 };
 
 enum Mode { kStep = 0, kRepack = 1, kInit = 2, kStatsOnly = 3 };
@@ -70,7 +74,8 @@ struct FastSched {
 
 // The main step kernel (stq_step_fast.cu) with `grid` CTAs.  err_flag is set to 1 if a bounded wait
 // inside the kernel ran out.
-cudaError_t launch_step_fast(int grad_dtype, bool stats, const TensorDesc* table, const uint32_t* tile_map,
+// amp: some tensor wants a low-precision copy, or the gradients are loss-scaled.
+cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, const TensorDesc* table, const uint32_t* tile_map,
                              FastSched* sched, const StepConsts& sc, double* partials, int* err_flag, int grid,
                              cudaStream_t stream);
 int fast_ctas_per_sm();

@@ -17,6 +17,9 @@
 // defined with them.  Round-half-even to integer is done by adding 1.5*2^23 (one FFMA on the exact
 // product), and the integer sits in the low mantissa bits of the result, which is also how the
 // codes are packed: sum_k bits_k << (k*b) minus a per-width constant.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
 #include "stq_internal.h"
 
 namespace stq {
@@ -278,6 +281,8 @@ template <>
 struct GradRow<0> { float4 v; };
 template <>
 struct GradRow<1> { uint2 v; };
+template <>
+struct GradRow<2> { uint2 v; };
 
 template <int GDT>
 __device__ __forceinline__ void load_grad(const void* grad, unsigned long long e, int nvl, GradRow<GDT>& g) {
@@ -308,11 +313,39 @@ template <int GDT>
 __device__ __forceinline__ void widen_grad(const GradRow<GDT>& g, float (&o)[4]) {
   if constexpr (GDT == 0) {
     o[0] = g.v.x; o[1] = g.v.y; o[2] = g.v.z; o[3] = g.v.w;
-  } else {
+  } else if constexpr (GDT == 1) {
     o[0] = __uint_as_float(g.v.x << 16);
     o[1] = __uint_as_float(g.v.x & 0xFFFF0000u);
     o[2] = __uint_as_float(g.v.y << 16);
     o[3] = __uint_as_float(g.v.y & 0xFFFF0000u);
+  } else {
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&g.v.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&g.v.y));
+    o[0] = a.x; o[1] = a.y; o[2] = b.x; o[3] = b.y;
+  }
+}
+
+// The low-precision copy of up to four updated parameters (nearest-even rounding).
+__device__ __forceinline__ void store_param_lp(void* lp, unsigned lp_dtype, unsigned long long e, int nvl,
+                                               const float (&x)[4]) {
+  uint16_t h[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    if (lp_dtype == 1u) {
+      const __nv_bfloat16 b = __float2bfloat16_rn(x[k]);
+      h[k] = *reinterpret_cast<const uint16_t*>(&b);
+    } else {
+      const __half b = __float2half_rn(x[k]);
+      h[k] = *reinterpret_cast<const uint16_t*>(&b);
+    }
+  }
+  uint16_t* p = reinterpret_cast<uint16_t*>(lp) + e;
+  if (nvl == 4) {
+    *reinterpret_cast<uint2*>(p) = make_uint2(h[0] | ((uint32_t)h[1] << 16), h[2] | ((uint32_t)h[3] << 16));
+  } else {
+    if (nvl > 0) p[0] = h[0];
+    if (nvl > 1) p[1] = h[1];
+    if (nvl > 2) p[2] = h[2];
   }
 }
 
@@ -343,6 +376,12 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
   constexpr bool kHasGrad = (MODE == kStep || MODE == kStatsOnly);
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
+  float grad_mul = 1.0f;
+  if constexpr (MODE == kStep) {
+    // a non-finite gradient somewhere in the model: the whole step is skipped
+    if (sc.found_inf != nullptr && __ldg(sc.found_inf) != 0.0f) return;
+    if (sc.inv_scale != nullptr) grad_mul = __ldg(sc.inv_scale);
+  }
 
   for (uint32_t tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
     const TensorDesc* __restrict__ T = table + __ldg(tile_map + tile);
@@ -452,6 +491,10 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
               th[r][0] = th4[r].x; th[r][1] = th4[r].y; th[r][2] = th4[r].z; th[r][3] = th4[r].w;
               float g[4];
               widen_grad<GDT>(graw[r], g);
+              if (sc.inv_scale != nullptr) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) g[k] = __fmul_rn(g[k], grad_mul);
+              }
 #pragma unroll
               for (int k = 0; k < 4; ++k) {
                 if constexpr (STATS) {
@@ -596,6 +639,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
               out[k] = __fadd_rn(th[r][k], -__fmaf_rn(th[r][k], lrwd, upd));
             }
             store_param(param + e_row + 4 * lane, nvl[r], out);
+            if (T->param_lp != nullptr) store_param_lp(T->param_lp, T->lp_dtype, e_row + 4 * lane, nvl[r], out);
           }
         }
       }
@@ -662,7 +706,15 @@ stq_grad_stats_kernel(const TensorDesc* __restrict__ table, const uint32_t* __re
           const float g = __uint_as_float(w[k]);
           a0 += g; a1 += fabsf(g); a2 = __fmaf_rn(g, g, a2);
         } else {
-          const float g0 = __uint_as_float(w[k] << 16), g1 = __uint_as_float(w[k] & 0xFFFF0000u);
+          float g0, g1;
+          if constexpr (GDT == 1) {
+            g0 = __uint_as_float(w[k] << 16);
+            g1 = __uint_as_float(w[k] & 0xFFFF0000u);
+          } else {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[k]));
+            g0 = f.x;
+            g1 = f.y;
+          }
           a0 += g0; a1 += fabsf(g0); a2 = __fmaf_rn(g0, g0, a2);
           a0 += g1; a1 += fabsf(g1); a2 = __fmaf_rn(g1, g1, a2);
         }
@@ -770,8 +822,11 @@ cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const
       if (grad_dtype == 0)
         return stats ? launch_w<kStep, 0, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream)
                      : launch_w<kStep, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
-      return stats ? launch_w<kStep, 1, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream)
-                   : launch_w<kStep, 1, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+      if (grad_dtype == 1)
+        return stats ? launch_w<kStep, 1, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream)
+                     : launch_w<kStep, 1, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+      return stats ? launch_w<kStep, 2, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream)
+                   : launch_w<kStep, 2, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
     case kRepack:
       return launch_w<kRepack, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
     case kInit:
@@ -782,8 +837,10 @@ cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const
       const int g = (int)(n < want ? n : want);
       if (grad_dtype == 0)
         stq_grad_stats_kernel<0><<<g, kThreads, 0, stream>>>(table, tile_map, tile_begin, tile_end, partials);
-      else
+      else if (grad_dtype == 1)
         stq_grad_stats_kernel<1><<<g, kThreads, 0, stream>>>(table, tile_map, tile_begin, tile_end, partials);
+      else
+        stq_grad_stats_kernel<2><<<g, kThreads, 0, stream>>>(table, tile_map, tile_begin, tile_end, partials);
       return cudaGetLastError();
     }
   }

@@ -16,6 +16,9 @@
 // specialised on the pair of widths (one dispatch per tile), so shifts and masks are immediates;
 // the per-block constants (a reciprocal or a logarithm of the block maximum) are computed by one
 // lane per row and broadcast.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
 #include "stq_internal.h"
 
 namespace stq {
@@ -56,8 +59,8 @@ struct __align__(16) TileInfo {
   uint8_t* vco;
   float* mso;
   float* vso;
-  uint32_t wim, wiv;   // width indices (0..4 for 2,3,4,8,16 bits)
-  uint32_t lgB;
+  uint16_t* lp;        // low-precision copy of the parameters (2 bytes per element), or nullptr
+  uint32_t packed;     // width index of m | of v << 8 (0..4 for 2,3,4,8,16 bits) | log2(block) << 16 | lp dtype << 24
   float wdx;           // fp32(lr*wd) (AdamW) or fp32(wd) (L2 mode)
   uint32_t tile;       // index of the tile in the launch's tile order; 0xFFFFFFFF closes the stream
   uint32_t pad;
@@ -317,13 +320,33 @@ __device__ __forceinline__ void lds_grad(const uint8_t* stage, int elem, float (
   if constexpr (GDT == 0) {
     const float4 v = *reinterpret_cast<const float4*>(stage + kOffGrad + 4 * elem);
     g[0] = v.x; g[1] = v.y; g[2] = v.z; g[3] = v.w;
-  } else {
+  } else if constexpr (GDT == 1) {
     const uint2 v = *reinterpret_cast<const uint2*>(stage + kOffGrad + 2 * elem);
     g[0] = __uint_as_float(v.x << 16);
     g[1] = __uint_as_float(v.x & 0xFFFF0000u);
     g[2] = __uint_as_float(v.y << 16);
     g[3] = __uint_as_float(v.y & 0xFFFF0000u);
+  } else {
+    const uint2 v = *reinterpret_cast<const uint2*>(stage + kOffGrad + 2 * elem);
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+    g[0] = a.x; g[1] = a.y; g[2] = b.x; g[3] = b.y;
   }
+}
+
+// Four updated parameters rounded (nearest-even) to the working precision of the model.
+__device__ __forceinline__ uint2 pack_lp(const float (&x)[4], uint32_t lp_dtype) {
+  uint2 r;
+  if (lp_dtype == 1u) {
+    const __nv_bfloat162 a = __floats2bfloat162_rn(x[0], x[1]), b = __floats2bfloat162_rn(x[2], x[3]);
+    r.x = *reinterpret_cast<const uint32_t*>(&a);
+    r.y = *reinterpret_cast<const uint32_t*>(&b);
+  } else {
+    const __half2 a = __floats2half2_rn(x[0], x[1]), b = __floats2half2_rn(x[2], x[3]);
+    r.x = *reinterpret_cast<const uint32_t*>(&a);
+    r.y = *reinterpret_cast<const uint32_t*>(&b);
+  }
+  return r;
 }
 
 // One staged tile, one warp: R rows of 128 elements, taken in passes of RP rows.  The pass loop is
@@ -331,11 +354,12 @@ __device__ __forceinline__ void lds_grad(const uint8_t* stage, int elem, float (
 // instruction cache, and halving it pays more than the lost overlap between passes.  Specialised on
 // both widths.
 constexpr int RP = kFastRowsPerPass;
-template <int BM, int BV, int GDT>
+template <int BM, int BV, int GDT, bool AMP>
 __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, const TileInfo& ti, const StepConsts& sc,
                                           const float* __restrict__ lut8, int lane, int warp, uint32_t empty_bar,
-                                          double* __restrict__ part) {
-  const int lgB = (int)ti.lgB;
+                                          double* __restrict__ part, float grad_mul) {
+  const int lgB = (int)((ti.packed >> 16) & 0xFFu);
+  [[maybe_unused]] const uint32_t lp_dtype = ti.packed >> 24;
   const float lrwd = sc.l2_mode ? 0.0f : ti.wdx;
   float a0 = 0.f, a1 = 0.f, a2 = 0.f;      // statistics over the raw gradient (decision steps)
 
@@ -365,6 +389,12 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
       if (lane == 0) mbar_arrive(empty_bar);
     }
 
+    if constexpr (AMP) {               // loss-scaled gradients: back to true scale first (x1 is exact)
+#pragma unroll
+      for (int r = 0; r < RP; ++r)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) g[r][k] = __fmul_rn(g[r][k], grad_mul);
+    }
     if (part != nullptr) {
 #pragma unroll
       for (int r = 0; r < RP; ++r)
@@ -474,6 +504,10 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
         out[k] = __fadd_rn(th[r][k], -__fmaf_rn(th[r][k], lrwd, upd));
       }
       *reinterpret_cast<float4*>(param + r * kRowElems) = make_float4(out[0], out[1], out[2], out[3]);
+      if constexpr (AMP) {
+        if (ti.lp != nullptr)
+          *reinterpret_cast<uint2*>(ti.lp + (row0 + r) * kRowElems + 4 * lane) = pack_lp(out, lp_dtype);
+      }
     }
   }
 
@@ -500,7 +534,9 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
 // streamed together, and the balance is dynamic.
 __device__ __forceinline__ uint32_t width_index(uint32_t b) { return b == 2 ? 0u : b == 3 ? 1u : b == 4 ? 2u : b == 8 ? 3u : 4u; }
 
-template <int GDT>
+// AMP: the mixed-precision extras (gradient unscaling, low-precision parameter copy) are compiled
+// in only for launches that use them, so the plain step pays nothing for them.
+template <int GDT, bool AMP>
 __global__ void __launch_bounds__(kFastThreads, kFastCtasPerSm)
 stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map,
                      FastSched* __restrict__ sched, const StepConsts sc, double* __restrict__ partials,
@@ -512,6 +548,9 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
   float* lut8 = reinterpret_cast<float*>(smem + kOffLut);
   constexpr uint32_t kEnd = 0xFFFFFFFFu;   // TileInfo.tile of the closing stage
   constexpr uint32_t gsz = GDT == 0 ? 4u : 2u;
+  // a non-finite gradient somewhere in the model: the whole step is skipped (every thread sees the same value)
+  if (sc.found_inf != nullptr && __ldg(sc.found_inf) != 0.0f) return;
+  const float grad_mul = sc.inv_scale != nullptr ? __ldg(sc.inv_scale) : 1.0f;
 
   if (tid == 0) {
 #pragma unroll
@@ -565,9 +604,8 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
         ti.vco = T->vc_out + (e0 >> 3) * bv;
         ti.mso = T->ms_out + (e0 >> lgB);
         ti.vso = T->vs_out + (e0 >> lgB);
-        ti.wim = width_index(bm);
-        ti.wiv = width_index(bv);
-        ti.lgB = lgB;
+        ti.lp = T->param_lp ? reinterpret_cast<uint16_t*>(T->param_lp) + e0 : nullptr;
+        ti.packed = width_index(bm) | (width_index(bv) << 8) | (lgB << 16) | (T->lp_dtype << 24);
         ti.wdx = sc.l2_mode ? T->wd : (float)(sc.lr * (double)T->wd);
         ti.tile = tile;
         ti.pad = 0u;
@@ -620,10 +658,10 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
     double* part = partials ? partials + ((size_t)ti.tile * kConsumerWarps + warp) * 3 : nullptr;
 
 #define STQ_CASE(IM, IV, BM, BV) \
-  case IM * 5 + IV: tile_body<BM, BV, GDT>(stage, ti, sc, lut8, lane, warp, ebar, part); break;
+  case IM * 5 + IV: tile_body<BM, BV, GDT, AMP>(stage, ti, sc, lut8, lane, warp, ebar, part, grad_mul); break;
 #define STQ_CASES_M(IM, BM) \
   STQ_CASE(IM, 0, BM, 2) STQ_CASE(IM, 1, BM, 3) STQ_CASE(IM, 2, BM, 4) STQ_CASE(IM, 3, BM, 8) STQ_CASE(IM, 4, BM, 16)
-    switch (ti.wim * 5 + ti.wiv) {
+    switch ((ti.packed & 0xFFu) * 5 + ((ti.packed >> 8) & 0xFFu)) {
       STQ_CASES_M(0, 2)
       STQ_CASES_M(1, 3)
       STQ_CASES_M(2, 4)
@@ -650,10 +688,10 @@ __global__ void stq_wait_timeout_selftest_kernel(int* __restrict__ err_flag, lon
   if (!done && threadIdx.x == 0) atomicExch(err_flag, 1);
 }
 
-template <int GDT>
+template <int GDT, bool AMP>
 cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, FastSched* sched, const StepConsts& sc,
                           double* partials, int* err_flag, int grid, cudaStream_t stream) {
-  auto kern = stq_step_fast_kernel<GDT>;
+  auto kern = stq_step_fast_kernel<GDT, AMP>;
   // per device and cheap, so simply repeated: the kernel needs more than the default 48 KB
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
@@ -666,12 +704,22 @@ cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, Fas
 
 }  // namespace
 
-cudaError_t launch_step_fast(int grad_dtype, bool stats, const TensorDesc* table, const uint32_t* tile_map,
+cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, const TensorDesc* table, const uint32_t* tile_map,
                              FastSched* sched, const StepConsts& sc, double* partials, int* err_flag, int grid,
                              cudaStream_t stream) {
   double* p = stats ? partials : nullptr;
-  return grad_dtype == 0 ? launch_fast_t<0>(table, tile_map, sched, sc, p, err_flag, grid, stream)
-                         : launch_fast_t<1>(table, tile_map, sched, sc, p, err_flag, grid, stream);
+  if (amp) {
+    switch (grad_dtype) {
+      case 0: return launch_fast_t<0, true>(table, tile_map, sched, sc, p, err_flag, grid, stream);
+      case 1: return launch_fast_t<1, true>(table, tile_map, sched, sc, p, err_flag, grid, stream);
+      default: return launch_fast_t<2, true>(table, tile_map, sched, sc, p, err_flag, grid, stream);
+    }
+  }
+  switch (grad_dtype) {
+    case 0: return launch_fast_t<0, false>(table, tile_map, sched, sc, p, err_flag, grid, stream);
+    case 1: return launch_fast_t<1, false>(table, tile_map, sched, sc, p, err_flag, grid, stream);
+    default: return launch_fast_t<2, false>(table, tile_map, sched, sc, p, err_flag, grid, stream);
+  }
 }
 
 cudaError_t launch_wait_timeout_selftest(int* err_flag, cudaStream_t stream) {
@@ -681,7 +729,7 @@ cudaError_t launch_wait_timeout_selftest(int* err_flag, cudaStream_t stream) {
 
 int fast_ctas_per_sm() {
   int n = 0;
-  auto kern = stq_step_fast_kernel<1>;
+  auto kern = stq_step_fast_kernel<1, false>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return 1;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kFastThreads, kSmemBytes) != cudaSuccess) return 1;
   return n > 0 ? n : 1;

@@ -17,7 +17,8 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libstq.so")
 
-GRAD_F32, GRAD_BF16 = 0, 1
+GRAD_F32, GRAD_BF16, GRAD_F16 = 0, 1, 2
+LP_NONE, LP_BF16, LP_F16 = 0, 1, 2
 WITH_STATS = 1
 WIDTHS = (2, 3, 4, 8, 16, 32)
 
@@ -38,14 +39,16 @@ class CTensor(C.Structure):
         ("v_codes_out", C.c_void_p), ("v_scales_out", C.c_void_p),
         ("numel", C.c_uint64), ("block", C.c_uint32),
         ("bits_m", C.c_uint8), ("bits_v", C.c_uint8), ("bits_m_out", C.c_uint8), ("bits_v_out", C.c_uint8),
-        ("weight_decay", C.c_float), ("reserved", C.c_uint32),
+        ("weight_decay", C.c_float), ("lp_dtype", C.c_uint32),
+        ("param_lp", C.c_void_p),
     ]
 
 
 class CHParams(C.Structure):
     """struct stq_hparams"""
     _fields_ = [("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
-                ("step", C.c_int64), ("decoupled_wd", C.c_int32), ("grad_dtype", C.c_int32)]
+                ("step", C.c_int64), ("decoupled_wd", C.c_int32), ("grad_dtype", C.c_int32),
+                ("inv_grad_scale", C.c_void_p), ("found_inf", C.c_void_p)]
 
 
 class CPolicyCfg(C.Structure):
@@ -146,9 +149,15 @@ def _ptr(t: torch.Tensor | None) -> int | None:
     return None if t is None or t.numel() == 0 else t.data_ptr()
 
 
+def grad_dtype_of(t: torch.Tensor) -> int:
+    return {torch.float32: GRAD_F32, torch.bfloat16: GRAD_BF16, torch.float16: GRAD_F16}[t.dtype]
+
+
 def make_row(numel: int, block: int, st_in: QState | None, st_out: QState, param: torch.Tensor | None = None,
-             grad: torch.Tensor | None = None, weight_decay: float = 0.0) -> CTensor:
-    """One table row.  st_out may be st_in (in-place) when the widths are unchanged."""
+             grad: torch.Tensor | None = None, weight_decay: float = 0.0,
+             param_lp: torch.Tensor | None = None) -> CTensor:
+    """One table row.  st_out may be st_in (in-place) when the widths are unchanged.  param_lp: an
+    optional bf16/fp16 tensor that receives the rounded copy of the updated parameters."""
     r = CTensor()
     r.param = _ptr(param)
     r.grad = _ptr(grad)
@@ -161,7 +170,12 @@ def make_row(numel: int, block: int, st_in: QState | None, st_out: QState, param
     r.m_codes_out, r.m_scales_out = _ptr(st_out.m_codes), _ptr(st_out.m_scales)
     r.v_codes_out, r.v_scales_out = _ptr(st_out.v_codes), _ptr(st_out.v_scales)
     r.bits_m_out, r.bits_v_out = st_out.bits_m, st_out.bits_v
-    r.numel, r.block, r.weight_decay, r.reserved = numel, block, weight_decay, 0
+    r.numel, r.block, r.weight_decay = numel, block, weight_decay
+    if param_lp is not None:
+        r.lp_dtype = LP_BF16 if param_lp.dtype == torch.bfloat16 else LP_F16
+        r.param_lp = param_lp.data_ptr()
+    else:
+        r.lp_dtype, r.param_lp = LP_NONE, None
     return r
 
 
@@ -222,8 +236,11 @@ class Handle:
     def init_state(self, tbl, stream=None):
         self._check(lib().stq_init_state(self._h, tbl, len(tbl), _stream_ptr(stream)), "stq_init_state")
 
-    def step(self, tbl, *, lr, beta1, beta2, eps, t, grad_dtype=GRAD_F32, decoupled_wd=True, flags=0, stream=None):
-        hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype)
+    def step(self, tbl, *, lr, beta1, beta2, eps, t, grad_dtype=GRAD_F32, decoupled_wd=True, flags=0, stream=None,
+             inv_grad_scale: torch.Tensor | None = None, found_inf: torch.Tensor | None = None):
+        """inv_grad_scale / found_inf: optional one-element float32 device tensors (loss-scaled training)."""
+        hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype,
+                      _ptr(inv_grad_scale), _ptr(found_inf))
         self._check(lib().stq_step(self._h, tbl, len(tbl), C.byref(hp), flags, _stream_ptr(stream)), "stq_step")
 
     def grad_stats(self, tbl, grad_dtype=GRAD_F32, stream=None):
@@ -239,7 +256,7 @@ class Handle:
         self._check(lib().stq_repack(self._h, tbl, len(tbl), _stream_ptr(stream)), "stq_repack")
 
     def step_host(self, tbl, *, lr, beta1, beta2, eps, t, grad_dtype=GRAD_F32, decoupled_wd=True, flags=0):
-        hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype)
+        hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype, None, None)
         h2d, d2h = C.c_uint64(0), C.c_uint64(0)
         self._check(lib().stq_step_host(self._h, tbl, len(tbl), C.byref(hp), flags, C.byref(h2d), C.byref(d2h)),
                     "stq_step_host")

@@ -16,7 +16,7 @@ from paper_2604_06836_b200.runner import Job
 def to_np(t: torch.Tensor) -> np.ndarray:
     """Device tensor -> numpy; bf16 comes back as its uint16 bit patterns."""
     t = t.detach().cpu().contiguous()
-    if t.dtype == torch.bfloat16:
+    if t.dtype in (torch.bfloat16, torch.float16):
         return t.view(torch.int16).numpy().view(np.uint16).copy()
     return t.numpy().copy()
 
@@ -38,7 +38,8 @@ class OracleJob:
                        for n, bm, bv in zip(self.numels, self.bits_m, self.bits_v)]
         self.wd = list(job.wd)
 
-    def step(self, grads, t: int, want_stats=False, new_bits=None, decoupled_wd=True):
+    def step(self, grads, t: int, want_stats=False, new_bits=None, decoupled_wd=True, fp16_grad=False,
+             inv_grad_scale=1.0, found_inf=False):
         w = self.w
         stats = np.zeros((len(self.numels), 4))
         bm, bv = (self.bits_m, self.bits_v) if new_bits is None else (np.asarray(a, np.uint8) for a in new_bits)
@@ -47,7 +48,8 @@ class OracleJob:
             self.states[i], s = O.step(self.theta[i], g, self.states[i], self.block, lr=w.lr, beta1=w.beta1,
                                        beta2=w.beta2, eps=w.eps, weight_decay=self.wd[i], t=t,
                                        bits_m_out=int(bm[i]), bits_v_out=int(bv[i]),
-                                       decoupled_wd=decoupled_wd, want_stats=want_stats)
+                                       decoupled_wd=decoupled_wd, want_stats=want_stats, fp16_grad=fp16_grad,
+                                       inv_grad_scale=inv_grad_scale, found_inf=found_inf)
             self.upd_mag[i] = np.maximum(self.upd_mag[i], np.maximum(np.abs(self.theta[i] - before), np.abs(self.theta[i])))
             if want_stats:
                 stats[i] = s

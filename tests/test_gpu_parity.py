@@ -225,3 +225,47 @@ def test_algorithm1_order_with_the_paper_policy_driving_the_widths(H, O):
         job.step(t, new_bits=new_bits)
         H.compare_job(job, oj, REL_1STEP * t if t <= 10 else REL_100, f"t={t}")
     assert len(seen) >= 2          # the policy did move layers between widths
+
+
+@pytest.mark.parametrize("gdt", [torch.float16, torch.bfloat16, torch.float32])
+def test_loss_scaled_gradients_skip_flag_and_low_precision_copy(H, O, gdt):
+    """Mixed-precision training plumbing fused into the step: gradients arrive multiplied by the loss
+    scale (fp16 here, as the paper trains), are brought back by *inv_grad_scale before anything else,
+    found_inf skips the step, and the updated parameters are also written as a bf16 / fp16 copy."""
+    import oracle
+    shapes = [("a", (4096 * 2 + 700,)), ("b", (333,)), ("c", (4096,))]
+    w = W.Workload("amp", tuple(shapes), 128, "fp32", "student_t", nu=4, scale_log10=(-4.0, -3.0), seed=21)
+    S = 1024.0
+    job = Job(w, [8, 4, 3], [4, 8, 2])
+    oj = H.OracleJob(job)
+    inv = torch.tensor([1.0 / S], dtype=torch.float32, device="cuda")
+    flag = torch.zeros(1, dtype=torch.float32, device="cuda")
+    lp_dt = torch.float16 if gdt == torch.float16 else torch.bfloat16
+    lps = [torch.zeros(n, dtype=lp_dt, device="cuda") for n in job.numels]
+    grads = [torch.zeros(n, dtype=gdt, device="cuda") for n in job.numels]
+    rows = lambda: stq.table([stq.make_row(n, job.block, job.states[i], job.states[i], job.params[i], grads[i],
+                                            job.wd[i], lps[i]) for i, n in enumerate(job.numels)])
+    for t in (1, 2, 3, 4):
+        job.draw_grads(t)
+        for i in range(job.L):
+            grads[i].copy_((job.grads[i] * S).to(gdt))
+        skip = (t == 3)
+        flag.fill_(1.0 if skip else 0.0)
+        before = [p.clone() for p in job.params]
+        codes_before = [s.m_codes.clone() for s in job.states]
+        st_o = oj.step([H.to_np(g) for g in grads], t, want_stats=True, fp16_grad=(gdt == torch.float16),
+                       inv_grad_scale=1.0 / S, found_inf=skip)
+        job.handle.step(rows(), flags=stq.WITH_STATS, inv_grad_scale=inv, found_inf=flag,
+                        **{**job.hp(t), "grad_dtype": stq.grad_dtype_of(grads[0])})
+        H.compare_job(job, oj, REL_1STEP * t, f"{gdt} t={t}")
+        if skip:
+            assert all(torch.equal(a, b) for a, b in zip(before, job.params))
+            assert all(torch.equal(a, s.m_codes) for a, s in zip(codes_before, job.states))
+        else:
+            H.assert_stats_close(job.handle.layer_stats(job.L), st_o, f"{gdt} t={t}")
+            for i in range(job.L):
+                # the copy is exactly the nearest-even rounding of the parameters the kernel wrote
+                assert torch.equal(lps[i], job.params[i].to(lp_dt)), (t, i)
+                want = oracle.round_lp(oj.theta[i], "fp16" if lp_dt == torch.float16 else "bf16")
+                got = H.to_np(lps[i])
+                assert (np.abs(got.astype(np.int32) - want.astype(np.int32)) <= 1).all()   # a last-bit tie at most

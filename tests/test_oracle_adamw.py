@@ -198,3 +198,35 @@ def test_bf16_grads_widen_exactly(O):
     st2, s2 = O.step(th2, widened, st2, 128, t=1, want_stats=True, **HP)
     assert (th1 == th2).all() and (st1.m_codes == st2.m_codes).all() and (st1.v_codes == st2.v_codes).all()
     assert (s1 == s2).all()
+
+
+def test_half_precision_conversions_match_the_library(O):
+    """fp16 widening and the nearest-even roundings to bf16 / fp16 against torch's conversions."""
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.normal(0, 1, 100000) * 10.0 ** rng.uniform(-9, 5, 100000),
+                        [0, -0.0, 65504, 65519.9, 65520, 6.1e-5, 5.96e-8, 2.98e-8, 2.99e-8, 1e-10, -3e-8]]).astype(np.float32)
+    t = torch.from_numpy(x)
+    assert (O.round_lp(x, "bf16") == t.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)).all()
+    assert (O.round_lp(x, "fp16") == t.to(torch.float16).view(torch.int16).numpy().view(np.uint16)).all()
+    allh = np.arange(65536, dtype=np.uint16)
+    want = torch.from_numpy(allh.view(np.int16)).view(torch.float16).float().numpy()
+    got = O.widen_f16(allh)
+    fin = np.isfinite(want)
+    assert (got[fin].view(np.uint32) == want[fin].view(np.uint32)).all()
+
+
+def test_loss_scale_and_skipped_step(O):
+    """Gradients scaled by S and multiplied back by 1/S (a power of two) give the unscaled step bit for
+    bit; a step with found_inf leaves everything untouched."""
+    rng = np.random.default_rng(9)
+    n = 128 * 3 + 17
+    g = (rng.standard_t(4, n) * 1e-3).astype(np.float32)
+    th1 = rng.normal(0, 0.02, n).astype(np.float32)
+    th2 = th1.copy()
+    st1, _ = O.step(th1, g, O.new_state(n, 128, 8, 4), 128, t=1, **HP)
+    st2, _ = O.step(th2, (g * np.float32(1024)).astype(np.float32), O.new_state(n, 128, 8, 4), 128, t=1,
+                    inv_grad_scale=1.0 / 1024, **HP)
+    assert (th1 == th2).all() and (st1.m_codes == st2.m_codes).all() and (st1.v_codes == st2.v_codes).all()
+    before = th1.copy()
+    st3, _ = O.step(th1, g, st1, 128, t=2, found_inf=True, **HP)
+    assert (th1 == before).all() and st3 is st1
