@@ -301,7 +301,8 @@ def run_ours(args, w, bits_m, bits_v):
                    "decision_interval": w.decision_interval, "decision_steps_timed": int(is_dec.sum()),
                    "l2": "inputs larger than L2 (%.1f GB touched per step)" % (alg_bytes / 1e9),
                    "parallelism": "replicas" if world > 1 else "single", "grid": job.handle.grid_size,
-                   "state_bytes": job.state_bytes(), "fp32_state_bytes": 8 * params},
+                   "state_bytes": job.state_bytes(), "fp32_state_bytes": 8 * params,
+                   "state_saved_frac": 1.0 - job.state_bytes() / (8.0 * params)},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": (NCU_TRAFFIC_BYTES_PER_PARAM[args.config] * params
                                  if args.config in NCU_TRAFFIC_BYTES_PER_PARAM else None),

@@ -177,14 +177,15 @@ bool row_is_wide(const stq_tensor& t, int kind) {
 int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStream_t stream) {
   if (!h || !tensors) return STQ_E_NULL;
   if (L <= 0 || L > (1 << 20)) return STQ_E_NUMEL;
+  STQ_CUDA(h, cudaSetDevice(h->device));
+  // the same table as last time (the usual case between decision steps) was validated and uploaded then
+  const bool same = h->cached_kind == kind && (int)h->cached.size() == L &&
+                    std::memcmp(h->cached.data(), tensors, sizeof(stq_tensor) * (size_t)L) == 0;
+  if (same) return STQ_OK;
   for (int l = 0; l < L; ++l) {
     int rc = validate_row(tensors[l], kind);
     if (rc != STQ_OK) return rc;
   }
-  STQ_CUDA(h, cudaSetDevice(h->device));
-  const bool same = h->cached_kind == kind && (int)h->cached.size() == L &&
-                    std::memcmp(h->cached.data(), tensors, sizeof(stq_tensor) * (size_t)L) == 0;
-  if (same) return STQ_OK;
 
   // Tile classes.  "Fast": full tiles of a step whose widths do not change (2..16 bits); they go to
   // the main kernel.  The rest (ragged last tile, width change, 32-bit state, other entry points)
