@@ -310,6 +310,8 @@ def run_ours(args, w, bits_m, bits_v):
                      "bytes_per_param": alg_bytes / params, "kernel_ms_mean": k_ms,
                      "kernel_ms_plain": float(kern_ms[~is_dec].mean()) if (~is_dec).any() else None,
                      "kernel_ms_with_stats": float(kern_ms[is_dec].mean()) if is_dec.any() else None,
+                     # the step runs at the board's power limit: the first steps see boost clocks, later ones do not
+                     "kernel_ms_first_10": float(kern_ms[:10].mean()), "kernel_ms_last_10": float(kern_ms[-10:].mean()),
                      "frac_of_nominal_8000": achieved / 8000.0},
         "clocks": clocks,
         "decision_step": decision,
