@@ -269,3 +269,55 @@ def test_loss_scaled_gradients_skip_flag_and_low_precision_copy(H, O, gdt):
                 want = oracle.round_lp(oj.theta[i], "fp16" if lp_dt == torch.float16 else "bf16")
                 got = H.to_np(lps[i])
                 assert (np.abs(got.astype(np.int32) - want.astype(np.int32)) <= 1).all()   # a last-bit tie at most
+
+
+def test_extreme_but_finite_values(H, O):
+    """Zero blocks, denormal gradients (the tiny-scale rule), huge gradients, one outlier per block,
+    alternating signs: codes and scales stay bit-exact and nothing faults."""
+    n = 4096 * 2 + 128 * 3
+    w = W.Workload("extreme", (("a", (n,)), ("b", (n,)), ("c", (n,))), 128, "fp32", "normal",
+                   scale_log10=(-3.0, -3.0), seed=31)
+    job = Job(w, [8, 3, 16], [4, 8, 2])
+    oj = H.OracleJob(job)
+    g = torch.Generator(device="cuda").manual_seed(3)
+    for t in range(1, 6):
+        for i in range(3):
+            x = torch.randn(n, generator=g, device="cuda") * 1e-3
+            blk = x.view(-1, 128)
+            blk[0::7] = 0.0                                    # all-zero blocks
+            blk[1::7] *= 1e-42                                 # denormal gradients
+            blk[2::7] *= 1e-25                                 # v below the tiny-scale rule, m above it
+            blk[3::7] *= 1e16                                  # large: v up to ~1e23
+            blk[4::7, 5] = 3e3                                 # one outlier dwarfs its block
+            blk[5::7] = blk[5::7].abs() * (1 - 2 * (torch.arange(128, device="cuda") % 2))   # +-+-
+            job.grads[i].copy_(x)
+        oj.step([H.to_np(gr) for gr in job.grads], t, want_stats=False)
+        job.step(t)
+        H.compare_job(job, oj, REL_1STEP * t, f"extreme t={t}")
+
+
+def test_non_finite_gradients_do_not_fault_or_leak_into_other_blocks(H, O):
+    """Inf / NaN gradients are outside the contract (use found_inf): the affected blocks hold garbage,
+    but the kernel neither faults nor disturbs any other block."""
+    n = 4096 + 512
+    w = W.Workload("nonfinite", (("a", (n,)),), 128, "fp32", "normal", scale_log10=(-3.0, -3.0), seed=32)
+    job = Job(w, [4], [4])
+    oj = H.OracleJob(job)
+    job.draw_grads(1)
+    bad_blocks = [3, 17, 35]
+    for b, val in zip(bad_blocks, (float("inf"), float("nan"), -float("inf"))):
+        job.grads[0][b * 128 + 7] = val
+    good = np.ones(n, bool)
+    for b in bad_blocks:
+        good[b * 128:(b + 1) * 128] = False
+    gnp = H.to_np(job.grads[0])
+    gnp_clean = np.where(good, gnp, 0).astype(np.float32)
+    oj.step([gnp_clean], 1)
+    job.step(1)
+    job.handle.device_status()
+    th = H.to_np(job.params[0])
+    assert np.allclose(th[good], oj.theta[0][good], rtol=2e-6, atol=1e-9)
+    gm = H.to_np(job.states[0].m_codes)
+    om = oj.states[0].m_codes
+    keep = np.repeat(good.reshape(-1, 128)[:, 0], 64)       # 4-bit codes: 64 bytes per block
+    assert (gm[:keep.size][keep] == om[:keep.size][keep]).all()
