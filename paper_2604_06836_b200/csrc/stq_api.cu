@@ -270,6 +270,11 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
       next_fast += nfast[l];
     }
     hs->grp_begin[hs->ng] = next_fast;
+    // chunk size: the usual one when every CTA gets several chunks, down to single tiles for small launches
+    {
+      const uint64_t per_cta = next_fast / (uint64_t)std::max(1, h->fast_grid);
+      hs->chunk = (uint32_t)std::min<uint64_t>(stq::kFastChunk, std::max<uint64_t>(1, per_cta / 4));
+    }
     // CTAs per group in proportion to cost (largest remainders), at least one each
     const int G = h->fast_grid;
     double total_cost = 0.0;

@@ -64,10 +64,11 @@ cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const
 // of equal width pair.  Lives in device memory; the counters are zeroed before every launch.
 constexpr int kFastMaxGroups = 32;     // 25 width pairs exist
 constexpr int kFastMaxGrid = 4096;
-constexpr uint32_t kFastChunk = 8;     // tiles handed out per counter increment
+constexpr uint32_t kFastChunk = 8;     // tiles handed out per counter increment (fewer for small launches)
 struct FastSched {
   uint32_t ctr[kFastMaxGroups];            // chunks handed out so far, per group
   uint32_t ng;                             // number of groups
+  uint32_t chunk;                          // tiles per counter increment for this launch
   uint32_t grp_begin[kFastMaxGroups + 1];  // tile range of group g: [grp_begin[g], grp_begin[g+1])
   uint16_t cta_group[kFastMaxGrid];        // group a CTA starts in
 };

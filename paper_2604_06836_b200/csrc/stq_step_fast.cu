@@ -528,7 +528,8 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
 }
 
 // Scheduling: the fast tiles are grouped by width pair (one body each).  A CTA starts in the group
-// the host assigned to it and takes chunks of kFastChunk consecutive tiles from that group's
+// the host assigned to it and takes chunks of consecutive tiles (kFastChunk of them, fewer when the
+// launch is small) from that group's
 // counter; when its group runs dry it moves on to the next one that still has work.  So a CTA runs
 // few different bodies (a change of body is an instruction-cache refill), the tiles of a group are
 // streamed together, and the balance is dynamic.
@@ -570,7 +571,7 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
   if (warp == kConsumerWarps) {
     // ================================ producer ========================================================
     if (lane != 0) return;
-    const uint32_t ng = sched->ng;
+    const uint32_t ng = sched->ng, chunk = sched->chunk;
     uint32_t grp = sched->cta_group[blockIdx.x];
     uint32_t dry = 0;          // consecutive groups found empty
     uint32_t issued = 0;
@@ -583,14 +584,14 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
     while (ok && dry < ng) {
       const uint32_t gbeg = sched->grp_begin[grp], gend = sched->grp_begin[grp + 1];
       const uint32_t c = atomicAdd(&sched->ctr[grp], 1u);
-      const unsigned long long t0 = (unsigned long long)gbeg + (unsigned long long)c * kFastChunk;
+      const unsigned long long t0 = (unsigned long long)gbeg + (unsigned long long)c * chunk;
       if (t0 >= gend) {        // this group has been handed out completely
         ++dry;
         grp = grp + 1 == ng ? 0u : grp + 1;
         continue;
       }
       dry = 0;
-      const uint32_t t1 = (uint32_t)(t0 + kFastChunk < gend ? t0 + kFastChunk : gend);
+      const uint32_t t1 = (uint32_t)(t0 + chunk < gend ? t0 + chunk : gend);
       for (uint32_t tile = (uint32_t)t0; tile < t1; ++tile) {
         if (issued >= (uint32_t)kStages && !mbar_wait(empty0 + 8 * s, phase ^ 1u)) { ok = false; break; }
         const TensorDesc* T = table + __ldg(tile_map + tile);
