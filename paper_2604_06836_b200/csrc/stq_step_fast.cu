@@ -459,11 +459,16 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
           if ((lane & (2 * RP - 1)) == RP + r) mine = mxv[r];
       }
       const float x = __uint_as_float(mine);
+      const bool zero = x < kTiny;
       const float mul = (BV <= 4 && (lane & RP)) ? kSqrt2 : (float)Wd<BM>::qmax;
-      const float val = x < kTiny ? 0.f : __fmul_rn(mul, __frcp_rn(x));
+      const float val = zero ? 0.f : __fmul_rn(mul, __frcp_rn(x));
+      // the same lanes store the new scales (a zero block stores 0), for the rows that open a block
+      const int e_mine = (row0 + (lane & (RP - 1))) * kRowElems;
+      const bool opens = (e_mine & ((1 << lgB) - 1)) == 0;
 #pragma unroll
       for (int r = 0; r < RP; ++r) inv_m[r] = __shfl_sync(kFull, val, r);
       if constexpr (BV <= 4) {
+        if (lane < 2 * RP && opens) ((lane & RP) ? ti.vso : ti.mso)[e_mine >> lgB] = zero ? 0.f : x;
 #pragma unroll
         for (int r = 0; r < RP; ++r) lgc[r] = __shfl_sync(kFull, val, RP + r);
       } else {
@@ -471,6 +476,10 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
 #pragma unroll
         for (int r = 1; r < RP; ++r)
           if ((lane & (RP - 1)) == r) mv = mxv[r];
+        if (lane < RP && opens) {
+          ti.mso[e_mine >> lgB] = zero ? 0.f : x;
+          ti.vso[e_mine >> lgB] = __uint_as_float(mv) < kTiny ? 0.f : __uint_as_float(mv);
+        }
         const float ps = lg_poly(mv);
 #pragma unroll
         for (int r = 0; r < RP; ++r) lgc[r] = __shfl_sync(kFull, ps, r);
@@ -481,21 +490,16 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
     float* param = ti.param + row0 * kRowElems + 4 * lane;
 #pragma unroll
     for (int r = 0; r < RP; ++r) {
+      // A zero block of m needs no special case here: its inv is 0, so every q is 0 and so is mq.
       const float sm_raw = __uint_as_float(mxm[r]);
-      const float s_m = sm_raw < kTiny ? 0.f : sm_raw;
       const float sv_raw = __uint_as_float(mxv[r]);
       const bool vzero = sv_raw < kTiny;
       const float s_v = vzero ? 0.f : sv_raw;
       const uint32_t ebase = kMagicBits - (vzero ? (uint32_t)kZeroBlockExp : (mxv[r] >> 23));
       float mq[4], vq[4];
       // mq comes out multiplied by lr/(1-beta1^t): the decode scale carries the factor
-      encode_lin_row<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], __fmul_rn(s_m, sc.step_size), inv_m[r], mq);
+      encode_lin_row<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], __fmul_rn(sm_raw, sc.step_size), inv_m[r], mq);
       encode_log_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], s_v, lgc[r], ebase, lut8, vq);
-      const int e_row = (row0 + r) * kRowElems;
-      if (lane == 0 && (e_row & ((1 << lgB) - 1)) == 0) {
-        ti.mso[e_row >> lgB] = s_m;
-        ti.vso[e_row >> lgB] = s_v;
-      }
       float out[4];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
