@@ -29,8 +29,8 @@ class Job:
         self.numels = w.numels
         self.L = len(self.numels)
         self.block = w.block
-        self.grad_dtype = stq.GRAD_BF16 if w.grad_dtype == "bf16" else stq.GRAD_F32
-        self.gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
+        self.gdt = {"fp32": torch.float32, "bf16": torch.bfloat16, "fp16": torch.float16}[w.grad_dtype]
+        self.grad_dtype = {"fp32": stq.GRAD_F32, "bf16": stq.GRAD_BF16, "fp16": stq.GRAD_F16}[w.grad_dtype]
         self.scales = tensor_scales(w)
         # parameters and gradients live in two flat buffers; every tensor starts 256-byte aligned
         offs, total = [], 0
@@ -42,6 +42,14 @@ class Job:
         self.grad_flat = torch.zeros(total, dtype=self.gdt, device=self.device)
         self.params = [self.param_flat[o:o + n] for o, n in zip(offs, self.numels)]
         self.grads = [self.grad_flat[o:o + n] for o, n in zip(offs, self.numels)]
+        # loss-scaled training: 1/scale and the found-inf flag are read by the kernel from device memory
+        self.inv_scale = (torch.tensor([1.0 / w.loss_scale], dtype=torch.float32, device=self.device)
+                          if w.loss_scale > 0 else None)
+        self.found_inf = torch.zeros(1, dtype=torch.float32, device=self.device) if w.loss_scale > 0 else None
+        self.lp_flat = (torch.zeros(total, dtype={"bf16": torch.bfloat16, "fp16": torch.float16}[w.lp_copy],
+                                    device=self.device) if w.lp_copy else None)
+        self.params_lp = ([self.lp_flat[o:o + n] for o, n in zip(offs, self.numels)]
+                          if w.lp_copy else [None] * self.L)
         if draw_params:
             for i in range(self.L):
                 self.params[i].copy_(draw_param(w, i, self.device))
@@ -59,7 +67,8 @@ class Job:
     def _make_table(self, st_in, st_out, with_inputs=True):
         rows = [stq.make_row(n, self.block, si if with_inputs else None, so,
                              self.params[i] if with_inputs else None,
-                             self.grads[i] if with_inputs else None, self.wd[i])
+                             self.grads[i] if with_inputs else None, self.wd[i],
+                             self.params_lp[i] if with_inputs else None)
                 for i, (n, si, so) in enumerate(zip(self.numels, st_in, st_out))]
         return stq.table(rows)
 
@@ -77,7 +86,8 @@ class Job:
     # ---- the path --------------------------------------------------------------------------------
     def hp(self, t: int) -> dict:
         w = self.w
-        return dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, t=t, grad_dtype=self.grad_dtype)
+        return dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, t=t, grad_dtype=self.grad_dtype,
+                    inv_grad_scale=self.inv_scale, found_inf=self.found_inf)
 
     def step(self, t: int | None = None, stats: bool = False, new_bits=None, stream=None):
         """One optimizer step.  new_bits = (bits_m, bits_v) arrays switches widths inside the step."""
@@ -131,8 +141,9 @@ class Job:
 
     # ---- accounting ------------------------------------------------------------------------------
     def algorithmic_bytes(self) -> int:
-        """Bytes one step must move: theta r+w, grad, codes r+w, scales r+w."""
-        gb = 2 if self.w.grad_dtype == "bf16" else 4
+        """Bytes one step must move: theta r+w, grad, codes r+w, scales r+w, the working copy if any."""
+        gb = 4 if self.w.grad_dtype == "fp32" else 2
+        gb += 2 if self.w.lp_copy else 0        # the working copy is written once per step
         total = 0
         for n, bm, bv in zip(self.numels, self.bits_m, self.bits_v):
             nb = (n + self.block - 1) // self.block

@@ -255,7 +255,10 @@ class Handle:
     def repack(self, tbl, stream=None):
         self._check(lib().stq_repack(self._h, tbl, len(tbl), _stream_ptr(stream)), "stq_repack")
 
-    def step_host(self, tbl, *, lr, beta1, beta2, eps, t, grad_dtype=GRAD_F32, decoupled_wd=True, flags=0):
+    def step_host(self, tbl, *, lr, beta1, beta2, eps, t, grad_dtype=GRAD_F32, decoupled_wd=True, flags=0,
+                  inv_grad_scale=None, found_inf=None):
+        if inv_grad_scale is not None or found_inf is not None:
+            raise ValueError("step_host takes host buffers only: unscale the gradients on the device path")
         hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype, None, None)
         h2d, d2h = C.c_uint64(0), C.c_uint64(0)
         self._check(lib().stq_step_host(self._h, tbl, len(tbl), C.byref(hp), flags, C.byref(h2d), C.byref(d2h)),

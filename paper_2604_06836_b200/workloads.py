@@ -52,6 +52,18 @@ def vit_shapes(n_layer: int = 12, d: int = 768, d_ff: int = 3072, patch: int = 1
     return s
 
 
+def roberta_shapes(n_layer: int = 24, d: int = 1024, vocab: int = 50265, positions: int = 514):
+    """RoBERTa (Table 1 fine-tunes RoBERTa-Large): embeddings with their norm, encoder blocks, and the
+    masked-LM head (dense, norm, output bias; the decoder matrix is tied to the word embeddings)."""
+    s = [("emb.word", (vocab, d)), ("emb.pos", (positions, d)), ("emb.type", (1, d)),
+         ("emb.ln.w", (d,)), ("emb.ln.b", (d,))]
+    for l in range(n_layer):
+        s += transformer_block_shapes(f"l{l}", d, 4 * d)
+    s += [("head.dense.w", (d, d)), ("head.dense.b", (d,)), ("head.ln.w", (d,)), ("head.ln.b", (d,)),
+          ("head.bias", (vocab,))]
+    return s
+
+
 # --------------------------------------------------------------------------------------------
 # workload configurations
 # --------------------------------------------------------------------------------------------
@@ -60,7 +72,7 @@ class Workload:
     name: str
     shapes: tuple                      # ((name, shape), ...)
     block: int
-    grad_dtype: str                    # "fp32" | "bf16"
+    grad_dtype: str                    # "fp32" | "bf16" | "fp16"
     grad_kind: str                     # "normal" | "student_t" | "normal_outliers"
     nu: int = 0                        # Student-t degrees of freedom
     scale_log10: tuple = (-3.0, -3.0)  # per-tensor scale is 10^U(lo, hi)
@@ -77,6 +89,8 @@ class Workload:
     beta2: float = 0.999
     eps: float = 1e-8
     weight_decay: float = 0.01
+    loss_scale: float = 0.0            # > 0: gradients arrive multiplied by it (fp16 training)
+    lp_copy: str = ""                  # "bf16" | "fp16": the step also writes the model's working copy
 
     @property
     def numels(self) -> list[int]:
@@ -111,6 +125,16 @@ def config(name: str) -> Workload:
         return Workload("cfg5s-gpt2-xl-6-layers", tuple(gpt2_shapes(6, 1600)), 128, "bf16", "student_t",
                         nu=3, scale_log10=(-5.0, -2.0), bits_mean=(4.9, 5.1), steps=20,
                         decision_interval=5, seed=5)
+    # Table 1's other models, trained the way Sec. 4 describes (fp16 with a loss scale): fp16 gradients
+    # times 2^12, unscaled inside the step, and an fp16 working copy of the parameters written by it.
+    amp = dict(block=128, grad_dtype="fp16", grad_kind="student_t", nu=4, scale_log10=(-5.0, -2.0),
+               steps=20, decision_interval=10, loss_scale=4096.0, lp_copy="fp16")
+    if name == "gpt2_medium":
+        return Workload("gpt2-medium-355M-fp16", tuple(gpt2_shapes(24, 1024)), seed=6, **amp)
+    if name == "roberta_large":
+        return Workload("roberta-large-356M-fp16", tuple(roberta_shapes()), seed=7, **amp)
+    if name == "vit_b32":
+        return Workload("vit-b32-88M-fp16", tuple(vit_shapes(patch=32, tokens=50)), seed=8, **amp)
     raise KeyError(name)
 
 
@@ -180,7 +204,8 @@ def draw_param(w: Workload, idx: int, device="cpu") -> torch.Tensor:
 
 def draw_grad(w: Workload, idx: int, step: int, device="cpu", scale: float | None = None,
               chunk: int = 1 << 24) -> torch.Tensor:
-    """Gradient of tensor ``idx`` at ``step`` (flattened; fp32 or bf16 per the workload)."""
+    """Gradient of tensor ``idx`` at ``step`` (flattened; fp32, bf16 or fp16 per the workload; times the
+    workload's loss scale when it has one)."""
     n = w.numels[idx]
     if scale is None:
         scale = float(tensor_scales(w)[idx])
@@ -198,7 +223,11 @@ def draw_grad(w: Workload, idx: int, step: int, device="cpu", scale: float | Non
             mask = torch.empty(m, dtype=torch.float32, device=device).uniform_(0.0, 1.0, generator=g) < 1e-3
             z = torch.where(mask, torch.sign(z) * 100.0, z)
         out[lo:lo + m] = z * scale
-    return out.to(torch.bfloat16) if w.grad_dtype == "bf16" else out
+    if w.loss_scale > 0:
+        out *= w.loss_scale
+    if w.grad_dtype == "bf16":
+        return out.to(torch.bfloat16)
+    return out.to(torch.float16) if w.grad_dtype == "fp16" else out
 
 
 def small_gpt2(d: int = 200, n_layer: int = 2, vocab: int = 1031, ctx: int = 64):

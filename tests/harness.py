@@ -154,6 +154,7 @@ class SampledOracle:
         self.states = [O.new_state(self.n_mini[i], self.block, int(job.bits_m[i]), int(job.bits_v[i]))
                        for i in range(job.L)]
         self.mag = [np.abs(t) for t in self.theta]
+        self.stepped = False      # the working copy exists only after the first step
 
     def _elem_index(self, i: int) -> torch.Tensor:
         blocks, tail, nb_full = self.sel[i]
@@ -185,6 +186,7 @@ class SampledOracle:
         """Oracle step on the sample, with the gradients currently held by the job.  new_bits =
         (bits_m, bits_v) arrays switches widths inside the step."""
         w = self.job.w
+        self.stepped = True
         for i in range(self.job.L):
             if self.n_mini[i] == 0:
                 continue
@@ -192,9 +194,10 @@ class SampledOracle:
             before = self.theta[i].copy()
             bm = None if new_bits is None else int(new_bits[0][i])
             bv = None if new_bits is None else int(new_bits[1][i])
+            amp = dict(fp16_grad=True, inv_grad_scale=1.0 / w.loss_scale) if w.grad_dtype == "fp16" else {}
             self.states[i], _ = O.step(self.theta[i], g, self.states[i], self.block, lr=w.lr, beta1=w.beta1,
                                        beta2=w.beta2, eps=w.eps, weight_decay=self.job.wd[i], t=t,
-                                       bits_m_out=bm, bits_v_out=bv)
+                                       bits_m_out=bm, bits_v_out=bv, **amp)
             self.mag[i] = np.maximum(self.mag[i], np.maximum(np.abs(self.theta[i]), np.abs(self.theta[i] - before)))
 
     def repack(self, new_bits):
@@ -227,3 +230,7 @@ class SampledOracle:
             o = self.theta[i].astype(np.float64)
             lim = rel * np.maximum(self.mag[i].astype(np.float64), 1e-3 * np.abs(o).max())
             assert (np.abs(g - o) <= lim).all(), name + f" theta: max err {np.abs(g - o).max():.3e}"
+            if job.w.lp_copy and self.stepped:   # the working copy is the kernel's own fp32 result, rounded to nearest even
+                idx = self._elem_index(i)
+                lp = job.params_lp[i]
+                assert torch.equal(lp[idx], job.params[i][idx].to(lp.dtype)), name + " working copy"

@@ -22,11 +22,13 @@ def _need(gb):
         pytest.skip(f"needs {gb} GiB of free device memory")
 
 
-@pytest.mark.parametrize("name,gib", [("cfg2", 4), ("cfg3", 3), ("cfg4", 14), ("cfg5", 26)])
+@pytest.mark.parametrize("name,gib", [("cfg2", 4), ("cfg3", 3), ("cfg4", 14), ("cfg5", 26),
+                                      ("gpt2_medium", 8), ("roberta_large", 8), ("vit_b32", 3)])
 def test_full_size_sampled_blocks(name, gib):
     """Each configuration as specified: its step count, its decision interval, statistics on the
     decision steps, and for cfg3 the width change of 10 % of the tensors on every decision step
-    (alternately by stq_repack between steps and fused into the step)."""
+    (alternately by stq_repack between steps and fused into the step).  The last three are the other
+    models of Table 1 under fp16 training: loss-scaled fp16 gradients and an fp16 working copy."""
     import harness as H
     import oracle
     _need(gib)
@@ -56,9 +58,9 @@ def test_full_size_sampled_blocks(name, gib):
             got = job.layer_stats()
     for i, g in enumerate(job.grads):     # statistics of the last decision step (the last step of every config)
         if g.numel() <= (1 << 21):
-            want = oracle.grad_stats(H.to_np(g))
+            want = oracle.grad_stats(H.to_np(g.float() / w.loss_scale if w.loss_scale > 0 else g))
         else:
-            g64 = g.double()
+            g64 = g.double() * (1.0 / w.loss_scale if w.loss_scale > 0 else 1.0)
             want = np.array([g64.sum().item(), g64.abs().sum().item(), (g64 * g64).sum().item(), g.numel()])
         H.assert_stats_close(got[i:i + 1], want[None, :], f"{name} stats tensor {i}")
     # memory accounting of the problem statement: sum over layers of N_l * (b_m + b_v) bits (+ scales)
