@@ -1,8 +1,14 @@
-"""Multi-process plumbing of the benchmark: replicas only, no data-path collective.
+"""Multi-process plumbing: replicas for the benchmark, and the host side of a sharded optimizer.
 
-The path does not shard (every rank steps its own replica), so the only exchange is the timing:
+The benchmark runs replicas (every rank steps its own copy), so its only exchange is the timing:
 the slowest rank defines the step time, and the job's throughput is the sum of the units all ranks
 processed divided by that time.
+
+A sharded optimizer (each rank keeps the quantized state of a slice of the parameters) needs no
+data-path collective either, because quantization blocks are independent: ``partition`` cuts the
+parameter list into per-rank element ranges on block boundaries, each rank steps its ranges as rows
+of its own table, and on decision steps the per-layer sums are added over ranks
+(``sync_layer_stats``, Sec. 3.1's distributed engine) so that every rank takes the same decision.
 """
 from __future__ import annotations
 
@@ -47,3 +53,36 @@ def sync_layer_stats(stats, device="cpu"):
     t = torch.as_tensor(np.ascontiguousarray(stats, dtype=np.float64), device=device).clone()
     dist.all_reduce(t, op=dist.ReduceOp.SUM)
     return t.cpu().numpy()
+
+
+def partition(numels, world: int, align: int = 4096):
+    """Cuts the concatenated parameter list into ``world`` contiguous shares of about equal size.
+
+    Returns one list per rank of (tensor index, first element, end element).  A cut inside a tensor
+    falls on a multiple of ``align`` elements from the tensor's start (the default, one kernel tile,
+    is a multiple of every block size, so no quantization block is split and every range starts on a
+    16-byte boundary of the packed codes for every width).  Ranges of one tensor on different ranks
+    are disjoint and cover it; a rank may get no range when there is less work than ranks."""
+    numels = [int(n) for n in numels]
+    total = sum(numels)
+    shares = [[] for _ in range(world)]
+    # units: whole align-sized pieces (the ragged tail of a tensor belongs to its last piece)
+    pieces = [max(1, (n + align - 1) // align) if n > 0 else 0 for n in numels]
+    npieces = sum(pieces)
+    done = 0            # pieces handed out so far
+    rank = 0
+    for l, (n, p) in enumerate(zip(numels, pieces)):
+        first = 0       # piece index inside the tensor
+        while first < p:
+            # the rank's share ends at piece index round((rank+1) * npieces / world) of the whole list
+            end_global = ((rank + 1) * npieces + world - 1) // world
+            take = min(p - first, end_global - done)
+            if take <= 0:
+                rank += 1
+                continue
+            lo, hi = first * align, min(n, (first + take) * align)
+            shares[rank].append((l, lo, hi))
+            first += take
+            done += take
+    assert done == npieces and sum(hi - lo for sh in shares for _, lo, hi in sh) == total
+    return shares

@@ -321,3 +321,46 @@ def test_non_finite_gradients_do_not_fault_or_leak_into_other_blocks(H, O):
     om = oj.states[0].m_codes
     keep = np.repeat(good.reshape(-1, 128)[:, 0], 64)       # 4-bit codes: 64 bytes per block
     assert (gm[:keep.size][keep] == om[:keep.size][keep]).all()
+
+
+@pytest.mark.parametrize("bits", [(4, 4), (3, 8), (8, 3), (16, 2)])
+def test_element_ranges_of_a_tensor_step_like_the_whole_tensor(H, O, bits):
+    """A sharded optimizer hands each rank ranges of a tensor cut on tile boundaries: stepping the
+    ranges as rows of their own (here: two handles, one after the other) writes the same bits as
+    stepping the whole tensor, and the per-layer sums of the ranges add up to the tensor's."""
+    from paper_2604_06836_b200 import multi, stq
+    bm, bv = bits
+    n, block, dev = 5 * 4096 + 777, 128, "cuda"
+    g0 = torch.Generator(device=dev).manual_seed(5)
+    theta = torch.empty(n, device=dev).normal_(0, 0.02, generator=g0)
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, grad_dtype=stq.GRAD_BF16)
+    cuts = [r for sh in multi.partition([n], 2) for r in sh]
+    assert len(cuts) == 2 and cuts[0][2] == cuts[1][1]
+
+    def view(st, lo, hi):     # the range's slice of a whole-tensor state (no copy: same device memory)
+        return stq.QState(st.m_codes[lo * bm // 8:], st.m_scales[lo // block:], bm,
+                          st.v_codes[lo * bv // 8:], st.v_scales[lo // block:], bv)
+
+    whole_p, split_p = theta.clone(), theta.clone()
+    whole_s, split_s = stq.alloc_state(n, block, bm, bv, dev), stq.alloc_state(n, block, bm, bv, dev)
+    h_whole, h_a, h_b = stq.Handle(), stq.Handle(), stq.Handle()
+    h_whole.init_state(stq.table([stq.make_row(n, block, None, whole_s)]))
+    for h, (_, lo, hi) in zip((h_a, h_b), cuts):
+        h.init_state(stq.table([stq.make_row(hi - lo, block, None, view(split_s, lo, hi))]))
+    for t in (1, 2, 3):
+        g = (torch.empty(n, device=dev).normal_(0, 1e-3, generator=g0)).to(torch.bfloat16)
+        h_whole.step(stq.table([stq.make_row(n, block, whole_s, whole_s, whole_p, g, 0.01)]), t=t,
+                     flags=stq.WITH_STATS, **hp)
+        total = np.zeros(4)
+        for h, (_, lo, hi) in zip((h_a, h_b), cuts):
+            v = view(split_s, lo, hi)
+            h.step(stq.table([stq.make_row(hi - lo, block, v, v, split_p[lo:hi], g[lo:hi], 0.01)]), t=t,
+                   flags=stq.WITH_STATS, **hp)
+            total += h.layer_stats(1)[0]
+        want = h_whole.layer_stats(1)[0]
+        assert torch.equal(whole_p, split_p)
+        for a, b in ((whole_s.m_codes, split_s.m_codes), (whole_s.v_codes, split_s.v_codes),
+                     (whole_s.m_scales, split_s.m_scales), (whole_s.v_scales, split_s.v_scales)):
+            assert torch.equal(a, b)
+        assert total[3] == want[3] == n
+        np.testing.assert_allclose(total[:3], want[:3], rtol=1e-6, atol=1e-12)
