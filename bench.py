@@ -203,8 +203,29 @@ def run_ours(args, w, bits_m, bits_v):
             dist.barrier()
         torch.cuda.synchronize()
 
+    # --shard: strong scaling.  Every rank keeps the optimizer state of a block-aligned slice of the
+    # parameter list and steps only that; the per-layer sums are added over ranks on decision steps.
+    w_global, L_global, layer_of_row = w, len(w.shapes), None
+    if args.shard:
+        from dataclasses import replace
+        from paper_2604_06836_b200 import multi as _multi
+        mine = _multi.partition(w.numels, world)[rank]
+        layer_of_row = np.array([l for l, _, _ in mine], dtype=np.int64)
+        w = replace(w, name=w.name + f"-shard{rank}of{world}",
+                    shapes=tuple((f"{w.shapes[l][0]}[{lo}:{hi}]", (hi - lo,)) for l, lo, hi in mine))
+        bits_m, bits_v = bits_m[layer_of_row], bits_v[layer_of_row]
+
     job = Job(w, bits_m, bits_v, device=dev)
     job.draw_grads(1)
+
+    def decide(t):
+        st = job.layer_stats()
+        if layer_of_row is not None:
+            from paper_2604_06836_b200 import multi as _multi
+            full = np.zeros((L_global, 4))
+            np.add.at(full, layer_of_row, st)
+            st = _multi.sync_layer_stats(full, dev)
+        pol.decide(st, t)                            # the paper's policy in shadow: widths stay the seeded ones
     pol = stq.Policy(alpha=0.1, tau=100.0, eps_stat=1e-8, interval=w.decision_interval)
     stream = torch.cuda.current_stream()
 
@@ -215,8 +236,7 @@ def run_ours(args, w, bits_m, bits_v):
         dec = one_step_is_decision(t)
         job.step(t, stats=dec)
         if dec:
-            st = job.layer_stats()
-            pol.decide(st, t)                        # the paper's policy in shadow: widths stay the seeded ones
+            decide(t)
         return dec
 
     t = 0
@@ -226,7 +246,7 @@ def run_ours(args, w, bits_m, bits_v):
             # the last warm-up step takes the decision path whatever its index, so that every kernel
             # variant the timed region launches has been loaded before the clock starts
             job.step(t, stats=True)
-            pol.decide(job.layer_stats(), t)
+            decide(t)
         else:
             one_step(t)
     barrier()
@@ -254,7 +274,7 @@ def run_ours(args, w, bits_m, bits_v):
         job.step(t, stats=dec)
         ev[i][1].record(stream)
         if dec:
-            pol.decide(job.layer_stats(), t)
+            decide(t)
         is_dec.append(dec)
     e1.record(stream)
     barrier()
@@ -300,22 +320,24 @@ def run_ours(args, w, bits_m, bits_v):
     from paper_2604_06836_b200 import multi
     params = w.total_params
     total_ms, e2e_ms = multi.max_over_ranks([total_ms, e2e["ms"] if e2e else 0.0], dev)   # slowest rank
-    value = world * params * args.steps / (total_ms * 1e-3)
+    job_params = w_global.total_params if args.shard else world * params     # what all ranks process per step
+    value = job_params * args.steps / (total_ms * 1e-3)
     alg_bytes = job.algorithmic_bytes()
     k_ms = float(kern_ms.mean())
     achieved = alg_bytes / (k_ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "params": params, "tensors": len(w.shapes), "block": w.block,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "strong" if args.shard else "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w_global.name, "params": job_params if args.shard else params, "tensors": len(w.shapes), "block": w.block,
                    "grad_dtype": w.grad_dtype, "loss_scale": w.loss_scale or None, "lp_copy": w.lp_copy or None,
                    "mean_bits": round(W.mean_bits(w, bits_m, bits_v), 3),
                    "decision_interval": w.decision_interval, "decision_steps_timed": int(is_dec.sum()),
                    "l2": ("flushed before every timed step (256 MB write; %.1f MB touched per step)" % (alg_bytes / 1e6)
                           if small else "inputs larger than L2 (%.1f GB touched per step)" % (alg_bytes / 1e9)),
-                   "parallelism": "replicas" if world > 1 else "single", "grid": job.handle.grid_size,
+                   "parallelism": ("sharded over %d ranks (this rank: %d parameters)" % (world, params) if args.shard
+                                   else "replicas" if world > 1 else "single"), "grid": job.handle.grid_size,
                    "state_bytes": job.state_bytes(), "fp32_state_bytes": 8 * params,
                    "state_saved_frac": 1.0 - job.state_bytes() / (8.0 * params)},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -334,7 +356,7 @@ def run_ours(args, w, bits_m, bits_v):
         "gpu_params_per_s_per_gpu": params * args.steps / (total_ms * 1e-3),
     }
     if e2e:
-        line["e2e"] = {"value": world * params * e2e["steps"] / (e2e_ms * 1e-3), "unit": UNIT,
+        line["e2e"] = {"value": job_params * e2e["steps"] / (e2e_ms * 1e-3), "unit": UNIT,
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"],
                        "ms_per_step": e2e_ms / e2e["steps"]}
     if rank == 0 and not args.no_cpu_baseline and world == 1 and not amp:
@@ -389,6 +411,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--shard", action="store_true",
+                    help="strong scaling: each rank owns a block-aligned slice of the parameter list "
+                         "(default: every rank steps a full replica)")
     args = ap.parse_args()
     w = W.config(args.config)
     bits_m, bits_v, _ = W.draw_bits(w)

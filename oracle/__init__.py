@@ -33,7 +33,8 @@ def build(force: bool = False) -> str:
 class HParams(C.Structure):
     _fields_ = [("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
                 ("weight_decay", C.c_double), ("step", C.c_int64), ("decoupled_wd", C.c_int),
-                ("grad_dtype", C.c_int), ("inv_grad_scale", C.c_float), ("found_inf", C.c_int)]
+                ("grad_dtype", C.c_int), ("inv_grad_scale", C.c_float), ("found_inf", C.c_int),
+                ("v_mode", C.c_int)]
 
 
 class Policy(C.Structure):
@@ -83,7 +84,7 @@ def lib():
     return _lib
 
 
-LINEAR, LOG = 0, 1
+LINEAR, LOG, LOG_PL = 0, 1, 2      # LOG_PL: the log quantizer with the piecewise-linear logarithm
 WIDTHS = (2, 3, 4, 8, 16, 32)
 
 
@@ -195,9 +196,10 @@ def new_state(n: int, block: int, bits_m: int, bits_v: int) -> State:
 def step(theta: np.ndarray, grad: np.ndarray, st: State, block: int, *, lr, beta1, beta2, eps,
          weight_decay, t: int, bits_m_out: int | None = None, bits_v_out: int | None = None,
          decoupled_wd: bool = True, want_stats: bool = False, fp16_grad: bool = False,
-         inv_grad_scale: float = 1.0, found_inf: bool = False):
+         inv_grad_scale: float = 1.0, found_inf: bool = False, v_mode: int = LOG):
     """One Algorithm-1 step on one tensor.  theta is updated in place; returns (new State, stats).
-    A uint16 grad holds bf16 bit patterns, or fp16 ones with fp16_grad=True."""
+    A uint16 grad holds bf16 bit patterns, or fp16 ones with fp16_grad=True.  v_mode: LOG or LOG_PL,
+    the quantizer of the second moment (the stored state must have been written with the same one)."""
     _chk(theta, np.float32)
     n = theta.size
     dt = _grad_dtype(grad, fp16_grad)
@@ -208,7 +210,8 @@ def step(theta: np.ndarray, grad: np.ndarray, st: State, block: int, *, lr, beta
     bv = st.bits_v if bits_v_out is None else bits_v_out
     mc, ms = alloc_state(n, bm, block)
     vc, vs = alloc_state(n, bv, block)
-    hp = HParams(lr, beta1, beta2, eps, weight_decay, t, 1 if decoupled_wd else 0, dt, inv_grad_scale, 0)
+    hp = HParams(lr, beta1, beta2, eps, weight_decay, t, 1 if decoupled_wd else 0, dt, inv_grad_scale, 0,
+                 v_mode)
     stats = np.zeros(4, dtype=np.float64) if want_stats else None
     rc = lib().orc_step(_p(theta), _p(grad), n, block,
                         _p(st.m_codes), _p(st.m_scales), st.bits_m,

@@ -129,8 +129,17 @@ inline float dequant_lin(uint32_t code, float s, int b) {
 //    c = fl(fl(1/s) * sqrt2): floor(log2(x*sqrt2/s)) is that exponent.
 //  * b = 8, 16: d = log-distance to the maximum in octaves from the split logarithm,
 //    q = clamp(K + round-half-even(d*K/R), 0, K).
+//
+// Variant "pl" (mode 2; an alternative reading of "logarithmic", integer-only at widths 8 and 16):
+// the logarithm is replaced by the piecewise-linear one that the fp32 bit pattern itself is,
+// pl(x) = bits(x) * 2^-23 - 127 (equal to log2 at powers of two, linear in the mantissa between them).
+//  * d = pl(x) - pl(s) = (bits(x) - bits(s)) * 2^-23, an integer subtraction, floored at -R octaves;
+//    q = clamp(K + round-half-even(fl32(bits(x) - bits(s)) * (K/R * 2^-23)), 0, K).
+//  * decode: bits(x^) = max(bits(s) + round-half-even(fl((q - K) * (fl(R/K) * 2^23))), 0).
+//  * widths <= 4 are the octave code above in both variants.
 const float kSqrt2 = 0x1.6a09e6p+0f;
-void quant_log_block(const float* x, uint64_t n, int b, uint32_t* code, float* scale) {
+const float kTwo23 = 8388608.0f;
+void quant_log_block(const float* x, uint64_t n, int b, uint32_t* code, float* scale, bool pl) {
   float s = 0.0f;
   for (uint64_t i = 0; i < n; ++i) if (x[i] > s) s = x[i];
   if (s < kTinyScale) {
@@ -153,6 +162,21 @@ void quant_log_block(const float* x, uint64_t n, int b, uint32_t* code, float* s
     return;
   }
   const float a_b = (float)K / (float)R;          // exact: 8.5, 2184.5
+  if (pl) {
+    const int64_t floor_d = -(int64_t)R * (int64_t)(1 << 23);
+    const float a_bits = a_b / kTwo23;            // exact scaling by a power of two
+    for (uint64_t i = 0; i < n; ++i) {
+      int64_t di = (int64_t)f2u(x[i]) - (int64_t)f2u(s);
+      if (di < floor_d) di = floor_d;
+      float df = (float)di;                       // nearest-even when the difference needs > 24 bits
+      double r = nearbyint((double)df * (double)a_bits);
+      double q = (double)K + r;
+      if (q < 0) q = 0;
+      if (q > K) q = K;
+      code[i] = (uint32_t)q;
+    }
+    return;
+  }
   const int Es = lg_E(s);
   const float Ps = lg_P(s);
   for (uint64_t i = 0; i < n; ++i) {
@@ -166,24 +190,32 @@ void quant_log_block(const float* x, uint64_t n, int b, uint32_t* code, float* s
     code[i] = (uint32_t)q;
   }
 }
-inline float dequant_log(uint32_t code, float s, int b) {
+inline float dequant_log(uint32_t code, float s, int b, bool pl) {
   const int K = K_of(b), R = R_of(b);
   const float c_b = (float)R / (float)K;
   float rf = (float)((int)code - K);
+  if (pl && b > 4) {
+    float step_bits = c_b * kTwo23;               // exact scaling by a power of two
+    float ef = rf * step_bits;
+    int64_t xb = (int64_t)f2u(s) + (int64_t)nearbyintf(ef);
+    if (xb < 0) xb = 0;
+    return u2f((uint32_t)xb);
+  }
   float e = rf * c_b;
   float y = ex2(e);
   return s * y;
 }
 
 // ---- state (de)coding over a whole range ------------------------------------------------------
-// mode 0 = linear (m), 1 = log (v).  Width 32 stores raw fp32 and no scales.
+// mode 0 = linear (m), 1 = log (v), 2 = log with the piecewise-linear logarithm (v, variant "pl").
+// Width 32 stores raw fp32 and no scales.
 void decode_state(const uint8_t* codes, const float* scales, uint64_t n, int b, uint32_t block,
                   int mode, float* out) {
   if (b == 32) { std::memcpy(out, codes, n * 4); return; }
   for (uint64_t i = 0; i < n; ++i) {
     uint32_t c = get_code(codes, i, b);
     float s = scales[i / block];
-    out[i] = mode == 0 ? dequant_lin(c, s, b) : dequant_log(c, s, b);
+    out[i] = mode == 0 ? dequant_lin(c, s, b) : dequant_log(c, s, b, mode == 2);
   }
 }
 void encode_state(const float* x, uint64_t n, int b, uint32_t block, int mode, uint8_t* codes,
@@ -194,7 +226,7 @@ void encode_state(const float* x, uint64_t n, int b, uint32_t block, int mode, u
   for (uint64_t j = 0, k = 0; j < n; j += block, ++k) {
     uint64_t len = n - j < block ? n - j : block;
     if (mode == 0) quant_lin_block(x + j, len, b, tmp.data(), scales + k);
-    else quant_log_block(x + j, len, b, tmp.data(), scales + k);
+    else quant_log_block(x + j, len, b, tmp.data(), scales + k, mode == 2);
     for (uint64_t i = 0; i < len; ++i) put_code(codes, j + i, b, tmp[i]);
   }
 }
@@ -250,6 +282,7 @@ struct orc_hparams {
   int grad_dtype;      // 0 = fp32, 1 = bf16, 2 = fp16
   float inv_grad_scale;  // loss-scaled training: every gradient is multiplied by this first (1 = off)
   int found_inf;         // non-zero: a non-finite gradient was found, the step is skipped
+  int v_mode;            // quantizer of the second moment: 1 = log, 2 = its "pl" variant
 };
 
 uint64_t orc_codes_bytes(uint64_t n, int bits) { return codes_bytes(n, bits); }
@@ -267,7 +300,7 @@ void orc_unpack(const uint8_t* in, uint64_t n, int bits, uint32_t* code) {
   for (uint64_t i = 0; i < n; ++i) code[i] = get_code(in, i, bits);
 }
 
-// Quantize / dequantize a whole tensor state.  mode 0 = linear (m), 1 = log (v).
+// Quantize / dequantize a whole tensor state.  mode 0 = linear (m), 1 = log (v), 2 = log "pl" (v).
 int orc_quantize(const float* x, uint64_t n, int bits, uint32_t block, int mode, uint8_t* codes,
                  float* scales) {
   if (!width_ok(bits) || block == 0) return -1;
@@ -313,12 +346,14 @@ int orc_step(float* theta, const void* grad, uint64_t n, uint32_t block,
   if (!width_ok(bits_m_in) || !width_ok(bits_v_in) || !width_ok(bits_m_out) || !width_ok(bits_v_out))
     return -1;
   if (block == 0 || hp->step < 1) return -1;
+  if (hp->v_mode != 1 && hp->v_mode != 2) return -1;
+  const int vmode = hp->v_mode;
   if (hp->found_inf) return 0;          // skipped step: nothing is touched
   std::vector<float> m(n), v(n), g(n);
 
   // stored m_{t-1}, v_{t-1}
   decode_state(m_codes_in, m_scales_in, n, bits_m_in, block, 0, m.data());
-  decode_state(v_codes_in, v_scales_in, n, bits_v_in, block, 1, v.data());
+  decode_state(v_codes_in, v_scales_in, n, bits_v_in, block, vmode, v.data());
 
   // gradient as fp32 (bf16 and fp16 widen exactly), brought back from the loss scale
   for (uint64_t i = 0; i < n; ++i) g[i] = grad_to_f32(grad, hp->grad_dtype, i) * hp->inv_grad_scale;
@@ -343,11 +378,11 @@ int orc_step(float* theta, const void* grad, uint64_t n, uint32_t block,
 
   // Quantize(m_t, linear), Quantize(v_t, log) at the widths assigned for this step
   encode_state(m.data(), n, bits_m_out, block, 0, m_codes_out, m_scales_out);
-  encode_state(v.data(), n, bits_v_out, block, 1, v_codes_out, v_scales_out);
+  encode_state(v.data(), n, bits_v_out, block, vmode, v_codes_out, v_scales_out);
 
   // the update consumes the quantized states
   decode_state(m_codes_out, m_scales_out, n, bits_m_out, block, 0, m.data());
-  decode_state(v_codes_out, v_scales_out, n, bits_v_out, block, 1, v.data());
+  decode_state(v_codes_out, v_scales_out, n, bits_v_out, block, vmode, v.data());
 
   const double b1 = hp->beta1, b2 = hp->beta2, lr = hp->lr, eps = hp->eps;
   const double bc1 = 1.0 - std::pow(b1, (double)hp->step);
