@@ -133,12 +133,20 @@ inline float dequant_lin(uint32_t code, float s, int b) {
 // Variant "pl" (mode 2; an alternative reading of "logarithmic", integer-only at widths 8 and 16):
 // the logarithm is replaced by the piecewise-linear one that the fp32 bit pattern itself is,
 // pl(x) = bits(x) * 2^-23 - 127 (equal to log2 at powers of two, linear in the mantissa between them).
-//  * d = pl(x) - pl(s) = (bits(x) - bits(s)) * 2^-23, an integer subtraction, floored at -R octaves;
-//    q = clamp(K + round-half-even(fl32(bits(x) - bits(s)) * (K/R * 2^-23)), 0, K).
-//  * decode: bits(x^) = max(bits(s) + round-half-even(fl((q - K) * (fl(R/K) * 2^23))), 0).
+// With D = R * 2^23 (R octaves in units of the bit pattern), all in exact integers:
+//  * n = min(bits(s) - bits(x), D), the distance below the block maximum;
+//    j = floor(n*K/D + 1/2) code steps below the maximum; q = K - j.
+//  * decode: j = K - q; n' = floor(j*B/2^S + 1/2) with B = round(D * 2^S / K) and S = 12 (8 bits),
+//    20 (16 bits), so that j*B fits 64 bits with B below 2^32; bits(x^) = max(bits(s) - n', 0).
+//    n' = k * 2^23 exactly whenever j is a whole number k of octaves.
 //  * widths <= 4 are the octave code above in both variants.
 const float kSqrt2 = 0x1.6a09e6p+0f;
-const float kTwo23 = 8388608.0f;
+inline int pl_shift(int b) { return b == 8 ? 12 : 20; }
+inline int64_t pl_octaves(int b) { return (int64_t)R_of(b) << 23; }                    // D
+inline int64_t pl_step(int b) {                                                        // B
+  const int64_t K = K_of(b), D = pl_octaves(b);
+  return (2 * (D << pl_shift(b)) + K) / (2 * K);
+}
 void quant_log_block(const float* x, uint64_t n, int b, uint32_t* code, float* scale, bool pl) {
   float s = 0.0f;
   for (uint64_t i = 0; i < n; ++i) if (x[i] > s) s = x[i];
@@ -163,17 +171,12 @@ void quant_log_block(const float* x, uint64_t n, int b, uint32_t* code, float* s
   }
   const float a_b = (float)K / (float)R;          // exact: 8.5, 2184.5
   if (pl) {
-    const int64_t floor_d = -(int64_t)R * (int64_t)(1 << 23);
-    const float a_bits = a_b / kTwo23;            // exact scaling by a power of two
+    const int64_t D = pl_octaves(b);
     for (uint64_t i = 0; i < n; ++i) {
-      int64_t di = (int64_t)f2u(x[i]) - (int64_t)f2u(s);
-      if (di < floor_d) di = floor_d;
-      float df = (float)di;                       // nearest-even when the difference needs > 24 bits
-      double r = nearbyint((double)df * (double)a_bits);
-      double q = (double)K + r;
-      if (q < 0) q = 0;
-      if (q > K) q = K;
-      code[i] = (uint32_t)q;
+      int64_t dist = (int64_t)f2u(s) - (int64_t)f2u(x[i]);
+      if (dist > D) dist = D;
+      int64_t j = (2 * dist * K + D) / (2 * D);   // floor(dist*K/D + 1/2)
+      code[i] = (uint32_t)(K - j);
     }
     return;
   }
@@ -195,9 +198,10 @@ inline float dequant_log(uint32_t code, float s, int b, bool pl) {
   const float c_b = (float)R / (float)K;
   float rf = (float)((int)code - K);
   if (pl && b > 4) {
-    float step_bits = c_b * kTwo23;               // exact scaling by a power of two
-    float ef = rf * step_bits;
-    int64_t xb = (int64_t)f2u(s) + (int64_t)nearbyintf(ef);
+    const int64_t j = (int64_t)K - (int64_t)code;
+    const int S = pl_shift(b);
+    const int64_t below = (j * pl_step(b) + ((int64_t)1 << (S - 1))) >> S;
+    int64_t xb = (int64_t)f2u(s) - below;
     if (xb < 0) xb = 0;
     return u2f((uint32_t)xb);
   }
