@@ -119,7 +119,8 @@ def oracle_sample_run(w: W.Workload, bits_m, bits_v, budget_s: float, repeats: i
     g = torch.from_numpy(g32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16).copy() \
         if w.grad_dtype == "bf16" else g32
     st = O.new_state(chunk, w.block, 4, 4)
-    kw = dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, weight_decay=w.weight_decay)
+    kw = dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, weight_decay=w.weight_decay,
+              v_mode=O.LOG_PL if w.v_log == "pl" else O.LOG)
     t0 = time.perf_counter()
     st, _ = O.step(th, g, st, w.block, t=1, **kw)
     rate1 = chunk / (time.perf_counter() - t0)
@@ -331,7 +332,7 @@ def run_ours(args, w, bits_m, bits_v):
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "strong" if args.shard else "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w_global.name, "params": job_params if args.shard else params, "tensors": len(w.shapes), "block": w.block,
-                   "grad_dtype": w.grad_dtype, "loss_scale": w.loss_scale or None, "lp_copy": w.lp_copy or None,
+                   "grad_dtype": w.grad_dtype, "loss_scale": w.loss_scale or None, "lp_copy": w.lp_copy or None, "v_log": w.v_log,
                    "mean_bits": round(W.mean_bits(w, bits_m, bits_v), 3),
                    "decision_interval": w.decision_interval, "decision_steps_timed": int(is_dec.sum()),
                    "l2": ("flushed before every timed step (256 MB write; %.1f MB touched per step)" % (alg_bytes / 1e6)
@@ -381,7 +382,7 @@ def run_e2e(job, w, args):
     for i, n in enumerate(job.numels):
         s = job.states[i]
         hs = stq.QState(s.m_codes.cpu().pin_memory(), s.m_scales.cpu().pin_memory(), s.bits_m,
-                        s.v_codes.cpu().pin_memory(), s.v_scales.cpu().pin_memory(), s.bits_v)
+                        s.v_codes.cpu().pin_memory(), s.v_scales.cpu().pin_memory(), s.bits_v, s.v_log)
         host_states.append(hs)
         o = job.offsets[i]
         rows.append(stq.make_row(n, job.block, hs, hs, host_p[o:o + n], host_g[o:o + n], job.wd[i]))
@@ -411,11 +412,16 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--v-log", default="poly", choices=["poly", "pl"],
+                    help="variant of the v quantizer at widths 8 and 16 (default: the polynomial logarithm)")
     ap.add_argument("--shard", action="store_true",
                     help="strong scaling: each rank owns a block-aligned slice of the parameter list "
                          "(default: every rank steps a full replica)")
     args = ap.parse_args()
     w = W.config(args.config)
+    if args.v_log != "poly":
+        from dataclasses import replace
+        w = replace(w, name=w.name + "-v" + args.v_log, v_log=args.v_log)
     bits_m, bits_v, _ = W.draw_bits(w)
     if args.impl == "reference":
         run_reference(args, w, bits_m, bits_v)

@@ -29,6 +29,15 @@
  *  - first moment: code u = q + 2^(b-1), q in [-qmax, qmax], qmax = 2^(b-1)-1, value scale*q/qmax.
  *  - second moment: code u in [0, 2^b-1]; value scale * 2^((u-K)*R/K), K = 2^b-1, R = min(K,30);
  *    code 0 is a floor level, never zero.  A block whose scale is 0 decodes to all zeros.
+ *  - second moment, variant STQ_VLOG_PL (per tensor, widths 8 and 16 only; the paper names
+ *    logarithmic quantization in Sec. 3.5 without a formula, and this is a second, integer-only
+ *    reading of it): log2 is replaced by the piecewise-linear logarithm that the fp32 bit pattern
+ *    is.  With D = 30 * 2^23: a value x of a block with scale s has distance
+ *    n = min(bits(s) - bits(x), D) and code u = K - floor(n*K/D + 1/2); code u decodes to the
+ *    float whose bit pattern is max(bits(s) - floor(j*B/2^S + 1/2), 0), j = K - u,
+ *    B = round(D*2^S/K), S = 12 (8 bits) or 20 (16 bits).  Exact at whole octaves below the
+ *    maximum; relative error at most 0.7214*30/K octaves.  A state must be read with the variant
+ *    it was written with.
  */
 #ifndef STQ_H_
 #define STQ_H_
@@ -65,6 +74,9 @@ enum { STQ_GRAD_F32 = 0, STQ_GRAD_BF16 = 1, STQ_GRAD_F16 = 2 };
 /* type of the optional low-precision copy of the updated parameters (stq_tensor.param_lp) */
 enum { STQ_LP_NONE = 0, STQ_LP_BF16 = 1, STQ_LP_F16 = 2 };
 
+/* quantizer of the second moment at widths 8 and 16 (stq_tensor.v_log); see "Stored layout" */
+enum { STQ_VLOG_POLY = 0, STQ_VLOG_PL = 1 };
+
 /* flags of stq_step */
 enum { STQ_WITH_STATS = 1u };
 
@@ -90,6 +102,9 @@ typedef struct stq_tensor {
                              /* rounded (nearest-even) to lp_dtype, the model's working copy   */
                              /* in mixed-precision training; 8-byte aligned; written by         */
                              /* stq_step only                                                  */
+  uint32_t v_log;            /* STQ_VLOG_*: how the second moment is coded at widths 8 and 16,  */
+                             /* on the way in and on the way out (ignored at other widths)     */
+  uint32_t reserved;         /* must be 0                                                      */
 } stq_tensor;
 
 typedef struct stq_hparams {

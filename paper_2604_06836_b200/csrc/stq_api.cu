@@ -116,6 +116,7 @@ bool overlap(const void* a, size_t na, const void* b, size_t nb) {
 int validate_row(const stq_tensor& t, int kind) {
   if (t.numel == 0 || t.numel > (1ull << 40)) return STQ_E_NUMEL;
   if (t.lp_dtype > STQ_LP_F16) return STQ_E_ARG;
+  if (t.v_log > STQ_VLOG_PL || t.reserved != 0) return STQ_E_ARG;
   if (kind == kKindStep && t.lp_dtype != STQ_LP_NONE) {
     if (!t.param_lp) return STQ_E_NULL;
     if (!aligned(t.param_lp, 8)) return STQ_E_ALIGN;
@@ -166,6 +167,13 @@ int validate_row(const stq_tensor& t, int kind) {
   return STQ_OK;
 }
 
+// Tensors with the same key run the same specialised body of the main kernel: the two widths, and
+// for v at 8 or 16 bits the variant of its quantizer.  Ordered from cheap to expensive v codes.
+int body_key(const stq_tensor& t) {
+  const int pl = t.v_log == STQ_VLOG_PL && (t.bits_v == 8 || t.bits_v == 16) ? 1 : 0;
+  return (t.bits_v * 2 + (1 - pl)) * 64 + t.bits_m;
+}
+
 bool row_is_wide(const stq_tensor& t, int kind) {
   if (kind == kKindStats) return false;
   if (t.bits_m_out == 32 || t.bits_v_out == 32) return true;
@@ -208,7 +216,8 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     fast += nf;
     if (!wide) slow_narrow += nt - nf;
     sig[l] = t.numel | (wide ? 1ull << 63 : 0ull) | (fast_ok ? 1ull << 62 : 0ull) |
-             ((uint64_t)t.bits_m << 56) | ((uint64_t)t.bits_v << 48);   // numel <= 2^40
+             ((uint64_t)t.bits_m << 56) | ((uint64_t)t.bits_v << 48) |
+             ((uint64_t)(t.v_log & 1u) << 47);                           // numel <= 2^40
   }
   if (total > 0xFFFFFFF0ull) return STQ_E_NUMEL;
   // the tile map depends only on sizes and classes: skip it when unchanged
@@ -238,8 +247,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   std::vector<int> order(L);
   for (int l = 0; l < L; ++l) order[l] = l;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
-    const int ka = tensors[a].bits_v * 64 + tensors[a].bits_m, kb = tensors[b].bits_v * 64 + tensors[b].bits_m;
-    return ka < kb;
+    return body_key(tensors[a]) < body_key(tensors[b]);
   });
   std::vector<uint32_t> fast0(L);
   stq::FastSched* hs = reinterpret_cast<stq::FastSched*>(st + off_sched);
@@ -256,12 +264,13 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
       fast0[l] = next_fast;
       if (nfast[l] == 0) continue;
       const stq_tensor& t = tensors[l];
-      const int key = t.bits_v * 64 + t.bits_m;
+      const int key = body_key(t);
       if (key != last_key && hs->ng < (uint32_t)stq::kFastMaxGroups) {
         hs->grp_begin[hs->ng++] = next_fast;
         last_key = key;
       }
       double w = t.bits_v == 16 ? 1.45 : t.bits_v == 8 ? 1.2 : 1.0;
+      if (t.v_log == STQ_VLOG_PL && t.bits_v >= 8) w = t.bits_v == 16 ? 1.1 : 1.0;
       if (t.bits_v == 3 || t.bits_m == 3) w += 0.06;
       if (t.bits_m == 16) w += 0.08;
       cost[hs->ng - 1] += w * nfast[l];
@@ -336,6 +345,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     d.bm_in = t.bits_m; d.bv_in = t.bits_v; d.bm_out = t.bits_m_out; d.bv_out = t.bits_v_out;
     d.wd = t.weight_decay;
     d.lp_dtype = kind == kKindStep ? t.lp_dtype : 0u;
+    d.v_pl = kind != kKindStats && t.v_log == STQ_VLOG_PL ? 1u : 0u;
     d.param_lp = kind == kKindStep && t.lp_dtype != STQ_LP_NONE ? t.param_lp : nullptr;
     ht[l] = d;
   }

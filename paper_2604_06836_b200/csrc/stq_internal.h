@@ -37,6 +37,7 @@ struct TensorDesc {
   unsigned char bm_in, bv_in, bm_out, bv_out;
   float wd;                 // fp32(lambda)
   unsigned int lp_dtype;    // 0: none, 1: bf16, 2: fp16
+  unsigned int v_pl;        // 1: the second moment uses the piecewise-linear logarithm at widths 8 and 16
   void* param_lp;           // low-precision copy of the updated parameters, or nullptr
 };
 
@@ -62,7 +63,7 @@ cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const
 
 // Work list of the main step kernel: the fast tiles [0, n_fast) of the tile order, cut into groups
 // of equal width pair.  Lives in device memory; the counters are zeroed before every launch.
-constexpr int kFastMaxGroups = 32;     // 25 width pairs exist
+constexpr int kFastMaxGroups = 64;     // 5 widths of m x (5 widths of v + 2 variants at 8 and 16 bits) = 35 bodies
 constexpr int kFastMaxGrid = 4096;
 constexpr uint32_t kFastChunk = 8;     // tiles handed out per counter increment (fewer for small launches)
 struct FastSched {

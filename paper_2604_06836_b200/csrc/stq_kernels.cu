@@ -267,10 +267,22 @@ __device__ __forceinline__ float decode_lin(uint32_t c, float s, const LinW& w) 
   const float q = __fadd_rn(__uint_as_float(kTwo23Bits | c), -(kTwo23 + w.halff));
   return __fmul_rn(s, __fmul_rn(q, w.invq));
 }
-__device__ __forceinline__ float decode_log(uint32_t c, float s, int b, const LogW& w) {
+// Variant with the piecewise-linear logarithm (widths 8, 16), in integers: code steps below the
+// maximum -> distance in units of the bit pattern, n' = floor(j*B/2^S + 1/2).
+__device__ __forceinline__ uint32_t pl_step(int b) { return b == 8 ? 4042322161u : 4026593281u; }   // round(30*2^23*2^S/K)
+__device__ __forceinline__ int pl_shift(int b) { return b == 8 ? 12 : 20; }
+__device__ __forceinline__ float decode_pl(uint32_t j, uint32_t s_bits, int b) {
+  const int S = pl_shift(b);
+  const unsigned long long below = ((unsigned long long)j * pl_step(b) + (1ull << (S - 1))) >> S;
+  const int xb = (int)s_bits - (int)(uint32_t)below;
+  return __uint_as_float((uint32_t)max(xb, 0));
+}
+
+__device__ __forceinline__ float decode_log(uint32_t c, float s, int b, const LogW& w, bool pl) {
   if (b <= 4) {   // one octave per code: 2^(c-K)
     return __fmul_rn(s, __uint_as_float((c + (uint32_t)(127 - w.K)) << 23));
   }
+  if (pl) return decode_pl((uint32_t)w.K - c, __float_as_uint(s), b);
   const float rf = __fadd_rn(__uint_as_float(kTwo23Bits | c), -(kTwo23 + (float)w.K));
   return __fmul_rn(s, ex2_poly(__fmul_rn(rf, w.c)));
 }
@@ -394,6 +406,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
       const uint32_t B = T->block;
       const int lgB = B == 128 ? 7 : B == 256 ? 8 : 9;
       const int bm_in = T->bm_in, bv_in = T->bv_in, bm_out = T->bm_out, bv_out = T->bv_out;
+      const bool pl = T->v_pl != 0u;
 
       int nvl[R];
 #pragma unroll
@@ -485,7 +498,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
               uint32_t c[4];
               split_codes<WIDE>(rawv[r], bv_in, lane, c);
 #pragma unroll
-              for (int k = 0; k < 4; ++k) vh[k] = decode_log(c[k], s_v_in[r], bv_in, gw_in);
+              for (int k = 0; k < 4; ++k) vh[k] = decode_log(c[k], s_v_in[r], bv_in, gw_in, pl);
             }
             if constexpr (MODE == kStep) {
               th[r][0] = th4[r].x; th[r][1] = th4[r].y; th[r][2] = th4[r].z; th[r][3] = th4[r].w;
@@ -608,6 +621,20 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
                 const uint32_t yb = __float_as_uint(fmaxf(__fmul_rn(vt[r][k], c), ymin));
                 x[k] = yb >> 23;
                 if constexpr (MODE == kStep) vq[k] = __fmul_rn(s, __uint_as_float(yb & 0x7F800000u));
+              }
+            } else if (pl) {
+              // distance below the block maximum in units of the bit pattern, at most 30 octaves;
+              // j = floor(n*K/D + 1/2) = (n * (512*K/30) + 2^31) >> 32, the factor being a whole number
+              const uint32_t s_enc = zero ? 0x7F800000u : mxv[r];     // zero block: every code is the floor
+              const uint32_t s_dec = zero ? 0u : mxv[r];
+              const uint32_t A = bv_out == 8 ? 4352u : 1118464u;
+              sub = 0u;
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const uint32_t n = min(s_enc - __float_as_uint(vt[r][k]), 30u << 23);
+                const uint32_t j = (uint32_t)(((unsigned long long)n * A + (1ull << 31)) >> 32);
+                x[k] = (uint32_t)gw.K - j;
+                if constexpr (MODE == kStep) vq[k] = decode_pl(j, s_dec, bv_out);
               }
             } else {
               const int Es = zero ? kZeroBlockExp : (int)(mxv[r] >> 23);

@@ -60,7 +60,8 @@ struct __align__(16) TileInfo {
   float* mso;
   float* vso;
   uint16_t* lp;        // low-precision copy of the parameters (2 bytes per element), or nullptr
-  uint32_t packed;     // width index of m | of v << 8 (0..4 for 2,3,4,8,16 bits) | log2(block) << 16 | lp dtype << 24
+  uint32_t packed;     // width index of m | of v << 8 (0..4 for 2,3,4,8,16 bits; 5, 6: 8, 16 bits in the
+                       // piecewise-linear variant) | log2(block) << 16 | lp dtype << 24
   float wdx;           // fp32(lr*wd) (AdamW) or fp32(wd) (L2 mode)
   uint32_t tile;       // index of the tile in the launch's tile order; 0xFFFFFFFF closes the stream
   uint32_t pad;
@@ -69,8 +70,8 @@ static_assert(sizeof(TileInfo) == 64, "TileInfo is read with four 128-bit loads"
 
 constexpr int kOffInfo = kStages * kStageBytes;
 constexpr int kOffBars = kOffInfo + kStages * 64;        // full[kStages], empty[kStages]
-constexpr int kOffLut = kOffBars + 16 * kStages;         // 256 floats: decode table of the 8-bit log code
-constexpr int kSmemBytes = kOffLut + 1024;
+constexpr int kOffLut = kOffBars + 16 * kStages;         // 256 floats: decode table of the 8-bit log code, then
+constexpr int kSmemBytes = kOffLut + 2048;               // 256 integers: the same for its piecewise-linear variant
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: far beyond any copy; then give up
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -227,6 +228,42 @@ __device__ __forceinline__ void decode_log_row(const uint32_t (&w)[2], float s, 
   }
 }
 
+// ---- variant of the log code with the piecewise-linear logarithm (widths 8 and 16), all integers ----
+// Distances are differences of fp32 bit patterns (2^23 units per octave); a block covers 30 octaves.
+template <int B>
+struct Pl {
+  static constexpr uint32_t A = B == 8 ? 4352u : 1118464u;               // 2^32 * K / (30 * 2^23), a whole number
+  static constexpr uint32_t step = B == 8 ? 4042322161u : 4026593281u;   // round(30 * 2^23 * 2^S / K)
+  static constexpr int S = B == 8 ? 12 : 20;
+};
+constexpr uint32_t kPlOctaves = 30u << 23;
+
+// distance below the block maximum of the level j code steps below it: floor(j * step / 2^S + 1/2)
+template <int B>
+__device__ __forceinline__ uint32_t pl_below(uint32_t j) {
+  return (uint32_t)(((unsigned long long)j * Pl<B>::step + (1ull << (Pl<B>::S - 1))) >> Pl<B>::S);
+}
+__device__ __forceinline__ float pl_value(uint32_t s_bits, uint32_t below) {
+  return __uint_as_float((uint32_t)max((int)s_bits - (int)below, 0));
+}
+
+// lutn: pl_below<8>(j) for j = 0..255
+template <int B>
+__device__ __forceinline__ void decode_pl_row(const uint32_t (&w)[2], uint32_t s_bits, const uint32_t* lutn,
+                                              float (&out)[4]) {
+  if constexpr (B == 8) {
+    const uint32_t nw = ~w[0];          // K - code per field
+#pragma unroll
+    for (int k = 0; k < 4; ++k) out[k] = pl_value(s_bits, lutn[(nw >> (8 * k)) & 255u]);
+  } else {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t nw = ~w[k >> 1];
+      out[k] = pl_value(s_bits, pl_below<16>((k & 1) ? nw >> 16 : nw & 0xFFFFu));
+    }
+  }
+}
+
 // Stores the lane's packed field(s) of one row.  f: the 4*B-bit field (two words at 16 bits).
 template <int B>
 __device__ __forceinline__ void store_fields(uint8_t* row_ptr, int lane, uint32_t f0, uint32_t f1) {
@@ -315,6 +352,26 @@ __device__ __forceinline__ void encode_log_row(uint8_t* row_ptr, int lane, const
   }
 }
 
+// The same in the piecewise-linear variant.  s_enc: bit pattern of the block maximum (+inf's for a
+// zero block, which floors every code); s_dec: the same, 0 for a zero block.
+template <int B>
+__device__ __forceinline__ void encode_pl_row(uint8_t* row_ptr, int lane, const float (&v)[4], uint32_t s_enc,
+                                              uint32_t s_dec, const uint32_t* lutn, float (&vq)[4]) {
+  uint32_t j[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t n = min(s_enc - __float_as_uint(v[k]), kPlOctaves);
+    j[k] = (uint32_t)(((unsigned long long)n * Pl<B>::A + (1ull << 31)) >> 32);   // floor(n*K/D + 1/2) <= K
+    uint32_t below;
+    if constexpr (B == 8) below = lutn[j[k]];
+    else below = pl_below<16>(j[k]);
+    vq[k] = pl_value(s_dec, below);
+  }
+  // code = K - j: the complement of j inside its field
+  if constexpr (B == 8) store_fields<8>(row_ptr, lane, ~(j[0] | (j[1] << 8) | (j[2] << 16) | (j[3] << 24)), 0u);
+  else store_fields<16>(row_ptr, lane, ~(j[0] | (j[1] << 16)), ~(j[2] | (j[3] << 16)));
+}
+
 template <int GDT>
 __device__ __forceinline__ void lds_grad(const uint8_t* stage, int elem, float (&g)[4]) {
   if constexpr (GDT == 0) {
@@ -354,10 +411,12 @@ __device__ __forceinline__ uint2 pack_lp(const float (&x)[4], uint32_t lp_dtype)
 // instruction cache, and halving it pays more than the lost overlap between passes.  Specialised on
 // both widths.
 constexpr int RP = kFastRowsPerPass;
-template <int BM, int BV, int GDT, bool AMP>
+template <int BM, int BV, bool VPL, int GDT, bool AMP>
 __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, const TileInfo& ti, const StepConsts& sc,
                                           const float* __restrict__ lut8, int lane, int warp, uint32_t empty_bar,
                                           double* __restrict__ part, float grad_mul) {
+  static_assert(!VPL || BV >= 8, "the piecewise-linear variant exists at 8 and 16 bits");
+  [[maybe_unused]] const uint32_t* lutn = reinterpret_cast<const uint32_t*>(lut8 + 256);
   const int lgB = (int)((ti.packed >> 16) & 0xFFu);
   [[maybe_unused]] const uint32_t lp_dtype = ti.packed >> 24;
   const float lrwd = sc.l2_mode ? 0.0f : ti.wdx;
@@ -382,7 +441,8 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
       lds_codes<BM>(stage + kOffMc + (row0 + r) * (16 * BM), lane, w);
       decode_lin_row<BM>(w, sm, mt[r]);
       lds_codes<BV>(stage + kOffVc + (row0 + r) * (16 * BV), lane, w);
-      decode_log_row<BV>(w, sv, lut8, vt[r]);
+      if constexpr (VPL) decode_pl_row<BV>(w, __float_as_uint(sv), lutn, vt[r]);
+      else decode_log_row<BV>(w, sv, lut8, vt[r]);
     }
     if (pass == R / RP - 1) {   // the last rows are in registers: this warp is done with the stage
       __syncwarp();
@@ -480,9 +540,14 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
           ti.mso[e_mine >> lgB] = zero ? 0.f : x;
           ti.vso[e_mine >> lgB] = __uint_as_float(mv) < kTiny ? 0.f : __uint_as_float(mv);
         }
-        const float ps = lg_poly(mv);
+        if constexpr (!VPL) {
+          const float ps = lg_poly(mv);
 #pragma unroll
-        for (int r = 0; r < RP; ++r) lgc[r] = __shfl_sync(kFull, ps, r);
+          for (int r = 0; r < RP; ++r) lgc[r] = __shfl_sync(kFull, ps, r);
+        } else {
+#pragma unroll
+          for (int r = 0; r < RP; ++r) lgc[r] = 0.f;
+        }
       }
     }
 
@@ -499,7 +564,11 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
       float mq[4], vq[4];
       // mq comes out multiplied by lr/(1-beta1^t): the decode scale carries the factor
       encode_lin_row<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], __fmul_rn(sm_raw, sc.step_size), inv_m[r], mq);
-      encode_log_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], s_v, lgc[r], ebase, lut8, vq);
+      if constexpr (VPL)
+        encode_pl_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], vzero ? 0x7F800000u : mxv[r],
+                          vzero ? 0u : mxv[r], lutn, vq);
+      else
+        encode_log_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], s_v, lgc[r], ebase, lut8, vq);
       float out[4];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
@@ -569,6 +638,7 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
   if (tid < 256) {   // decode table of the 8-bit log code: ex((q - 255) * fl(30/255))
     constexpr float cb = (float)Wd<8>::Roct / (float)Wd<8>::K;
     lut8[tid] = ex2_poly(__fmul_rn((float)(tid - 255), cb));
+    reinterpret_cast<uint32_t*>(lut8 + 256)[tid] = pl_below<8>((uint32_t)tid);
   }
   __syncthreads();
 
@@ -610,7 +680,8 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
         ti.mso = T->ms_out + (e0 >> lgB);
         ti.vso = T->vs_out + (e0 >> lgB);
         ti.lp = T->param_lp ? reinterpret_cast<uint16_t*>(T->param_lp) + e0 : nullptr;
-        ti.packed = width_index(bm) | (width_index(bv) << 8) | (lgB << 16) | (T->lp_dtype << 24);
+        ti.packed = width_index(bm) | ((width_index(bv) + (T->v_pl != 0u && bv >= 8u ? 2u : 0u)) << 8) | (lgB << 16) |
+                    (T->lp_dtype << 24);
         ti.wdx = sc.l2_mode ? T->wd : (float)(sc.lr * (double)T->wd);
         ti.tile = tile;
         ti.pad = 0u;
@@ -662,11 +733,12 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
     const uint32_t ebar = empty0 + 8 * s;
     double* part = partials ? partials + ((size_t)ti.tile * kConsumerWarps + warp) * 3 : nullptr;
 
-#define STQ_CASE(IM, IV, BM, BV) \
-  case IM * 5 + IV: tile_body<BM, BV, GDT, AMP>(stage, ti, sc, lut8, lane, warp, ebar, part, grad_mul); break;
-#define STQ_CASES_M(IM, BM) \
-  STQ_CASE(IM, 0, BM, 2) STQ_CASE(IM, 1, BM, 3) STQ_CASE(IM, 2, BM, 4) STQ_CASE(IM, 3, BM, 8) STQ_CASE(IM, 4, BM, 16)
-    switch ((ti.packed & 0xFFu) * 5 + ((ti.packed >> 8) & 0xFFu)) {
+#define STQ_CASE(IM, IV, BM, BV, VPL) \
+  case IM * 7 + IV: tile_body<BM, BV, VPL, GDT, AMP>(stage, ti, sc, lut8, lane, warp, ebar, part, grad_mul); break;
+#define STQ_CASES_M(IM, BM)                                                                                   \
+  STQ_CASE(IM, 0, BM, 2, false) STQ_CASE(IM, 1, BM, 3, false) STQ_CASE(IM, 2, BM, 4, false) STQ_CASE(IM, 3, BM, 8, false) \
+  STQ_CASE(IM, 4, BM, 16, false) STQ_CASE(IM, 5, BM, 8, true) STQ_CASE(IM, 6, BM, 16, true)
+    switch ((ti.packed & 0xFFu) * 7 + ((ti.packed >> 8) & 0xFFu)) {
       STQ_CASES_M(0, 2)
       STQ_CASES_M(1, 3)
       STQ_CASES_M(2, 4)

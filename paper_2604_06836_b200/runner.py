@@ -55,7 +55,8 @@ class Job:
                 self.params[i].copy_(draw_param(w, i, self.device))
         self.bits_m = np.asarray(bits_m, dtype=np.uint8).copy()
         self.bits_v = np.asarray(bits_v, dtype=np.uint8).copy()
-        self.states = [stq.alloc_state(n, self.block, int(bm), int(bv), self.device)
+        self.v_log = stq.VLOG_PL if w.v_log == "pl" else stq.VLOG_POLY
+        self.states = [stq.alloc_state(n, self.block, int(bm), int(bv), self.device, self.v_log)
                        for n, bm, bv in zip(self.numels, self.bits_m, self.bits_v)]
         self.wd = [w.weight_decay] * self.L
         self._tbl = None
@@ -131,7 +132,7 @@ class Job:
             stq.alloc_codes(n, bm, self.device), stq.alloc_scales(n, bm, self.block, self.device))
         vc, vs = (old.v_codes, old.v_scales) if bv == old.bits_v else (
             stq.alloc_codes(n, bv, self.device), stq.alloc_scales(n, bv, self.block, self.device))
-        return stq.QState(mc, ms, bm, vc, vs, bv)
+        return stq.QState(mc, ms, bm, vc, vs, bv, self.v_log)
 
     def _adopt(self, new_states, bm, bv):
         torch.cuda.current_stream().synchronize()   # old buffers are released below

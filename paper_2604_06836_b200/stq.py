@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libstq.so")
 GRAD_F32, GRAD_BF16, GRAD_F16 = 0, 1, 2
 LP_NONE, LP_BF16, LP_F16 = 0, 1, 2
 WITH_STATS = 1
+VLOG_POLY, VLOG_PL = 0, 1
 WIDTHS = (2, 3, 4, 8, 16, 32)
 
 
@@ -41,6 +42,7 @@ class CTensor(C.Structure):
         ("bits_m", C.c_uint8), ("bits_v", C.c_uint8), ("bits_m_out", C.c_uint8), ("bits_v_out", C.c_uint8),
         ("weight_decay", C.c_float), ("lp_dtype", C.c_uint32),
         ("param_lp", C.c_void_p),
+        ("v_log", C.c_uint32), ("reserved", C.c_uint32),
     ]
 
 
@@ -129,6 +131,7 @@ class QState:
     v_codes: torch.Tensor
     v_scales: torch.Tensor
     bits_v: int
+    v_log: int = 0          # VLOG_POLY | VLOG_PL: how v is coded at widths 8 and 16
 
 
 def alloc_codes(numel: int, bits: int, device) -> torch.Tensor:
@@ -140,9 +143,9 @@ def alloc_scales(numel: int, bits: int, block: int, device) -> torch.Tensor:
     return torch.zeros(n, dtype=torch.float32, device=device)
 
 
-def alloc_state(numel: int, block: int, bits_m: int, bits_v: int, device) -> QState:
+def alloc_state(numel: int, block: int, bits_m: int, bits_v: int, device, v_log: int = 0) -> QState:
     return QState(alloc_codes(numel, bits_m, device), alloc_scales(numel, bits_m, block, device), bits_m,
-                  alloc_codes(numel, bits_v, device), alloc_scales(numel, bits_v, block, device), bits_v)
+                  alloc_codes(numel, bits_v, device), alloc_scales(numel, bits_v, block, device), bits_v, v_log)
 
 
 def _ptr(t: torch.Tensor | None) -> int | None:
@@ -170,6 +173,9 @@ def make_row(numel: int, block: int, st_in: QState | None, st_out: QState, param
     r.m_codes_out, r.m_scales_out = _ptr(st_out.m_codes), _ptr(st_out.m_scales)
     r.v_codes_out, r.v_scales_out = _ptr(st_out.v_codes), _ptr(st_out.v_scales)
     r.bits_m_out, r.bits_v_out = st_out.bits_m, st_out.bits_v
+    if st_in is not None and st_in.v_log != st_out.v_log:
+        raise ValueError("a state is read and written with the same variant of the v quantizer")
+    r.v_log, r.reserved = st_out.v_log, 0
     r.numel, r.block, r.weight_decay = numel, block, weight_decay
     if param_lp is not None:
         r.lp_dtype = LP_BF16 if param_lp.dtype == torch.bfloat16 else LP_F16

@@ -91,6 +91,7 @@ class Workload:
     weight_decay: float = 0.01
     loss_scale: float = 0.0            # > 0: gradients arrive multiplied by it (fp16 training)
     lp_copy: str = ""                  # "bf16" | "fp16": the step also writes the model's working copy
+    v_log: str = "poly"                # "poly" | "pl": variant of the v quantizer at widths 8 and 16
 
     @property
     def numels(self) -> list[int]:

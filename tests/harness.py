@@ -37,6 +37,7 @@ class OracleJob:
         self.states = [O.new_state(n, self.block, int(bm), int(bv))
                        for n, bm, bv in zip(self.numels, self.bits_m, self.bits_v)]
         self.wd = list(job.wd)
+        self.v_mode = O.LOG_PL if job.w.v_log == "pl" else O.LOG
 
     def step(self, grads, t: int, want_stats=False, new_bits=None, decoupled_wd=True, fp16_grad=False,
              inv_grad_scale=1.0, found_inf=False):
@@ -49,7 +50,7 @@ class OracleJob:
                                        beta2=w.beta2, eps=w.eps, weight_decay=self.wd[i], t=t,
                                        bits_m_out=int(bm[i]), bits_v_out=int(bv[i]),
                                        decoupled_wd=decoupled_wd, want_stats=want_stats, fp16_grad=fp16_grad,
-                                       inv_grad_scale=inv_grad_scale, found_inf=found_inf)
+                                       inv_grad_scale=inv_grad_scale, found_inf=found_inf, v_mode=self.v_mode)
             self.upd_mag[i] = np.maximum(self.upd_mag[i], np.maximum(np.abs(self.theta[i] - before), np.abs(self.theta[i])))
             if want_stats:
                 stats[i] = s
@@ -64,7 +65,8 @@ class OracleJob:
                 st.m_codes, st.m_scales = O.repack(st.m_codes, st.m_scales, st.bits_m, int(bm[i]), n, self.block, O.LINEAR)
                 st.bits_m = int(bm[i])
             if bv[i] != st.bits_v:
-                st.v_codes, st.v_scales = O.repack(st.v_codes, st.v_scales, st.bits_v, int(bv[i]), n, self.block, O.LOG)
+                st.v_codes, st.v_scales = O.repack(st.v_codes, st.v_scales, st.bits_v, int(bv[i]), n, self.block,
+                                                   self.v_mode)
                 st.bits_v = int(bv[i])
         self.bits_m, self.bits_v = bm.copy(), bv.copy()
 
@@ -155,6 +157,7 @@ class SampledOracle:
                        for i in range(job.L)]
         self.mag = [np.abs(t) for t in self.theta]
         self.stepped = False      # the working copy exists only after the first step
+        self.v_mode = O.LOG_PL if job.w.v_log == "pl" else O.LOG
 
     def _elem_index(self, i: int) -> torch.Tensor:
         blocks, tail, nb_full = self.sel[i]
@@ -197,7 +200,7 @@ class SampledOracle:
             amp = dict(fp16_grad=True, inv_grad_scale=1.0 / w.loss_scale) if w.grad_dtype == "fp16" else {}
             self.states[i], _ = O.step(self.theta[i], g, self.states[i], self.block, lr=w.lr, beta1=w.beta1,
                                        beta2=w.beta2, eps=w.eps, weight_decay=self.job.wd[i], t=t,
-                                       bits_m_out=bm, bits_v_out=bv, **amp)
+                                       bits_m_out=bm, bits_v_out=bv, v_mode=self.v_mode, **amp)
             self.mag[i] = np.maximum(self.mag[i], np.maximum(np.abs(self.theta[i]), np.abs(self.theta[i] - before)))
 
     def repack(self, new_bits):
@@ -211,7 +214,7 @@ class SampledOracle:
                 st.m_codes, st.m_scales = O.repack(st.m_codes, st.m_scales, st.bits_m, bm, n, self.block, O.LINEAR)
                 st.bits_m = bm
             if bv != st.bits_v:
-                st.v_codes, st.v_scales = O.repack(st.v_codes, st.v_scales, st.bits_v, bv, n, self.block, O.LOG)
+                st.v_codes, st.v_scales = O.repack(st.v_codes, st.v_scales, st.bits_v, bv, n, self.block, self.v_mode)
                 st.bits_v = bv
 
     def compare(self, rel: float, tag=""):

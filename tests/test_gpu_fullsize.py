@@ -23,7 +23,8 @@ def _need(gb):
 
 
 @pytest.mark.parametrize("name,gib", [("cfg2", 4), ("cfg3", 3), ("cfg4", 14), ("cfg5", 26),
-                                      ("gpt2_medium", 8), ("roberta_large", 8), ("vit_b32", 3)])
+                                      ("gpt2_medium", 8), ("roberta_large", 8), ("vit_b32", 3),
+                                      ("cfg3:pl", 3), ("cfg5:pl", 26)])
 def test_full_size_sampled_blocks(name, gib):
     """Each configuration as specified: its step count, its decision interval, statistics on the
     decision steps, and for cfg3 the width change of 10 % of the tensors on every decision step
@@ -32,7 +33,10 @@ def test_full_size_sampled_blocks(name, gib):
     import harness as H
     import oracle
     _need(gib)
-    w = W.config(name)
+    w = W.config(name.split(":")[0])
+    if name.endswith(":pl"):      # the same configuration with the piecewise-linear variant of the v quantizer
+        from dataclasses import replace
+        w = replace(w, v_log="pl")
     bm, bv, _ = W.draw_bits(w)
     job = Job(w, bm, bv)
     so = H.SampledOracle(job, per_tensor=4, seed=1)
@@ -149,7 +153,7 @@ def test_host_buffer_step_matches_device_step():
     for i, n in enumerate(job.numels):
         s = job.states[i]
         hs = stq.QState(s.m_codes.cpu().pin_memory(), s.m_scales.cpu().pin_memory(), s.bits_m,
-                        s.v_codes.cpu().pin_memory(), s.v_scales.cpu().pin_memory(), s.bits_v)
+                        s.v_codes.cpu().pin_memory(), s.v_scales.cpu().pin_memory(), s.bits_v, s.v_log)
         hstates.append(hs)
         o = job.offsets[i]
         rows.append(stq.make_row(n, job.block, hs, hs, hp_[o:o + n], hg[o:o + n], job.wd[i]))

@@ -255,8 +255,9 @@ def test_loss_scaled_gradients_skip_flag_and_low_precision_copy(H, O, gdt):
         codes_before = [s.m_codes.clone() for s in job.states]
         st_o = oj.step([H.to_np(g) for g in grads], t, want_stats=True, fp16_grad=(gdt == torch.float16),
                        inv_grad_scale=1.0 / S, found_inf=skip)
-        job.handle.step(rows(), flags=stq.WITH_STATS, inv_grad_scale=inv, found_inf=flag,
-                        **{**job.hp(t), "grad_dtype": stq.grad_dtype_of(grads[0])})
+        job.handle.step(rows(), flags=stq.WITH_STATS,
+                        **{**job.hp(t), "grad_dtype": stq.grad_dtype_of(grads[0]), "inv_grad_scale": inv,
+                           "found_inf": flag})
         H.compare_job(job, oj, REL_1STEP * t, f"{gdt} t={t}")
         if skip:
             assert all(torch.equal(a, b) for a, b in zip(before, job.params))
@@ -364,3 +365,88 @@ def test_element_ranges_of_a_tensor_step_like_the_whole_tensor(H, O, bits):
             assert torch.equal(a, b)
         assert total[3] == want[3] == n
         np.testing.assert_allclose(total[:3], want[:3], rtol=1e-6, atol=1e-12)
+
+
+# ---- the piecewise-linear variant of the v quantizer -----------------------------------------------------
+@pytest.mark.parametrize("gdt", ["fp32", "bf16"])
+@pytest.mark.parametrize("block", [128, 256, 512])
+@pytest.mark.parametrize("bm", [2, 3, 4, 8, 16])
+@pytest.mark.parametrize("bv", [8, 16])
+def test_pl_variant_every_width_pair(H, O, bm, bv, block, gdt):
+    from dataclasses import replace
+    n = 4096 * 3 + 128 * 5 + 52
+    w = replace(_single(n, block, gdt, seed=bm * 100 + bv), v_log="pl")
+    job = Job(w, [bm], [bv])
+    oj = H.OracleJob(job)
+    H.compare_job(job, oj, 0.0, "init")
+    for t in (1, 2, 3):
+        job.draw_grads(t)
+        st = oj.step([H.to_np(g) for g in job.grads], t, want_stats=True)
+        job.step(t, stats=True)
+        H.compare_job(job, oj, REL_1STEP * t, f"pl t={t}")
+        H.assert_stats_close(job.layer_stats(), st, "pl")
+
+
+@pytest.mark.parametrize("n", [1, 5, 129, 1000, 4095, 4097, 12289])
+def test_pl_variant_ragged_sizes(H, O, n):
+    from dataclasses import replace
+    for bits, block, gdt in (((8, 8), 128, "fp32"), ((3, 16), 256, "bf16")):
+        w = replace(_single(n, block, gdt, seed=n), v_log="pl")
+        job = Job(w, [bits[0]], [bits[1]])
+        oj = H.OracleJob(job)
+        for t in (1, 2):
+            job.draw_grads(t)
+            oj.step([H.to_np(g) for g in job.grads], t)
+            job.step(t)
+            H.compare_job(job, oj, REL_1STEP * t, f"pl n={n} t={t}")
+
+
+def test_pl_variant_small_vit_with_width_churn(H, O):
+    """100 steps with width changes between and inside steps (the octave widths are shared by both
+    variants, so a change 4 -> 8 bits moves a state into the variant's code and back)."""
+    from dataclasses import replace
+    w = replace(W.scaled(W.config("cfg3"), W.small_vit(), steps=100), v_log="pl")
+    _run_config(H, w, 100)
+
+
+def test_pl_variant_small_gpt2_xl_recipe_bf16(H, O):
+    from dataclasses import replace
+    w = replace(W.scaled(W.config("cfg5"), W.small_gpt2(d=100, n_layer=4, vocab=523), steps=20), v_log="pl")
+    _run_config(H, w, 20)
+
+
+def test_pl_variant_extreme_values_and_mixed_tables(H, O):
+    """Zero, denormal and huge blocks in the variant; and a table that mixes tensors of both variants."""
+    n, block, dev = 4096 * 2 + 300, 128, "cuda"
+    import oracle
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
+    g = torch.zeros(n, device=dev)
+    g[:128] = 0.0
+    g[128:256] = 1e-30            # squares underflow: a zero block of v
+    g[256:384] = 1e18             # v near the top of the fp32 range
+    g[384:512] = torch.linspace(1e-12, 1e-3, 128, device=dev)
+    g[4096:] = torch.empty(n - 4096, device=dev).normal_(0, 1e-3, generator=torch.Generator(device=dev).manual_seed(1))
+    h = stq.Handle()
+    states, thetas = [], []
+    for v_log, bv in ((stq.VLOG_PL, 8), (stq.VLOG_POLY, 16), (stq.VLOG_PL, 16), (stq.VLOG_POLY, 8)):
+        st = stq.alloc_state(n, block, 4, bv, dev, v_log)
+        th = torch.full((n,), 0.01, device=dev)
+        states.append(st)
+        thetas.append(th)
+    h.init_state(stq.table([stq.make_row(n, block, None, s) for s in states]))
+    o_states = [oracle.new_state(n, block, s.bits_m, s.bits_v) for s in states]
+    o_thetas = [H.to_np(t) for t in thetas]
+    for t in (1, 2, 3):
+        h.step(stq.table([stq.make_row(n, block, s, s, th, g, 0.01) for s, th in zip(states, thetas)]), t=t, **hp)
+        h.device_status()
+        for i, s in enumerate(states):
+            o_states[i], _ = oracle.step(o_thetas[i], H.to_np(g), o_states[i], block, t=t, weight_decay=0.01,
+                                         v_mode=oracle.LOG_PL if s.v_log == stq.VLOG_PL else oracle.LOG, **hp)
+            H.assert_states_equal(s, o_states[i], f"mixed table row {i} t={t}")
+            H.assert_theta_close(thetas[i], o_thetas[i], REL_1STEP * t * 4, f"mixed table row {i} t={t}",
+                                 upd=np.full(n, 0.01))
+    # a bad variant id is refused before anything runs
+    bad = stq.make_row(n, block, states[0], states[0], thetas[0], g, 0.01)
+    bad.v_log = 7
+    with pytest.raises(stq.StqError):
+        h.step(stq.table([bad]), t=4, **hp)
