@@ -374,19 +374,8 @@ def run_e2e(job, w, args):
     """The same step through stq_step_host: pinned host buffers in, host buffers out, copies timed."""
     from paper_2604_06836_b200 import stq
     steps = max(1, min(args.e2e_steps, args.steps))
-    torch.cuda.synchronize()
-    host_p = job.param_flat.cpu().pin_memory()
-    host_g = job.grad_flat.cpu().pin_memory()
-    rows = []
-    host_states = []
-    for i, n in enumerate(job.numels):
-        s = job.states[i]
-        hs = stq.QState(s.m_codes.cpu().pin_memory(), s.m_scales.cpu().pin_memory(), s.bits_m,
-                        s.v_codes.cpu().pin_memory(), s.v_scales.cpu().pin_memory(), s.bits_v, s.v_log)
-        host_states.append(hs)
-        o = job.offsets[i]
-        rows.append(stq.make_row(n, job.block, hs, hs, host_p[o:o + n], host_g[o:o + n], job.wd[i]))
-    tbl = stq.table(rows)
+    # the caller's side of the host path: every kind of buffer in one flat pinned allocation
+    tbl, host_states, host_p, host_g = job.host_table(flat=True)
     hp = job.hp(job.t + 1)
     job.handle.step_host(tbl, **hp)          # warm-up: grows the device arena
     torch.cuda.synchronize()

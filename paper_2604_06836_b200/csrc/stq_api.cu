@@ -9,6 +9,8 @@
 #include <utility>
 #include <vector>
 
+#include <cuda.h>   // types of the one driver query below; the entry point is fetched at run time, nothing links libcuda
+
 #include "../../include/stq.h"
 #include "stq_internal.h"
 
@@ -105,6 +107,28 @@ int grow_stage(stq_handle* h, size_t bytes) {
   if (e != cudaSuccess) { h->cuda_err = cudaGetErrorString(e); h->h_stage = nullptr; return STQ_E_WORKSPACE; }
   h->h_stage_cap = want;
   return STQ_OK;
+}
+
+// True if [p, p + len) lies inside ONE allocation known to the driver.  Buffers that are neighbours in
+// the address space may still be separate allocations, and a copy must not span two of them.
+bool one_allocation(const void* p, size_t len) {
+  typedef CUresult (*get_attr_t)(void*, CUpointer_attribute, CUdeviceptr);
+  static const get_attr_t get = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuPointerGetAttribute", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    (void)cudaGetLastError();
+    return reinterpret_cast<get_attr_t>(f);
+  }();
+  if (!get) return false;
+  CUdeviceptr base = 0;
+  size_t size = 0;
+  const CUdeviceptr q = reinterpret_cast<CUdeviceptr>(p);
+  if (get(&base, CU_POINTER_ATTRIBUTE_RANGE_START_ADDR, q) != CUDA_SUCCESS) return false;
+  if (get(&size, CU_POINTER_ATTRIBUTE_RANGE_SIZE, q) != CUDA_SUCCESS) return false;
+  return q >= base && q + len <= base + size;
 }
 
 bool overlap(const void* a, size_t na, const void* b, size_t nb) {
@@ -596,6 +620,7 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
     if (t.bits_m_out != t.bits_m) need += up(stq_codes_bytes(t.numel, t.bits_m_out));
     if (t.bits_v_out != t.bits_v) need += up(stq_codes_bytes(t.numel, t.bits_v_out));
     if (t.lp_dtype != STQ_LP_NONE) need += up(t.numel * 2);
+    need += 6 * (4096 + 512);   // padding carried along when buffers travel as one run
   }
   if (hp->inv_grad_scale || hp->found_inf) return STQ_E_ARG;   // device pointers have no place in the host-buffer call
   rc = grow(h, h->d_arena, h->d_arena_cap, need);
@@ -625,22 +650,107 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
     *ev = h->host_events[n_events++];
     return cudaSuccess;
   };
+  // Buffers of one kind (parameters, gradients, codes or scales of one state) that lie back to back in
+  // host memory over the tensors of a chunk, with nothing but alignment padding between them, travel
+  // as ONE copy into a device image of the whole run: under a concurrent copy in the other direction
+  // every separate host-to-device copy costs tens of microseconds of start-up, which a table of
+  // hundreds of tensors cannot afford.  Callers that keep each kind in one flat pinned buffer get this
+  // path; separately allocated buffers (even when they happen to be neighbours) are copied one by one.
+  constexpr size_t kMaxGap = 4096;
+  struct Run { const uint8_t* lo; size_t len; uint8_t* dev; };
+  enum { kParam, kGrad, kMc, kVc, kMs, kVs, kKinds };
+  auto in_ptr = [&](const stq_tensor& t, int kind) -> const uint8_t* {
+    switch (kind) {
+      case kParam: return reinterpret_cast<const uint8_t*>(t.param);
+      case kGrad: return static_cast<const uint8_t*>(t.grad);
+      case kMc: return static_cast<const uint8_t*>(t.m_codes_in);
+      case kVc: return static_cast<const uint8_t*>(t.v_codes_in);
+      case kMs: return reinterpret_cast<const uint8_t*>(t.m_scales_in);
+      default: return reinterpret_cast<const uint8_t*>(t.v_scales_in);
+    }
+  };
+  auto in_size = [&](const stq_tensor& t, int kind) -> size_t {
+    switch (kind) {
+      case kParam: return t.numel * 4;
+      case kGrad: return t.numel * gsz;
+      case kMc: return stq_codes_bytes(t.numel, t.bits_m);
+      case kVc: return stq_codes_bytes(t.numel, t.bits_v);
+      case kMs: return t.bits_m != 32 ? stq_scales_bytes(t.numel, t.block) : 0;
+      default: return t.bits_v != 32 ? stq_scales_bytes(t.numel, t.block) : 0;
+    }
+  };
+  // the run of kind `kind` over tensors [a, b), or len 0 if the buffers do not lie back to back
+  auto find_run = [&](int a, int b, int kind) -> Run {
+    Run r{nullptr, 0, nullptr};
+    if (b - a < 2) return r;
+    const uint8_t* end = nullptr;
+    for (int l = a; l < b; ++l) {
+      const uint8_t* p = in_ptr(tensors[l], kind);
+      const size_t n = in_size(tensors[l], kind);
+      if (!p || n == 0) return r;
+      if (l == a) r.lo = p;
+      else if (p < end || (size_t)(p - end) > kMaxGap) return r;
+      end = p + n;
+    }
+    r.len = (size_t)(end - r.lo);
+    if (!one_allocation(r.lo, r.len)) r.len = 0;
+    return r;
+  };
   int a = 0;
   while (a < L) {
-    // ---- copies in (stream s_in) ----
+    // ---- the chunk: consecutive tensors up to the byte budget ----
     size_t moved = 0;
     int b = a;
-    for (; b < L && (b == a || moved < chunk_bytes); ++b) {
-      const stq_tensor& t = tensors[b];
-      stq_tensor& d = dev[b];
+    for (; b < L && (b == a || moved < chunk_bytes); ++b)
+      for (int k = 0; k < kKinds; ++k) moved += in_size(tensors[b], k);
+    // ---- copies in (stream s_in) ----
+    Run run[kKinds];
+    for (int k = 0; k < kKinds; ++k) {
+      run[k] = find_run(a, b, k);
+      if (run[k].len) {
+        // the image keeps the host run's offset inside a 256-byte line, so every buffer keeps its alignment
+        uint8_t* base = place(run[k].len + 256);
+        run[k].dev = base + (reinterpret_cast<uintptr_t>(run[k].lo) & 255u);
+        STQ_CUDA(h, cudaMemcpyAsync(run[k].dev, run[k].lo, run[k].len, cudaMemcpyHostToDevice, s_in));
+        h2d += run[k].len;
+      }
+    }
+    auto dev_in = [&](const stq_tensor& t, int kind, size_t always_bytes) -> uint8_t* {
+      const size_t n = in_size(t, kind);
+      if (run[kind].len) return run[kind].dev + (in_ptr(t, kind) - run[kind].lo);
+      uint8_t* p = place(n ? n : always_bytes);
+      if (n) {
+        cudaError_t e = cudaMemcpyAsync(p, in_ptr(t, kind), n, cudaMemcpyHostToDevice, s_in);
+        if (e != cudaSuccess) { h->cuda_err = cudaGetErrorString(e); return nullptr; }
+        h2d += n;
+      }
+      return p;
+    };
+    // which outputs may go back as one copy of the run they came in with: written in place on the host too
+    bool out_run[kKinds];
+    for (int k = 0; k < kKinds; ++k) out_run[k] = run[k].len != 0;
+    out_run[kGrad] = false;
+    for (int l = a; l < b; ++l) {
+      const stq_tensor& t = tensors[l];
+      if (t.bits_m_out != t.bits_m || t.m_codes_out != t.m_codes_in) out_run[kMc] = false;
+      if (t.bits_v_out != t.bits_v || t.v_codes_out != t.v_codes_in) out_run[kVc] = false;
+      if (t.bits_m_out == 32 || t.m_scales_out != t.m_scales_in) out_run[kMs] = false;
+      if (t.bits_v_out == 32 || t.v_scales_out != t.v_scales_in) out_run[kVs] = false;
+    }
+    for (int l = a; l < b; ++l) {
+      const stq_tensor& t = tensors[l];
+      stq_tensor& d = dev[l];
       const size_t sb = stq_scales_bytes(t.numel, t.block);
-      const size_t mi = stq_codes_bytes(t.numel, t.bits_m), vi = stq_codes_bytes(t.numel, t.bits_v);
-      d.param = reinterpret_cast<float*>(place(t.numel * 4));
-      d.grad = place(t.numel * gsz);
-      d.m_codes_in = place(mi);
-      d.v_codes_in = place(vi);
-      d.m_scales_in = reinterpret_cast<float*>(place(sb));
-      d.v_scales_in = reinterpret_cast<float*>(place(sb));
+      d.param = reinterpret_cast<float*>(dev_in(t, kParam, 0));
+      d.grad = dev_in(t, kGrad, 0);
+      d.m_codes_in = dev_in(t, kMc, 0);
+      d.v_codes_in = dev_in(t, kVc, 0);
+      d.m_scales_in = reinterpret_cast<float*>(dev_in(t, kMs, sb));   // placed even at 32 bits: the step may write scales
+      d.v_scales_in = reinterpret_cast<float*>(dev_in(t, kVs, sb));
+      if (!d.param || !d.grad || !d.m_codes_in || !d.v_codes_in || !d.m_scales_in || !d.v_scales_in) {
+        cudaDeviceSynchronize();
+        return STQ_E_CUDA;
+      }
       d.m_codes_out = t.bits_m_out != t.bits_m ? place(stq_codes_bytes(t.numel, t.bits_m_out))
                                                : const_cast<void*>(d.m_codes_in);
       d.v_codes_out = t.bits_v_out != t.bits_v ? place(stq_codes_bytes(t.numel, t.bits_v_out))
@@ -648,21 +758,6 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
       d.m_scales_out = const_cast<float*>(d.m_scales_in);
       d.v_scales_out = const_cast<float*>(d.v_scales_in);
       if (t.lp_dtype != STQ_LP_NONE) d.param_lp = place(t.numel * 2);
-      STQ_CUDA(h, cudaMemcpyAsync(d.param, t.param, t.numel * 4, cudaMemcpyHostToDevice, s_in));
-      STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.grad), t.grad, t.numel * gsz, cudaMemcpyHostToDevice, s_in));
-      STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.m_codes_in), t.m_codes_in, mi, cudaMemcpyHostToDevice, s_in));
-      STQ_CUDA(h, cudaMemcpyAsync(const_cast<void*>(d.v_codes_in), t.v_codes_in, vi, cudaMemcpyHostToDevice, s_in));
-      size_t bytes = t.numel * 4 + t.numel * gsz + mi + vi;
-      if (t.bits_m != 32) {
-        STQ_CUDA(h, cudaMemcpyAsync(const_cast<float*>(d.m_scales_in), t.m_scales_in, sb, cudaMemcpyHostToDevice, s_in));
-        bytes += sb;
-      }
-      if (t.bits_v != 32) {
-        STQ_CUDA(h, cudaMemcpyAsync(const_cast<float*>(d.v_scales_in), t.v_scales_in, sb, cudaMemcpyHostToDevice, s_in));
-        bytes += sb;
-      }
-      h2d += bytes;
-      moved += bytes;
     }
     cudaEvent_t ev_in, ev_run;
     STQ_CUDA(h, next_event(&ev_in));
@@ -675,24 +770,38 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
     STQ_CUDA(h, cudaEventRecord(ev_run, s_run));
     // ---- copies out (stream s_out) ----
     STQ_CUDA(h, cudaStreamWaitEvent(s_out, ev_run, 0));
+    for (int k = 0; k < kKinds; ++k) {
+      if (!out_run[k]) continue;
+      // (the padding between the buffers goes back as it came)
+      STQ_CUDA(h, cudaMemcpyAsync(const_cast<uint8_t*>(run[k].lo), run[k].dev, run[k].len, cudaMemcpyDeviceToHost, s_out));
+      d2h += run[k].len;
+    }
     for (int l = a; l < b; ++l) {
       const stq_tensor& t = tensors[l];
       const stq_tensor& d = dev[l];
       const size_t sb = stq_scales_bytes(t.numel, t.block);
       const size_t mo = stq_codes_bytes(t.numel, t.bits_m_out), vo = stq_codes_bytes(t.numel, t.bits_v_out);
-      STQ_CUDA(h, cudaMemcpyAsync(t.param, d.param, t.numel * 4, cudaMemcpyDeviceToHost, s_out));
-      STQ_CUDA(h, cudaMemcpyAsync(t.m_codes_out, d.m_codes_out, mo, cudaMemcpyDeviceToHost, s_out));
-      STQ_CUDA(h, cudaMemcpyAsync(t.v_codes_out, d.v_codes_out, vo, cudaMemcpyDeviceToHost, s_out));
-      d2h += t.numel * 4 + mo + vo;
+      if (!out_run[kParam]) {
+        STQ_CUDA(h, cudaMemcpyAsync(t.param, d.param, t.numel * 4, cudaMemcpyDeviceToHost, s_out));
+        d2h += t.numel * 4;
+      }
+      if (!out_run[kMc]) {
+        STQ_CUDA(h, cudaMemcpyAsync(t.m_codes_out, d.m_codes_out, mo, cudaMemcpyDeviceToHost, s_out));
+        d2h += mo;
+      }
+      if (!out_run[kVc]) {
+        STQ_CUDA(h, cudaMemcpyAsync(t.v_codes_out, d.v_codes_out, vo, cudaMemcpyDeviceToHost, s_out));
+        d2h += vo;
+      }
       if (t.lp_dtype != STQ_LP_NONE) {
         STQ_CUDA(h, cudaMemcpyAsync(t.param_lp, d.param_lp, t.numel * 2, cudaMemcpyDeviceToHost, s_out));
         d2h += t.numel * 2;
       }
-      if (t.bits_m_out != 32) {
+      if (t.bits_m_out != 32 && !out_run[kMs]) {
         STQ_CUDA(h, cudaMemcpyAsync(t.m_scales_out, d.m_scales_out, sb, cudaMemcpyDeviceToHost, s_out));
         d2h += sb;
       }
-      if (t.bits_v_out != 32) {
+      if (t.bits_v_out != 32 && !out_run[kVs]) {
         STQ_CUDA(h, cudaMemcpyAsync(t.v_scales_out, d.v_scales_out, sb, cudaMemcpyDeviceToHost, s_out));
         d2h += sb;
       }

@@ -140,6 +140,40 @@ class Job:
         self.bits_m, self.bits_v = bm.copy(), bv.copy()
         self._tbl = None
 
+    # ---- host mirror (for the host-buffer entry point) ------------------------------------------------
+    def host_table(self, flat: bool = True):
+        """Pinned host copies of everything a step reads and writes, and the table over them.
+
+        flat: each kind of buffer (parameters, gradients, codes and scales of either state) lives in
+        one pinned allocation, tensor after tensor at 256-byte aligned offsets, so that
+        ``stq_step_host`` can move a chunk of tensors as one copy per kind.  Otherwise every state
+        buffer is its own allocation.  Returns (table, host states, host parameters, host gradients)."""
+        torch.cuda.synchronize(self.device)
+        host_p = self.param_flat.cpu().pin_memory()
+        host_g = self.grad_flat.cpu().pin_memory()
+
+        def mirror(tensors):
+            if not flat:
+                return [t.cpu().pin_memory() for t in tensors]
+            offs, total = [], 0
+            for t in tensors:
+                offs.append(total)
+                total += _round_up(t.numel() * t.element_size(), 256)
+            buf = torch.empty(max(total, 1), dtype=torch.uint8).pin_memory()
+            out = []
+            for t, o in zip(tensors, offs):
+                v = buf[o:o + t.numel() * t.element_size()].view(t.dtype)
+                v.copy_(t)
+                out.append(v)
+            return out
+
+        mc, ms = mirror([s.m_codes for s in self.states]), mirror([s.m_scales for s in self.states])
+        vc, vs = mirror([s.v_codes for s in self.states]), mirror([s.v_scales for s in self.states])
+        states = [stq.QState(mc[i], ms[i], s.bits_m, vc[i], vs[i], s.bits_v, s.v_log) for i, s in enumerate(self.states)]
+        rows = [stq.make_row(n, self.block, states[i], states[i], host_p[o:o + n], host_g[o:o + n], self.wd[i])
+                for i, (n, o) in enumerate(zip(self.numels, self.offsets))]
+        return stq.table(rows), states, host_p, host_g
+
     # ---- accounting ------------------------------------------------------------------------------
     def algorithmic_bytes(self) -> int:
         """Bytes one step must move: theta r+w, grad, codes r+w, scales r+w, the working copy if any."""

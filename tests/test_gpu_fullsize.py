@@ -137,8 +137,17 @@ def test_checkpoint_resume_is_bit_identical():
         assert torch.equal(sa.m_scales, sb.m_scales) and torch.equal(sa.v_scales, sb.v_scales)
 
 
-def test_host_buffer_step_matches_device_step():
-    """stq_step_host (host pointers, copies inside the call) against stq_step on device buffers."""
+def _whole(t):
+    """All bytes of the allocation a host tensor lives in."""
+    return torch.empty(0, dtype=torch.uint8).set_(t.untyped_storage())
+
+
+@pytest.mark.parametrize("flat", [True, False])
+@pytest.mark.parametrize("stats", [False, True])
+def test_host_buffer_step_matches_device_step(flat, stats):
+    """stq_step_host (host pointers, copies inside the call) against stq_step on device buffers, with
+    the host buffers of each kind in one flat allocation (a chunk then travels as one copy per kind)
+    and allocated one by one.  The padding between flat buffers comes back untouched."""
     from paper_2604_06836_b200 import stq
     w = W.scaled(W.config("cfg4"), W.small_gpt2(d=136, n_layer=2), steps=2)
     bm, bv, _ = W.draw_bits(w)
@@ -146,26 +155,70 @@ def test_host_buffer_step_matches_device_step():
     job.draw_grads(1)
     job.step(1)
     job.draw_grads(2)
-    torch.cuda.synchronize()
-    hp_ = job.param_flat.cpu().pin_memory()
-    hg = job.grad_flat.cpu().pin_memory()
-    rows, hstates = [], []
-    for i, n in enumerate(job.numels):
-        s = job.states[i]
-        hs = stq.QState(s.m_codes.cpu().pin_memory(), s.m_scales.cpu().pin_memory(), s.bits_m,
-                        s.v_codes.cpu().pin_memory(), s.v_scales.cpu().pin_memory(), s.bits_v, s.v_log)
-        hstates.append(hs)
-        o = job.offsets[i]
-        rows.append(stq.make_row(n, job.block, hs, hs, hp_[o:o + n], hg[o:o + n], job.wd[i]))
-    h2d, d2h = job.handle.step_host(stq.table(rows), **job.hp(2))
+    tbl, hstates, hp_, hg = job.host_table(flat=flat)
+    wholes = [_whole(t) for t in (hstates[0].m_codes, hstates[0].v_codes, hstates[0].m_scales, hstates[0].v_scales)]
+    if flat:       # a pattern in the padding between the buffers
+        for wh, ts in zip(wholes, ([s.m_codes for s in hstates], [s.v_codes for s in hstates],
+                                   [s.m_scales for s in hstates], [s.v_scales for s in hstates])):
+            keep = [t.clone() for t in ts]
+            wh.fill_(0xA5)
+            for t, k in zip(ts, keep):
+                t.copy_(k)
+    before = [wh.clone() for wh in wholes]
+    flags = stq.WITH_STATS if stats else 0
+    h2d, d2h = job.handle.step_host(tbl, flags=flags, **job.hp(2))
+    got_stats = job.layer_stats() if stats else None
     job._tbl = None
-    job.step(2)
+    job.step(2, stats=stats)
     torch.cuda.synchronize()
     assert h2d > 0 and d2h > 0
     assert torch.equal(hp_, job.param_flat.cpu())
     for hs, s in zip(hstates, job.states):
         assert torch.equal(hs.m_codes, s.m_codes.cpu()) and torch.equal(hs.v_codes, s.v_codes.cpu())
         assert torch.equal(hs.m_scales, s.m_scales.cpu()) and torch.equal(hs.v_scales, s.v_scales.cpu())
+    if stats:
+        np.testing.assert_array_equal(got_stats, job.layer_stats())
+    if flat:
+        for wh, b4, ts in zip(wholes, before, ([s.m_codes for s in hstates], [s.v_codes for s in hstates],
+                                               [s.m_scales for s in hstates], [s.v_scales for s in hstates])):
+            covered = torch.zeros(wh.numel(), dtype=torch.bool)
+            base = wh.data_ptr()
+            for t in ts:
+                o = t.data_ptr() - base
+                covered[o:o + t.numel() * t.element_size()] = True
+            assert torch.equal(wh[~covered], b4[~covered])
+            assert (wh[~covered] == 0xA5).all()
+
+
+def test_host_buffer_step_with_a_width_change_and_mixed_layouts():
+    """Flat parameters and gradients, states allocated one by one, and new widths written to separate
+    host buffers: the run path and the one-by-one path serve the same call."""
+    from paper_2604_06836_b200 import stq
+    w = W.scaled(W.config("cfg2"), W.small_gpt2(d=72, n_layer=1, vocab=301, ctx=16), steps=2)
+    bm, bv, _ = W.draw_bits(w)
+    job = Job(w, bm, bv)
+    job.draw_grads(1)
+    job.step(1)
+    job.draw_grads(2)
+    _, hstates, hp_, hg = job.host_table(flat=False)
+    from dataclasses import replace
+    nbm, nbv, _ = W.churn_bits(replace(w, churn=0.5), job.bits_m, job.bits_v, 0)
+    new_h = [stq.QState(torch.zeros(stq.codes_bytes(n, int(a)), dtype=torch.uint8).pin_memory(),
+                        torch.zeros(max(1, (n + w.block - 1) // w.block), dtype=torch.float32).pin_memory(), int(a),
+                        torch.zeros(stq.codes_bytes(n, int(b)), dtype=torch.uint8).pin_memory(),
+                        torch.zeros(max(1, (n + w.block - 1) // w.block), dtype=torch.float32).pin_memory(), int(b))
+             for n, a, b in zip(job.numels, nbm, nbv)]
+    rows = [stq.make_row(n, job.block, hstates[i], new_h[i], hp_[o:o + n], hg[o:o + n], job.wd[i])
+            for i, (n, o) in enumerate(zip(job.numels, job.offsets))]
+    job.handle.step_host(stq.table(rows), **job.hp(2))
+    job._tbl = None
+    job.step(2, new_bits=(nbm, nbv))
+    torch.cuda.synchronize()
+    assert torch.equal(hp_, job.param_flat.cpu())
+    for hs, s in zip(new_h, job.states):
+        assert torch.equal(hs.m_codes, s.m_codes.cpu()) and torch.equal(hs.v_codes, s.v_codes.cpu())
+        nb = s.m_scales.numel()
+        assert torch.equal(hs.m_scales[:nb], s.m_scales.cpu()) and torch.equal(hs.v_scales[:nb], s.v_scales.cpu())
 
 
 def test_a_wait_that_runs_out_is_reported_and_the_context_survives():
