@@ -264,10 +264,10 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   uint8_t* st = static_cast<uint8_t*>(h->h_stage);
   TensorDesc* ht = reinterpret_cast<TensorDesc*>(st);
   uint32_t* hm = reinterpret_cast<uint32_t*>(st + off_map);
-  // Fast tiles are laid out grouped by width pair: the main kernel runs a body specialised on the
-  // pair, and a change of body costs an instruction-cache refill on every SM, so tensors that share
-  // a pair are made neighbours in the tile order (at most 25 changes per launch).  The order of the
-  // table itself is untouched.
+  // Fast tiles are laid out grouped by body (width pair, variant of the v code): the main kernel runs
+  // one specialised body per group, and a change of body costs an instruction-cache refill on every
+  // SM, so tensors that share a body are made neighbours in the tile order (at most 35 changes per
+  // launch).  The order of the table itself is untouched.
   std::vector<int> order(L);
   for (int l = 0; l < L; ++l) order[l] = l;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
@@ -277,7 +277,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   stq::FastSched* hs = reinterpret_cast<stq::FastSched*>(st + off_sched);
   std::memset(hs, 0, sizeof(*hs));
   {
-    // groups of equal width pair, and an estimate of their cost for the initial spread of the CTAs
+    // groups of equal body, and an estimate of their cost for the initial spread of the CTAs
     // (relative cost per tile from measurement: 8- and 16-bit log codes and 3-bit packing cost more;
     // the estimate only decides where CTAs start, the balance itself is dynamic)
     double cost[stq::kFastMaxGroups] = {0.0};

@@ -62,7 +62,7 @@ cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const
                          const StepConsts& sc, double* partials, int grid, cudaStream_t stream);
 
 // Work list of the main step kernel: the fast tiles [0, n_fast) of the tile order, cut into groups
-// of equal width pair.  Lives in device memory; the counters are zeroed before every launch.
+// of equal body (width pair, variant of the v code).  Lives in device memory; the counters are zeroed before every launch.
 constexpr int kFastMaxGroups = 64;     // 5 widths of m x (5 widths of v + 2 variants at 8 and 16 bits) = 35 bodies
 constexpr int kFastMaxGrid = 4096;
 constexpr uint32_t kFastChunk = 8;     // tiles handed out per counter increment (fewer for small launches)

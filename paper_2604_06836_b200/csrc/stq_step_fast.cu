@@ -600,7 +600,7 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
   }
 }
 
-// Scheduling: the fast tiles are grouped by width pair (one body each).  A CTA starts in the group
+// Scheduling: the fast tiles are grouped by body (width pair and variant of the v code).  A CTA starts in the group
 // the host assigned to it and takes chunks of consecutive tiles (kFastChunk of them, fewer when the
 // launch is small) from that group's
 // counter; when its group runs dry it moves on to the next one that still has work.  So a CTA runs

@@ -53,7 +53,7 @@ def test_paper_policy_trains_and_resumes_bit_for_bit():
         loss = torch.nn.functional.mse_loss(model(x), y)
         loss.backward()
         opt.step()
-        losses.append(float(loss))
+        losses.append(float(loss.detach()))
     assert np.mean(losses[-5:]) < 0.7 * np.mean(losses[:5])
     assert set(opt.bits_m.tolist()) <= {4, 8, 16, 32} and (opt.bits_m == opt.bits_v).all()
     assert opt.last_scores is not None and opt.state_bytes() > 0

@@ -450,3 +450,23 @@ def test_pl_variant_extreme_values_and_mixed_tables(H, O):
     bad.v_log = 7
     with pytest.raises(stq.StqError):
         h.step(stq.table([bad]), t=4, **hp)
+
+
+@pytest.mark.parametrize("v_log", ["poly", "pl"])
+def test_fp16_training_recipe_on_a_small_model(H, O, v_log):
+    """Table 1's fp16 recipe (loss-scaled fp16 gradients, fp16 working copy) on a small GPT-2-shaped list,
+    in both variants of the v code: the mixed-precision bodies of the step kernel against the oracle."""
+    from dataclasses import replace
+    w = replace(W.scaled(W.config("gpt2_medium"), W.small_gpt2(d=136, n_layer=2), steps=6), v_log=v_log)
+    bm, bv, _ = W.draw_bits(w)
+    job = Job(w, bm, bv)
+    oj = H.OracleJob(job)
+    for t in range(1, 7):
+        job.draw_grads(t)
+        st = oj.step([H.to_np(g) for g in job.grads], t, want_stats=True, fp16_grad=True,
+                     inv_grad_scale=1.0 / w.loss_scale)
+        job.step(t, stats=True)
+        H.compare_job(job, oj, REL_1STEP * t, f"fp16 {v_log} t={t}")
+        H.assert_stats_close(job.layer_stats(), st, f"fp16 {v_log} t={t}")
+        for p, lp in zip(job.params, job.params_lp):
+            assert torch.equal(lp, p.to(torch.float16))
