@@ -16,6 +16,7 @@ HEADERS = [os.path.join(CSRC, "stq_internal.h"), os.path.join(os.path.dirname(HE
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-fmad=false", "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
+    "-diag-suppress", "177",     # unused members of the per-width constant tables
 ]
 
 

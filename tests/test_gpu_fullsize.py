@@ -283,3 +283,51 @@ def test_nothing_is_written_outside_the_callers_buffers():
 
 def _r16(x):
     return (x + 15) // 16 * 16
+
+
+def test_one_tensor_beyond_two_to_the_31_elements():
+    """Element indices past 2^31 and byte offsets past 2^33: one tensor of 2^31 + 20,813 elements (fast
+    tiles plus a ragged tail in the generic kernel), checked on sampled blocks (first, last, tail, random)."""
+    import harness as H
+    _need(40)
+    n = (1 << 31) + 4096 * 5 + 333
+    w = W.Workload("one-tensor-2^31", (("w", (n,)),), 128, "bf16", "student_t", nu=3, scale_log10=(-3.0, -3.0),
+                   bits_kind="fixed", bits_fixed=(4, 8), seed=11)
+    job = Job(w, [4], [8])
+    so = H.SampledOracle(job, per_tensor=12, seed=2)
+    for t in (1, 2):
+        job.draw_grads(t)
+        so.step(t)
+        job.step(t, stats=True)
+        so.compare(1e-6 * t, f"2^31 t={t}")
+        got = job.layer_stats()
+        g = job.grads[0]
+        want = np.zeros(4)
+        for lo in range(0, n, 1 << 28):          # float64 sums, a slice at a time
+            x = g[lo:lo + (1 << 28)].double()
+            want += np.array([x.sum().item(), x.abs().sum().item(), (x * x).sum().item(), x.numel()])
+        H.assert_stats_close(got, want[None, :], f"2^31 t={t}")
+
+
+def test_one_tensor_beyond_two_to_the_32_elements():
+    """The largest class of tensor the table accepts on one GPU: more than 2^32 elements, which the main
+    kernel leaves to the generic one (its tile counters are 32-bit); 64-bit element indices throughout."""
+    import harness as H
+    _need(90)
+    n = (1 << 32) + 4096 * 3 + 77
+    w = W.Workload("one-tensor-2^32", (("w", (n,)),), 256, "bf16", "normal", scale_log10=(-3.0, -3.0),
+                   bits_kind="fixed", bits_fixed=(3, 4), seed=12)
+    job = Job(w, [3], [4])
+    so = H.SampledOracle(job, per_tensor=12, seed=3)
+    job.draw_grads(1)
+    so.step(1)
+    job.step(1, stats=True)
+    so.compare(1e-6, "2^32 t=1")
+    got = job.layer_stats()
+    assert got[0, 3] == n
+    g = job.grads[0]
+    want = np.zeros(4)
+    for lo in range(0, n, 1 << 28):
+        x = g[lo:lo + (1 << 28)].double()
+        want += np.array([x.sum().item(), x.abs().sum().item(), (x * x).sum().item(), x.numel()])
+    H.assert_stats_close(got, want[None, :], "2^32")
