@@ -33,10 +33,11 @@ struct stq_handle {
   uint32_t* d_tile_map = nullptr;
   size_t d_tile_cap = 0;
   uint32_t n_tiles = 0, n_fast = 0, n_narrow = 0;   // n_narrow counts fast + remaining narrow
+  uint32_t n_main = 0;                              // fast tiles of the fused bodies; [n_main, n_fast) change width
   int fast_grid = 0;
   bool any_lp = false;              // some tensor of the current table wants a low-precision copy
   int* d_err = nullptr;             // raised by a kernel whose bounded wait ran out
-  stq::FastSched* d_sched = nullptr;   // work list of the main step kernel
+  stq::FastSched* d_sched = nullptr;   // two work lists of the main step kernel (fused bodies, width changes)
 
   // pinned staging for uploads
   void* h_stage = nullptr;
@@ -193,7 +194,9 @@ int validate_row(const stq_tensor& t, int kind) {
 
 // Tensors with the same key run the same specialised body of the main kernel: the two widths, and
 // for v at 8 or 16 bits the variant of its quantizer.  Ordered from cheap to expensive v codes.
+constexpr int kSplitKey = 1 << 20;
 int body_key(const stq_tensor& t) {
+  if (t.bits_m != t.bits_m_out || t.bits_v != t.bits_v_out) return kSplitKey;   // one runtime-width body for all of them
   const int pl = t.v_log == STQ_VLOG_PL && (t.bits_v == 8 || t.bits_v == 16) ? 1 : 0;
   return (t.bits_v * 2 + (1 - pl)) * 64 + t.bits_m;
 }
@@ -230,7 +233,8 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     const uint64_t nt = (t.numel + stq::kTile - 1) / stq::kTile;
     const bool wide = row_is_wide(t, kind);
     // (the main kernel moves the scales with 16-byte bulk copies as well)
-    const bool fast_ok = kind == kKindStep && !wide && t.bits_m == t.bits_m_out && t.bits_v == t.bits_v_out &&
+    // (a tensor whose widths change inside the step takes the main kernel's runtime-width body)
+    const bool fast_ok = kind == kKindStep && !wide &&
                          t.numel < (1ull << 32) && aligned(t.m_scales_in, 16) && aligned(t.v_scales_in, 16) &&
                          t.block <= (uint32_t)stq::kFastMaxBlock;
     const uint64_t nf = fast_ok ? t.numel / stq::kTile : 0;
@@ -241,7 +245,8 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     if (!wide) slow_narrow += nt - nf;
     sig[l] = t.numel | (wide ? 1ull << 63 : 0ull) | (fast_ok ? 1ull << 62 : 0ull) |
              ((uint64_t)t.bits_m << 56) | ((uint64_t)t.bits_v << 48) |
-             ((uint64_t)(t.v_log & 1u) << 47);                           // numel <= 2^40
+             ((uint64_t)(t.v_log & 1u) << 47) |
+             ((uint64_t)(t.bits_m != t.bits_m_out || t.bits_v != t.bits_v_out) << 46);   // numel <= 2^40
   }
   if (total > 0xFFFFFFF0ull) return STQ_E_NUMEL;
   // the tile map depends only on sizes and classes: skip it when unchanged
@@ -253,7 +258,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   const size_t off_sched = (off_map + bytes_map + 255) & ~size_t(255);
   uint64_t n_seg = 0;
   for (int l = 0; l < L; ++l) n_seg += ((uint64_t)nfast[l] + nslow[l] + stq::kStatSegTiles - 1) / stq::kStatSegTiles;
-  const size_t off_seg = (off_sched + sizeof(stq::FastSched) + 255) & ~size_t(255);
+  const size_t off_seg = (off_sched + 2 * sizeof(stq::FastSched) + 255) & ~size_t(255);
   int rc;
   if ((rc = grow_stage(h, off_seg + sizeof(uint32_t) * (size_t)n_seg)) != STQ_OK) return rc;
   if ((rc = grow(h, h->d_seg_map, h->d_seg_map_cap, (size_t)n_seg)) != STQ_OK) return rc;
@@ -274,8 +279,11 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     return body_key(tensors[a]) < body_key(tensors[b]);
   });
   std::vector<uint32_t> fast0(L);
+  // two work lists: hs for the fused bodies, hs2 (one group) for the tensors that change width in this step
   stq::FastSched* hs = reinterpret_cast<stq::FastSched*>(st + off_sched);
-  std::memset(hs, 0, sizeof(*hs));
+  stq::FastSched* hs2 = hs + 1;
+  std::memset(hs, 0, 2 * sizeof(*hs));
+  uint32_t split_begin = 0;
   {
     // groups of equal body, and an estimate of their cost for the initial spread of the CTAs
     // (relative cost per tile from measurement: 8- and 16-bit log codes and 3-bit packing cost more;
@@ -283,12 +291,20 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     double cost[stq::kFastMaxGroups] = {0.0};
     uint32_t next_fast = 0;
     int last_key = -1;
+    bool in_split = false;
     for (int i = 0; i < L; ++i) {
       const int l = order[i];
       fast0[l] = next_fast;
       if (nfast[l] == 0) continue;
       const stq_tensor& t = tensors[l];
       const int key = body_key(t);
+      if (key == kSplitKey) {           // sorted last: everything from here on belongs to the second work list
+        if (!in_split) { in_split = true; split_begin = next_fast; }
+        if (!same_map)
+          for (uint32_t k = 0; k < nfast[l]; ++k) hm[next_fast + k] = (uint32_t)l;
+        next_fast += nfast[l];
+        continue;
+      }
       if (key != last_key && hs->ng < (uint32_t)stq::kFastMaxGroups) {
         hs->grp_begin[hs->ng++] = next_fast;
         last_key = key;
@@ -302,12 +318,18 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
         for (uint32_t k = 0; k < nfast[l]; ++k) hm[next_fast + k] = (uint32_t)l;
       next_fast += nfast[l];
     }
-    hs->grp_begin[hs->ng] = next_fast;
+    if (!in_split) split_begin = next_fast;
+    hs->grp_begin[hs->ng] = split_begin;
     // chunk size: the usual one when every CTA gets several chunks, down to single tiles for small launches
-    {
-      const uint64_t per_cta = next_fast / (uint64_t)std::max(1, h->fast_grid);
-      hs->chunk = (uint32_t)std::min<uint64_t>(stq::kFastChunk, std::max<uint64_t>(1, per_cta / 4));
-    }
+    auto chunk_for = [&](uint64_t tiles) {
+      const uint64_t per_cta = tiles / (uint64_t)std::max(1, h->fast_grid);
+      return (uint32_t)std::min<uint64_t>(stq::kFastChunk, std::max<uint64_t>(1, per_cta / 4));
+    };
+    hs->chunk = chunk_for(split_begin);
+    hs2->ng = 1;
+    hs2->grp_begin[0] = split_begin;
+    hs2->grp_begin[1] = next_fast;
+    hs2->chunk = chunk_for(next_fast - split_begin);     // (cta_group stays 0: every CTA starts in the one group)
     // CTAs per group in proportion to cost (largest remainders), at least one each
     const int G = h->fast_grid;
     double total_cost = 0.0;
@@ -376,7 +398,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   STQ_CUDA(h, cudaMemcpyAsync(h->d_table, ht, bytes_table, cudaMemcpyHostToDevice, stream));
   if (!same_map)
     STQ_CUDA(h, cudaMemcpyAsync(h->d_tile_map, hm, bytes_map, cudaMemcpyHostToDevice, stream));
-  STQ_CUDA(h, cudaMemcpyAsync(h->d_sched, hs, sizeof(stq::FastSched), cudaMemcpyHostToDevice, stream));
+  STQ_CUDA(h, cudaMemcpyAsync(h->d_sched, hs, 2 * sizeof(stq::FastSched), cudaMemcpyHostToDevice, stream));
   if (!same_map)
     STQ_CUDA(h, cudaMemcpyAsync(h->d_seg_map, hseg, sizeof(uint32_t) * (size_t)n_seg, cudaMemcpyHostToDevice, stream));
   h->n_seg = (uint32_t)n_seg;
@@ -389,6 +411,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   for (int l = 0; l < L; ++l) h->any_lp = h->any_lp || (kind == kKindStep && tensors[l].lp_dtype != STQ_LP_NONE);
   h->n_tiles = (uint32_t)total;
   h->n_fast = (uint32_t)fast;
+  h->n_main = split_begin;
   h->n_narrow = (uint32_t)(fast + slow_narrow);
   return STQ_OK;
 }
@@ -401,10 +424,16 @@ int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::St
     if (rc != STQ_OK) return rc;
     partials = h->d_partials;
   }
-  if (h->n_fast > 0) {   // only a step table has fast tiles
+  if (h->n_main > 0) {   // only a step table has fast tiles
     const bool amp = h->any_lp || sc.inv_scale != nullptr;
-    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, amp, h->d_table, h->d_tile_map, h->d_sched, sc, partials,
-                                      h->d_err, h->fast_grid, stream));
+    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, amp, false, h->d_table, h->d_tile_map, h->d_sched, sc,
+                                      partials, h->d_err, h->fast_grid, stream));
+    h->launches++;
+  }
+  if (h->n_fast > h->n_main) {   // tensors that change width inside this step
+    const int grid = (int)std::min<uint32_t>((uint32_t)h->fast_grid, h->n_fast - h->n_main);
+    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, true, true, h->d_table, h->d_tile_map, h->d_sched + 1, sc,
+                                      partials, h->d_err, grid, stream));
     h->launches++;
   }
   if (h->n_narrow > h->n_fast) {
@@ -473,7 +502,7 @@ int stq_create(stq_handle** out, int device) {
   if (h->fast_grid > stq::kFastMaxGrid) h->fast_grid = stq::kFastMaxGrid;
   if (cudaMalloc(reinterpret_cast<void**>(&h->d_err), sizeof(int)) != cudaSuccess ||
       cudaMemset(h->d_err, 0, sizeof(int)) != cudaSuccess ||
-      cudaMalloc(reinterpret_cast<void**>(&h->d_sched), sizeof(stq::FastSched)) != cudaSuccess) {
+      cudaMalloc(reinterpret_cast<void**>(&h->d_sched), 2 * sizeof(stq::FastSched)) != cudaSuccess) {
     cudaEventDestroy(h->stage_ev);
     delete h;
     return STQ_E_WORKSPACE;

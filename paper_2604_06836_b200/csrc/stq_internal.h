@@ -77,9 +77,10 @@ struct FastSched {
 // The main step kernel (stq_step_fast.cu) with `grid` CTAs.  err_flag is set to 1 if a bounded wait
 // inside the kernel ran out.
 // amp: some tensor wants a low-precision copy, or the gradients are loss-scaled.
-cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, const TensorDesc* table, const uint32_t* tile_map,
-                             FastSched* sched, const StepConsts& sc, double* partials, int* err_flag, int grid,
-                             cudaStream_t stream);
+// split: the launch over the tiles of tensors whose widths change inside the step (its own work list).
+cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, bool split, const TensorDesc* table,
+                             const uint32_t* tile_map, FastSched* sched, const StepConsts& sc, double* partials,
+                             int* err_flag, int grid, cudaStream_t stream);
 int fast_ctas_per_sm();
 // Launches the time-out self-test (see stq_step_fast.cu): sets *err_flag after a ~0.1 ms bounded wait.
 cudaError_t launch_wait_timeout_selftest(int* err_flag, cudaStream_t stream);

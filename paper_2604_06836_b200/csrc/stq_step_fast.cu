@@ -19,6 +19,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "stq_internal.h"
 
 namespace stq {
@@ -64,7 +66,8 @@ struct __align__(16) TileInfo {
                        // piecewise-linear variant) | log2(block) << 16 | lp dtype << 24
   float wdx;           // fp32(lr*wd) (AdamW) or fp32(wd) (L2 mode)
   uint32_t tile;       // index of the tile in the launch's tile order; 0xFFFFFFFF closes the stream
-  uint32_t pad;
+  uint32_t out;        // width indices to write, m | v << 8 (same coding); equal to the low half of `packed`
+                       // unless the step changes the widths of this tensor
 };
 static_assert(sizeof(TileInfo) == 64, "TileInfo is read with four 128-bit loads");
 
@@ -600,6 +603,183 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
   }
 }
 
+// Calls f with the width behind a width index as a compile-time constant (warp-uniform switch).
+template <class F>
+__device__ __forceinline__ void with_m_width(uint32_t idx, F&& f) {
+  switch (idx) {
+    case 0: f(std::integral_constant<int, 2>{}); break;
+    case 1: f(std::integral_constant<int, 3>{}); break;
+    case 2: f(std::integral_constant<int, 4>{}); break;
+    case 3: f(std::integral_constant<int, 8>{}); break;
+    default: f(std::integral_constant<int, 16>{}); break;
+  }
+}
+template <class F>
+__device__ __forceinline__ void with_v_width(uint32_t idx, F&& f) {   // f(width, piecewise-linear variant?)
+  switch (idx) {
+    case 0: f(std::integral_constant<int, 2>{}, std::false_type{}); break;
+    case 1: f(std::integral_constant<int, 3>{}, std::false_type{}); break;
+    case 2: f(std::integral_constant<int, 4>{}, std::false_type{}); break;
+    case 3: f(std::integral_constant<int, 8>{}, std::false_type{}); break;
+    case 4: f(std::integral_constant<int, 16>{}, std::false_type{}); break;
+    case 5: f(std::integral_constant<int, 8>{}, std::true_type{}); break;
+    default: f(std::integral_constant<int, 16>{}, std::true_type{}); break;
+  }
+}
+
+// A tile whose tensor changes width inside the step (Algorithm 1 writes the states of a decision step
+// at the new widths): the stored widths and the widths to write are runtime values here, so every
+// row decode and encode goes through a warp-uniform switch into the same specialised row functions
+// the fused bodies use.  One body serves all combinations; it is slower than a fused body and far
+// faster than leaving these tiles to the generic kernel.
+template <int GDT, bool AMP>
+__device__ __forceinline__ void tile_body_split(const uint8_t* __restrict__ stage, const TileInfo& ti, const StepConsts& sc,
+                                             const float* __restrict__ lut8, int lane, int warp, uint32_t empty_bar,
+                                             double* __restrict__ part, float grad_mul) {
+  const uint32_t* lutn = reinterpret_cast<const uint32_t*>(lut8 + 256);
+  const int lgB = (int)((ti.packed >> 16) & 0xFFu);
+  [[maybe_unused]] const uint32_t lp_dtype = ti.packed >> 24;
+  const uint32_t im = ti.packed & 0xFFu, iv = (ti.packed >> 8) & 0xFFu;
+  const uint32_t om = ti.out & 0xFFu, ov = (ti.out >> 8) & 0xFFu;
+  const uint32_t bm_out = om == 0 ? 2u : om == 1 ? 3u : om == 2 ? 4u : om == 3 ? 8u : 16u;
+  const float qmax_out = (float)((1u << (bm_out - 1u)) - 1u);
+  const float lrwd = sc.l2_mode ? 0.0f : ti.wdx;
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f;
+
+#pragma unroll 1
+  for (int pass = 0; pass < R / RP; ++pass) {
+    const int row0 = warp * R + pass * RP;
+    float th[RP][4], g[RP][4], mt[RP][4], vt[RP][4];
+#pragma unroll
+    for (int r = 0; r < RP; ++r) {
+      const int row = row0 + r;
+      const int elem = row * kRowElems + 4 * lane;
+      const float4 t4 = *reinterpret_cast<const float4*>(stage + kOffTheta + 4 * elem);
+      th[r][0] = t4.x; th[r][1] = t4.y; th[r][2] = t4.z; th[r][3] = t4.w;
+      lds_grad<GDT>(stage, elem, g[r]);
+      const int blk = (row * kRowElems) >> lgB;
+      const float sm = *reinterpret_cast<const float*>(stage + kOffMs + 4 * blk);
+      const float sv = *reinterpret_cast<const float*>(stage + kOffVs + 4 * blk);
+      with_m_width(im, [&](auto B) {
+        uint32_t w[2];
+        lds_codes<decltype(B)::value>(stage + kOffMc + row * (16 * decltype(B)::value), lane, w);
+        decode_lin_row<decltype(B)::value>(w, sm, mt[r]);
+      });
+      with_v_width(iv, [&](auto B, auto pl) {
+        uint32_t w[2];
+        lds_codes<decltype(B)::value>(stage + kOffVc + row * (16 * decltype(B)::value), lane, w);
+        if constexpr (decltype(pl)::value) decode_pl_row<decltype(B)::value>(w, __float_as_uint(sv), lutn, vt[r]);
+        else decode_log_row<decltype(B)::value>(w, sv, lut8, vt[r]);
+      });
+    }
+    if (pass == R / RP - 1) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar);
+    }
+    if constexpr (AMP) {
+#pragma unroll
+      for (int r = 0; r < RP; ++r)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) g[r][k] = __fmul_rn(g[r][k], grad_mul);
+    }
+    if (part != nullptr) {
+#pragma unroll
+      for (int r = 0; r < RP; ++r)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          a0 += g[r][k];
+          a1 += fabsf(g[r][k]);
+          a2 = __fmaf_rn(g[r][k], g[r][k], a2);
+        }
+    }
+    if (sc.l2_mode) {
+#pragma unroll
+      for (int r = 0; r < RP; ++r)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) g[r][k] = __fadd_rn(g[r][k], __fmul_rn(ti.wdx, th[r][k]));
+    }
+#pragma unroll
+    for (int r = 0; r < RP; ++r)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float gk = g[r][k];
+        mt[r][k] = __fmaf_rn(sc.b1, mt[r][k], __fmul_rn(sc.c1, gk));
+        vt[r][k] = __fmaf_rn(sc.b2, vt[r][k], __fmul_rn(__fmul_rn(sc.c2, gk), gk));
+      }
+    uint32_t mxm[RP], mxv[RP];
+#pragma unroll
+    for (int r = 0; r < RP; ++r) {
+      const float am = fmaxf(fmaxf(fabsf(mt[r][0]), fabsf(mt[r][1])), fmaxf(fabsf(mt[r][2]), fabsf(mt[r][3])));
+      const float av = fmaxf(fmaxf(vt[r][0], vt[r][1]), fmaxf(vt[r][2], vt[r][3]));
+      mxm[r] = __reduce_max_sync(kFull, __float_as_uint(am));
+      mxv[r] = __reduce_max_sync(kFull, __float_as_uint(av));
+    }
+    if (RP >= 2 && lgB >= 8) {
+#pragma unroll
+      for (int r = 0; r + 1 < RP; r += 2) {
+        mxm[r] = mxm[r + 1] = max(mxm[r], mxm[r + 1]);
+        mxv[r] = mxv[r + 1] = max(mxv[r], mxv[r + 1]);
+      }
+    }
+    float* param = ti.param + row0 * kRowElems + 4 * lane;
+#pragma unroll
+    for (int r = 0; r < RP; ++r) {
+      const int row = row0 + r;
+      const float sm_raw = __uint_as_float(mxm[r]);
+      const bool mzero = sm_raw < kTiny;
+      const float sv_raw = __uint_as_float(mxv[r]);
+      const bool vzero = sv_raw < kTiny;
+      const float s_v = vzero ? 0.f : sv_raw;
+      // (this body computes the block constants in every lane: it runs on decision steps only)
+      const float inv_m = mzero ? 0.f : __fmul_rn(qmax_out, __frcp_rn(sm_raw));
+      float mq[4], vq[4];
+      with_m_width(om, [&](auto B) {
+        encode_lin_row<decltype(B)::value>(ti.mco + row * (16 * decltype(B)::value), lane, mt[r], __fmul_rn(sm_raw, sc.step_size), inv_m, mq);
+      });
+      with_v_width(ov, [&](auto B, auto pl) {
+        uint8_t* dst = ti.vco + row * (16 * decltype(B)::value);
+        if constexpr (decltype(pl)::value) {
+          encode_pl_row<decltype(B)::value>(dst, lane, vt[r], vzero ? 0x7F800000u : mxv[r], vzero ? 0u : mxv[r], lutn, vq);
+        } else if constexpr (decltype(B)::value <= 4) {
+          const float c = vzero ? 0.f : __fmul_rn(kSqrt2, __frcp_rn(sv_raw));
+          encode_log_row<decltype(B)::value>(dst, lane, vt[r], s_v, c, 0u, lut8, vq);
+        } else {
+          const uint32_t ebase = kMagicBits - (vzero ? (uint32_t)kZeroBlockExp : (mxv[r] >> 23));
+          encode_log_row<decltype(B)::value>(dst, lane, vt[r], s_v, lg_poly(mxv[r]), ebase, lut8, vq);
+        }
+      });
+      const int e_row = row * kRowElems;
+      if (lane == 0 && (e_row & ((1 << lgB) - 1)) == 0) {
+        ti.mso[e_row >> lgB] = mzero ? 0.f : sm_raw;
+        ti.vso[e_row >> lgB] = s_v;
+      }
+      float out[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float den = __fmaf_rn(sqrt_fast(vq[k]), sc.rsqrt_bc2, sc.eps);
+        const float upd = __fmul_rn(mq[k], rcp_fast(den));
+        out[k] = __fadd_rn(th[r][k], -__fmaf_rn(th[r][k], lrwd, upd));
+      }
+      *reinterpret_cast<float4*>(param + r * kRowElems) = make_float4(out[0], out[1], out[2], out[3]);
+      if constexpr (AMP) {
+        if (ti.lp != nullptr)
+          *reinterpret_cast<uint2*>(ti.lp + row * kRowElems + 4 * lane) = pack_lp(out, lp_dtype);
+      }
+    }
+  }
+  if (part != nullptr) {
+    const bool hi = lane & 16;
+    float x = (hi ? a2 : a0) + __shfl_xor_sync(kFull, hi ? a0 : a2, 16);
+    float y = (hi ? 0.f : a1) + __shfl_xor_sync(kFull, hi ? a1 : 0.f, 16);
+    const bool q = lane & 8;
+    float z = (q ? y : x) + __shfl_xor_sync(kFull, q ? x : y, 8);
+    z += __shfl_xor_sync(kFull, z, 4);
+    z += __shfl_xor_sync(kFull, z, 2);
+    z += __shfl_xor_sync(kFull, z, 1);
+    if ((lane & 7) == 0 && lane < 24) part[lane >> 3] = (double)z;
+  }
+}
+
 // Scheduling: the fast tiles are grouped by body (width pair and variant of the v code).  A CTA starts in the group
 // the host assigned to it and takes chunks of consecutive tiles (kFastChunk of them, fewer when the
 // launch is small) from that group's
@@ -610,7 +790,9 @@ __device__ __forceinline__ uint32_t width_index(uint32_t b) { return b == 2 ? 0u
 
 // AMP: the mixed-precision extras (gradient unscaling, low-precision parameter copy) are compiled
 // in only for launches that use them, so the plain step pays nothing for them.
-template <int GDT, bool AMP>
+// SPLIT: the launch over the tiles of tensors that change width inside the step (one runtime-width
+// body); compiled apart from the fused bodies so that it cannot disturb their register allocation.
+template <int GDT, bool AMP, bool SPLIT>
 __global__ void __launch_bounds__(kFastThreads, kFastCtasPerSm)
 stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map,
                      FastSched* __restrict__ sched, const StepConsts sc, double* __restrict__ partials,
@@ -667,16 +849,18 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
       dry = 0;
       const uint32_t t1 = (uint32_t)(t0 + chunk < gend ? t0 + chunk : gend);
       for (uint32_t tile = (uint32_t)t0; tile < t1; ++tile) {
-        if (issued >= (uint32_t)kStages && !mbar_wait(empty0 + 8 * s, phase ^ 1u)) { ok = false; break; }
+        // Everything that can be prepared without the stage (table look-ups, addresses) comes before the
+        // wait for it, so that the copies leave the moment the consumers release the stage: in the
+        // memory-bound bodies the time from release to issue adds to every tile's turnaround.
         const TensorDesc* T = table + __ldg(tile_map + tile);
         const unsigned long long e0 = (unsigned long long)(tile - T->tile0) * kTile;
-        const uint32_t bm = T->bm_in, bv = T->bv_in;
+        const uint32_t bm = T->bm_in, bv = T->bv_in, bmo = T->bm_out, bvo = T->bv_out;
         const uint32_t lgB = T->block == 128 ? 7u : T->block == 256 ? 8u : 9u;
         const uint32_t nb_m = (kTile / 8) * bm, nb_v = (kTile / 8) * bv, nb_s = (uint32_t)(kTile * 4) >> lgB;
         TileInfo ti;
         ti.param = T->param + e0;
-        ti.mco = T->mc_out + (e0 >> 3) * bm;
-        ti.vco = T->vc_out + (e0 >> 3) * bv;
+        ti.mco = T->mc_out + (e0 >> 3) * bmo;
+        ti.vco = T->vc_out + (e0 >> 3) * bvo;
         ti.mso = T->ms_out + (e0 >> lgB);
         ti.vso = T->vs_out + (e0 >> lgB);
         ti.lp = T->param_lp ? reinterpret_cast<uint16_t*>(T->param_lp) + e0 : nullptr;
@@ -684,17 +868,23 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
                     (T->lp_dtype << 24);
         ti.wdx = sc.l2_mode ? T->wd : (float)(sc.lr * (double)T->wd);
         ti.tile = tile;
-        ti.pad = 0u;
+        ti.out = width_index(bmo) | ((width_index(bvo) + (T->v_pl != 0u && bvo >= 8u ? 2u : 0u)) << 8);
+        const uint8_t* src_g = reinterpret_cast<const uint8_t*>(T->grad) + e0 * gsz;
+        const uint8_t* src_mc = T->mc_in + (e0 >> 3) * bm;
+        const uint8_t* src_vc = T->vc_in + (e0 >> 3) * bv;
+        const float* src_ms = T->ms_in + (e0 >> lgB);
+        const float* src_vs = T->vs_in + (e0 >> lgB);
+        if (issued >= (uint32_t)kStages && !mbar_wait(empty0 + 8 * s, phase ^ 1u)) { ok = false; break; }
         *reinterpret_cast<TileInfo*>(smem + kOffInfo + 64 * s) = ti;
         const uint32_t bar = full0 + 8 * s;
         const uint32_t dst = smem_u32(smem + s * kStageBytes);
         mbar_expect_tx(bar, kTile * 4 + kTile * gsz + nb_m + nb_v + 2 * nb_s);
-        bulk_g2s(dst + kOffTheta, T->param + e0, kTile * 4, bar);
-        bulk_g2s(dst + kOffGrad, reinterpret_cast<const uint8_t*>(T->grad) + e0 * gsz, kTile * gsz, bar);
-        bulk_g2s(dst + kOffMc, T->mc_in + (e0 >> 3) * bm, nb_m, bar);
-        bulk_g2s(dst + kOffVc, T->vc_in + (e0 >> 3) * bv, nb_v, bar);
-        bulk_g2s(dst + kOffMs, T->ms_in + (e0 >> lgB), nb_s, bar);
-        bulk_g2s(dst + kOffVs, T->vs_in + (e0 >> lgB), nb_s, bar);
+        bulk_g2s(dst + kOffTheta, ti.param, kTile * 4, bar);
+        bulk_g2s(dst + kOffGrad, src_g, kTile * gsz, bar);
+        bulk_g2s(dst + kOffMc, src_mc, nb_m, bar);
+        bulk_g2s(dst + kOffVc, src_vc, nb_v, bar);
+        bulk_g2s(dst + kOffMs, src_ms, nb_s, bar);
+        bulk_g2s(dst + kOffVs, src_vs, nb_s, bar);
         ++issued;
 #pragma unroll
         for (int k = 0; k < kStages; ++k)
@@ -738,13 +928,22 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
 #define STQ_CASES_M(IM, BM)                                                                                   \
   STQ_CASE(IM, 0, BM, 2, false) STQ_CASE(IM, 1, BM, 3, false) STQ_CASE(IM, 2, BM, 4, false) STQ_CASE(IM, 3, BM, 8, false) \
   STQ_CASE(IM, 4, BM, 16, false) STQ_CASE(IM, 5, BM, 8, true) STQ_CASE(IM, 6, BM, 16, true)
-    switch ((ti.packed & 0xFFu) * 7 + ((ti.packed >> 8) & 0xFFu)) {
-      STQ_CASES_M(0, 2)
-      STQ_CASES_M(1, 3)
-      STQ_CASES_M(2, 4)
-      STQ_CASES_M(3, 8)
-      STQ_CASES_M(4, 16)
-      default: break;
+    if constexpr (SPLIT) {
+      tile_body_split<GDT, AMP>(stage, ti, sc, lut8, lane, warp, ebar, part, grad_mul);
+    } else {
+#define STQ_CASE(IM, IV, BM, BV, VPL) \
+  case IM * 7 + IV: tile_body<BM, BV, VPL, GDT, AMP>(stage, ti, sc, lut8, lane, warp, ebar, part, grad_mul); break;
+#define STQ_CASES_M(IM, BM)                                                                                   \
+  STQ_CASE(IM, 0, BM, 2, false) STQ_CASE(IM, 1, BM, 3, false) STQ_CASE(IM, 2, BM, 4, false) STQ_CASE(IM, 3, BM, 8, false) \
+  STQ_CASE(IM, 4, BM, 16, false) STQ_CASE(IM, 5, BM, 8, true) STQ_CASE(IM, 6, BM, 16, true)
+      switch ((ti.packed & 0xFFu) * 7 + ((ti.packed >> 8) & 0xFFu)) {
+        STQ_CASES_M(0, 2)
+        STQ_CASES_M(1, 3)
+        STQ_CASES_M(2, 4)
+        STQ_CASES_M(3, 8)
+        STQ_CASES_M(4, 16)
+        default: break;
+      }
     }
     if (++s == kStages) { s = 0; phase ^= 1u; }
   }
@@ -765,10 +964,10 @@ __global__ void stq_wait_timeout_selftest_kernel(int* __restrict__ err_flag, lon
   if (!done && threadIdx.x == 0) atomicExch(err_flag, 1);
 }
 
-template <int GDT, bool AMP>
+template <int GDT, bool AMP, bool SPLIT>
 cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, FastSched* sched, const StepConsts& sc,
                           double* partials, int* err_flag, int grid, cudaStream_t stream) {
-  auto kern = stq_step_fast_kernel<GDT, AMP>;
+  auto kern = stq_step_fast_kernel<GDT, AMP, SPLIT>;
   // per device and cheap, so simply repeated: the kernel needs more than the default 48 KB
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
@@ -781,22 +980,27 @@ cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, Fas
 
 }  // namespace
 
-cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, const TensorDesc* table, const uint32_t* tile_map,
-                             FastSched* sched, const StepConsts& sc, double* partials, int* err_flag, int grid,
-                             cudaStream_t stream) {
+cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, bool split, const TensorDesc* table,
+                             const uint32_t* tile_map, FastSched* sched, const StepConsts& sc, double* partials,
+                             int* err_flag, int grid, cudaStream_t stream) {
   double* p = stats ? partials : nullptr;
+#define STQ_LAUNCH(G, A, S) return launch_fast_t<G, A, S>(table, tile_map, sched, sc, p, err_flag, grid, stream)
+#define STQ_LAUNCH_G(A, S)              \
+  switch (grad_dtype) {                 \
+    case 0: STQ_LAUNCH(0, A, S);        \
+    case 1: STQ_LAUNCH(1, A, S);        \
+    default: STQ_LAUNCH(2, A, S);       \
+  }
+  if (split) {
+    // the mixed-precision extras cost this body nothing measurable: one variant serves both
+    STQ_LAUNCH_G(true, true)
+  }
   if (amp) {
-    switch (grad_dtype) {
-      case 0: return launch_fast_t<0, true>(table, tile_map, sched, sc, p, err_flag, grid, stream);
-      case 1: return launch_fast_t<1, true>(table, tile_map, sched, sc, p, err_flag, grid, stream);
-      default: return launch_fast_t<2, true>(table, tile_map, sched, sc, p, err_flag, grid, stream);
-    }
+    STQ_LAUNCH_G(true, false)
   }
-  switch (grad_dtype) {
-    case 0: return launch_fast_t<0, false>(table, tile_map, sched, sc, p, err_flag, grid, stream);
-    case 1: return launch_fast_t<1, false>(table, tile_map, sched, sc, p, err_flag, grid, stream);
-    default: return launch_fast_t<2, false>(table, tile_map, sched, sc, p, err_flag, grid, stream);
-  }
+  STQ_LAUNCH_G(false, false)
+#undef STQ_LAUNCH_G
+#undef STQ_LAUNCH
 }
 
 cudaError_t launch_wait_timeout_selftest(int* err_flag, cudaStream_t stream) {
@@ -806,7 +1010,7 @@ cudaError_t launch_wait_timeout_selftest(int* err_flag, cudaStream_t stream) {
 
 int fast_ctas_per_sm() {
   int n = 0;
-  auto kern = stq_step_fast_kernel<1, false>;
+  auto kern = stq_step_fast_kernel<1, false, false>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return 1;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kFastThreads, kSmemBytes) != cudaSuccess) return 1;
   return n > 0 ? n : 1;
