@@ -331,3 +331,36 @@ def test_one_tensor_beyond_two_to_the_32_elements():
         x = g[lo:lo + (1 << 28)].double()
         want += np.array([x.sum().item(), x.abs().sum().item(), (x * x).sum().item(), x.numel()])
     H.assert_stats_close(got, want[None, :], "2^32")
+
+
+def test_full_size_runs_are_identical_bit_for_bit():
+    """The tile order a CTA sees depends on dynamic scheduling (atomic chunk counters), the results must
+    not: two runs of cfg2 (30 steps, statistics every 10th, a width change on the way) end in the same
+    parameters, codes, scales and statistics."""
+    _need(6)
+    w = W.config("cfg2")
+    bm, bv, _ = W.draw_bits(w)
+
+    def run():
+        job = Job(w, bm, bv)
+        stats = []
+        for t in range(1, 31):
+            job.draw_grads(t)
+            new_bits = None
+            if t == 20:
+                new_bits = W.churn_bits(__import__("dataclasses").replace(w, churn=0.2), job.bits_m, job.bits_v, 0)[:2]
+            job.step(t, stats=(t % 10 == 0), new_bits=new_bits)
+            if t % 10 == 0:
+                stats.append(job.layer_stats())
+        job.handle.device_status()
+        return job, stats
+
+    a, sa = run()
+    b, sb = run()
+    assert torch.equal(a.param_flat, b.param_flat)
+    for x, y in zip(a.states, b.states):
+        assert x.bits_m == y.bits_m and x.bits_v == y.bits_v
+        assert torch.equal(x.m_codes, y.m_codes) and torch.equal(x.v_codes, y.v_codes)
+        assert torch.equal(x.m_scales, y.m_scales) and torch.equal(x.v_scales, y.v_scales)
+    for x, y in zip(sa, sb):
+        np.testing.assert_array_equal(x, y)
