@@ -43,6 +43,9 @@ struct stq_handle {
   void* h_stage = nullptr;
   size_t h_stage_cap = 0;
   cudaEvent_t stage_ev = nullptr;
+  // the generic kernel's share of a step (ragged tails, 32-bit states) runs beside the main kernel:
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   bool stage_busy = false;
 
   // statistics
@@ -424,6 +427,27 @@ int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::St
     if (rc != STQ_OK) return rc;
     partials = h->d_partials;
   }
+  // The tiles of the generic kernel are independent of the main kernel's.  When a step has both, the
+  // generic launches go to a side stream forked from the caller's and joined back into it, so that they
+  // fill the SMs the persistent CTAs leave free at the ends of the main kernel instead of waiting for it.
+  const bool both = h->n_fast > 0 && h->n_tiles > h->n_fast && h->side != nullptr;
+  cudaStream_t gs = stream;
+  if (both) {
+    STQ_CUDA(h, cudaEventRecord(h->ev_fork, stream));
+    STQ_CUDA(h, cudaStreamWaitEvent(h->side, h->ev_fork, 0));
+    gs = h->side;
+  }
+  if (h->n_narrow > h->n_fast) {
+    STQ_CUDA(h, stq::launch_tiles(mode, false, grad_dtype, stats, h->d_table, h->d_tile_map, h->n_fast,
+                                  h->n_narrow, sc, partials, h->grid, gs));
+    h->launches++;
+  }
+  if (h->n_tiles > h->n_narrow) {
+    STQ_CUDA(h, stq::launch_tiles(mode, true, grad_dtype, stats, h->d_table, h->d_tile_map, h->n_narrow,
+                                  h->n_tiles, sc, partials, h->grid, gs));
+    h->launches++;
+  }
+  if (both) STQ_CUDA(h, cudaEventRecord(h->ev_join, h->side));
   if (h->n_main > 0) {   // only a step table has fast tiles
     const bool amp = h->any_lp || sc.inv_scale != nullptr;
     STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, amp, false, h->d_table, h->d_tile_map, h->d_sched, sc,
@@ -436,16 +460,7 @@ int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::St
                                       partials, h->d_err, grid, stream));
     h->launches++;
   }
-  if (h->n_narrow > h->n_fast) {
-    STQ_CUDA(h, stq::launch_tiles(mode, false, grad_dtype, stats, h->d_table, h->d_tile_map, h->n_fast,
-                                  h->n_narrow, sc, partials, h->grid, stream));
-    h->launches++;
-  }
-  if (h->n_tiles > h->n_narrow) {
-    STQ_CUDA(h, stq::launch_tiles(mode, true, grad_dtype, stats, h->d_table, h->d_tile_map, h->n_narrow,
-                                  h->n_tiles, sc, partials, h->grid, stream));
-    h->launches++;
-  }
+  if (both) STQ_CUDA(h, cudaStreamWaitEvent(stream, h->ev_join, 0));
   return STQ_OK;
 }
 
@@ -507,6 +522,14 @@ int stq_create(stq_handle** out, int device) {
     delete h;
     return STQ_E_WORKSPACE;
   }
+  // (without the side stream everything simply runs in order on the caller's stream)
+  if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+    (void)cudaGetLastError();
+    if (h->side) cudaStreamDestroy(h->side);
+    h->side = nullptr;
+  }
   *out = h;
   return STQ_OK;
 }
@@ -530,6 +553,9 @@ int stq_destroy(stq_handle* h) {
   if (h->h_stage) cudaFreeHost(h->h_stage);
   if (h->h_stats) cudaFreeHost(h->h_stats);
   if (h->stage_ev) cudaEventDestroy(h->stage_ev);
+  if (h->side) cudaStreamDestroy(h->side);
+  if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+  if (h->ev_join) cudaEventDestroy(h->ev_join);
   delete h;
   return STQ_OK;
 }
