@@ -140,7 +140,12 @@ int stq_init_state(stq_handle* h, const stq_tensor* tensors, int L, void* stream
  *   param = param*(1 - lr*wd) - lr * (mq/(1-beta1^t)) / (sqrt(vq/(1-beta2^t)) + eps)
  * where mq, vq are the values the new codes decode to.  With STQ_WITH_STATS the per-tensor sums
  * sum g, sum |g|, sum g^2 (Eq. 2, 3, 8) are accumulated in the same pass; fetch them with
- * stq_layer_stats. */
+ * stq_layer_stats.
+ * Stream capture: the first call with a given table validates it and uploads it (host work that
+ * may synchronise); a later call with the byte-identical table only enqueues work on `stream` and on
+ * an internal side stream forked from and joined back into it, so it can be captured into a CUDA
+ * graph.  The scalars derived from `hp` (bias corrections, learning rate) are launch parameters:
+ * a replay repeats the captured step t. */
 int stq_step(stq_handle* h, const stq_tensor* tensors, int L, const stq_hparams* hp, unsigned flags,
              void* stream);
 

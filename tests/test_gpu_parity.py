@@ -470,3 +470,36 @@ def test_fp16_training_recipe_on_a_small_model(H, O, v_log):
         H.assert_stats_close(job.layer_stats(), st, f"fp16 {v_log} t={t}")
         for p, lp in zip(job.params, job.params_lp):
             assert torch.equal(lp, p.to(torch.float16))
+
+
+def test_a_step_can_be_captured_into_a_cuda_graph(H, O):
+    """A step over a table the handle has already seen enqueues only stream work (a counter reset, the
+    kernels, the fork and join of the side stream), so it can be captured and replayed.  The scalars
+    of the step (bias corrections, learning rate) are baked in at capture: a replay repeats step t."""
+    w = W.scaled(W.config("cfg5"), W.small_gpt2(d=136, n_layer=2, vocab=777), steps=3)
+    bm, bv, _ = W.draw_bits(w)
+
+    def make():
+        job = Job(w, bm, bv)
+        job.draw_grads(1)
+        job.step(1)
+        return job
+
+    eager, graphed = make(), make()
+    for _ in range(3):
+        eager.step(5)
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        graphed.handle.step(graphed.table(), **graphed.hp(5))      # step 1 of 3, and the table's first use
+        s.synchronize()
+        with torch.cuda.graph(g, stream=s):
+            graphed.handle.step(graphed.table(), **graphed.hp(5))  # captured, not run
+        g.replay()                                                  # steps 2 and 3
+        g.replay()
+        s.synchronize()
+    graphed.handle.device_status()
+    assert torch.equal(eager.param_flat, graphed.param_flat)
+    for x, y in zip(eager.states, graphed.states):
+        assert torch.equal(x.m_codes, y.m_codes) and torch.equal(x.v_codes, y.v_codes)
+        assert torch.equal(x.m_scales, y.m_scales) and torch.equal(x.v_scales, y.v_scales)
