@@ -49,7 +49,9 @@ _lib = None
 def lib():
     global _lib
     if _lib is None:
-        L = C.CDLL(build())
+        # STQ_ORACLE_LIB: the pin suite can be pointed at another build of the oracle source (the mutation
+        # check in tests/ runs it against deliberately broken copies to see that the pins notice)
+        L = C.CDLL(os.environ.get("STQ_ORACLE_LIB") or build())
         L.orc_codes_bytes.restype = C.c_uint64
         L.orc_codes_bytes.argtypes = [C.c_uint64, C.c_int]
         L.orc_num_blocks.restype = C.c_uint64
@@ -204,20 +206,20 @@ def step(theta: np.ndarray, grad: np.ndarray, st: State, block: int, *, lr, beta
     n = theta.size
     dt = _grad_dtype(grad, fp16_grad)
     assert grad.size == n
-    if found_inf:
-        return st, (np.zeros(4) if want_stats else None)
     bm = st.bits_m if bits_m_out is None else bits_m_out
     bv = st.bits_v if bits_v_out is None else bits_v_out
     mc, ms = alloc_state(n, bm, block)
     vc, vs = alloc_state(n, bv, block)
-    hp = HParams(lr, beta1, beta2, eps, weight_decay, t, 1 if decoupled_wd else 0, dt, inv_grad_scale, 0,
-                 v_mode)
+    hp = HParams(lr, beta1, beta2, eps, weight_decay, t, 1 if decoupled_wd else 0, dt, inv_grad_scale,
+                 1 if found_inf else 0, v_mode)
     stats = np.zeros(4, dtype=np.float64) if want_stats else None
     rc = lib().orc_step(_p(theta), _p(grad), n, block,
                         _p(st.m_codes), _p(st.m_scales), st.bits_m,
                         _p(st.v_codes), _p(st.v_scales), st.bits_v,
                         _p(mc), _p(ms), bm, _p(vc), _p(vs), bv, C.byref(hp), _p(stats))
     assert rc == 0
+    if found_inf:      # the skipped step touched nothing: the stored state stands, no statistics
+        return st, (np.zeros(4) if want_stats else None)
     return State(mc, ms, bm, vc, vs, bv), stats
 
 
