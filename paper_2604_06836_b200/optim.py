@@ -10,7 +10,9 @@ the CUDA library, the decision in its host policy.  One optimizer step is
     other steps:
         stq_step in place
 
-which is the order Algorithm 1 prints.  Every tensor starts at ``init_bits`` (16 in the paper).
+which is the order Algorithm 1 prints.  With ``order="fused"`` the statistics ride on the update of
+the step before a decision step instead (``STQ_WITH_STATS``), which saves the extra pass over the
+gradients.  Every tensor starts at ``init_bits`` (16 in the paper).
 """
 from __future__ import annotations
 
@@ -29,6 +31,10 @@ class STQAdamW(torch.optim.Optimizer):
     the other hyper-parameters are shared).  Gradients may be fp32, bf16 or fp16, one type for all.
     policy: "paper" lets the transition decision pick widths in {4, 8, 16, 32} every ``interval`` steps
     (and while t < 5); "fixed" keeps ``init_bits`` (an int, or a pair (bits_m, bits_v)) for good.
+    order: "paper" takes the statistics of a decision step from that step's own gradients in a pass
+    before the update (Algorithm 1 as printed, one more read of the gradients on decision steps);
+    "fused" lets them ride on the update of the step before (no extra pass; the decision then sees
+    gradients that are one step old, except at t = 1).
     v_log: "poly" or "pl", the variant of the second-moment code at 8 and 16 bits.
     grad_scaler_inv / found_inf: optional one-element float32 CUDA tensors for loss-scaled training.
     """
@@ -36,9 +42,13 @@ class STQAdamW(torch.optim.Optimizer):
     def __init__(self, params: Iterable, lr: float = 1e-3, betas=(0.9, 0.999), eps: float = 1e-8,
                  weight_decay: float = 0.01, *, block: int = 128, init_bits=16, policy: str = "paper",
                  interval: int = 10, alpha: float = 0.1, tau: float = 100.0, eps_stat: float = 1e-8,
-                 v_log: str = "poly", decoupled_weight_decay: bool = True):
+                 v_log: str = "poly", decoupled_weight_decay: bool = True, order: str = "paper"):
         if policy not in ("paper", "fixed"):
             raise ValueError("policy is 'paper' or 'fixed'")
+        if order not in ("paper", "fused"):
+            raise ValueError("order is 'paper' or 'fused'")
+        self.order = order
+        self._pending_stats = False       # the last step carried statistics that have not been fetched
         if block not in (128, 256, 512):
             raise ValueError("block is 128, 256 or 512")
         defaults = dict(lr=lr, weight_decay=weight_decay)
@@ -119,17 +129,24 @@ class STQAdamW(torch.optim.Optimizer):
                   inv_grad_scale=self.grad_scaler_inv, found_inf=self.found_inf)
         new_m = new_v = None
         if self.policy_kind == "paper" and self.policy.is_decision_step(t):
-            tbl = self._table()
-            self.handle.grad_stats(tbl, hp["grad_dtype"])
-            stats = self.handle.layer_stats(len(self._params))
-            if self.grad_scaler_inv is not None:       # the pre-pass sees the scaled gradients: unscale the sums
-                s = float(self.grad_scaler_inv.item())
-                stats[:, 0:2] *= s
-                stats[:, 2] *= s * s
+            if self._pending_stats:                    # fused order: the sums rode on the previous step
+                stats = self.handle.layer_stats(len(self._params))
+            else:
+                tbl = self._table()
+                self.handle.grad_stats(tbl, hp["grad_dtype"])
+                stats = self.handle.layer_stats(len(self._params))
+                if self.grad_scaler_inv is not None:   # the pre-pass sees the scaled gradients: unscale the sums
+                    s = float(self.grad_scaler_inv.item())
+                    stats[:, 0:2] *= s
+                    stats[:, 2] *= s * s
             bits, self.last_scores = self.policy.decide(stats, t)
             new_m = new_v = bits                       # Algorithm 1: one width per layer for both states
+        # fused order: if the next step decides, this one carries the statistics
+        flags = stq.WITH_STATS if (self.order == "fused" and self.policy_kind == "paper" and
+                                   self.policy.is_decision_step(t + 1)) else 0
+        self._pending_stats = bool(flags)
         if new_m is None or ((new_m == self.bits_m).all() and (new_v == self.bits_v).all()):
-            self.handle.step(self._table(), **hp)
+            self.handle.step(self._table(), flags=flags, **hp)
             return loss
         out = []
         for k, p in enumerate(self._params):
@@ -144,7 +161,7 @@ class STQAdamW(torch.optim.Optimizer):
             vc, vs = (old.v_codes, old.v_scales) if bv == old.bits_v else (
                 stq.alloc_codes(n, bv, self.device), stq.alloc_scales(n, bv, self.block, self.device))
             out.append(stq.QState(mc, ms, bm, vc, vs, bv, self.v_log))
-        self.handle.step(stq.table(self._rows(out)), **hp)
+        self.handle.step(stq.table(self._rows(out)), flags=flags, **hp)
         torch.cuda.current_stream(self.device).synchronize()     # the old buffers are released below
         self.states = out
         self.bits_m, self.bits_v = np.array(new_m, np.uint8), np.array(new_v, np.uint8)

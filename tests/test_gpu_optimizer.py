@@ -110,3 +110,39 @@ def test_wrapper_matches_the_oracle_run_of_algorithm_1(v_log):
             H.assert_theta_close(params[i].data, theta[i], 1e-6 * t, f"t={t} tensor {i}", upd=upd[i])
         if bits is not None:
             assert (opt.bits_m == bits).all()
+
+
+def test_fused_order_decides_on_the_previous_steps_gradients():
+    """order="fused": the statistics of a decision step ride on the update before it, so the decision at
+    step t sees the gradients of step t - 1 (t = 1 has none and takes a pre-pass).  Against the oracle."""
+    import harness as H
+    import oracle
+    torch.manual_seed(6)
+    sizes = [4096 * 2 + 300, 777, 4096]
+    params = [torch.nn.Parameter(torch.randn(n, device="cuda") * 0.02) for n in sizes]
+    opt = STQAdamW(params, lr=1e-3, weight_decay=0.01, policy="paper", interval=4, tau=8.0, order="fused")
+    theta = [H.to_np(p.data) for p in params]
+    states = [oracle.new_state(n, 128, 16, 16) for n in sizes]
+    pol = oracle.new_policy(0.1, 8.0, 1e-8)
+    upd = [np.abs(t) for t in theta]
+    prev = None
+    for t in range(1, 14):
+        g = torch.Generator(device="cuda").manual_seed(50 + t)
+        for k, p in enumerate(params):
+            p.grad = torch.randn(p.numel(), device="cuda", generator=g) * (1e-3 * 10.0 ** (-k)) * (1.0 + 2.0 * (t % 4))
+        grads = [H.to_np(p.grad) for p in params]
+        bits = None
+        if oracle.is_decision_step(t, 4):
+            src = grads if t == 1 else prev
+            st = np.stack([oracle.grad_stats(x) for x in src])
+            bits, _ = oracle.decide(pol, st, t)
+        opt.step()
+        for i in range(len(sizes)):
+            before = theta[i].copy()
+            b = None if bits is None else int(bits[i])
+            states[i], _ = oracle.step(theta[i], grads[i], states[i], 128, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8,
+                                       weight_decay=0.01, t=t, bits_m_out=b, bits_v_out=b)
+            upd[i] = np.maximum(upd[i], np.maximum(np.abs(theta[i]), np.abs(theta[i] - before)))
+            H.assert_states_equal(opt.states[i], states[i], f"fused t={t} tensor {i}")
+            H.assert_theta_close(params[i].data, theta[i], 1e-6 * t, f"fused t={t} tensor {i}", upd=upd[i])
+        prev = grads
