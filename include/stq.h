@@ -117,6 +117,11 @@ typedef struct stq_hparams {
                                /* before anything else (statistics included)                         */
   const float* found_inf;      /* if *found_inf != 0 the step is skipped: no buffer is touched, and   */
                                /* statistics requested with the step are not produced                */
+  /* Step count and learning rate kept on the DEVICE (both optional, NULL = use `step` and `lr` above):  */
+  /* a step captured into a CUDA graph then advances with the caller's counter instead of repeating     */
+  /* the captured t.  The bias corrections 1 - beta^t are formed on the device in double precision.     */
+  const int64_t* step_dev;     /* device pointer to t >= 1 (values below 1 are read as 1)              */
+  const float* lr_dev;         /* device pointer to the learning rate                                  */
 } stq_hparams;
 
 /* Handle: device copy of the tensor table, tile map and statistics workspace.

@@ -36,7 +36,8 @@ struct stq_handle {
   uint32_t n_main = 0;                              // fast tiles of the fused bodies; [n_main, n_fast) change width
   int fast_grid = 0;
   bool any_lp = false;              // some tensor of the current table wants a low-precision copy
-  int* d_err = nullptr;             // raised by a kernel whose bounded wait ran out
+  int* d_err = nullptr;
+  float* d_scalars = nullptr;   // {step_size, rsqrt_bc2, lr} when the step count lives on the device             // raised by a kernel whose bounded wait ran out
   stq::FastSched* d_sched = nullptr;   // two work lists of the main step kernel (fused bodies, width changes)
 
   // pinned staging for uploads
@@ -449,7 +450,7 @@ int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::St
   }
   if (both) STQ_CUDA(h, cudaEventRecord(h->ev_join, h->side));
   if (h->n_main > 0) {   // only a step table has fast tiles
-    const bool amp = h->any_lp || sc.inv_scale != nullptr;
+    const bool amp = h->any_lp || sc.inv_scale != nullptr || sc.dev_scalars != nullptr;
     STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, amp, false, h->d_table, h->d_tile_map, h->d_sched, sc,
                                       partials, h->d_err, h->fast_grid, stream));
     h->launches++;
@@ -470,6 +471,7 @@ int check_hparams(const stq_hparams* hp, unsigned flags) {
   if (hp->grad_dtype < STQ_GRAD_F32 || hp->grad_dtype > STQ_GRAD_F16) return STQ_E_ARG;
   if (flags & ~(unsigned)STQ_WITH_STATS) return STQ_E_ARG;
   if (!aligned(hp->inv_grad_scale, 4) || !aligned(hp->found_inf, 4)) return STQ_E_ALIGN;
+  if (!aligned(hp->step_dev, 8) || !aligned(hp->lr_dev, 4)) return STQ_E_ALIGN;
   if (!(hp->beta1 >= 0.0 && hp->beta1 < 1.0 && hp->beta2 >= 0.0 && hp->beta2 < 1.0)) return STQ_E_ARG;
   return STQ_OK;
 }
@@ -489,6 +491,7 @@ stq::StepConsts make_consts(const stq_hparams* hp) {
   sc.lr = hp->lr;
   sc.inv_scale = hp->inv_grad_scale;
   sc.found_inf = hp->found_inf;
+  sc.dev_scalars = nullptr;
   return sc;
 }
 
@@ -517,6 +520,7 @@ int stq_create(stq_handle** out, int device) {
   if (h->fast_grid > stq::kFastMaxGrid) h->fast_grid = stq::kFastMaxGrid;
   if (cudaMalloc(reinterpret_cast<void**>(&h->d_err), sizeof(int)) != cudaSuccess ||
       cudaMemset(h->d_err, 0, sizeof(int)) != cudaSuccess ||
+      cudaMalloc(reinterpret_cast<void**>(&h->d_scalars), 4 * sizeof(float)) != cudaSuccess ||
       cudaMalloc(reinterpret_cast<void**>(&h->d_sched), 2 * sizeof(stq::FastSched)) != cudaSuccess) {
     cudaEventDestroy(h->stage_ev);
     delete h;
@@ -542,6 +546,7 @@ int stq_destroy(stq_handle* h) {
   cudaFree(h->d_tile_map);
   cudaFree(h->d_err);
   cudaFree(h->d_sched);
+  cudaFree(h->d_scalars);
   cudaFree(h->d_partials);
   cudaFree(h->d_stats);
   cudaFree(h->d_seg_map);
@@ -588,7 +593,17 @@ int stq_step(stq_handle* h, const stq_tensor* tensors, int L, const stq_hparams*
   rc = prepare(h, tensors, L, kKindStep, s);
   if (rc != STQ_OK) return rc;
   const bool stats = (flags & STQ_WITH_STATS) != 0;
-  rc = run(h, stq::kStep, hp->grad_dtype, stats, make_consts(hp), s);
+  stq::StepConsts sc = make_consts(hp);
+  if (hp->step_dev != nullptr || hp->lr_dev != nullptr) {
+    // step count and / or learning rate on the device: a one-thread kernel derives the step's scalars
+    // ahead of the step kernels, which then read them instead of their launch parameters
+    if (hp->step_dev == nullptr) return STQ_E_ARG;       // (a device learning rate comes with a device step count)
+    STQ_CUDA(h, stq::launch_step_scalars(reinterpret_cast<const long long*>(hp->step_dev), hp->lr_dev, hp->lr,
+                                         hp->beta1, hp->beta2, h->d_scalars, s));
+    h->launches++;
+    sc.dev_scalars = h->d_scalars;
+  }
+  rc = run(h, stq::kStep, hp->grad_dtype, stats, sc, s);
   if (rc == STQ_OK && stats) h->stats_L = L;
   return rc;
 }
@@ -677,7 +692,8 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
     if (t.lp_dtype != STQ_LP_NONE) need += up(t.numel * 2);
     need += 6 * (4096 + 512);   // padding carried along when buffers travel as one run
   }
-  if (hp->inv_grad_scale || hp->found_inf) return STQ_E_ARG;   // device pointers have no place in the host-buffer call
+  if (hp->inv_grad_scale || hp->found_inf || hp->step_dev || hp->lr_dev)
+    return STQ_E_ARG;   // device pointers have no place in the host-buffer call
   rc = grow(h, h->d_arena, h->d_arena_cap, need);
   if (rc != STQ_OK) return rc;
 

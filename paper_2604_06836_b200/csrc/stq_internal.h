@@ -51,7 +51,14 @@ struct StepConsts {
   double lr;                // decoupled decay factor is fp32(1 - lr*wd), formed per tile
   const float* inv_scale;   // device: gradients are multiplied by *inv_scale first (nullptr: no)
   const float* found_inf;   // device: a non-zero value skips the whole step (nullptr: never)
+  const float* dev_scalars; // device: {step_size, rsqrt_bc2, lr} written by the scalars kernel for this launch
+                            // (nullptr: the three values above are the ones to use)
 };
+
+// Derives the step's scalars from a step count (and optionally a learning rate) held on the device:
+// out = {lr / (1 - beta1^t), 1 / sqrt(1 - beta2^t), lr}, in double precision, one thread.
+cudaError_t launch_step_scalars(const long long* step_dev, const float* lr_dev, double lr_host, double beta1,
+                                double beta2, float* out, cudaStream_t stream);
 
 enum Mode { kStep = 0, kRepack = 1, kInit = 2, kStatsOnly = 3 };
 

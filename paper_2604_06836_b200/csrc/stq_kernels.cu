@@ -383,7 +383,15 @@ __device__ __forceinline__ void store_param(float* p, int nvl, const float (&x)[
 template <int MODE, int GDT, bool STATS, bool WIDE>
 __global__ void __launch_bounds__(kThreads, 2)
 stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map,
-                uint32_t tile_begin, uint32_t tile_end, const StepConsts sc, double* __restrict__ partials) {
+                uint32_t tile_begin, uint32_t tile_end, const StepConsts sc_in, double* __restrict__ partials) {
+  StepConsts sc = sc_in;
+  if constexpr (MODE == kStep) {
+    if (sc_in.dev_scalars != nullptr) {     // step count / learning rate live on the device
+      sc.step_size = __ldg(sc_in.dev_scalars + 0);
+      sc.rsqrt_bc2 = __ldg(sc_in.dev_scalars + 1);
+      sc.lr = (double)__ldg(sc_in.dev_scalars + 2);
+    }
+  }
   constexpr int R = kRowsPerWarp;
   constexpr bool kHasGrad = (MODE == kStep || MODE == kStatsOnly);
   const int lane = threadIdx.x & 31;
@@ -880,6 +888,24 @@ cudaError_t launch_stats_finish(const TensorDesc* table, int L, const uint32_t* 
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   stq_stats_finish_kernel<<<L, 256, 0, stream>>>(table, L, seg_sums, out);
+  return cudaGetLastError();
+}
+
+__global__ void stq_step_scalars_kernel(const long long* __restrict__ step_dev, const float* __restrict__ lr_dev,
+                                        double lr_host, double beta1, double beta2, float* __restrict__ out) {
+  long long t = *step_dev;
+  if (t < 1) t = 1;
+  const double lr = lr_dev != nullptr ? (double)*lr_dev : lr_host;
+  const double bc1 = 1.0 - pow(beta1, (double)t);
+  const double bc2 = 1.0 - pow(beta2, (double)t);
+  out[0] = (float)(lr / bc1);
+  out[1] = (float)(1.0 / sqrt(bc2));
+  out[2] = (float)lr;
+}
+
+cudaError_t launch_step_scalars(const long long* step_dev, const float* lr_dev, double lr_host, double beta1,
+                                double beta2, float* out, cudaStream_t stream) {
+  stq_step_scalars_kernel<<<1, 1, 0, stream>>>(step_dev, lr_dev, lr_host, beta1, beta2, out);
   return cudaGetLastError();
 }
 

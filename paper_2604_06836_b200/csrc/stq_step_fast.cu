@@ -795,8 +795,22 @@ __device__ __forceinline__ uint32_t width_index(uint32_t b) { return b == 2 ? 0u
 template <int GDT, bool AMP, bool SPLIT>
 __global__ void __launch_bounds__(kFastThreads, kFastCtasPerSm)
 stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map,
-                     FastSched* __restrict__ sched, const StepConsts sc, double* __restrict__ partials,
+                     FastSched* __restrict__ sched, const StepConsts sc_in, double* __restrict__ partials,
                      int* __restrict__ err_flag) {
+  // The launches with the mixed-precision extras also accept the step's scalars from device memory
+  // (a step count and learning rate that advance between replays of a captured graph).
+  StepConsts sc_dev;
+  const StepConsts* scp = &sc_in;
+  if constexpr (AMP) {
+    if (sc_in.dev_scalars != nullptr) {
+      sc_dev = sc_in;
+      sc_dev.step_size = __ldg(sc_in.dev_scalars + 0);
+      sc_dev.rsqrt_bc2 = __ldg(sc_in.dev_scalars + 1);
+      sc_dev.lr = (double)__ldg(sc_in.dev_scalars + 2);
+      scp = &sc_dev;
+    }
+  }
+  const StepConsts& sc = *scp;
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t full0 = smem_u32(smem + kOffBars);

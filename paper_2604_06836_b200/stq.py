@@ -50,7 +50,8 @@ class CHParams(C.Structure):
     """struct stq_hparams"""
     _fields_ = [("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
                 ("step", C.c_int64), ("decoupled_wd", C.c_int32), ("grad_dtype", C.c_int32),
-                ("inv_grad_scale", C.c_void_p), ("found_inf", C.c_void_p)]
+                ("inv_grad_scale", C.c_void_p), ("found_inf", C.c_void_p),
+                ("step_dev", C.c_void_p), ("lr_dev", C.c_void_p)]
 
 
 class CPolicyCfg(C.Structure):
@@ -243,10 +244,17 @@ class Handle:
         self._check(lib().stq_init_state(self._h, tbl, len(tbl), _stream_ptr(stream)), "stq_init_state")
 
     def step(self, tbl, *, lr, beta1, beta2, eps, t, grad_dtype=GRAD_F32, decoupled_wd=True, flags=0, stream=None,
-             inv_grad_scale: torch.Tensor | None = None, found_inf: torch.Tensor | None = None):
-        """inv_grad_scale / found_inf: optional one-element float32 device tensors (loss-scaled training)."""
+             inv_grad_scale: torch.Tensor | None = None, found_inf: torch.Tensor | None = None,
+             step_dev: torch.Tensor | None = None, lr_dev: torch.Tensor | None = None):
+        """inv_grad_scale / found_inf: optional one-element float32 device tensors (loss-scaled training).
+        step_dev (one int64) / lr_dev (one float32): optional device tensors that replace t and lr, for steps
+        replayed from a CUDA graph."""
+        if step_dev is not None and step_dev.dtype != torch.int64:
+            raise ValueError("step_dev holds one int64")
+        if lr_dev is not None and lr_dev.dtype != torch.float32:
+            raise ValueError("lr_dev holds one float32")
         hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype,
-                      _ptr(inv_grad_scale), _ptr(found_inf))
+                      _ptr(inv_grad_scale), _ptr(found_inf), _ptr(step_dev), _ptr(lr_dev))
         self._check(lib().stq_step(self._h, tbl, len(tbl), C.byref(hp), flags, _stream_ptr(stream)), "stq_step")
 
     def grad_stats(self, tbl, grad_dtype=GRAD_F32, stream=None):
@@ -265,7 +273,7 @@ class Handle:
                   inv_grad_scale=None, found_inf=None):
         if inv_grad_scale is not None or found_inf is not None:
             raise ValueError("step_host takes host buffers only: unscale the gradients on the device path")
-        hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype, None, None)
+        hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype, None, None, None, None)
         h2d, d2h = C.c_uint64(0), C.c_uint64(0)
         self._check(lib().stq_step_host(self._h, tbl, len(tbl), C.byref(hp), flags, C.byref(h2d), C.byref(d2h)),
                     "stq_step_host")

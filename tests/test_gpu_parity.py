@@ -503,3 +503,41 @@ def test_a_step_can_be_captured_into_a_cuda_graph(H, O):
     for x, y in zip(eager.states, graphed.states):
         assert torch.equal(x.m_codes, y.m_codes) and torch.equal(x.v_codes, y.v_codes)
         assert torch.equal(x.m_scales, y.m_scales) and torch.equal(x.v_scales, y.v_scales)
+
+
+def test_graph_replays_advance_with_a_step_count_on_the_device(H, O):
+    """The step count and the learning rate may live on the device (hparams.step_dev / lr_dev): a step
+    captured once then runs steps t, t+1, ... as the caller's counter advances inside the graph, with new
+    gradients copied into the same buffers before every replay.  Codes and scales are those of eager
+    steps; the parameters agree to rounding (the device forms lr / (1 - beta1^t) from a float32 lr)."""
+    w = W.scaled(W.config("cfg2"), W.small_gpt2(d=136, n_layer=2, vocab=777), steps=8)
+    bm, bv, _ = W.draw_bits(w)
+    eager, graphed = Job(w, bm, bv), Job(w, bm, bv)
+    oj = H.OracleJob(eager)
+    step_dev = torch.zeros(1, dtype=torch.int64, device="cuda")
+    lr_dev = torch.full((1,), w.lr, dtype=torch.float32, device="cuda")
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    hp = {**graphed.hp(1), "step_dev": step_dev, "lr_dev": lr_dev}
+    with torch.cuda.stream(s):
+        graphed.draw_grads(1)
+        step_dev.fill_(1)
+        graphed.handle.step(graphed.table(), **hp)          # t = 1 eagerly: the table's first use
+        s.synchronize()
+        with torch.cuda.graph(g, stream=s):
+            step_dev.add_(1)
+            graphed.handle.step(graphed.table(), **hp)
+    for t in range(1, 8):
+        eager.draw_grads(t)
+        oj.step([H.to_np(x) for x in eager.grads], t)
+        eager.step(t)
+        if t > 1:
+            with torch.cuda.stream(s):
+                graphed.draw_grads(t)
+                g.replay()
+                s.synchronize()
+        graphed.handle.device_status()
+        assert int(step_dev.item()) == t
+        H.compare_job(graphed, oj, REL_1STEP * t * 2, f"graph t={t}")
+        for x, y in zip(eager.states, graphed.states):
+            assert torch.equal(x.m_codes, y.m_codes) and torch.equal(x.v_codes, y.v_codes)
