@@ -72,7 +72,9 @@ cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const
 // of equal body (width pair, variant of the v code).  Lives in device memory; the counters are zeroed before every launch.
 constexpr int kFastMaxGroups = 64;     // 5 widths of m x (5 widths of v + 2 variants at 8 and 16 bits) = 35 bodies
 constexpr int kFastMaxGrid = 4096;
-constexpr uint32_t kFastChunk = 8;     // tiles handed out per counter increment (fewer for small launches)
+constexpr uint32_t kFastChunk = 2;     // tiles handed out per counter increment (one for small launches); measured:
+                                       // 2-3 beat 1 and 8 by 1-4 % on the small and medium configurations (shorter tail
+                                       // when a group runs dry), no difference on the largest
 struct FastSched {
   uint32_t ctr[kFastMaxGroups];            // chunks handed out so far, per group
   uint32_t ng;                             // number of groups

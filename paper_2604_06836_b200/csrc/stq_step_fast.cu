@@ -781,7 +781,7 @@ __device__ __forceinline__ void tile_body_split(const uint8_t* __restrict__ stag
 }
 
 // Scheduling: the fast tiles are grouped by body (width pair and variant of the v code).  A CTA starts in the group
-// the host assigned to it and takes chunks of consecutive tiles (kFastChunk of them, fewer when the
+// the host assigned to it and takes chunks of consecutive tiles (kFastChunk of them, single tiles when the
 // launch is small) from that group's
 // counter; when its group runs dry it moves on to the next one that still has work.  So a CTA runs
 // few different bodies (a change of body is an instruction-cache refill), the tiles of a group are
