@@ -198,6 +198,24 @@ int validate_row(const stq_tensor& t, int kind) {
 
 // Tensors with the same key run the same specialised body of the main kernel: the two widths, and
 // for v at 8 or 16 bits the variant of its quantizer.  Ordered from cheap to expensive v codes.
+// Relative time per tile of the fused bodies, from the measured throughput of each on one large tensor
+// (rows: m at 2, 3, 4, 8, 16 bits; columns: v at 2, 3, 4, 8, 16 bits, then 8 and 16 bits in the
+// piecewise-linear variant; 1.0 = the 4/4-bit body).  Only the initial spread of the CTAs over the
+// groups uses it; the balance itself is dynamic.
+double body_cost(const stq_tensor& t) {
+  static const double kRate[5][7] = {
+      {490, 458, 480, 392, 345, 440, 411},
+      {454, 426, 455, 370, 323, 424, 401},
+      {470, 462, 483, 389, 345, 437, 413},
+      {476, 458, 466, 389, 340, 435, 396},
+      {436, 426, 422, 379, 332, 396, 355},
+  };
+  auto idx = [](int b) { return b == 2 ? 0 : b == 3 ? 1 : b == 4 ? 2 : b == 8 ? 3 : 4; };
+  int iv = idx(t.bits_v);
+  if (t.v_log == STQ_VLOG_PL && iv >= 3) iv += 2;
+  return 483.0 / kRate[idx(t.bits_m)][iv];
+}
+
 constexpr int kSplitKey = 1 << 20;
 int body_key(const stq_tensor& t) {
   if (t.bits_m != t.bits_m_out || t.bits_v != t.bits_v_out) return kSplitKey;   // one runtime-width body for all of them
@@ -313,11 +331,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
         hs->grp_begin[hs->ng++] = next_fast;
         last_key = key;
       }
-      double w = t.bits_v == 16 ? 1.45 : t.bits_v == 8 ? 1.2 : 1.0;
-      if (t.v_log == STQ_VLOG_PL && t.bits_v >= 8) w = t.bits_v == 16 ? 1.1 : 1.0;
-      if (t.bits_v == 3 || t.bits_m == 3) w += 0.06;
-      if (t.bits_m == 16) w += 0.08;
-      cost[hs->ng - 1] += w * nfast[l];
+      cost[hs->ng - 1] += body_cost(t) * nfast[l];
       if (!same_map)
         for (uint32_t k = 0; k < nfast[l]; ++k) hm[next_fast + k] = (uint32_t)l;
       next_fast += nfast[l];
