@@ -1,11 +1,13 @@
-// The main kernel of the quantized AdamW step: full tiles of tensors whose widths stay the same
-// this step (2..16 bits).  Everything else (ragged last tiles, 32-bit states, width changes inside
-// the step, init, repack) goes through the generic kernel in stq_kernels.cu.
+// The main kernel of the quantized AdamW step: full tiles of tensors with packed states (2..16 bits)
+// on both sides of the step.  Tensors that keep their widths run bodies fused and specialised on the
+// width pair; tensors that change width inside the step run one runtime-width body in a second launch
+// (template flag SPLIT).  Everything else (ragged last tiles, 32-bit states, block 512, init, repack)
+// goes through the generic kernel in stq_kernels.cu.
 //
 // Data movement: a persistent CTA walks its tiles through a shared-memory ring.  A producer warp
 // (one elected lane) runs ahead: per tile it writes a small descriptor and issues six bulk
 // asynchronous copies (parameters, gradients, m codes, v codes, m scales, v scales: each a contiguous,
-// 16-byte aligned range because a tile starts at a multiple of 2048 elements) that complete on the
+// 16-byte aligned range because a tile starts at a multiple of 4096 elements) that complete on the
 // stage's "full" mbarrier.  The eight consumer warps never synchronise with each other: each waits
 // on "full", pulls its rows into registers with conflict-free 128/64/32-bit shared loads, arrives on
 // the stage's "empty" mbarrier (which lets the producer refill it) and computes.  Results go
