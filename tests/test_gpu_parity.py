@@ -541,3 +541,61 @@ def test_graph_replays_advance_with_a_step_count_on_the_device(H, O):
         H.compare_job(graphed, oj, REL_1STEP * t * 2, f"graph t={t}")
         for x, y in zip(eager.states, graphed.states):
             assert torch.equal(x.m_codes, y.m_codes) and torch.equal(x.v_codes, y.v_codes)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_tables_against_the_oracle(H, O, seed):
+    """Randomised tables: sizes from 1 element to a few tiles, every block size, widths 2..32 on both
+    sides of the step (so width changes, raw fp32 states and packed states mix in one call), all three
+    gradient types, both variants of the v code, per-tensor weight decay, AdamW and L2 mode, with and
+    without statistics.  Three steps each, codes and scales bit for bit."""
+    import oracle
+    rng = np.random.RandomState(1000 + seed)
+    widths = [2, 3, 4, 8, 16, 32]
+    for case in range(6):
+        L = int(rng.randint(1, 7))
+        block = int(rng.choice([128, 256, 512]))
+        gdt = [torch.float32, torch.bfloat16, torch.float16][int(rng.randint(0, 3))]
+        decoupled = bool(rng.randint(0, 2))
+        sizes = [int(rng.choice([1, 7, 127, 128, 129, 1000, 4095, 4096, 4097, 4096 * 2 + 333, 4096 * 3])) if rng.rand() < 0.6
+                 else int(rng.randint(1, 20000)) for _ in range(L)]
+        vlog = [int(rng.randint(0, 2)) for _ in range(L)]
+        wds = [float(rng.choice([0.0, 0.01, 0.1])) for _ in range(L)]
+        bits = [(int(rng.choice(widths)), int(rng.choice(widths))) for _ in range(L)]
+        gen = torch.Generator(device="cuda").manual_seed(int(rng.randint(0, 2 ** 31)))
+        params = [torch.empty(n, device="cuda").normal_(0, 0.02, generator=gen) for n in sizes]
+        states = [stq.alloc_state(n, block, bm, bv, "cuda", vl) for n, (bm, bv), vl in zip(sizes, bits, vlog)]
+        h = stq.Handle()
+        h.init_state(stq.table([stq.make_row(n, block, None, s) for n, s in zip(sizes, states)]))
+        theta = [H.to_np(p) for p in params]
+        ostates = [oracle.new_state(n, block, bm, bv) for n, (bm, bv) in zip(sizes, bits)]
+        upd = [np.abs(t) for t in theta]
+        for t in (1, 2, 3):
+            scale = 10.0 ** rng.uniform(-5, -2)
+            grads = [(torch.empty(n, device="cuda").normal_(0, 1.0, generator=gen) * scale).to(gdt) for n in sizes]
+            new_bits = [(int(rng.choice(widths)), int(rng.choice(widths))) if rng.rand() < 0.3 else b for b in bits]
+            out = [s if nb == b else stq.alloc_state(n, block, nb[0], nb[1], "cuda", vl)
+                   for s, nb, b, n, vl in zip(states, new_bits, bits, sizes, vlog)]
+            want_stats = bool(rng.randint(0, 2))
+            rows = [stq.make_row(n, block, s, o, p, g, wd) for n, s, o, p, g, wd in zip(sizes, states, out, params, grads, wds)]
+            h.step(stq.table(rows), lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, t=t, grad_dtype=stq.grad_dtype_of(grads[0]),
+                   decoupled_wd=decoupled, flags=stq.WITH_STATS if want_stats else 0)
+            got_stats = h.layer_stats(L) if want_stats else None
+            h.device_status()
+            states, bits = out, new_bits
+            for i in range(L):
+                before = theta[i].copy()
+                ostates[i], st = oracle.step(theta[i], H.to_np(grads[i]), ostates[i], block, lr=1e-3, beta1=0.9, beta2=0.999,
+                                             eps=1e-8, weight_decay=wds[i], t=t, bits_m_out=bits[i][0], bits_v_out=bits[i][1],
+                                             decoupled_wd=decoupled, want_stats=want_stats, fp16_grad=(gdt == torch.float16),
+                                             v_mode=oracle.LOG_PL if vlog[i] else oracle.LOG)
+                upd[i] = np.maximum(upd[i], np.maximum(np.abs(theta[i]), np.abs(theta[i] - before)))
+                tag = f"seed {seed} case {case} t={t} tensor {i} n={sizes[i]} B={block} bits {bits[i]} {gdt}"
+                H.assert_states_equal(states[i], ostates[i], tag)
+                H.assert_theta_close(params[i], theta[i], REL_1STEP * t * 2, tag, upd=upd[i])
+                if want_stats:
+                    H.assert_stats_close(got_stats[i:i + 1], st[None, :], tag)
+                if not decoupled:
+                    # L2 mode feeds the parameters back into the moments (g + lambda * theta), and the parameters
+                    # agree to rounding, not to the bit: each step is checked from identical inputs
+                    theta[i] = H.to_np(params[i])
