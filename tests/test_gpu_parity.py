@@ -599,3 +599,58 @@ def test_random_tables_against_the_oracle(H, O, seed):
                     # L2 mode feeds the parameters back into the moments (g + lambda * theta), and the parameters
                     # agree to rounding, not to the bit: each step is checked from identical inputs
                     theta[i] = H.to_np(params[i])
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_repacks_and_statistics_against_the_oracle(H, O, seed):
+    """Randomised width transitions without a step (stq_repack, including to and from raw fp32 states and
+    in both variants of the v code) and the statistics-only pass, on states that two steps have filled."""
+    import oracle
+    rng = np.random.RandomState(2000 + seed)
+    widths = [2, 3, 4, 8, 16, 32]
+    for case in range(6):
+        L = int(rng.randint(1, 6))
+        block = int(rng.choice([128, 256, 512]))
+        gdt = [torch.float32, torch.bfloat16, torch.float16][int(rng.randint(0, 3))]
+        sizes = [int(rng.choice([1, 129, 4095, 4096, 4097, 4096 * 2 + 333])) if rng.rand() < 0.5 else int(rng.randint(1, 15000))
+                 for _ in range(L)]
+        vlog = [int(rng.randint(0, 2)) for _ in range(L)]
+        bits = [(int(rng.choice(widths)), int(rng.choice(widths))) for _ in range(L)]
+        gen = torch.Generator(device="cuda").manual_seed(int(rng.randint(0, 2 ** 31)))
+        params = [torch.empty(n, device="cuda").normal_(0, 0.02, generator=gen) for n in sizes]
+        states = [stq.alloc_state(n, block, bm, bv, "cuda", vl) for n, (bm, bv), vl in zip(sizes, bits, vlog)]
+        h = stq.Handle()
+        h.init_state(stq.table([stq.make_row(n, block, None, s) for n, s in zip(sizes, states)]))
+        theta = [H.to_np(p) for p in params]
+        ostates = [oracle.new_state(n, block, bm, bv) for n, (bm, bv) in zip(sizes, bits)]
+        for t in (1, 2):
+            grads = [(torch.empty(n, device="cuda").normal_(0, 1.0, generator=gen) * 10.0 ** rng.uniform(-4, -2)).to(gdt)
+                     for n in sizes]
+            rows = [stq.make_row(n, block, s, s, p, g, 0.01) for n, s, p, g in zip(sizes, states, params, grads)]
+            h.step(stq.table(rows), lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, t=t, grad_dtype=stq.grad_dtype_of(grads[0]))
+            for i in range(L):
+                ostates[i], _ = oracle.step(theta[i], H.to_np(grads[i]), ostates[i], block, lr=1e-3, beta1=0.9, beta2=0.999,
+                                            eps=1e-8, weight_decay=0.01, t=t, fp16_grad=(gdt == torch.float16),
+                                            v_mode=oracle.LOG_PL if vlog[i] else oracle.LOG)
+        # statistics alone, on the last gradients
+        h.grad_stats(stq.table([stq.make_row(n, block, s, s, p, g) for n, s, p, g in zip(sizes, states, params, grads)]),
+                     stq.grad_dtype_of(grads[0]))
+        got = h.layer_stats(L)
+        want = np.stack([oracle.grad_stats(H.to_np(g), fp16=(gdt == torch.float16)) for g in grads])
+        H.assert_stats_close(got, want, f"seed {seed} case {case} statistics")
+        # two repacks in a row
+        for hop in range(2):
+            new_bits = [(int(rng.choice(widths)), int(rng.choice(widths))) for _ in range(L)]
+            out = [stq.alloc_state(n, block, nb[0], nb[1], "cuda", vl) for n, nb, vl in zip(sizes, new_bits, vlog)]
+            h.repack(stq.table([stq.make_row(n, block, s, o) for n, s, o in zip(sizes, states, out)]))
+            h.device_status()
+            for i in range(L):
+                st = ostates[i]
+                n = sizes[i]
+                vm = oracle.LOG_PL if vlog[i] else oracle.LOG
+                mc, ms = oracle.repack(st.m_codes, st.m_scales, st.bits_m, new_bits[i][0], n, block, oracle.LINEAR)
+                vc, vs = oracle.repack(st.v_codes, st.v_scales, st.bits_v, new_bits[i][1], n, block, vm)
+                ostates[i] = oracle.State(mc, ms, new_bits[i][0], vc, vs, new_bits[i][1])
+                H.assert_states_equal(out[i], ostates[i], f"seed {seed} case {case} hop {hop} tensor {i} n={n} B={block} "
+                                                          f"{bits[i]} -> {new_bits[i]} pl={vlog[i]}")
+            states, bits = out, new_bits
