@@ -570,16 +570,23 @@ def test_random_tables_against_the_oracle(H, O, seed):
         theta = [H.to_np(p) for p in params]
         ostates = [oracle.new_state(n, block, bm, bv) for n, (bm, bv) in zip(sizes, bits)]
         upd = [np.abs(t) for t in theta]
+        # mixed-precision extras on some tables: a loss scale (not always a power of two) and a working copy
+        amp = rng.rand() < 0.4
+        S = float(rng.choice([1024.0, 3.0, 65536.0])) if amp else 1.0
+        inv = torch.tensor([np.float32(1.0 / S)], dtype=torch.float32, device="cuda") if amp else None
+        lp_dt = [None, torch.bfloat16, torch.float16][int(rng.randint(0, 3))] if amp else None
+        lps = [torch.zeros(n, dtype=lp_dt, device="cuda") if lp_dt is not None else None for n in sizes]
         for t in (1, 2, 3):
-            scale = 10.0 ** rng.uniform(-5, -2)
+            scale = 10.0 ** rng.uniform(-5, -2) * (S if gdt != torch.float16 else min(S, 1024.0))
             grads = [(torch.empty(n, device="cuda").normal_(0, 1.0, generator=gen) * scale).to(gdt) for n in sizes]
             new_bits = [(int(rng.choice(widths)), int(rng.choice(widths))) if rng.rand() < 0.3 else b for b in bits]
             out = [s if nb == b else stq.alloc_state(n, block, nb[0], nb[1], "cuda", vl)
                    for s, nb, b, n, vl in zip(states, new_bits, bits, sizes, vlog)]
             want_stats = bool(rng.randint(0, 2))
-            rows = [stq.make_row(n, block, s, o, p, g, wd) for n, s, o, p, g, wd in zip(sizes, states, out, params, grads, wds)]
+            rows = [stq.make_row(n, block, s, o, p, g, wd, lp)
+                    for n, s, o, p, g, wd, lp in zip(sizes, states, out, params, grads, wds, lps)]
             h.step(stq.table(rows), lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, t=t, grad_dtype=stq.grad_dtype_of(grads[0]),
-                   decoupled_wd=decoupled, flags=stq.WITH_STATS if want_stats else 0)
+                   decoupled_wd=decoupled, flags=stq.WITH_STATS if want_stats else 0, inv_grad_scale=inv)
             got_stats = h.layer_stats(L) if want_stats else None
             h.device_status()
             states, bits = out, new_bits
@@ -588,13 +595,16 @@ def test_random_tables_against_the_oracle(H, O, seed):
                 ostates[i], st = oracle.step(theta[i], H.to_np(grads[i]), ostates[i], block, lr=1e-3, beta1=0.9, beta2=0.999,
                                              eps=1e-8, weight_decay=wds[i], t=t, bits_m_out=bits[i][0], bits_v_out=bits[i][1],
                                              decoupled_wd=decoupled, want_stats=want_stats, fp16_grad=(gdt == torch.float16),
-                                             v_mode=oracle.LOG_PL if vlog[i] else oracle.LOG)
+                                             v_mode=oracle.LOG_PL if vlog[i] else oracle.LOG,
+                                             inv_grad_scale=float(np.float32(1.0 / S)))
                 upd[i] = np.maximum(upd[i], np.maximum(np.abs(theta[i]), np.abs(theta[i] - before)))
                 tag = f"seed {seed} case {case} t={t} tensor {i} n={sizes[i]} B={block} bits {bits[i]} {gdt}"
                 H.assert_states_equal(states[i], ostates[i], tag)
                 H.assert_theta_close(params[i], theta[i], REL_1STEP * t * 2, tag, upd=upd[i])
                 if want_stats:
                     H.assert_stats_close(got_stats[i:i + 1], st[None, :], tag)
+                if lps[i] is not None:
+                    assert torch.equal(lps[i], params[i].to(lp_dt)), tag + " working copy"
                 if not decoupled:
                     # L2 mode feeds the parameters back into the moments (g + lambda * theta), and the parameters
                     # agree to rounding, not to the bit: each step is checked from identical inputs
