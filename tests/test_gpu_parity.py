@@ -664,3 +664,51 @@ def test_random_repacks_and_statistics_against_the_oracle(H, O, seed):
                 H.assert_states_equal(out[i], ostates[i], f"seed {seed} case {case} hop {hop} tensor {i} n={n} B={block} "
                                                           f"{bits[i]} -> {new_bits[i]} pl={vlog[i]}")
             states, bits = out, new_bits
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_random_medium_tables_many_bodies_in_one_launch(H, O, seed):
+    """Forty tensors of tens to hundreds of tiles with random widths, so that one launch runs many fused
+    bodies, the runtime-width body (a third of the tensors change width every step) and the generic
+    kernel side by side; five steps with statistics on every other one."""
+    import oracle
+    rng = np.random.RandomState(3000 + seed)
+    widths = [2, 3, 4, 8, 16]
+    L = 40
+    block = [128, 256, 128][seed]
+    gdt = [torch.bfloat16, torch.float32, torch.float16][seed]
+    sizes = [int(rng.randint(20000, 200000)) for _ in range(L)]
+    vlog = [int(rng.randint(0, 2)) for _ in range(L)]
+    bits = [(int(rng.choice(widths)), int(rng.choice(widths))) for _ in range(L)]
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    params = [torch.empty(n, device="cuda").normal_(0, 0.02, generator=gen) for n in sizes]
+    states = [stq.alloc_state(n, block, bm, bv, "cuda", vl) for n, (bm, bv), vl in zip(sizes, bits, vlog)]
+    h = stq.Handle()
+    h.init_state(stq.table([stq.make_row(n, block, None, s) for n, s in zip(sizes, states)]))
+    theta = [H.to_np(p) for p in params]
+    ostates = [oracle.new_state(n, block, bm, bv) for n, (bm, bv) in zip(sizes, bits)]
+    upd = [np.abs(t) for t in theta]
+    for t in range(1, 6):
+        grads = [(torch.empty(n, device="cuda").normal_(0, 1.0, generator=gen) * 10.0 ** rng.uniform(-4, -2)).to(gdt) for n in sizes]
+        new_bits = [(int(rng.choice(widths)), int(rng.choice(widths))) if rng.rand() < 0.33 else b for b in bits]
+        out = [s if nb == b else stq.alloc_state(n, block, nb[0], nb[1], "cuda", vl)
+               for s, nb, b, n, vl in zip(states, new_bits, bits, sizes, vlog)]
+        want_stats = t % 2 == 0
+        h.step(stq.table([stq.make_row(n, block, s, o, p, g, 0.01) for n, s, o, p, g in zip(sizes, states, out, params, grads)]),
+               lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, t=t, grad_dtype=stq.grad_dtype_of(grads[0]),
+               flags=stq.WITH_STATS if want_stats else 0)
+        got = h.layer_stats(L) if want_stats else None
+        h.device_status()
+        states, bits = out, new_bits
+        for i in range(L):
+            before = theta[i].copy()
+            ostates[i], st = oracle.step(theta[i], H.to_np(grads[i]), ostates[i], block, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8,
+                                         weight_decay=0.01, t=t, bits_m_out=bits[i][0], bits_v_out=bits[i][1],
+                                         want_stats=want_stats, fp16_grad=(gdt == torch.float16),
+                                         v_mode=oracle.LOG_PL if vlog[i] else oracle.LOG)
+            upd[i] = np.maximum(upd[i], np.maximum(np.abs(theta[i]), np.abs(theta[i] - before)))
+            tag = f"seed {seed} t={t} tensor {i} n={sizes[i]} bits {bits[i]} pl={vlog[i]}"
+            H.assert_states_equal(states[i], ostates[i], tag)
+            H.assert_theta_close(params[i], theta[i], REL_1STEP * t * 2, tag, upd=upd[i])
+            if want_stats:
+                H.assert_stats_close(got[i:i + 1], st[None, :], tag)
