@@ -154,7 +154,7 @@ def oracle_sample_run(w: W.Workload, bits_m, bits_v, budget_s: float, repeats: i
             t0 = time.perf_counter()
             list(ex.map(lambda tk: one(tk, 2 + r), tasks))
             times.append(time.perf_counter() - t0)
-    return {"params": taken, "seconds": times, "cores": min(cores, len(tasks)),
+    return {"params": taken, "seconds": times, "cores": min(cores, len(tasks)), "single_thread": rate1,
             "sample": f"{taken} params in {len(tasks)} block-aligned chunks of <= {chunk} drawn from the "
                       f"largest tensors of the workload at their widths, one oracle step each, "
                       f"{min(cores, len(tasks))} threads"}
@@ -396,7 +396,8 @@ def run_ours(args, w, bits_m, bits_v):
     if rank == 0 and not args.no_cpu_baseline and world == 1 and not amp:
         res = oracle_sample_run(w, bits_m, bits_v, budget_s=8.0, repeats=1)
         line["cpu_baseline"] = {"value": res["params"] / res["seconds"][0], "unit": UNIT, "cores": res["cores"],
-                                "kind": "oracle", "sample": res["sample"]}
+                                "kind": "oracle", "sample": res["sample"],
+                                "single_thread_value": res["single_thread"]}   # one 4/4-bit chunk of 2^18 elements
     if rank == 0:
         print(json.dumps(line), flush=True)
     if use_dist:
