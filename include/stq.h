@@ -116,7 +116,9 @@ typedef struct stq_hparams {
   const float* inv_grad_scale; /* every gradient is multiplied by *inv_grad_scale (1 / loss scale)   */
                                /* before anything else (statistics included)                         */
   const float* found_inf;      /* if *found_inf != 0 the step is skipped: no buffer is touched, and   */
-                               /* statistics requested with the step are not produced                */
+                               /* statistics requested with the step are not produced (the next      */
+                               /* stq_layer_stats returns STQ_E_STATE; the value is read when the     */
+                               /* step runs, so the caller may reuse the flag afterwards)            */
   /* Step count and learning rate kept on the DEVICE (both optional, NULL = use `step` and `lr` above):  */
   /* a step captured into a CUDA graph then advances with the caller's counter instead of repeating     */
   /* the captured t.  The bias corrections 1 - beta^t are formed on the device in double precision.     */
@@ -160,7 +162,12 @@ int stq_grad_stats(stq_handle* h, const stq_tensor* tensors, int L, int grad_dty
 
 /* Finishes the reduction started by the last stq_step(STQ_WITH_STATS) or stq_grad_stats on this
  * handle and copies it to HOST memory: out[l] = {sum g, sum |g|, sum g^2, numel} for l < L.
- * Synchronises `stream`.  The reduction order is fixed, so results are run-to-run identical. */
+ * Synchronises `stream`.  The reduction order is fixed, so results are run-to-run identical.
+ * Call order: the sums stay pending while the handle keeps seeing the table they were taken with
+ * (further steps over the byte-identical table are fine).  Any call with another table on the same
+ * handle (stq_repack, stq_init_state, a step with other pointers or widths) drops them, and so does a
+ * step that found_inf skipped: this call then returns STQ_E_STATE and writes nothing.  Fetch the sums
+ * before re-packing or changing widths. */
 int stq_layer_stats(stq_handle* h, double* out, int L, void* stream);
 
 /* The same sums as stq_grad_stats + stq_layer_stats for ONE gradient tensor, for callers that must

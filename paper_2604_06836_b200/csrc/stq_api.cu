@@ -36,8 +36,9 @@ struct stq_handle {
   uint32_t n_main = 0;                              // fast tiles of the fused bodies; [n_main, n_fast) change width
   int fast_grid = 0;
   bool any_lp = false;              // some tensor of the current table wants a low-precision copy
-  int* d_err = nullptr;
-  float* d_scalars = nullptr;   // {step_size, rsqrt_bc2, lr} when the step count lives on the device             // raised by a kernel whose bounded wait ran out
+  int* d_err = nullptr;         // [0] raised by a kernel whose bounded wait ran out; [1] non-zero if the last call
+                                // that carried statistics really produced them (a skipped step does not)
+  float* d_scalars = nullptr;   // {step_size, rsqrt_bc2, lr} when the step count lives on the device
   stq::FastSched* d_sched = nullptr;   // two work lists of the main step kernel (fused bodies, width changes)
 
   // pinned staging for uploads
@@ -239,6 +240,9 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   const bool same = h->cached_kind == kind && (int)h->cached.size() == L &&
                     std::memcmp(h->cached.data(), tensors, sizeof(stq_tensor) * (size_t)L) == 0;
   if (same) return STQ_OK;
+  // Pending statistics belong to the table they were taken with (its tile map and segment map finish the
+  // reduction): a call with another table drops them, and stq_layer_stats then reports STQ_E_STATE.
+  h->stats_L = 0;
   for (int l = 0; l < L; ++l) {
     int rc = validate_row(tensors[l], kind);
     if (rc != STQ_OK) return rc;
@@ -532,8 +536,8 @@ int stq_create(stq_handle** out, int device) {
   h->grid = h->sm_count * stq::step_ctas_per_sm();
   h->fast_grid = h->sm_count * stq::fast_ctas_per_sm();
   if (h->fast_grid > stq::kFastMaxGrid) h->fast_grid = stq::kFastMaxGrid;
-  if (cudaMalloc(reinterpret_cast<void**>(&h->d_err), sizeof(int)) != cudaSuccess ||
-      cudaMemset(h->d_err, 0, sizeof(int)) != cudaSuccess ||
+  if (cudaMalloc(reinterpret_cast<void**>(&h->d_err), 2 * sizeof(int)) != cudaSuccess ||
+      cudaMemset(h->d_err, 0, 2 * sizeof(int)) != cudaSuccess ||
       cudaMalloc(reinterpret_cast<void**>(&h->d_scalars), 4 * sizeof(float)) != cudaSuccess ||
       cudaMalloc(reinterpret_cast<void**>(&h->d_sched), 2 * sizeof(stq::FastSched)) != cudaSuccess) {
     cudaEventDestroy(h->stage_ev);
@@ -617,6 +621,10 @@ int stq_step(stq_handle* h, const stq_tensor* tensors, int L, const stq_hparams*
     h->launches++;
     sc.dev_scalars = h->d_scalars;
   }
+  if (stats) {   // a step skipped through found_inf writes no partial sums: record whether this one will
+    STQ_CUDA(h, stq::launch_stats_valid(hp->found_inf, h->d_err + 1, s));
+    h->launches++;
+  }
   rc = run(h, stq::kStep, hp->grad_dtype, stats, sc, s);
   if (rc == STQ_OK && stats) h->stats_L = L;
   return rc;
@@ -630,6 +638,8 @@ int stq_grad_stats(stq_handle* h, const stq_tensor* tensors, int L, int grad_dty
   if (rc != STQ_OK) return rc;
   stq::StepConsts sc;
   std::memset(&sc, 0, sizeof(sc));
+  STQ_CUDA(h, stq::launch_stats_valid(nullptr, h->d_err + 1, s));
+  h->launches++;
   rc = run(h, stq::kStatsOnly, grad_dtype, true, sc, s);
   if (rc == STQ_OK) h->stats_L = L;
   return rc;
@@ -646,7 +656,8 @@ int stq_layer_stats(stq_handle* h, double* out, int L, void* stream) {
     if (h->h_stats) cudaFreeHost(h->h_stats);
     h->h_stats = nullptr;
     h->h_stats_cap = 0;
-    cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&h->h_stats), sizeof(double) * 4 * (size_t)L);
+    // (one more slot: the "statistics were produced" word travels with the sums)
+    cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&h->h_stats), sizeof(double) * (4 * (size_t)L + 1));
     if (e != cudaSuccess) { h->cuda_err = cudaGetErrorString(e); return STQ_E_WORKSPACE; }
     h->h_stats_cap = (size_t)L * 4;
   }
@@ -656,7 +667,13 @@ int stq_layer_stats(stq_handle* h, double* out, int L, void* stream) {
                                        h->d_stats, s));
   h->launches += 2;
   STQ_CUDA(h, cudaMemcpyAsync(h->h_stats, h->d_stats, sizeof(double) * 4 * (size_t)L, cudaMemcpyDeviceToHost, s));
+  int* h_valid = reinterpret_cast<int*>(h->h_stats + 4 * (size_t)L);
+  STQ_CUDA(h, cudaMemcpyAsync(h_valid, h->d_err + 1, sizeof(int), cudaMemcpyDeviceToHost, s));
   STQ_CUDA(h, cudaStreamSynchronize(s));
+  if (*h_valid == 0) {        // the step that was to carry the sums was skipped (found_inf): nothing to report
+    h->stats_L = 0;
+    return STQ_E_STATE;
+  }
   std::memcpy(out, h->h_stats, sizeof(double) * 4 * (size_t)L);
   return STQ_OK;
 }
@@ -927,7 +944,7 @@ const char* stq_strerror(int code) {
     case STQ_E_CUDA: return "CUDA runtime error";
     case STQ_E_WORKSPACE: return "could not allocate library workspace";
     case STQ_E_ARG: return "invalid scalar argument";
-    case STQ_E_STATE: return "no statistics pending for this table";
+    case STQ_E_STATE: return "no statistics pending for this table (none requested, another table since, or the step was skipped)";
     case STQ_E_TIMEOUT: return "a bounded wait inside a kernel ran out (results of that launch are invalid)";
     case STQ_E_TOO_LARGE: return "tensor larger than the fixed capacity of this non-allocating entry point";
     default: return "unknown error";

@@ -11,9 +11,9 @@ constexpr int kRowsPerWarp = 4;  // a warp owns this many consecutive rows of a 
 constexpr int kTile = (kThreads / 32) * kRowsPerWarp * kRowElems;   // elements per tile; a tile lies inside one tensor
 constexpr int kMaxBlock = kRowsPerWarp * kRowElems;                 // a quantization block never leaves its warp
 constexpr int kFastCtasPerSm = 2;   // resident CTAs per SM of the main step kernel
-constexpr int kFastStages = 2;
+constexpr int kFastStages = 2;      // depth of its shared-memory ring
 constexpr int kFastRowsPerPass = 2; // rows a warp handles per pass over its kRowsPerWarp rows (see the kernel)
-constexpr int kFastMaxBlock = kFastRowsPerPass * kRowElems;   // larger blocks take the generic path      // depth of its shared-memory ring
+constexpr int kFastMaxBlock = kFastRowsPerPass * kRowElems;   // larger blocks take the generic path
 
 // Device-side row of the tensor table.
 struct TensorDesc {
@@ -59,6 +59,10 @@ struct StepConsts {
 // out = {lr / (1 - beta1^t), 1 / sqrt(1 - beta2^t), lr}, in double precision, one thread.
 cudaError_t launch_step_scalars(const long long* step_dev, const float* lr_dev, double lr_host, double beta1,
                                 double beta2, float* out, cudaStream_t stream);
+
+// Records whether a call that is to carry statistics will produce them: *valid = 1 unless *found_inf (device,
+// may be nullptr) is non-zero, in which case the step kernels return without writing a partial sum.
+cudaError_t launch_stats_valid(const float* found_inf, int* valid, cudaStream_t stream);
 
 enum Mode { kStep = 0, kRepack = 1, kInit = 2, kStatsOnly = 3 };
 

@@ -909,6 +909,15 @@ cudaError_t launch_step_scalars(const long long* step_dev, const float* lr_dev, 
   return cudaGetLastError();
 }
 
+__global__ void stq_stats_valid_kernel(const float* __restrict__ found_inf, int* __restrict__ valid) {
+  *valid = (found_inf == nullptr || *found_inf == 0.0f) ? 1 : 0;
+}
+
+cudaError_t launch_stats_valid(const float* found_inf, int* valid, cudaStream_t stream) {
+  stq_stats_valid_kernel<<<1, 1, 0, stream>>>(found_inf, valid);
+  return cudaGetLastError();
+}
+
 int step_ctas_per_sm() {
   int n = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, stq_tile_kernel<kStep, 1, false, false>, kThreads, 0) !=

@@ -90,7 +90,10 @@ stq_static_stats_kernel(const void* __restrict__ grad, unsigned long long numel,
   if (tid < 3) part[(size_t)blockIdx.x * 3 + tid] = sh[0][tid];
   __threadfence();
   __syncthreads();
-  if (tid == 0) is_last = (atomicAdd(counter, 1u) == gridDim.x - 1);
+  if (tid == 0) {
+    __threadfence();   // the publishing thread itself orders the three stores (seen through the barrier) before its ticket
+    is_last = (atomicAdd(counter, 1u) == gridDim.x - 1);
+  }
   __syncthreads();
   if (!is_last) return;
   __threadfence();

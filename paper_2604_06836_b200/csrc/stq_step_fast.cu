@@ -947,11 +947,6 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
     if constexpr (SPLIT) {
       tile_body_split<GDT, AMP>(stage, ti, sc, lut8, lane, warp, ebar, part, grad_mul);
     } else {
-#define STQ_CASE(IM, IV, BM, BV, VPL) \
-  case IM * 7 + IV: tile_body<BM, BV, VPL, GDT, AMP>(stage, ti, sc, lut8, lane, warp, ebar, part, grad_mul); break;
-#define STQ_CASES_M(IM, BM)                                                                                   \
-  STQ_CASE(IM, 0, BM, 2, false) STQ_CASE(IM, 1, BM, 3, false) STQ_CASE(IM, 2, BM, 4, false) STQ_CASE(IM, 3, BM, 8, false) \
-  STQ_CASE(IM, 4, BM, 16, false) STQ_CASE(IM, 5, BM, 8, true) STQ_CASE(IM, 6, BM, 16, true)
       switch ((ti.packed & 0xFFu) * 7 + ((ti.packed >> 8) & 0xFFu)) {
         STQ_CASES_M(0, 2)
         STQ_CASES_M(1, 3)

@@ -37,6 +37,9 @@ class STQAdamW(torch.optim.Optimizer):
     gradients that are one step old, except at t = 1).
     v_log: "poly" or "pl", the variant of the second-moment code at 8 and 16 bits.
     grad_scaler_inv / found_inf: optional one-element float32 CUDA tensors for loss-scaled training.
+    With ``found_inf`` set, ``step()`` reads it on the host first (one small synchronising copy): a step
+    with a non-finite gradient is left out entirely, so the step count t, the bias corrections and the
+    decision schedule follow the steps actually taken and no statistics of a skipped step reach the policy.
     """
 
     def __init__(self, params: Iterable, lr: float = 1e-3, betas=(0.9, 0.999), eps: float = 1e-8,
@@ -48,7 +51,7 @@ class STQAdamW(torch.optim.Optimizer):
         if order not in ("paper", "fused"):
             raise ValueError("order is 'paper' or 'fused'")
         self.order = order
-        self._pending_stats = False       # the last step carried statistics that have not been fetched
+        self._carried_stats = None        # sums that rode on the last step (fused order), fetched right after it
         if block not in (128, 256, 512):
             raise ValueError("block is 128, 256 or 512")
         defaults = dict(lr=lr, weight_decay=weight_decay)
@@ -72,6 +75,7 @@ class STQAdamW(torch.optim.Optimizer):
         self.bits_v = np.full(len(self._params), bv, dtype=np.uint8)
         self.states = [stq.alloc_state(p.numel(), block, int(bm), int(bv), dev, self.v_log) for p in self._params]
         self.t = 0
+        self.skipped_steps = 0
         self.last_scores = None
         self.grad_scaler_inv = None      # torch tensor [1] float32 on the device, or None
         self.found_inf = None
@@ -122,6 +126,9 @@ class STQAdamW(torch.optim.Optimizer):
         if closure is not None:
             with torch.enable_grad():
                 loss = closure()
+        if self.found_inf is not None and float(self.found_inf.item()) != 0.0:
+            self.skipped_steps += 1       # nothing is launched, t does not advance, carried statistics are kept
+            return loss
         self.t += 1
         t = self.t
         hp = dict(lr=self.param_groups[0]["lr"], beta1=self.betas[0], beta2=self.betas[1], eps=self.eps, t=t,
@@ -129,9 +136,8 @@ class STQAdamW(torch.optim.Optimizer):
                   inv_grad_scale=self.grad_scaler_inv, found_inf=self.found_inf)
         new_m = new_v = None
         if self.policy_kind == "paper" and self.policy.is_decision_step(t):
-            if self._pending_stats:                    # fused order: the sums rode on the previous step
-                stats = self.handle.layer_stats(len(self._params))
-            else:
+            stats, self._carried_stats = self._carried_stats, None    # fused order: they rode on the previous step
+            if stats is None:
                 tbl = self._table()
                 self.handle.grad_stats(tbl, hp["grad_dtype"])
                 stats = self.handle.layer_stats(len(self._params))
@@ -144,9 +150,9 @@ class STQAdamW(torch.optim.Optimizer):
         # fused order: if the next step decides, this one carries the statistics
         flags = stq.WITH_STATS if (self.order == "fused" and self.policy_kind == "paper" and
                                    self.policy.is_decision_step(t + 1)) else 0
-        self._pending_stats = bool(flags)
         if new_m is None or ((new_m == self.bits_m).all() and (new_v == self.bits_v).all()):
             self.handle.step(self._table(), flags=flags, **hp)
+            self._fetch_carried(flags)
             return loss
         out = []
         for k, p in enumerate(self._params):
@@ -162,11 +168,18 @@ class STQAdamW(torch.optim.Optimizer):
                 stq.alloc_codes(n, bv, self.device), stq.alloc_scales(n, bv, self.block, self.device))
             out.append(stq.QState(mc, ms, bm, vc, vs, bv, self.v_log))
         self.handle.step(stq.table(self._rows(out)), flags=flags, **hp)
+        self._fetch_carried(flags)
         torch.cuda.current_stream(self.device).synchronize()     # the old buffers are released below
         self.states = out
         self.bits_m, self.bits_v = np.array(new_m, np.uint8), np.array(new_v, np.uint8)
         self._tbl = None
         return loss
+
+    def _fetch_carried(self, flags: int):
+        # The sums are finished with the table they were taken with, and the next step's table may differ
+        # (fresh gradient buffers), so they are brought to the host right away.
+        if flags:
+            self._carried_stats = self.handle.layer_stats(len(self._params))
 
     # ---- bookkeeping --------------------------------------------------------------------------------
     def state_bytes(self) -> int:
@@ -181,6 +194,7 @@ class STQAdamW(torch.optim.Optimizer):
         d = super().state_dict()
         d["stq"] = dict(t=self.t, bits_m=self.bits_m.copy(), bits_v=self.bits_v.copy(), v_log=self.v_log,
                         block=self.block, policy=self.policy.state.copy(),
+                        carried_stats=None if self._carried_stats is None else self._carried_stats.copy(),
                         states=[dict(m_codes=s.m_codes.clone(), m_scales=s.m_scales.clone(),
                                      v_codes=s.v_codes.clone(), v_scales=s.v_scales.clone()) for s in self.states])
         return d
@@ -194,6 +208,8 @@ class STQAdamW(torch.optim.Optimizer):
         self.t = int(q["t"])
         self.bits_m, self.bits_v = np.array(q["bits_m"], np.uint8), np.array(q["bits_v"], np.uint8)
         self.policy.state = q["policy"]
+        carried = q.get("carried_stats")
+        self._carried_stats = None if carried is None else np.array(carried, dtype=np.float64)
         self.states = [stq.QState(s["m_codes"].to(self.device).clone(), s["m_scales"].to(self.device).clone(), int(bm),
                                   s["v_codes"].to(self.device).clone(), s["v_scales"].to(self.device).clone(), int(bv),
                                   self.v_log)

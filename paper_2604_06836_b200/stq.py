@@ -22,6 +22,7 @@ LP_NONE, LP_BF16, LP_F16 = 0, 1, 2
 WITH_STATS = 1
 VLOG_POLY, VLOG_PL = 0, 1
 WIDTHS = (2, 3, 4, 8, 16, 32)
+E_STATE, E_TIMEOUT, E_TOO_LARGE = -10, -11, -12     # the STQ_E_* codes callers test for
 
 
 class StqError(RuntimeError):
@@ -199,6 +200,20 @@ def _stream_ptr(stream) -> int | None:
 STATIC_STATS_MAX_NUMEL = 64 * 1024 * 1024
 
 
+def check_static_stats_args(grad: torch.Tensor, out: torch.Tensor) -> None:
+    """The C entry point sees only pointers and a count: what it cannot check is checked here, before
+    anything is launched.  A gradient of another type would be read as numel fp32 values (twice the
+    length of an fp16 buffer), a strided one as if it were dense."""
+    if grad.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError(f"grad_stats_static takes float32 or bfloat16 gradients, not {grad.dtype}")
+    if not grad.is_contiguous():
+        raise ValueError("grad_stats_static needs a contiguous gradient")
+    if out.dtype != torch.float64 or out.numel() < 4 or not out.is_contiguous():
+        raise ValueError("out is a contiguous float64 tensor of at least 4 elements")
+    if grad.device.type != "cuda" or out.device != grad.device:
+        raise ValueError("grad and out live on the same CUDA device")
+
+
 def grad_stats_static(grad: torch.Tensor, out: torch.Tensor, stream=None) -> int:
     """Gradient sums of one tensor through the entry point that allocates nothing.
 
@@ -207,9 +222,10 @@ def grad_stats_static(grad: torch.Tensor, out: torch.Tensor, stream=None) -> int
     static array inside libstq.  ``out`` is a caller-owned float64[4] tensor on the same device; the
     call is asynchronous on the stream.  Returns the C status code (0 = ok) instead of raising, so
     that callers can test for STQ_E_TOO_LARGE (-12) and fall back to splitting the tensor."""
-    assert out.dtype == torch.float64 and out.numel() >= 4 and out.is_cuda and grad.is_cuda
+    check_static_stats_args(grad, out)
     dt = GRAD_BF16 if grad.dtype == torch.bfloat16 else GRAD_F32
-    return int(lib().stq_grad_stats_static(grad.device.index or 0, grad.data_ptr(), grad.numel(), dt,
+    return int(lib().stq_grad_stats_static(grad.device.index if grad.device.index is not None else
+                                           torch.cuda.current_device(), grad.data_ptr(), grad.numel(), dt,
                                            out.data_ptr(), _stream_ptr(stream)))
 
 

@@ -95,3 +95,23 @@ def test_policy_schedule_and_anchor(stq_lib):
     row = [0.0, 0.8e-3 * N, 1e-6 * N, N]
     bits, score = p.decide(np.array([row] * 5), 10 ** 6)
     assert np.allclose(score, 7.2, atol=1e-9) and (bits == 8).all()   # an average layer lands on 8 bits
+
+
+def test_static_stats_binding_rejects_what_the_c_call_cannot_see():
+    """The C entry point gets a pointer and a count; a gradient of another type or layout would be read as
+    dense fp32 (twice the length of an fp16 buffer).  The binding refuses those before any launch."""
+    import torch
+    from paper_2604_06836_b200 import stq
+    out = torch.zeros(4, dtype=torch.float64)
+    for bad in (torch.zeros(64, dtype=torch.float16), torch.zeros(64, dtype=torch.float64),
+                torch.zeros(64, dtype=torch.int32)):
+        with pytest.raises(ValueError, match="float32 or bfloat16"):
+            stq.grad_stats_static(bad, out)
+    with pytest.raises(ValueError, match="contiguous"):
+        stq.grad_stats_static(torch.zeros(8, 8)[:, ::2], out)
+    with pytest.raises(ValueError, match="float64"):
+        stq.grad_stats_static(torch.zeros(64), torch.zeros(4))
+    with pytest.raises(ValueError, match="float64"):
+        stq.grad_stats_static(torch.zeros(64), torch.zeros(3, dtype=torch.float64))
+    with pytest.raises(ValueError, match="same CUDA device"):
+        stq.grad_stats_static(torch.zeros(64), out)          # host tensors never reach the library

@@ -146,3 +146,39 @@ def test_fused_order_decides_on_the_previous_steps_gradients():
             H.assert_states_equal(opt.states[i], states[i], f"fused t={t} tensor {i}")
             H.assert_theta_close(params[i].data, theta[i], 1e-6 * t, f"fused t={t} tensor {i}", upd=upd[i])
         prev = grads
+
+
+@pytest.mark.parametrize("order", ["paper", "fused"])
+def test_a_skipped_step_leaves_no_trace(order):
+    """Loss-scaled training: a step whose gradients overflowed is left out.  The step count, the bias
+    corrections, the decision schedule and the running averages of the policy then follow the steps actually
+    taken, so a run with overflow steps sprinkled in ends exactly where the run without them ends."""
+    def run(skip_at):
+        model = _mlp(5)
+        opt = STQAdamW(model.parameters(), lr=2e-3, weight_decay=0.01, policy="paper", interval=4, tau=20.0,
+                       order=order)
+        opt.found_inf = torch.zeros(1, dtype=torch.float32, device="cuda")
+        real = 0
+        for it in range(14 + len(skip_at)):
+            x, y = _batch(real)
+            opt.zero_grad()
+            torch.nn.functional.mse_loss(model(x), y).backward()
+            if it in skip_at:
+                for p in model.parameters():          # what an overflow leaves behind
+                    p.grad.fill_(float("inf"))
+                opt.found_inf.fill_(1.0)
+            else:
+                opt.found_inf.fill_(0.0)
+                real += 1
+            opt.step()
+        return model, opt
+
+    (ma, oa), (mb, ob) = run(()), run((2, 3, 7, 11))      # 3 and 7 sit right before decision steps (t = 4, 8)
+    assert oa.t == ob.t == 14 and ob.skipped_steps == 4 and oa.skipped_steps == 0
+    assert (oa.bits_m == ob.bits_m).all() and np.array_equal(oa.policy.state, ob.policy.state)
+    assert np.isfinite(ob.policy.state).all()
+    for pa, pb in zip(ma.parameters(), mb.parameters()):
+        assert torch.equal(pa, pb)
+    for sa, sb in zip(oa.states, ob.states):
+        assert torch.equal(sa.m_codes, sb.m_codes) and torch.equal(sa.v_codes, sb.v_codes)
+        assert torch.equal(sa.m_scales, sb.m_scales) and torch.equal(sa.v_scales, sb.v_scales)

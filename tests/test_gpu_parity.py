@@ -262,6 +262,11 @@ def test_loss_scaled_gradients_skip_flag_and_low_precision_copy(H, O, gdt):
         if skip:
             assert all(torch.equal(a, b) for a, b in zip(before, job.params))
             assert all(torch.equal(a, s.m_codes) for a, s in zip(codes_before, job.states))
+            # the skipped step produced no sums: asking for them is a call-order error, not stale numbers
+            flag.fill_(0.0)                        # (the flag was read when the step ran; reusing it changes nothing)
+            with pytest.raises(stq.StqError) as err:
+                job.handle.layer_stats(job.L)
+            assert err.value.code == stq.E_STATE
         else:
             H.assert_stats_close(job.handle.layer_stats(job.L), st_o, f"{gdt} t={t}")
             for i in range(job.L):
@@ -712,3 +717,26 @@ def test_random_medium_tables_many_bodies_in_one_launch(H, O, seed):
             H.assert_theta_close(params[i], theta[i], REL_1STEP * t * 2, tag, upd=upd[i])
             if want_stats:
                 H.assert_stats_close(got[i:i + 1], st[None, :], tag)
+
+
+def test_pending_statistics_are_dropped_when_the_table_changes(H, O):
+    """Sums taken with one table cannot be finished with another table's tile and segment maps: a call with
+    a different table in between makes stq_layer_stats report the call order instead of wrong sums."""
+    shapes = [("a", (4096 * 3 + 5,)), ("b", (4096,)), ("c", (900,))]
+    w = W.Workload("order", tuple(shapes), 128, "fp32", "normal", scale_log10=(-3.0, -3.0), seed=5)
+    job = Job(w, [4, 8, 4], [4, 4, 8])
+    oj = H.OracleJob(job)
+    job.draw_grads(1)
+    st_o = oj.step([H.to_np(g) for g in job.grads], 1, want_stats=True)
+    job.step(1, stats=True)
+    job.step(2)                                   # the same table again: the sums of step 1 stay pending
+    H.assert_stats_close(job.layer_stats(), st_o, "still pending after a plain step")
+    job.step(3, stats=True)
+    job.repack(([8, 8, 4], [4, 4, 8]))            # another table through the same handle
+    with pytest.raises(stq.StqError) as err:
+        job.layer_stats()
+    assert err.value.code == stq.E_STATE
+    job.draw_grads(4)
+    job.step(4, stats=True)                       # and the next request works as usual
+    want = np.stack([O.grad_stats(H.to_np(g)) for g in job.grads])
+    H.assert_stats_close(job.layer_stats(), want, "after the drop")

@@ -47,6 +47,28 @@ def test_two_calls_in_a_row_match_the_regular_path(dtype):
         _close(out.cpu().numpy(), _reference(g)[0])
 
 
+def test_calls_leave_device_memory_as_it_was():
+    """The point of the entry point: no call allocates.  After a warm-up call (which loads the kernel and
+    looks the scratch address up) the free device memory reported by the driver does not move over a
+    series of calls of different sizes, and the torch allocator is not involved either."""
+    from paper_2604_06836_b200 import stq
+    out = torch.zeros(4, dtype=torch.float64, device="cuda")
+    grads = [torch.randn(n, device="cuda") for n in (1_000_003, 4096, 9_999_999)]
+    grads.append(grads[0].to(torch.bfloat16))
+    for g in grads:                                # warm-up: both kernel variants, every size
+        assert stq.grad_stats_static(g, out) == 0
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    reserved0, alloc0 = torch.cuda.memory_reserved(), torch.cuda.memory_allocated()
+    for _ in range(5):
+        for g in grads:
+            assert stq.grad_stats_static(g, out) == 0
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert torch.cuda.memory_reserved() == reserved0 and torch.cuda.memory_allocated() == alloc0
+
+
 def test_tiny_and_ragged_sizes():
     from paper_2604_06836_b200 import stq
     out = torch.zeros(4, dtype=torch.float64, device="cuda")
