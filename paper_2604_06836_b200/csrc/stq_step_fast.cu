@@ -377,6 +377,78 @@ __device__ __forceinline__ void encode_pl_row(uint8_t* row_ptr, int lane, const 
   else store_fields<16>(row_ptr, lane, ~(j[0] | (j[1] << 16)), ~(j[2] | (j[3] << 16)));
 }
 
+__device__ __forceinline__ float ex2_fast(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---- the update's share of the fused bodies ----------------------------------------------------------
+// The parameter update is held to 1e-6, not to the bit, so the fused bodies do not decode the new codes
+// again: they take what the update needs straight from the encode.
+//
+// First moment: q = code - 2^(B-1) as a float (the caller multiplies by scale * lr/(1-beta1^t) / qmax).
+template <int B>
+__device__ __forceinline__ void encode_lin_row_q(uint8_t* row_ptr, int lane, const float (&m)[4], float inv,
+                                                 float (&q)[4]) {
+  constexpr float mg = kMagic + (float)Wd<B>::half;
+  uint32_t x[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const float t = __fmaf_rn(m[k], inv, mg);
+    x[k] = __float_as_uint(t);
+    q[k] = __fadd_rn(t, -mg);
+  }
+  pack_store_row<B>(row_ptr, lane, x, kMagicBits);
+}
+
+// Octave code (B <= 4) of one row of new second moments.  A block has only 2^B levels, so the factor
+// every level contributes to the update is worked out once per row by 2^B lanes (tile_body) and fetched
+// with a shuffle.  The shuffle takes its source lane from the low five bits of its operand, so the
+// products are scaled by a power of two chosen per row (c_up = sqrt2/s * 2^u, ymin_up = 2^(u-K)) such
+// that the exponent field of y itself ends in (row's first lane + code): e[k] is that operand.  u is a
+// multiple of 2^B, so the code (the low B bits of the exponent) is what it was; scaling up cannot
+// overflow (c <= sqrt2 * 2^100, u <= 16) and is exact, and whatever underflows is below the floor
+// level in either scaling.
+template <int B>
+struct Oct {
+  static constexpr int NL = 1 << B;
+  static constexpr int up0 = (64 - (int)(Wd<B>::emin & 31u)) & 31;        // first row of the pass: lanes 0 .. NL-1
+  static constexpr int up1 = (NL + 64 - (int)(Wd<B>::emin & 31u)) & 31;   // second row: lanes NL .. 2 NL-1
+};
+template <int B>
+__device__ __forceinline__ void encode_oct_row(uint8_t* row_ptr, int lane, const float (&v)[4], float c_up,
+                                               float ymin_up, uint32_t (&e)[4]) {
+  uint32_t f = 0u;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t yb = __float_as_uint(fmaxf(__fmul_rn(v[k], c_up), ymin_up));
+    f |= (yb >> (23 - B * k)) & (Wd<B>::mask << (B * k));
+    e[k] = yb >> 23;
+  }
+  store_fields<B>(row_ptr, lane, f, 0u);
+}
+
+// Polynomial log code (B = 8, 16): r = code - K as a float (the update forms 2^(r * R/K / 2) itself).
+template <int B>
+__device__ __forceinline__ void encode_log_row_r(uint8_t* row_ptr, int lane, const float (&v)[4], float lgc,
+                                                 uint32_t ebase, float (&r)[4]) {
+  constexpr float a = (float)Wd<B>::K / (float)Wd<B>::Roct;
+  constexpr float negR = -(float)Wd<B>::Roct;
+  uint32_t x[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t xb = __float_as_uint(v[k]);
+    const float de = __fadd_rn(__uint_as_float(ebase + (xb >> 23)), -kMagic);
+    const float dp = __fadd_rn(lg_poly(xb), -lgc);
+    const float d = fmaxf(__fadd_rn(de, dp), negR);
+    const float t = __fmaf_rn(d, a, kMagic);
+    x[k] = __float_as_uint(t);
+    r[k] = __fadd_rn(t, -kMagic);
+  }
+  pack_store_row<B>(row_ptr, lane, x, kMagicBits - (uint32_t)Wd<B>::K);
+}
+
 template <int GDT>
 __device__ __forceinline__ void lds_grad(const uint8_t* stage, int elem, float (&g)[4]) {
   if constexpr (GDT == 0) {
@@ -426,6 +498,8 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
   [[maybe_unused]] const uint32_t lp_dtype = ti.packed >> 24;
   const float lrwd = sc.l2_mode ? 0.0f : ti.wdx;
   float a0 = 0.f, a1 = 0.f, a2 = 0.f;      // statistics over the raw gradient (decision steps)
+  // octave v codes: 2^(level - K) of the level this lane tabulates for the update (see below)
+  [[maybe_unused]] const float lvl = __uint_as_float((((uint32_t)lane & Wd<BV <= 4 ? BV : 2>::mask) + Wd<BV <= 4 ? BV : 2>::emin) << 23);
 
 #pragma unroll 1
   for (int pass = 0; pass < R / RP; ++pass) {
@@ -511,7 +585,8 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
     }
 
     // ---- per-block constants: one lane per (row, state) works them out, then they are broadcast --------
-    // lanes 0..RP-1: inv = fl(qmax * fl(1/s_m));  lanes RP..2RP-1 (octave widths): c = fl(sqrt2 * fl(1/s_v))
+    // lanes 0..RP-1: inv = fl(qmax * fl(1/s_m));  lanes RP..2RP-1 (octave widths): c = fl(sqrt2 * fl(1/s_v)),
+    // times the power of two that steers the level shuffle of its row (encode_oct_row)
     float inv_m[RP], lgc[RP];
     {
       uint32_t mine = mxm[0];
@@ -525,7 +600,13 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
       }
       const float x = __uint_as_float(mine);
       const bool zero = x < kTiny;
-      const float mul = (BV <= 4 && (lane & RP)) ? kSqrt2 : (float)Wd<BM>::qmax;
+      float mul = (float)Wd<BM>::qmax;
+      if constexpr (BV <= 4) {
+        static_assert(BV > 4 || RP == 2, "the level shuffle is laid out for two rows per pass");
+        constexpr float up0 = kSqrt2 * (float)(1 << Oct<BV <= 4 ? BV : 2>::up0);
+        constexpr float up1 = kSqrt2 * (float)(1 << Oct<BV <= 4 ? BV : 2>::up1);
+        if (lane & RP) mul = (lane & 1) ? up1 : up0;
+      }
       const float val = zero ? 0.f : __fmul_rn(mul, __frcp_rn(x));
       // the same lanes store the new scales (a zero block stores 0), for the rows that open a block
       const int e_mine = (row0 + (lane & (RP - 1))) * kRowElems;
@@ -556,30 +637,69 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
       }
     }
 
-    // ---- quantize, pack, store; decode the new codes; update the parameters --------------------------
+    // ---- octave v codes: what each level of each row contributes to the update, one level per lane -----
+    // lane l: level (l mod 2^BV) of row (l div 2^BV) of the pass; value lr/(1-beta1^t) * s_m/qmax /
+    // (sqrt(s_v * 2^(level-K) / (1-beta2^t)) + eps), so that the update of an element is q_m times the
+    // entry of its level.  (An all-zero block of v has s_v = 0: every level gives 1/eps, as its decode would.)
+    [[maybe_unused]] float lut_upd = 0.f;
+    if constexpr (BV <= 4) {
+      constexpr float invq = 1.0f / (float)Wd<BM>::qmax;
+      const bool second = (lane >> (BV <= 4 ? BV : 0)) & 1;
+      const float svr = __uint_as_float(second ? mxv[1] : mxv[0]);
+      const float smr = __uint_as_float(second ? mxm[1] : mxm[0]);
+      const float vl = __fmul_rn(svr < kTiny ? 0.f : svr, lvl);
+      const float den = __fmaf_rn(sqrt_fast(vl), sc.rsqrt_bc2, sc.eps);
+      lut_upd = __fmul_rn(__fmul_rn(__fmul_rn(smr, sc.step_size), invq), rcp_fast(den));
+    }
+
+    // ---- quantize, pack, store; update the parameters ---------------------------------------------------
     float* param = ti.param + row0 * kRowElems + 4 * lane;
 #pragma unroll
     for (int r = 0; r < RP; ++r) {
-      // A zero block of m needs no special case here: its inv is 0, so every q is 0 and so is mq.
+      // A zero block of m needs no special case here: its inv is 0, so every q is 0 and so is the update.
       const float sm_raw = __uint_as_float(mxm[r]);
       const float sv_raw = __uint_as_float(mxv[r]);
       const bool vzero = sv_raw < kTiny;
-      const float s_v = vzero ? 0.f : sv_raw;
-      const uint32_t ebase = kMagicBits - (vzero ? (uint32_t)kZeroBlockExp : (mxv[r] >> 23));
-      float mq[4], vq[4];
-      // mq comes out multiplied by lr/(1-beta1^t): the decode scale carries the factor
-      encode_lin_row<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], __fmul_rn(sm_raw, sc.step_size), inv_m[r], mq);
-      if constexpr (VPL)
+      float out[4];
+      if constexpr (BV <= 4) {
+        float q[4];
+        uint32_t e[4];
+        encode_lin_row_q<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], inv_m[r], q);
+        const float ymin_up = __uint_as_float((Wd<BV>::emin + (uint32_t)(r == 0 ? Oct<BV>::up0 : Oct<BV>::up1)) << 23);
+        encode_oct_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], lgc[r], ymin_up, e);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float base = __fmaf_rn(th[r][k], -lrwd, th[r][k]);
+          out[k] = __fmaf_rn(-q[k], __shfl_sync(kFull, lut_upd, e[k]), base);
+        }
+      } else if constexpr (!VPL) {
+        // 2^((code-K) * R/K / 2) by the special-function unit: sqrt of the decoded level, to 2^-22
+        constexpr float half_cb = 0.5f * ((float)Wd<BV>::Roct / (float)Wd<BV>::K);
+        constexpr float invq = 1.0f / (float)Wd<BM>::qmax;
+        const uint32_t ebase = kMagicBits - (vzero ? (uint32_t)kZeroBlockExp : (mxv[r] >> 23));
+        const float unit = __fmul_rn(__fmul_rn(sm_raw, sc.step_size), invq);
+        const float srt = __fmul_rn(sqrt_fast(vzero ? 0.f : sv_raw), sc.rsqrt_bc2);
+        float q[4], rr[4];
+        encode_lin_row_q<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], inv_m[r], q);
+        encode_log_row_r<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], lgc[r], ebase, rr);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float den = __fmaf_rn(ex2_fast(__fmul_rn(rr[k], half_cb)), srt, sc.eps);
+          const float base = __fmaf_rn(th[r][k], -lrwd, th[r][k]);
+          out[k] = __fmaf_rn(-__fmul_rn(q[k], unit), rcp_fast(den), base);
+        }
+      } else {
+        float mq[4], vq[4];
+        // mq comes out multiplied by lr/(1-beta1^t): the decode scale carries the factor
+        encode_lin_row<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], __fmul_rn(sm_raw, sc.step_size), inv_m[r], mq);
         encode_pl_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], vzero ? 0x7F800000u : mxv[r],
                           vzero ? 0u : mxv[r], lutn, vq);
-      else
-        encode_log_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], s_v, lgc[r], ebase, lut8, vq);
-      float out[4];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const float den = __fmaf_rn(sqrt_fast(vq[k]), sc.rsqrt_bc2, sc.eps);
-        const float upd = __fmul_rn(mq[k], rcp_fast(den));
-        out[k] = __fadd_rn(th[r][k], -__fmaf_rn(th[r][k], lrwd, upd));
+        for (int k = 0; k < 4; ++k) {
+          const float den = __fmaf_rn(sqrt_fast(vq[k]), sc.rsqrt_bc2, sc.eps);
+          const float base = __fmaf_rn(th[r][k], -lrwd, th[r][k]);
+          out[k] = __fmaf_rn(-mq[k], rcp_fast(den), base);
+        }
       }
       *reinterpret_cast<float4*>(param + r * kRowElems) = make_float4(out[0], out[1], out[2], out[3]);
       if constexpr (AMP) {
