@@ -505,6 +505,7 @@ stq::StepConsts make_consts(const stq_hparams* hp) {
   sc.step_size = (float)(hp->lr / bc1);
   sc.rsqrt_bc2 = (float)(1.0 / std::sqrt(bc2));
   sc.eps = (float)hp->eps;
+  sc.one = 1.0f;
   sc.l2_mode = hp->decoupled_wd ? 0 : 1;
   sc.lr = hp->lr;
   sc.inv_scale = hp->inv_grad_scale;

@@ -47,6 +47,7 @@ struct StepConsts {
   float step_size;          // lr / (1 - beta1^t)
   float rsqrt_bc2;          // 1 / sqrt(1 - beta2^t)
   float eps;
+  float one;                // 1.0f as a run-time value (see the packed arithmetic of the main step kernel)
   int l2_mode;              // 1: g += wd*theta before the moments, no decoupled decay
   double lr;                // decoupled decay factor is fp32(1 - lr*wd), formed per tile
   const float* inv_scale;   // device: gradients are multiplied by *inv_scale first (nullptr: no)

@@ -483,6 +483,142 @@ __device__ __forceinline__ uint2 pack_lp(const float (&x)[4], uint32_t lp_dtype)
   return r;
 }
 
+// ---- two elements per instruction ----------------------------------------------------------------------
+// sm_100 executes fp32 add, multiply and fused multiply-add on register pairs (two independent IEEE
+// operations per instruction, each rounded exactly as the scalar one).  The step is bound by instruction
+// issue as much as by memory, and a third of its instructions are fp32 arithmetic on a lane's four
+// elements, so the fused bodies keep those as two pairs and do the per-element arithmetic pairwise
+// (PTX add / mul / fma .rn.f32x2 through the toolkit's intrinsics).
+// One trap: the assembler contracts a packed multiply whose only use is a packed add into one packed fused
+// multiply-add, explicit rounding modifiers and -fmad=false notwithstanding (measured: 0.35 % of random
+// operands change).  The quantizers are defined with separate roundings, so wherever a packed product
+// meets a sum the sum is written as fma(x, one, y) with `one` = 1.0f that the assembler cannot know (a
+// launch parameter): the same value as x + y, and nothing to contract.
+using f2 = float2;
+__device__ __forceinline__ f2 splat(float x) { return make_float2(x, x); }
+__device__ __forceinline__ f2 add2(f2 a, f2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ f2 mul2(f2 a, f2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ f2 bits2(uint32_t a, uint32_t b) { return make_float2(__uint_as_float(a), __uint_as_float(b)); }
+
+template <int B>
+__device__ __forceinline__ f2 code_pair(const uint32_t (&w)[2], int h) {
+  return make_float2(code_as_float<B>(w, 2 * h), code_as_float<B>(w, 2 * h + 1));
+}
+
+template <int B>
+__device__ __forceinline__ void decode_lin_pairs(const uint32_t (&w)[2], float s, f2 (&out)[2]) {
+  constexpr float invq = 1.0f / (float)Wd<B>::qmax;
+  constexpr float off = kTwo23 + (float)Wd<B>::half;
+  const f2 s2 = splat(s);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) out[h] = mul2(s2, mul2(add2(code_pair<B>(w, h), splat(-off)), splat(invq)));
+}
+
+// 2^e (e <= 0) of a pair, the same operations as ex2_poly (e is a product: its sum goes through `one`)
+__device__ __forceinline__ f2 ex2_poly_pair(f2 e, f2 one) {
+  const f2 ti = fma2(e, one, splat(kMagic));
+  const f2 fi = add2(ti, splat(-kMagic));
+  const f2 f = fma2(fi, splat(-1.0f), e);          // e - fi, exact
+  f2 a = splat(kE4);
+  a = fma2(a, f, splat(kE3));
+  a = fma2(a, f, splat(kE2));
+  a = fma2(a, f, splat(kE1));
+  a = fma2(a, f, splat(kE0));
+  const f2 p = fma2(a, f, splat(1.0f));
+  return bits2(__float_as_uint(p.x) + (__float_as_uint(ti.x) << 23), __float_as_uint(p.y) + (__float_as_uint(ti.y) << 23));
+}
+// P(mantissa) of a pair of bit patterns, the same operations as lg_poly
+__device__ __forceinline__ f2 lg_poly_pair(uint32_t b0, uint32_t b1) {
+  const f2 mant = bits2((b0 & 0x007FFFFFu) | 0x3F800000u, (b1 & 0x007FFFFFu) | 0x3F800000u);
+  const f2 t = add2(mant, splat(-1.0f));
+  f2 a = splat(kP6);
+  a = fma2(a, t, splat(kP5));
+  a = fma2(a, t, splat(kP4));
+  a = fma2(a, t, splat(kP3));
+  a = fma2(a, t, splat(kP2));
+  a = fma2(a, t, splat(kP1));
+  return mul2(a, t);
+}
+
+template <int B>
+__device__ __forceinline__ void decode_log_pairs(const uint32_t (&w)[2], float s, const float* lut8, f2 one,
+                                                 f2 (&out)[2]) {
+  const f2 s2 = splat(s);
+  if constexpr (B == 8) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+      out[h] = mul2(s2, make_float2(lut8[(w[0] >> (16 * h)) & 255u], lut8[(w[0] >> (16 * h + 8)) & 255u]));
+  } else if constexpr (B <= 4) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint32_t e0 = ((w[0] << (23 - B * (2 * h))) & (Wd<B>::mask << 23)) | (Wd<B>::emin << 23);
+      const uint32_t e1 = ((w[0] << (23 - B * (2 * h + 1))) & (Wd<B>::mask << 23)) | (Wd<B>::emin << 23);
+      out[h] = mul2(s2, bits2(e0, e1));
+    }
+  } else {
+    constexpr float cb = (float)Wd<B>::Roct / (float)Wd<B>::K;
+    constexpr float off = kTwo23 + (float)Wd<B>::K;
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+      out[h] = mul2(s2, ex2_poly_pair(mul2(add2(code_pair<B>(w, h), splat(-off)), splat(cb)), one));
+  }
+}
+
+// Quantize one row of new first moments and store the codes; nq = 2^(B-1) - code = -q as floats.
+template <int B>
+__device__ __forceinline__ void encode_lin_pairs(uint8_t* row_ptr, int lane, const f2 (&m)[2], float inv, f2 (&nq)[2]) {
+  constexpr float mg = kMagic + (float)Wd<B>::half;
+  uint32_t x[4];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const f2 t = fma2(m[h], splat(inv), splat(mg));
+    x[2 * h] = __float_as_uint(t.x);
+    x[2 * h + 1] = __float_as_uint(t.y);
+    nq[h] = fma2(t, splat(-1.0f), splat(mg));       // mg - t, exact
+  }
+  pack_store_row<B>(row_ptr, lane, x, kMagicBits);
+}
+
+// Octave code of one row of new second moments (see encode_oct_row): codes stored, e = exponent fields.
+template <int B>
+__device__ __forceinline__ void encode_oct_pairs(uint8_t* row_ptr, int lane, const f2 (&v)[2], float c_up, float ymin_up,
+                                                 uint32_t (&e)[4]) {
+  uint32_t f = 0u;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const f2 y = mul2(v[h], splat(c_up));
+    const uint32_t y0 = __float_as_uint(fmaxf(y.x, ymin_up)), y1 = __float_as_uint(fmaxf(y.y, ymin_up));
+    f |= (y0 >> (23 - B * (2 * h))) & (Wd<B>::mask << (B * (2 * h)));
+    f |= (y1 >> (23 - B * (2 * h + 1))) & (Wd<B>::mask << (B * (2 * h + 1)));
+    e[2 * h] = y0 >> 23;
+    e[2 * h + 1] = y1 >> 23;
+  }
+  store_fields<B>(row_ptr, lane, f, 0u);
+}
+
+// Polynomial log code (8, 16 bits) of one row; r = code - K as floats.
+template <int B>
+__device__ __forceinline__ void encode_log_pairs(uint8_t* row_ptr, int lane, const f2 (&v)[2], float lgc, uint32_t ebase,
+                                                 f2 one, f2 (&r)[2]) {
+  constexpr float a = (float)Wd<B>::K / (float)Wd<B>::Roct;
+  constexpr float negR = -(float)Wd<B>::Roct;
+  uint32_t x[4];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const uint32_t b0 = __float_as_uint(v[h].x), b1 = __float_as_uint(v[h].y);
+    const f2 de = add2(bits2(ebase + (b0 >> 23), ebase + (b1 >> 23)), splat(-kMagic));
+    const f2 dp = fma2(lg_poly_pair(b0, b1), one, splat(-lgc));      // P(x) - P(s): a product meets a sum
+    f2 d = add2(de, dp);
+    d = make_float2(fmaxf(d.x, negR), fmaxf(d.y, negR));
+    const f2 t = fma2(d, splat(a), splat(kMagic));
+    x[2 * h] = __float_as_uint(t.x);
+    x[2 * h + 1] = __float_as_uint(t.y);
+    r[h] = add2(t, splat(-kMagic));
+  }
+  pack_store_row<B>(row_ptr, lane, x, kMagicBits - (uint32_t)Wd<B>::K);
+}
+
 // One staged tile, one warp: R rows of 128 elements, taken in passes of RP rows.  The pass loop is
 // a real loop (not unrolled): the straight-line body of a pass is what the warps stream through the
 // instruction cache, and halving it pays more than the lost overlap between passes.  Specialised on
@@ -493,35 +629,48 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
                                           const float* __restrict__ lut8, int lane, int warp, uint32_t empty_bar,
                                           double* __restrict__ part, float grad_mul) {
   static_assert(!VPL || BV >= 8, "the piecewise-linear variant exists at 8 and 16 bits");
+  static_assert(RP == 2, "the level shuffle of the octave codes is laid out for two rows per pass");
   [[maybe_unused]] const uint32_t* lutn = reinterpret_cast<const uint32_t*>(lut8 + 256);
   const int lgB = (int)((ti.packed >> 16) & 0xFFu);
   [[maybe_unused]] const uint32_t lp_dtype = ti.packed >> 24;
-  const float lrwd = sc.l2_mode ? 0.0f : ti.wdx;
-  float a0 = 0.f, a1 = 0.f, a2 = 0.f;      // statistics over the raw gradient (decision steps)
+  const float nlrwd = sc.l2_mode ? 0.0f : -ti.wdx;
+  f2 a0 = splat(0.f), a1 = splat(0.f), a2 = splat(0.f);      // statistics over the raw gradient (decision steps)
+  const f2 one2 = splat(sc.one);
   // octave v codes: 2^(level - K) of the level this lane tabulates for the update (see below)
-  [[maybe_unused]] const float lvl = __uint_as_float((((uint32_t)lane & Wd<BV <= 4 ? BV : 2>::mask) + Wd<BV <= 4 ? BV : 2>::emin) << 23);
+  constexpr int LV = BV <= 4 ? BV : 2;
+  [[maybe_unused]] const float lvl = __uint_as_float((((uint32_t)lane & Wd<LV>::mask) + Wd<LV>::emin) << 23);
 
 #pragma unroll 1
   for (int pass = 0; pass < R / RP; ++pass) {
     const int row0 = warp * R + pass * RP;
 
     // ---- staged rows -> registers, decode -----------------------------------------------------------
-    float th[RP][4], g[RP][4], mt[RP][4], vt[RP][4];
+    f2 th[RP][2], g[RP][2], mt[RP][2], vt[RP][2];
 #pragma unroll
     for (int r = 0; r < RP; ++r) {
       const int elem = (row0 + r) * kRowElems + 4 * lane;
       const float4 t4 = *reinterpret_cast<const float4*>(stage + kOffTheta + 4 * elem);
-      th[r][0] = t4.x; th[r][1] = t4.y; th[r][2] = t4.z; th[r][3] = t4.w;
-      lds_grad<GDT>(stage, elem, g[r]);
+      th[r][0] = make_float2(t4.x, t4.y);
+      th[r][1] = make_float2(t4.z, t4.w);
+      float gs[4];
+      lds_grad<GDT>(stage, elem, gs);
+      g[r][0] = make_float2(gs[0], gs[1]);
+      g[r][1] = make_float2(gs[2], gs[3]);
       const int blk = ((row0 + r) * kRowElems) >> lgB;
       const float sm = *reinterpret_cast<const float*>(stage + kOffMs + 4 * blk);
       const float sv = *reinterpret_cast<const float*>(stage + kOffVs + 4 * blk);
       uint32_t w[2];
       lds_codes<BM>(stage + kOffMc + (row0 + r) * (16 * BM), lane, w);
-      decode_lin_row<BM>(w, sm, mt[r]);
+      decode_lin_pairs<BM>(w, sm, mt[r]);
       lds_codes<BV>(stage + kOffVc + (row0 + r) * (16 * BV), lane, w);
-      if constexpr (VPL) decode_pl_row<BV>(w, __float_as_uint(sv), lutn, vt[r]);
-      else decode_log_row<BV>(w, sv, lut8, vt[r]);
+      if constexpr (VPL) {
+        float vs[4];
+        decode_pl_row<BV>(w, __float_as_uint(sv), lutn, vs);
+        vt[r][0] = make_float2(vs[0], vs[1]);
+        vt[r][1] = make_float2(vs[2], vs[3]);
+      } else {
+        decode_log_pairs<BV>(w, sv, lut8, one2, vt[r]);
+      }
     }
     if (pass == R / RP - 1) {   // the last rows are in registers: this warp is done with the stage
       __syncwarp();
@@ -532,16 +681,16 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
 #pragma unroll
       for (int r = 0; r < RP; ++r)
 #pragma unroll
-        for (int k = 0; k < 4; ++k) g[r][k] = __fmul_rn(g[r][k], grad_mul);
+        for (int h = 0; h < 2; ++h) g[r][h] = mul2(g[r][h], splat(grad_mul));
     }
     if (part != nullptr) {
 #pragma unroll
       for (int r = 0; r < RP; ++r)
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          a0 += g[r][k];
-          a1 += fabsf(g[r][k]);
-          a2 = __fmaf_rn(g[r][k], g[r][k], a2);
+        for (int h = 0; h < 2; ++h) {
+          a0 = fma2(g[r][h], one2, a0);       // (g may be a product: the unscaled gradient)
+          a1 = add2(a1, make_float2(fabsf(g[r][h].x), fabsf(g[r][h].y)));
+          a2 = fma2(g[r][h], g[r][h], a2);
         }
     }
 
@@ -550,15 +699,15 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
 #pragma unroll
       for (int r = 0; r < RP; ++r)
 #pragma unroll
-        for (int k = 0; k < 4; ++k) g[r][k] = __fadd_rn(g[r][k], __fmul_rn(ti.wdx, th[r][k]));
+        for (int h = 0; h < 2; ++h) g[r][h] = fma2(g[r][h], one2, mul2(splat(ti.wdx), th[r][h]));
     }
 #pragma unroll
     for (int r = 0; r < RP; ++r) {
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const float gk = g[r][k];
-        mt[r][k] = __fmaf_rn(sc.b1, mt[r][k], __fmul_rn(sc.c1, gk));
-        vt[r][k] = __fmaf_rn(sc.b2, vt[r][k], __fmul_rn(__fmul_rn(sc.c2, gk), gk));
+      for (int h = 0; h < 2; ++h) {
+        const f2 gk = g[r][h];
+        mt[r][h] = fma2(splat(sc.b1), mt[r][h], mul2(splat(sc.c1), gk));
+        vt[r][h] = fma2(splat(sc.b2), vt[r][h], mul2(mul2(splat(sc.c2), gk), gk));
       }
     }
 
@@ -566,22 +715,14 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
     uint32_t mxm[RP], mxv[RP];
 #pragma unroll
     for (int r = 0; r < RP; ++r) {
-      const float am = fmaxf(fmaxf(fabsf(mt[r][0]), fabsf(mt[r][1])), fmaxf(fabsf(mt[r][2]), fabsf(mt[r][3])));
-      const float av = fmaxf(fmaxf(vt[r][0], vt[r][1]), fmaxf(vt[r][2], vt[r][3]));
+      const float am = fmaxf(fmaxf(fabsf(mt[r][0].x), fabsf(mt[r][0].y)), fmaxf(fabsf(mt[r][1].x), fabsf(mt[r][1].y)));
+      const float av = fmaxf(fmaxf(vt[r][0].x, vt[r][0].y), fmaxf(vt[r][1].x, vt[r][1].y));
       mxm[r] = __reduce_max_sync(kFull, __float_as_uint(am));
       mxv[r] = __reduce_max_sync(kFull, __float_as_uint(av));
     }
-    if (RP >= 2 && lgB >= 8) {
-#pragma unroll
-      for (int r = 0; r + 1 < RP; r += 2) {
-        mxm[r] = mxm[r + 1] = max(mxm[r], mxm[r + 1]);
-        mxv[r] = mxv[r + 1] = max(mxv[r], mxv[r + 1]);
-      }
-    }
-    if (RP >= 4 && lgB >= 9) {
-      const uint32_t a = max(mxm[0], mxm[RP - 2]), b = max(mxv[0], mxv[RP - 2]);
-#pragma unroll
-      for (int r = 0; r < RP; ++r) { mxm[r] = a; mxv[r] = b; }
+    if (lgB >= 8) {
+      mxm[0] = mxm[1] = max(mxm[0], mxm[1]);
+      mxv[0] = mxv[1] = max(mxv[0], mxv[1]);
     }
 
     // ---- per-block constants: one lane per (row, state) works them out, then they are broadcast --------
@@ -589,22 +730,16 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
     // times the power of two that steers the level shuffle of its row (encode_oct_row)
     float inv_m[RP], lgc[RP];
     {
-      uint32_t mine = mxm[0];
-#pragma unroll
-      for (int r = 1; r < RP; ++r)
-        if ((lane & (RP - 1)) == r) mine = mxm[r];
+      uint32_t mine = (lane & 1) ? mxm[1] : mxm[0];
       if constexpr (BV <= 4) {
-#pragma unroll
-        for (int r = 0; r < RP; ++r)
-          if ((lane & (2 * RP - 1)) == RP + r) mine = mxv[r];
+        if (lane & RP) mine = (lane & 1) ? mxv[1] : mxv[0];
       }
       const float x = __uint_as_float(mine);
       const bool zero = x < kTiny;
       float mul = (float)Wd<BM>::qmax;
       if constexpr (BV <= 4) {
-        static_assert(BV > 4 || RP == 2, "the level shuffle is laid out for two rows per pass");
-        constexpr float up0 = kSqrt2 * (float)(1 << Oct<BV <= 4 ? BV : 2>::up0);
-        constexpr float up1 = kSqrt2 * (float)(1 << Oct<BV <= 4 ? BV : 2>::up1);
+        constexpr float up0 = kSqrt2 * (float)(1 << Oct<LV>::up0);
+        constexpr float up1 = kSqrt2 * (float)(1 << Oct<LV>::up1);
         if (lane & RP) mul = (lane & 1) ? up1 : up0;
       }
       const float val = zero ? 0.f : __fmul_rn(mul, __frcp_rn(x));
@@ -618,10 +753,7 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
 #pragma unroll
         for (int r = 0; r < RP; ++r) lgc[r] = __shfl_sync(kFull, val, RP + r);
       } else {
-        uint32_t mv = mxv[0];
-#pragma unroll
-        for (int r = 1; r < RP; ++r)
-          if ((lane & (RP - 1)) == r) mv = mxv[r];
+        const uint32_t mv = (lane & 1) ? mxv[1] : mxv[0];
         if (lane < RP && opens) {
           ti.mso[e_mine >> lgB] = zero ? 0.f : x;
           ti.vso[e_mine >> lgB] = __uint_as_float(mv) < kTiny ? 0.f : __uint_as_float(mv);
@@ -644,7 +776,7 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
     [[maybe_unused]] float lut_upd = 0.f;
     if constexpr (BV <= 4) {
       constexpr float invq = 1.0f / (float)Wd<BM>::qmax;
-      const bool second = (lane >> (BV <= 4 ? BV : 0)) & 1;
+      const bool second = (lane >> LV) & 1;
       const float svr = __uint_as_float(second ? mxv[1] : mxv[0]);
       const float smr = __uint_as_float(second ? mxm[1] : mxm[0]);
       const float vl = __fmul_rn(svr < kTiny ? 0.f : svr, lvl);
@@ -653,6 +785,8 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
     }
 
     // ---- quantize, pack, store; update the parameters ---------------------------------------------------
+    // theta - lr*wd*theta - update as fma(-q, factor, fma(theta, -lr*wd, theta)): the decay keeps its own
+    // precision (a factor 1 - lr*wd rounded to fp32 would be off by ~1e-3 of the decay it applies)
     float* param = ti.param + row0 * kRowElems + 4 * lane;
 #pragma unroll
     for (int r = 0; r < RP; ++r) {
@@ -660,51 +794,60 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
       const float sm_raw = __uint_as_float(mxm[r]);
       const float sv_raw = __uint_as_float(mxv[r]);
       const bool vzero = sv_raw < kTiny;
-      float out[4];
+      f2 out[2];
       if constexpr (BV <= 4) {
-        float q[4];
+        f2 nq[2];
         uint32_t e[4];
-        encode_lin_row_q<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], inv_m[r], q);
-        const float ymin_up = __uint_as_float((Wd<BV>::emin + (uint32_t)(r == 0 ? Oct<BV>::up0 : Oct<BV>::up1)) << 23);
-        encode_oct_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], lgc[r], ymin_up, e);
+        encode_lin_pairs<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], inv_m[r], nq);
+        const float ymin_up = __uint_as_float((Wd<LV>::emin + (uint32_t)(r == 0 ? Oct<LV>::up0 : Oct<LV>::up1)) << 23);
+        encode_oct_pairs<LV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], lgc[r], ymin_up, e);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float base = __fmaf_rn(th[r][k], -lrwd, th[r][k]);
-          out[k] = __fmaf_rn(-q[k], __shfl_sync(kFull, lut_upd, e[k]), base);
+        for (int h = 0; h < 2; ++h) {
+          const f2 base = fma2(th[r][h], splat(nlrwd), th[r][h]);
+          const f2 fac = make_float2(__shfl_sync(kFull, lut_upd, e[2 * h]), __shfl_sync(kFull, lut_upd, e[2 * h + 1]));
+          out[h] = fma2(nq[h], fac, base);
         }
       } else if constexpr (!VPL) {
         // 2^((code-K) * R/K / 2) by the special-function unit: sqrt of the decoded level, to 2^-22
-        constexpr float half_cb = 0.5f * ((float)Wd<BV>::Roct / (float)Wd<BV>::K);
+        constexpr int LB = BV >= 8 ? BV : 8;
+        constexpr float half_cb = 0.5f * ((float)Wd<LB>::Roct / (float)Wd<LB>::K);
         constexpr float invq = 1.0f / (float)Wd<BM>::qmax;
         const uint32_t ebase = kMagicBits - (vzero ? (uint32_t)kZeroBlockExp : (mxv[r] >> 23));
         const float unit = __fmul_rn(__fmul_rn(sm_raw, sc.step_size), invq);
         const float srt = __fmul_rn(sqrt_fast(vzero ? 0.f : sv_raw), sc.rsqrt_bc2);
-        float q[4], rr[4];
-        encode_lin_row_q<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], inv_m[r], q);
-        encode_log_row_r<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], lgc[r], ebase, rr);
+        f2 nq[2], rr[2];
+        encode_lin_pairs<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], inv_m[r], nq);
+        encode_log_pairs<LB>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], lgc[r], ebase, one2, rr);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float den = __fmaf_rn(ex2_fast(__fmul_rn(rr[k], half_cb)), srt, sc.eps);
-          const float base = __fmaf_rn(th[r][k], -lrwd, th[r][k]);
-          out[k] = __fmaf_rn(-__fmul_rn(q[k], unit), rcp_fast(den), base);
+        for (int h = 0; h < 2; ++h) {
+          const f2 arg = mul2(rr[h], splat(half_cb));
+          const f2 den = fma2(make_float2(ex2_fast(arg.x), ex2_fast(arg.y)), splat(srt), splat(sc.eps));
+          const f2 base = fma2(th[r][h], splat(nlrwd), th[r][h]);
+          out[h] = fma2(mul2(nq[h], splat(unit)), make_float2(rcp_fast(den.x), rcp_fast(den.y)), base);
         }
       } else {
-        float mq[4], vq[4];
-        // mq comes out multiplied by lr/(1-beta1^t): the decode scale carries the factor
-        encode_lin_row<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], __fmul_rn(sm_raw, sc.step_size), inv_m[r], mq);
-        encode_pl_row<BV>(ti.vco + (row0 + r) * (16 * BV), lane, vt[r], vzero ? 0x7F800000u : mxv[r],
+        constexpr int LB = BV >= 8 ? BV : 8;
+        constexpr float invq = 1.0f / (float)Wd<BM>::qmax;
+        const float unit = __fmul_rn(__fmul_rn(sm_raw, sc.step_size), invq);
+        f2 nq[2];
+        float vs[4], vq[4];
+        encode_lin_pairs<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], inv_m[r], nq);
+        vs[0] = vt[r][0].x; vs[1] = vt[r][0].y; vs[2] = vt[r][1].x; vs[3] = vt[r][1].y;
+        encode_pl_row<LB>(ti.vco + (row0 + r) * (16 * BV), lane, vs, vzero ? 0x7F800000u : mxv[r],
                           vzero ? 0u : mxv[r], lutn, vq);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float den = __fmaf_rn(sqrt_fast(vq[k]), sc.rsqrt_bc2, sc.eps);
-          const float base = __fmaf_rn(th[r][k], -lrwd, th[r][k]);
-          out[k] = __fmaf_rn(-mq[k], rcp_fast(den), base);
+        for (int h = 0; h < 2; ++h) {
+          const f2 den = fma2(make_float2(sqrt_fast(vq[2 * h]), sqrt_fast(vq[2 * h + 1])), splat(sc.rsqrt_bc2), splat(sc.eps));
+          const f2 base = fma2(th[r][h], splat(nlrwd), th[r][h]);
+          out[h] = fma2(mul2(nq[h], splat(unit)), make_float2(rcp_fast(den.x), rcp_fast(den.y)), base);
         }
       }
-      *reinterpret_cast<float4*>(param + r * kRowElems) = make_float4(out[0], out[1], out[2], out[3]);
+      *reinterpret_cast<float4*>(param + r * kRowElems) = make_float4(out[0].x, out[0].y, out[1].x, out[1].y);
       if constexpr (AMP) {
-        if (ti.lp != nullptr)
-          *reinterpret_cast<uint2*>(ti.lp + (row0 + r) * kRowElems + 4 * lane) = pack_lp(out, lp_dtype);
+        if (ti.lp != nullptr) {
+          const float o4[4] = {out[0].x, out[0].y, out[1].x, out[1].y};
+          *reinterpret_cast<uint2*>(ti.lp + (row0 + r) * kRowElems + 4 * lane) = pack_lp(o4, lp_dtype);
+        }
       }
     }
   }
@@ -713,9 +856,10 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
     // Pairwise fp32 butterfly that spreads the three sums over the lanes on the way down:
     // after xor 16 the low half carries (sum0, sum1) and the high half (sum2, -); after xor 8
     // lanes 0-7 / 8-15 / 16-23 carry sum0 / sum1 / sum2; three more steps finish each group.
+    const float s0 = a0.x + a0.y, s1 = a1.x + a1.y, s2 = a2.x + a2.y;
     const bool hi = lane & 16;
-    float x = (hi ? a2 : a0) + __shfl_xor_sync(kFull, hi ? a0 : a2, 16);
-    float y = (hi ? 0.f : a1) + __shfl_xor_sync(kFull, hi ? a1 : 0.f, 16);
+    float x = (hi ? s2 : s0) + __shfl_xor_sync(kFull, hi ? s0 : s2, 16);
+    float y = (hi ? 0.f : s1) + __shfl_xor_sync(kFull, hi ? s1 : 0.f, 16);
     const bool q = lane & 8;
     float z = (q ? y : x) + __shfl_xor_sync(kFull, q ? x : y, 8);
     z += __shfl_xor_sync(kFull, z, 4);
