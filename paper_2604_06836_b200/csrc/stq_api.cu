@@ -205,16 +205,16 @@ int validate_row(const stq_tensor& t, int kind) {
 // groups uses it; the balance itself is dynamic.
 double body_cost(const stq_tensor& t) {
   static const double kRate[5][7] = {
-      {490, 458, 480, 392, 345, 440, 411},
-      {454, 426, 455, 370, 323, 424, 401},
-      {470, 462, 483, 389, 345, 437, 413},
-      {476, 458, 466, 389, 340, 435, 396},
-      {436, 426, 422, 379, 332, 396, 355},
+      {581, 550, 564, 488, 445, 480, 430},
+      {550, 523, 540, 454, 417, 450, 400},
+      {567, 536, 551, 488, 439, 480, 425},
+      {531, 520, 510, 471, 414, 465, 405},
+      {458, 450, 443, 414, 369, 410, 360},
   };
   auto idx = [](int b) { return b == 2 ? 0 : b == 3 ? 1 : b == 4 ? 2 : b == 8 ? 3 : 4; };
   int iv = idx(t.bits_v);
   if (t.v_log == STQ_VLOG_PL && iv >= 3) iv += 2;
-  return 483.0 / kRate[idx(t.bits_m)][iv];
+  return 551.0 / kRate[idx(t.bits_m)][iv];
 }
 
 constexpr int kSplitKey = 1 << 20;
