@@ -104,68 +104,117 @@ class ClockSampler(threading.Thread):
 # ------------------------------------------------------------------------------------------------
 # the oracle arm (CPU baseline / --impl reference)
 # ------------------------------------------------------------------------------------------------
-def oracle_sample_run(w: W.Workload, bits_m, bits_v, budget_s: float, repeats: int = 1):
-    """Times the CPU oracle, as it stands, on a bounded sample of the workload: block-aligned chunks
-    taken round-robin from the tensor list, one chunk per task, tasks spread over the host cores."""
+FULL_ORACLE_PARAMS = 1 << 27     # workloads up to this size get a full oracle step on their real tensors
+
+
+def _to_np(t: torch.Tensor) -> np.ndarray:
+    if t.dtype in (torch.bfloat16, torch.float16):
+        return t.contiguous().view(torch.int16).numpy().view(np.uint16).copy()
+    return t.contiguous().numpy().copy()
+
+
+def oracle_run(w: W.Workload, bits_m, bits_v, budget_s: float, repeats: int = 1):
+    """Times the CPU oracle, as it stands, on the machine's host cores.
+
+    Workloads of up to 2^27 parameters (cfg1-cfg3): one full oracle step over the workload's real tensors
+    (the seeded parameter and gradient draws of the workload, every tensor at its width), all cores, and the
+    same full step again on one thread.  Larger workloads (cfg4, cfg5): a bounded sample, i.e. block-aligned
+    chunks of at most 2^18 elements of tensors drawn in proportion to their size (so the sample has the
+    workload's numel-weighted width mix), sized for about `budget_s` seconds of all-core work, and a
+    single-thread timing on every k-th chunk of the same sample.  Work is spread over host threads
+    range by range; the oracle's C code runs outside the interpreter lock."""
     import oracle as O
     from concurrent.futures import ThreadPoolExecutor
 
     cores = os.cpu_count() or 1
     chunk = 1 << 18
-    # calibrate the single-thread rate on one chunk
-    rng = np.random.default_rng(0)
-    th = rng.normal(0, 0.02, chunk).astype(np.float32)
-    g32 = (rng.standard_t(3, chunk) * 1e-3).astype(np.float32)
-    g = torch.from_numpy(g32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16).copy() \
-        if w.grad_dtype == "bf16" else g32
-    st = O.new_state(chunk, w.block, 4, 4)
+    block = w.block
     kw = dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, weight_decay=w.weight_decay,
               v_mode=O.LOG_PL if w.v_log == "pl" else O.LOG)
-    t0 = time.perf_counter()
-    st, _ = O.step(th, g, st, w.block, t=1, **kw)
-    rate1 = chunk / (time.perf_counter() - t0)
-    want = int(min(w.total_params, 1 << 27, max(chunk, rate1 * cores * budget_s)))
-    # build the sample: chunks of the real tensors' sizes and widths
-    tasks, taken = [], 0
+    if w.grad_dtype == "fp16":
+        kw.update(fp16_grad=True, inv_grad_scale=1.0 / w.loss_scale if w.loss_scale > 0 else 1.0)
+    full = w.total_params <= FULL_ORACLE_PARAMS
+    if full and w.total_params < 4 * cores * chunk:        # a small workload still gets a few ranges per thread
+        chunk = max(1024, w.total_params // (4 * cores) // 1024 * 1024)
     numels = w.numels
-    order = np.argsort(numels)[::-1]
-    i = 0
-    while taken < want and i < 100000:
-        l = int(order[i % len(order)])
-        n = int(min(chunk, numels[l], want - taken))
-        if n <= 0:
-            break
-        n = max(w.block, n // w.block * w.block) if n >= w.block else n
-        th = rng.normal(0, 0.02, n).astype(np.float32)
-        g32 = (rng.standard_t(3, n) * 1e-3).astype(np.float32)
-        g = torch.from_numpy(g32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16).copy() \
-            if w.grad_dtype == "bf16" else g32
-        tasks.append([th, g, O.new_state(n, w.block, int(bits_m[l]), int(bits_v[l]))])
-        taken += n
-        i += 1
+    rng = np.random.default_rng(0)
+    tensors = {}        # tensor index -> [theta, grad, state in, state out]
 
-    def one(task, t):
-        task[2], _ = O.step(task[0], task[1], task[2], w.block, t=t, **kw)
+    def materialise(l: int, n: int, real: bool):
+        if real:
+            th, g = _to_np(W.draw_param(w, l, "cpu")), _to_np(W.draw_grad(w, l, 1, "cpu"))
+        else:   # a chunk-sized stand-in with the value distributions of the recipe (the timing does not depend on values)
+            th = rng.normal(0, 0.02, n).astype(np.float32)
+            g32 = torch.from_numpy((rng.standard_t(3, n) * 1e-3).astype(np.float32))
+            g = _to_np(g32.to({"fp32": torch.float32, "bf16": torch.bfloat16, "fp16": torch.float16}[w.grad_dtype]))
+        bm, bv = int(bits_m[l]), int(bits_v[l])
+        return [th, g, O.new_state(n, block, bm, bv), O.new_state(n, block, bm, bv)]
+
+    tasks = []          # (key, e0, e1)
+    if full:
+        for l, n in enumerate(numels):
+            tensors[l] = materialise(l, n, True)
+            tasks += [(l, e0, min(n, e0 + chunk)) for e0 in range(0, n, chunk)]
+        taken = w.total_params
+    else:
+        st = O.new_state(chunk, block, 4, 4)
+        t0 = time.perf_counter()
+        O.step(rng.normal(0, 0.02, chunk).astype(np.float32), (rng.standard_t(3, chunk) * 1e-3).astype(np.float32),
+               st, block, t=1, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, weight_decay=w.weight_decay)
+        rate1 = chunk / (time.perf_counter() - t0)        # calibration only: sizes the sample
+        want = int(min(FULL_ORACLE_PARAMS, max(chunk, rate1 * cores * budget_s)))
+        prob = np.asarray(numels, dtype=np.float64) / float(sum(numels))
+        taken, k = 0, 0
+        while taken < want:
+            l = int(rng.choice(len(numels), p=prob))
+            n = int(min(chunk, numels[l]))
+            n = n // block * block if n >= block else n
+            tensors[("s", k)] = materialise(l, n, False)
+            tasks.append((("s", k), 0, n))
+            taken += n
+            k += 1
+
+    def run(task, t):
+        key, e0, e1 = task
+        th, g, a, b = tensors[key]
+        O.step_range(th, g, e0, e1, block, a, b, t=t, **kw)
+
+    def swap():
+        for v in tensors.values():
+            v[2], v[3] = v[3], v[2]
 
     times = []
     with ThreadPoolExecutor(max_workers=cores) as ex:
-        list(ex.map(lambda tk: one(tk, 1), tasks))          # populate the states (untimed)
+        list(ex.map(lambda tk: run(tk, 1), tasks))          # step 1 populates the states (untimed)
+        swap()
         for r in range(repeats):
             t0 = time.perf_counter()
-            list(ex.map(lambda tk: one(tk, 2 + r), tasks))
+            list(ex.map(lambda tk: run(tk, 2 + r), tasks))
             times.append(time.perf_counter() - t0)
-    return {"params": taken, "seconds": times, "cores": min(cores, len(tasks)), "single_thread": rate1,
-            "sample": f"{taken} params in {len(tasks)} block-aligned chunks of <= {chunk} drawn from the "
-                      f"largest tensors of the workload at their widths, one oracle step each, "
-                      f"{min(cores, len(tasks))} threads"}
+            swap()
+    # one thread, same width mix: the whole step for the small workloads, every k-th chunk of the sample otherwise
+    sub = tasks if full else tasks[::max(1, len(tasks) // 16)]
+    n_sub = sum(e1 - e0 for _, e0, e1 in sub)
+    t0 = time.perf_counter()
+    for tk in sub:
+        run(tk, 2 + repeats)
+    single = n_sub / (time.perf_counter() - t0)
+    used = min(cores, len(tasks))
+    what = (f"one full oracle step over the workload's {len(numels)} real tensors ({taken} params, ranges of <= {chunk} "
+            f"elements over {used} threads)" if full else
+            f"{taken} params in {len(tasks)} block-aligned chunks of <= {chunk} elements of tensors drawn in proportion "
+            f"to their size at their widths, one oracle step each, {used} threads")
+    return {"params": taken, "seconds": times, "cores": used, "single_thread": single,
+            "single_thread_sample": f"{n_sub} params ({len(sub)} of the same chunks), 1 thread", "sample": what,
+            "host_cores": cores}
 
 
 def run_reference(args, w, bits_m, bits_v):
     rank, _, world = dist_env()
     if rank != 0:
         return
-    res = oracle_sample_run(w, bits_m, bits_v, budget_s=max(2.0, 60.0 / max(1, args.steps + args.warmup)),
-                            repeats=args.steps + args.warmup)
+    res = oracle_run(w, bits_m, bits_v, budget_s=max(2.0, 60.0 / max(1, args.steps + args.warmup)),
+                     repeats=args.steps + args.warmup)
     timed = res["seconds"][args.warmup:]
     sec = float(np.mean(timed))
     value = res["params"] / sec
@@ -174,8 +223,12 @@ def run_reference(args, w, bits_m, bits_v):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "params": w.total_params, "block": w.block, "grad_dtype": w.grad_dtype,
-                   "mean_bits": W.mean_bits(w, bits_m, bits_v), "step_is": "one oracle step over the sample"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": res["cores"], "kind": "oracle", "sample": res["sample"]},
+                   "mean_bits": W.mean_bits(w, bits_m, bits_v),
+                   "step_is": ("one full oracle step over the workload" if w.total_params <= FULL_ORACLE_PARAMS
+                               else "one oracle step over the bounded sample")},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": res["cores"], "kind": "oracle", "sample": res["sample"],
+                         "host_cores": res["host_cores"], "single_thread_value": res["single_thread"],
+                         "single_thread_sample": res["single_thread_sample"]},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -393,11 +446,12 @@ def run_ours(args, w, bits_m, bits_v):
             del jv
         except Exception as exc:          # an extra must never cost the line
             line["variants"] = {"error": f"{type(exc).__name__}: {exc}"[:200]}
-    if rank == 0 and not args.no_cpu_baseline and world == 1 and not amp:
-        res = oracle_sample_run(w, bits_m, bits_v, budget_s=8.0, repeats=1)
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        res = oracle_run(w, bits_m, bits_v, budget_s=8.0, repeats=1)
         line["cpu_baseline"] = {"value": res["params"] / res["seconds"][0], "unit": UNIT, "cores": res["cores"],
-                                "kind": "oracle", "sample": res["sample"],
-                                "single_thread_value": res["single_thread"]}   # one 4/4-bit chunk of 2^18 elements
+                                "kind": "oracle", "sample": res["sample"], "host_cores": res["host_cores"],
+                                "single_thread_value": res["single_thread"],
+                                "single_thread_sample": res["single_thread_sample"]}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if use_dist:

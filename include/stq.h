@@ -56,7 +56,7 @@ enum {
   STQ_OK = 0,
   STQ_E_NULL = -1,      /* a required pointer is NULL                                         */
   STQ_E_BITS = -2,      /* a width outside {2,3,4,8,16,32}                                    */
-  STQ_E_BLOCK = -3,     /* block not in {128, 256, 512}                                       */
+  STQ_E_BLOCK = -3,     /* block is not a power of two in 32..1024                            */
   STQ_E_ALIGN = -4,     /* a buffer is not aligned as required                                */
   STQ_E_ALIAS = -5,     /* in/out buffers overlap in a way the step cannot honour             */
   STQ_E_NUMEL = -6,     /* numel == 0, or the table is empty or too large                     */
@@ -93,7 +93,8 @@ typedef struct stq_tensor {
   void* v_codes_out;         /* scales_out may equal scales_in                                 */
   float* v_scales_out;
   uint64_t numel;
-  uint32_t block;            /* quantization block: 128, 256 or 512                            */
+  uint32_t block;            /* quantization block: a power of two, 32..1024 (128 and 256 run   */
+                             /* in the main kernel, the others in the generic one)             */
   uint8_t bits_m, bits_v;          /* widths stored now                                        */
   uint8_t bits_m_out, bits_v_out;  /* widths to write                                          */
   float weight_decay;        /* per-tensor lambda                                              */

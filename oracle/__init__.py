@@ -223,6 +223,32 @@ def step(theta: np.ndarray, grad: np.ndarray, st: State, block: int, *, lr, beta
     return State(mc, ms, bm, vc, vs, bv), stats
 
 
+def step_range(theta: np.ndarray, grad: np.ndarray, e0: int, e1: int, block: int, st_in: State, st_out: State, *,
+               lr, beta1, beta2, eps, weight_decay, t: int, decoupled_wd: bool = True, fp16_grad: bool = False,
+               inv_grad_scale: float = 1.0, v_mode: int = LOG, stats: np.ndarray | None = None) -> None:
+    """The same Algorithm-1 step on the elements [e0, e1) of one tensor, e0 a multiple of the block size (blocks
+    are independent given their inputs, so a tensor may be stepped range by range, in any order or in
+    parallel).  theta, grad and the buffers of st_in / st_out belong to the whole tensor; theta and st_out are
+    written in place for the range only.  stats: float64[4] for this range's sums, or None."""
+    assert e0 % block == 0 and 0 <= e0 < e1 <= theta.size
+    n = e1 - e0
+    dt = _grad_dtype(grad, fp16_grad)
+
+    def cut(st: State):
+        def codes(c, b):
+            return c[e0 * 4:] if b == 32 else c[e0 * b // 8:]          # a block is a whole number of bytes
+        return (codes(st.m_codes, st.bits_m), st.m_scales[e0 // block:] if st.bits_m != 32 else st.m_scales,
+                codes(st.v_codes, st.bits_v), st.v_scales[e0 // block:] if st.bits_v != 32 else st.v_scales)
+
+    mci, msi, vci, vsi = cut(st_in)
+    mco, mso, vco, vso = cut(st_out)
+    hp = HParams(lr, beta1, beta2, eps, weight_decay, t, 1 if decoupled_wd else 0, dt, inv_grad_scale, 0, v_mode)
+    rc = lib().orc_step(_p(theta[e0:]), _p(grad[e0:]), n, block, _p(mci), _p(msi), st_in.bits_m, _p(vci), _p(vsi),
+                        st_in.bits_v, _p(mco), _p(mso), st_out.bits_m, _p(vco), _p(vso), st_out.bits_v,
+                        C.byref(hp), _p(stats))
+    assert rc == 0
+
+
 def round_lp(x: np.ndarray, lp: str) -> np.ndarray:
     """Nearest-even rounding of fp32 values to "bf16" or "fp16"; returns the uint16 bit patterns."""
     x = _chk(np.ascontiguousarray(x), np.float32)

@@ -76,7 +76,7 @@ namespace {
 enum Kind { kKindStep = 0, kKindRepack = 1, kKindInit = 2, kKindStats = 3 };
 
 bool width_ok(int b) { return b == 2 || b == 3 || b == 4 || b == 8 || b == 16 || b == 32; }
-bool block_ok(uint32_t b) { return b >= 128 && b <= (uint32_t)stq::kMaxBlock && (b & (b - 1)) == 0; }
+bool block_ok(uint32_t b) { return b >= (uint32_t)stq::kMinBlock && b <= (uint32_t)stq::kMaxBlock && (b & (b - 1)) == 0; }
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 int fail_cuda(stq_handle* h, cudaError_t e) {
@@ -262,7 +262,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     // (a tensor whose widths change inside the step takes the main kernel's runtime-width body)
     const bool fast_ok = kind == kKindStep && !wide &&
                          t.numel < (1ull << 32) && aligned(t.m_scales_in, 16) && aligned(t.v_scales_in, 16) &&
-                         t.block <= (uint32_t)stq::kFastMaxBlock;
+                         t.block >= 128 && t.block <= (uint32_t)stq::kFastMaxBlock;   // (one or two rows of a warp)
     const uint64_t nf = fast_ok ? t.numel / stq::kTile : 0;
     nfast[l] = (uint32_t)nf;
     nslow[l] = (uint32_t)(nt - nf);
@@ -938,7 +938,7 @@ const char* stq_strerror(int code) {
     case STQ_OK: return "ok";
     case STQ_E_NULL: return "a required pointer is NULL";
     case STQ_E_BITS: return "bit-width not in {2,3,4,8,16,32}";
-    case STQ_E_BLOCK: return "block not in {128,256,512}";
+    case STQ_E_BLOCK: return "block is not a power of two in 32..1024";
     case STQ_E_ALIGN: return "buffer not aligned (16 bytes for param/grad/codes, 4 for scales)";
     case STQ_E_ALIAS: return "in/out buffers overlap (in-place needs the same pointer and width)";
     case STQ_E_NUMEL: return "numel is 0, or the table is empty or too large";

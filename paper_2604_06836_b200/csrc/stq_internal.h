@@ -9,7 +9,8 @@ constexpr int kThreads = 256;    // 8 warps per CTA
 constexpr int kRowElems = 128;   // one row: lane l holds elements 4l .. 4l+3
 constexpr int kRowsPerWarp = 4;  // a warp owns this many consecutive rows of a tile
 constexpr int kTile = (kThreads / 32) * kRowsPerWarp * kRowElems;   // elements per tile; a tile lies inside one tensor
-constexpr int kMaxBlock = kRowsPerWarp * kRowElems;                 // a quantization block never leaves its warp
+constexpr int kMinBlock = 32;                                       // a lane's four elements never straddle blocks
+constexpr int kMaxBlock = 2 * kRowsPerWarp * kRowElems;             // a quantization block spans at most two warps of a tile
 constexpr int kFastCtasPerSm = 2;   // resident CTAs per SM of the main step kernel
 constexpr int kFastStages = 2;      // depth of its shared-memory ring
 constexpr int kFastRowsPerPass = 2; // rows a warp handles per pass over its kRowsPerWarp rows (see the kernel)
@@ -33,7 +34,7 @@ struct TensorDesc {
   unsigned int tile0s;      // first tile of the rest (ragged tail, or the whole tensor if it is not fast)
   unsigned int nslow;
   unsigned int seg0;        // first statistics segment (kStatSegTiles tiles each) of this tensor
-  unsigned int block;       // 128 / 256 / 512
+  unsigned int block;       // power of two, 32 .. 1024
   unsigned char bm_in, bv_in, bm_out, bv_out;
   float wd;                 // fp32(lambda)
   unsigned int lp_dtype;    // 0: none, 1: bf16, 2: fp16

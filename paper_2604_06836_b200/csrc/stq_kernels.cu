@@ -403,16 +403,26 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
     if (sc.inv_scale != nullptr) grad_mul = __ldg(sc.inv_scale);
   }
 
+  // blocks of 1024 elements: maxima of neighbouring warps meet here (two buffers, used alternately: a warp
+  // that runs ahead is held by the next tile's barrier before it can overwrite what a slower one still reads)
+  __shared__ uint32_t xchg[2][2 * (kThreads / 32)];
+  int xchg_parity = 0;
+
   for (uint32_t tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
     const TensorDesc* __restrict__ T = table + __ldg(tile_map + tile);
     const unsigned long long numel = T->numel;
     const unsigned long long e_warp =
         (unsigned long long)(T->nfast + (tile - T->tile0s)) * kTile + (unsigned)warp * (R * kRowElems);
     float st_g = 0.f, st_a = 0.f, st_q = 0.f;
+    const bool wide_block = MODE != kStatsOnly && T->block == 1024u;
 
+    if (e_warp >= numel && wide_block) {     // nothing to do here, but the neighbour may wait for this warp
+      if (lane == 0) { xchg[xchg_parity][2 * warp] = 0u; xchg[xchg_parity][2 * warp + 1] = 0u; }
+      asm volatile("bar.sync 1, %0;" ::"r"(kThreads) : "memory");
+    }
     if (e_warp < numel) {
-      const uint32_t B = T->block;
-      const int lgB = B == 128 ? 7 : B == 256 ? 8 : 9;
+      const uint32_t B = T->block;              // a power of two, 32 .. 1024
+      const int lgB = 31 - __clz((int)B);
       const int bm_in = T->bm_in, bv_in = T->bv_in, bm_out = T->bm_out, bv_out = T->bv_out;
       const bool pl = T->v_pl != 0u;
 
@@ -452,10 +462,11 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
         const float* vs = T->vs_in;
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-          const unsigned long long e_row = e_warp + r * kRowElems;
-          const bool live = e_row < numel;
-          s_m_in[r] = (live && bm_in != 32) ? ms[e_row >> lgB] : 0.f;
-          s_v_in[r] = (live && bv_in != 32) ? vs[e_row >> lgB] : 0.f;
+          // (blocks of 32 or 64 elements: a row holds several, each lane reads the scale of its own)
+          const unsigned long long e_lane = e_warp + r * kRowElems + 4 * lane;
+          const bool live = e_lane < numel;
+          s_m_in[r] = (live && bm_in != 32) ? ms[e_lane >> lgB] : 0.f;
+          s_v_in[r] = (live && bv_in != 32) ? vs[e_lane >> lgB] : 0.f;
         }
       }
 
@@ -543,12 +554,15 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
 
         // ---- block maxima: lane max of 4, warp REDUX on the bit patterns, rows merged per block ----
         uint32_t mxm[R], mxv[R];
+        // lanes that share a block with this one: the whole warp, or 8 / 16 neighbours for blocks of 32 / 64
+        const unsigned seg_lanes = B >= 128 ? 32u : B / 4;
+        const unsigned seg_mask = B >= 128 ? kFull : ((1u << seg_lanes) - 1u) << (lane & ~(seg_lanes - 1u));
 #pragma unroll
         for (int r = 0; r < R; ++r) {
           const float am = fmaxf(fmaxf(fabsf(mt[r][0]), fabsf(mt[r][1])), fmaxf(fabsf(mt[r][2]), fabsf(mt[r][3])));
           const float av = fmaxf(fmaxf(vt[r][0], vt[r][1]), fmaxf(vt[r][2], vt[r][3]));
-          mxm[r] = __reduce_max_sync(kFull, __float_as_uint(am));
-          mxv[r] = __reduce_max_sync(kFull, __float_as_uint(av));
+          mxm[r] = __reduce_max_sync(seg_mask, __float_as_uint(am));
+          mxv[r] = __reduce_max_sync(seg_mask, __float_as_uint(av));
         }
         if (B >= 256) {
 #pragma unroll
@@ -561,6 +575,17 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
           const uint32_t a = max(mxm[0], mxm[R - 2]), b = max(mxv[0], mxv[R - 2]);
 #pragma unroll
           for (int r = 0; r < R; ++r) { mxm[r] = a; mxv[r] = b; }
+        }
+        if (B == 1024) {
+          // a block of 1024 spans this warp and its neighbour: the two exchange their maxima through shared
+          // memory.  Every warp of the CTA takes part in the barrier (the ones past the end of the tensor from
+          // the branch below), which the whole CTA reaches because the block size is a property of the tile.
+          uint32_t* slot = xchg[xchg_parity];
+          if (lane == 0) { slot[2 * warp] = mxm[0]; slot[2 * warp + 1] = mxv[0]; }
+          asm volatile("bar.sync 1, %0;" ::"r"(kThreads) : "memory");
+          const uint32_t pm = slot[2 * (warp ^ 1)], pv = slot[2 * (warp ^ 1) + 1];
+#pragma unroll
+          for (int r = 0; r < R; ++r) { mxm[r] = max(mxm[r], pm); mxv[r] = max(mxv[r], pv); }
         }
 
         // ---- quantize, pack, store; decode the new codes; update the parameters -------------------
@@ -603,7 +628,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
               mq[k] = __fmul_rn(s, __fmul_rn(__fadd_rn(t, -mg), lw.invq));
             }
             store_codes(mco, e_row, bm_out, lane, lim_mo, x, kMagicBits, nvl[r]);
-            if (lane == 0 && (e_row & (B - 1)) == 0) mso[e_row >> lgB] = s;
+            if (((e_row + 4 * lane) & (B - 1)) == 0 && e_row + 4 * lane < numel) mso[(e_row + 4 * lane) >> lgB] = s;
           }
 
           // second moment, logarithmic
@@ -662,7 +687,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
               }
             }
             store_codes(vco, e_row, bv_out, lane, lim_vo, x, sub, nvl[r]);
-            if (lane == 0 && (e_row & (B - 1)) == 0) vso[e_row >> lgB] = s;
+            if (((e_row + 4 * lane) & (B - 1)) == 0 && e_row + 4 * lane < numel) vso[(e_row + 4 * lane) >> lgB] = s;
           }
 
           if constexpr (MODE == kStep) {
@@ -680,6 +705,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
       }
     }
 
+    if (wide_block) xchg_parity ^= 1;
     if constexpr (STATS || MODE == kStatsOnly) {
       // one partial per warp and tile; the finishing kernel adds them in a fixed order
       double dg = (double)st_g, da = (double)st_a, dq = (double)st_q;

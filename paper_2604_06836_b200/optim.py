@@ -52,8 +52,8 @@ class STQAdamW(torch.optim.Optimizer):
             raise ValueError("order is 'paper' or 'fused'")
         self.order = order
         self._carried_stats = None        # sums that rode on the last step (fused order), fetched right after it
-        if block not in (128, 256, 512):
-            raise ValueError("block is 128, 256 or 512")
+        if block not in (32, 64, 128, 256, 512, 1024):
+            raise ValueError("block is a power of two in 32..1024")
         defaults = dict(lr=lr, weight_decay=weight_decay)
         super().__init__(params, defaults)
         self.betas, self.eps = (float(betas[0]), float(betas[1])), float(eps)

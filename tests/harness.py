@@ -237,3 +237,108 @@ class SampledOracle:
                 idx = self._elem_index(i)
                 lp = job.params_lp[i]
                 assert torch.equal(lp[idx], job.params[i][idx].to(lp.dtype)), name + " working copy"
+
+
+class FullOracle:
+    """Oracle on EVERY element of a full-size Job.
+
+    Quantization blocks are independent given their inputs, so each tensor is cut into ranges that start
+    on block boundaries and the ranges are stepped by a pool of host threads (the oracle's C code runs
+    outside the interpreter lock).  The oracle's own state starts from its own zero initialisation and is
+    never fed from the CUDA path; only the seeded parameter and gradient draws are shared.  The comparison
+    covers whole buffers (every code byte, every scale, every parameter) and runs on the device to keep
+    the test short."""
+
+    def __init__(self, job: Job, range_elems: int = 1 << 21, threads: int | None = None):
+        import os
+        from concurrent.futures import ThreadPoolExecutor
+        self.job, self.w, self.block = job, job.w, job.block
+        assert range_elems % 1024 == 0
+        self.range_elems = range_elems
+        self.pool = ThreadPoolExecutor(max_workers=threads or os.cpu_count() or 4)
+        self.theta = [to_np(p) for p in job.params]
+        self.states = [O.new_state(n, self.block, int(bm), int(bv))
+                       for n, bm, bv in zip(job.numels, job.bits_m, job.bits_v)]
+        self.mag = [p.abs() for p in job.params]          # device: largest magnitude an element or its step has had
+        self.v_mode = O.LOG_PL if job.w.v_log == "pl" else O.LOG
+
+    def _ranges(self):
+        for i, n in enumerate(self.job.numels):
+            for e0 in range(0, n, self.range_elems):
+                yield i, e0, min(n, e0 + self.range_elems)
+
+    def step(self, t: int, new_bits=None, want_stats: bool = False) -> np.ndarray:
+        """One oracle step on the gradients the job currently holds.  Returns [L, 4] sums (zeros unless asked)."""
+        job, w = self.job, self.w
+        grads = [to_np(g) for g in job.grads]
+        out = []
+        for i, n in enumerate(job.numels):
+            bm = self.states[i].bits_m if new_bits is None else int(new_bits[0][i])
+            bv = self.states[i].bits_v if new_bits is None else int(new_bits[1][i])
+            mc, ms = O.alloc_state(n, bm, self.block)
+            vc, vs = O.alloc_state(n, bv, self.block)
+            out.append(O.State(mc, ms, bm, vc, vs, bv))
+        amp = dict(fp16_grad=True, inv_grad_scale=1.0 / w.loss_scale) if w.grad_dtype == "fp16" else {}
+        tasks = list(self._ranges())
+        part = np.zeros((len(tasks), 4))
+
+        def run(k):
+            i, e0, e1 = tasks[k]
+            O.step_range(self.theta[i], grads[i], e0, e1, self.block, self.states[i], out[i], lr=w.lr, beta1=w.beta1,
+                         beta2=w.beta2, eps=w.eps, weight_decay=job.wd[i], t=t, v_mode=self.v_mode,
+                         stats=part[k] if want_stats else None, **amp)
+
+        before = [torch.from_numpy(th).to(job.device) for th in self.theta]
+        list(self.pool.map(run, range(len(tasks))))
+        self.states = out
+        for i in range(job.L):
+            now = torch.from_numpy(self.theta[i]).to(job.device)
+            self.mag[i] = torch.maximum(self.mag[i], torch.maximum(now.abs(), (now - before[i]).abs()))
+        stats = np.zeros((job.L, 4))
+        for k, (i, _, _) in enumerate(tasks):
+            stats[i] += part[k]
+        return stats
+
+    def repack(self, new_bits):
+        def run(i):
+            st, n = self.states[i], self.job.numels[i]
+            bm, bv = int(new_bits[0][i]), int(new_bits[1][i])
+            if bm != st.bits_m:
+                st.m_codes, st.m_scales = O.repack(st.m_codes, st.m_scales, st.bits_m, bm, n, self.block, O.LINEAR)
+                st.bits_m = bm
+            if bv != st.bits_v:
+                st.v_codes, st.v_scales = O.repack(st.v_codes, st.v_scales, st.bits_v, bv, n, self.block, self.v_mode)
+                st.bits_v = bv
+        list(self.pool.map(run, range(self.job.L)))
+
+    def compare(self, rel: float, tag=""):
+        """Whole buffers: codes and scales byte for byte, parameters to rel * max(|b|, largest magnitude the
+        element or its step has had, 1e-3 * absmax of the tensor)."""
+        job = self.job
+        job.handle.device_status()
+        dev = job.device
+        for i in range(job.L):
+            gs, os_ = job.states[i], self.states[i]
+            name = f"{tag} tensor {i} ({job.w.shapes[i][0]}, bits {gs.bits_m}/{gs.bits_v})"
+            assert gs.bits_m == os_.bits_m and gs.bits_v == os_.bits_v, name
+            for what, g, o in (("m codes", gs.m_codes, os_.m_codes), ("v codes", gs.v_codes, os_.v_codes)):
+                o_d = torch.from_numpy(o).to(dev)
+                if not torch.equal(g, o_d):
+                    bad = torch.nonzero(g != o_d).flatten()[:8].tolist()
+                    raise AssertionError(f"{name}: {what} differ at bytes {bad}")
+            for what, g, o, b in (("m scales", gs.m_scales, os_.m_scales, gs.bits_m),
+                                  ("v scales", gs.v_scales, os_.v_scales, gs.bits_v)):
+                if b == 32:
+                    continue
+                o_d = torch.from_numpy(o).to(dev)
+                if not torch.equal(g.view(torch.int32), o_d.view(torch.int32)):
+                    bad = torch.nonzero(g.view(torch.int32) != o_d.view(torch.int32)).flatten()[:8].tolist()
+                    raise AssertionError(f"{name}: {what} differ at blocks {bad}")
+            o = torch.from_numpy(self.theta[i]).to(dev).double()
+            g = job.params[i].double()
+            lim = rel * torch.maximum(self.mag[i].double(), 1e-3 * o.abs().max())
+            err = (g - o).abs()
+            if not bool((err <= lim).all()):
+                k = int(torch.argmax(err / lim.clamp_min(1e-300)))
+                raise AssertionError(f"{name}: theta differs at {k}: gpu {float(g[k])!r} oracle {float(o[k])!r} "
+                                     f"err {float(err[k]):.3e} lim {float(lim[k]):.3e}")

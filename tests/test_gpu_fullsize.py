@@ -1,10 +1,13 @@
 """The benchmark configurations at full size, in the launch configuration bench.py times.
 
-The oracle cannot step 1.5e9 parameters in seconds, so it follows a sample of quantization blocks of
-every tensor (first, last, ragged tail, blocks next to tile boundaries, random ones): blocks are
-independent given their inputs, so the sampled blocks are checked exactly as the small cases are
-(codes and scales bit for bit, parameters to 1e-6 per step).  Statistics of tensors small enough are
-checked against the oracle, the large ones against a float64 library reduction.
+Two kinds of comparison.  Every element: the oracle, spread over the host cores range by range, steps the
+whole parameter list and every code byte, scale and parameter is compared (all steps of the two small
+configurations; the first three steps of the two large ones, all three decision steps with statistics).
+Sampled blocks: for the remaining steps of the large configurations, the fp16 workloads and the second
+variant of the v quantizer the oracle follows a sample of quantization blocks of every tensor (first, last,
+ragged tail, blocks next to tile boundaries, random ones); blocks are independent given their inputs, so
+they are checked exactly as the small cases are.  Statistics of tensors small enough are checked against the
+oracle, the large ones against a float64 library reduction.
 """
 import numpy as np
 import pytest
@@ -72,6 +75,40 @@ def test_full_size_sampled_blocks(name, gib):
     code_bytes = sum(s.m_codes.numel() + s.v_codes.numel() for s in job.states)
     assert bits / 8 <= code_bytes <= bits / 8 + 32 * job.L
     assert job.state_bytes() < 0.25 * 8 * w.total_params     # far below the fp32 states
+
+
+@pytest.mark.parametrize("name,gib,full_steps", [("cfg2", 8, None), ("cfg3", 6, None), ("cfg4", 30, 3), ("cfg5", 60, 3)])
+def test_full_size_every_element(name, gib, full_steps):
+    """Whole buffers against the oracle: every code byte, every scale, every parameter, on every step
+    run (all of them for cfg2 and cfg3; steps 1-3 for cfg4 and cfg5, which are decision steps with fused
+    statistics).  cfg3 changes the widths of 10 % of its tensors on every decision step from t = 5 on,
+    alternately by stq_repack and inside the step."""
+    import harness as H
+    _need(gib)
+    w = W.config(name)
+    bm, bv, _ = W.draw_bits(w)
+    job = Job(w, bm, bv)
+    fo = H.FullOracle(job)
+    fo.compare(0.0, f"{name} init")
+    decisions = 0
+    for t in range(1, (full_steps or w.steps) + 1):
+        job.draw_grads(t)
+        dec = t % w.decision_interval == 0 or t < 5
+        new_bits = None
+        if dec and w.churn > 0 and t >= 5:
+            nbm, nbv, _ = W.churn_bits(w, job.bits_m, job.bits_v, decisions)
+            decisions += 1
+            if decisions % 2 == 0:
+                new_bits = (nbm, nbv)
+            else:
+                job.repack((nbm, nbv))
+                fo.repack((nbm, nbv))
+        st_o = fo.step(t, new_bits=new_bits, want_stats=dec)
+        job.step(t, stats=dec, new_bits=new_bits)
+        fo.compare(1e-6 * t if t <= 10 else 1e-4, f"{name} t={t}")
+        if dec:
+            H.assert_stats_close(job.layer_stats(), st_o, f"{name} t={t}")
+    assert job.handle.launch_count > 0
 
 
 def test_errors_are_reported_before_anything_runs():

@@ -740,3 +740,59 @@ def test_pending_statistics_are_dropped_when_the_table_changes(H, O):
     job.step(4, stats=True)                       # and the next request works as usual
     want = np.stack([O.grad_stats(H.to_np(g)) for g in job.grads])
     H.assert_stats_close(job.layer_stats(), want, "after the drop")
+
+
+@pytest.mark.parametrize("block", [32, 64, 512, 1024])
+@pytest.mark.parametrize("bits", [(4, 4), (3, 8), (8, 2), (16, 3), (2, 16), (32, 4), (8, 32)])
+def test_blocks_from_32_to_1024(H, O, block, bits):
+    """The block sizes that the generic kernel serves: a row of 128 elements holds four or two blocks (32, 64),
+    or a block spans a whole warp (512) or two neighbouring warps (1024), including ragged last blocks that
+    end inside a lane group, a width change inside a step and a re-pack."""
+    import oracle
+    for n, gdt, v_log in ((4096 * 2 + 1024 + 333, "fp32", "poly"), (4096 + 37, "bf16", "pl"), (29, "bf16", "poly"),
+                          (1024 * 3, "fp32", "poly")):
+        if v_log == "pl" and 32 in bits:
+            continue
+        from dataclasses import replace
+        w = replace(_single(n, block, gdt, seed=block + n), v_log=v_log)
+        job = Job(w, [bits[0]], [bits[1]])
+        oj = H.OracleJob(job)
+        H.compare_job(job, oj, 0.0, f"B={block} n={n} init")
+        for t in (1, 2, 3):
+            job.draw_grads(t)
+            new_bits = ([8], [4]) if t == 3 else None          # step 3 writes other widths
+            st = oj.step([H.to_np(g) for g in job.grads], t, want_stats=True, new_bits=new_bits)
+            job.step(t, stats=True, new_bits=new_bits)
+            H.compare_job(job, oj, REL_1STEP * t, f"B={block} n={n} t={t}")
+            H.assert_stats_close(job.layer_stats(), st, f"B={block} n={n}")
+        job.repack(([bits[0]], [bits[1]]))
+        oj.repack(([bits[0]], [bits[1]]))
+        H.compare_job(job, oj, REL_1STEP * 3, f"B={block} n={n} repack")
+
+
+def test_blocks_of_every_size_in_one_table(H, O):
+    """One table whose tensors differ in block size cannot exist (the block is a property of the workload's
+    table rows, and each row carries its own): mix them and check every row against the oracle."""
+    import oracle
+    dev = "cuda"
+    sizes = [(4096 * 2 + 77, 32), (4096 + 512, 64), (4096 * 3, 128), (9000, 256), (4096 * 2 + 600, 512), (4096 * 2 + 1500, 1024)]
+    h = stq.Handle()
+    gen = torch.Generator(device=dev).manual_seed(11)
+    params = [torch.randn(n, device=dev, generator=gen) * 0.02 for n, _ in sizes]
+    states = [stq.alloc_state(n, b, 4, 8, dev) for n, b in sizes]
+    h.init_state(stq.table([stq.make_row(n, b, None, s) for (n, b), s in zip(sizes, states)]))
+    o_theta = [H.to_np(p) for p in params]
+    o_states = [oracle.new_state(n, b, 4, 8) for n, b in sizes]
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
+    for t in (1, 2, 3):
+        grads = [torch.randn(n, device=dev, generator=gen) * 1e-3 for n, _ in sizes]
+        h.step(stq.table([stq.make_row(n, b, s, s, p, g, 0.01) for (n, b), s, p, g in zip(sizes, states, params, grads)]),
+               t=t, flags=stq.WITH_STATS, **hp)
+        got = h.layer_stats(len(sizes))
+        for i, (n, b) in enumerate(sizes):
+            o_states[i], st = oracle.step(o_theta[i], H.to_np(grads[i]), o_states[i], b, weight_decay=0.01, t=t,
+                                          want_stats=True, **hp)
+            H.assert_states_equal(states[i], o_states[i], f"B={b} t={t}")
+            H.assert_theta_close(params[i], o_theta[i], REL_1STEP * t, f"B={b} t={t}", upd=np.abs(o_theta[i]) + 1e-3)
+            H.assert_stats_close(got[i:i + 1], st[None, :], f"B={b} t={t}")
+    h.close()

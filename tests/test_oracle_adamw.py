@@ -230,3 +230,33 @@ def test_loss_scale_and_skipped_step(O):
     before = th1.copy()
     st3, _ = O.step(th1, g, st1, 128, t=2, found_inf=True, **HP)
     assert (th1 == before).all() and st3 is st1
+
+
+@pytest.mark.parametrize("bits_m,bits_v,v_mode", [(4, 8, "log"), (3, 16, "pl"), (32, 4, "log"), (8, 32, "log"), (2, 2, "log")])
+def test_a_tensor_stepped_range_by_range_equals_the_tensor_stepped_whole(O, bits_m, bits_v, v_mode):
+    """Blocks are independent given their inputs: stepping block-aligned ranges one by one (as the full-size
+    GPU tests do, over a thread pool) writes the same bytes as one call over the tensor, ragged tail included."""
+    rng = np.random.RandomState(7)
+    n, block = 128 * 37 + 55, 128
+    vm = O.LOG_PL if v_mode == "pl" else O.LOG
+    th = (rng.randn(n) * 0.02).astype(np.float32)
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    whole_t, parts_t = th.copy(), th.copy()
+    whole = parts = O.new_state(n, block, bits_m, bits_v)
+    for t in (1, 2, 3):
+        g = (rng.standard_t(4, n) * 1e-3).astype(np.float32)
+        whole, stats = O.step(whole_t, g, whole, block, t=t, want_stats=True, v_mode=vm, **hp)
+        mc, ms = O.alloc_state(n, bits_m, block)
+        vc, vs = O.alloc_state(n, bits_v, block)
+        nxt = O.State(mc, ms, bits_m, vc, vs, bits_v)
+        total = np.zeros(4)
+        for e0 in reversed(range(0, n, block * 10)):          # any order
+            s4 = np.zeros(4)
+            O.step_range(parts_t, g, e0, min(n, e0 + block * 10), block, parts, nxt, t=t, v_mode=vm, stats=s4, **hp)
+            total += s4
+        parts = nxt
+        assert (whole_t == parts_t).all()
+        assert (whole.m_codes == parts.m_codes).all() and (whole.v_codes == parts.v_codes).all()
+        assert (whole.m_scales.view(np.uint32) == parts.m_scales.view(np.uint32)).all()
+        assert (whole.v_scales.view(np.uint32) == parts.v_scales.view(np.uint32)).all()
+        np.testing.assert_allclose(total, stats, rtol=1e-12)
