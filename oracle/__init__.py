@@ -34,7 +34,8 @@ class HParams(C.Structure):
     _fields_ = [("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
                 ("weight_decay", C.c_double), ("step", C.c_int64), ("decoupled_wd", C.c_int),
                 ("grad_dtype", C.c_int), ("inv_grad_scale", C.c_float), ("found_inf", C.c_int),
-                ("v_mode", C.c_int)]
+                ("v_mode", C.c_int), ("sr_seed", C.c_uint64), ("tensor_index", C.c_uint32),
+                ("elem_offset", C.c_uint64)]
 
 
 class Policy(C.Structure):
@@ -56,6 +57,22 @@ def lib():
         L.orc_codes_bytes.argtypes = [C.c_uint64, C.c_int]
         L.orc_num_blocks.restype = C.c_uint64
         L.orc_num_blocks.argtypes = [C.c_uint64, C.c_uint32]
+        L.orc_num_scales.restype = C.c_uint64
+        L.orc_num_scales.argtypes = [C.c_uint64, C.c_uint32, C.c_int]
+        L.orc_mix32.restype = C.c_uint32
+        L.orc_mix32.argtypes = [C.c_uint32]
+        L.orc_sr_key.restype = C.c_uint32
+        L.orc_sr_key.argtypes = [C.c_uint64, C.c_uint64, C.c_uint32]
+        L.orc_sr_word.restype = C.c_uint32
+        L.orc_sr_word.argtypes = [C.c_uint32, C.c_uint64]
+        L.orc_sr_code.restype = C.c_uint32
+        L.orc_sr_code.argtypes = [C.c_float, C.c_float, C.c_int, C.c_uint32]
+        L.orc_sr_level.restype = C.c_float
+        L.orc_sr_level.argtypes = [C.c_uint32, C.c_int]
+        L.orc_sr_enumerate.restype = None
+        L.orc_sr_enumerate.argtypes = [C.c_float, C.c_float, C.c_int, C.c_void_p, C.c_void_p]
+        L.orc_quantize_keyed.argtypes = [C.c_void_p, C.c_uint64, C.c_int, C.c_uint32, C.c_int, C.c_uint32,
+                                         C.c_void_p, C.c_void_p]
         L.orc_lg_P.restype = C.c_float
         L.orc_lg_P.argtypes = [C.c_float]
         L.orc_lg_E.restype = C.c_int
@@ -87,6 +104,7 @@ def lib():
 
 
 LINEAR, LOG, LOG_PL = 0, 1, 2      # LOG_PL: the log quantizer with the piecewise-linear logarithm
+LOG_SR, LOG_TS = 3, 4              # LOG_SR: stochastic rounding (normalised piecewise-linear log); LOG_TS: two scales
 WIDTHS = (2, 3, 4, 8, 16, 32)
 
 
@@ -133,18 +151,55 @@ def unpack(buf: np.ndarray, n: int, bits: int) -> np.ndarray:
     return out
 
 
-def alloc_state(n: int, bits: int, block: int):
+def num_scales(n: int, block: int, mode: int) -> int:
+    """Stored fp32 scales of a state: one per block, two in the two-scale variant."""
+    return int(lib().orc_num_scales(n, block, mode))
+
+
+def alloc_state(n: int, bits: int, block: int, mode: int = LOG):
     """Zero-filled (codes, scales) buffers of the stored sizes."""
     return (np.zeros(codes_bytes(n, bits), dtype=np.uint8),
-            np.zeros(num_blocks(n, block) if bits != 32 else 0, dtype=np.float32))
+            np.zeros(num_scales(n, block, mode) if bits != 32 else 0, dtype=np.float32))
 
 
-def quantize(x: np.ndarray, bits: int, block: int, mode: int):
+def quantize(x: np.ndarray, bits: int, block: int, mode: int, key: int | None = None):
+    """key: the 32-bit key of the stochastic-rounding variant (None: it rounds to nearest)."""
     x = _chk(np.ascontiguousarray(x), np.float32)
-    codes, scales = alloc_state(x.size, bits, block)
-    rc = lib().orc_quantize(_p(x), x.size, bits, block, mode, _p(codes), _p(scales))
+    codes, scales = alloc_state(x.size, bits, block, mode)
+    if key is None:
+        rc = lib().orc_quantize(_p(x), x.size, bits, block, mode, _p(codes), _p(scales))
+    else:
+        rc = lib().orc_quantize_keyed(_p(x), x.size, bits, block, mode, key, _p(codes), _p(scales))
     assert rc == 0
     return codes, scales
+
+
+def mix32(h: int) -> int:
+    return int(lib().orc_mix32(h & 0xFFFFFFFF))
+
+
+def sr_key(seed: int, step: int, tensor: int) -> int:
+    return int(lib().orc_sr_key(seed, step, tensor))
+
+
+def sr_word(key: int, element: int) -> int:
+    return int(lib().orc_sr_word(key, element))
+
+
+def sr_code(x: float, s: float, bits: int, word: int) -> int:
+    return int(lib().orc_sr_code(float(np.float32(x)), float(np.float32(s)), bits, word))
+
+
+def sr_level(code: int, bits: int) -> float:
+    return float(lib().orc_sr_level(code, bits))
+
+
+def sr_enumerate(x: float, s: float, bits: int):
+    """Over all 2^32 random words: ((lower code, count), (upper code, count)) of element x in a block of maximum s."""
+    codes = np.zeros(2, dtype=np.uint32)
+    counts = np.zeros(2, dtype=np.uint64)
+    lib().orc_sr_enumerate(float(np.float32(x)), float(np.float32(s)), bits, _p(codes), _p(counts))
+    return (int(codes[0]), int(counts[0])), (int(codes[1]), int(counts[1]))
 
 
 def dequantize(codes: np.ndarray, scales: np.ndarray, n: int, bits: int, block: int, mode: int):
@@ -190,18 +245,22 @@ class State:
     bits_v: int
 
 
-def new_state(n: int, block: int, bits_m: int, bits_v: int) -> State:
+def new_state(n: int, block: int, bits_m: int, bits_v: int, v_mode: int = LOG) -> State:
     mc, ms, vc, vs = init_state(n, block, bits_m, bits_v)
+    if v_mode == LOG_TS and bits_v != 32:
+        vs = np.zeros(num_scales(n, block, LOG_TS), dtype=np.float32)     # zero state: both scales 0
     return State(mc, ms, bits_m, vc, vs, bits_v)
 
 
 def step(theta: np.ndarray, grad: np.ndarray, st: State, block: int, *, lr, beta1, beta2, eps,
          weight_decay, t: int, bits_m_out: int | None = None, bits_v_out: int | None = None,
          decoupled_wd: bool = True, want_stats: bool = False, fp16_grad: bool = False,
-         inv_grad_scale: float = 1.0, found_inf: bool = False, v_mode: int = LOG):
+         inv_grad_scale: float = 1.0, found_inf: bool = False, v_mode: int = LOG, sr_seed: int = 0,
+         tensor_index: int = 0):
     """One Algorithm-1 step on one tensor.  theta is updated in place; returns (new State, stats).
-    A uint16 grad holds bf16 bit patterns, or fp16 ones with fp16_grad=True.  v_mode: LOG or LOG_PL,
-    the quantizer of the second moment (the stored state must have been written with the same one)."""
+    A uint16 grad holds bf16 bit patterns, or fp16 ones with fp16_grad=True.  v_mode: LOG, LOG_PL, LOG_SR or
+    LOG_TS, the quantizer of the second moment (the stored state must have been written with the same one);
+    sr_seed and tensor_index key the random words of LOG_SR."""
     _chk(theta, np.float32)
     n = theta.size
     dt = _grad_dtype(grad, fp16_grad)
@@ -209,9 +268,9 @@ def step(theta: np.ndarray, grad: np.ndarray, st: State, block: int, *, lr, beta
     bm = st.bits_m if bits_m_out is None else bits_m_out
     bv = st.bits_v if bits_v_out is None else bits_v_out
     mc, ms = alloc_state(n, bm, block)
-    vc, vs = alloc_state(n, bv, block)
+    vc, vs = alloc_state(n, bv, block, v_mode)
     hp = HParams(lr, beta1, beta2, eps, weight_decay, t, 1 if decoupled_wd else 0, dt, inv_grad_scale,
-                 1 if found_inf else 0, v_mode)
+                 1 if found_inf else 0, v_mode, sr_seed, tensor_index, 0)
     stats = np.zeros(4, dtype=np.float64) if want_stats else None
     rc = lib().orc_step(_p(theta), _p(grad), n, block,
                         _p(st.m_codes), _p(st.m_scales), st.bits_m,
@@ -225,7 +284,8 @@ def step(theta: np.ndarray, grad: np.ndarray, st: State, block: int, *, lr, beta
 
 def step_range(theta: np.ndarray, grad: np.ndarray, e0: int, e1: int, block: int, st_in: State, st_out: State, *,
                lr, beta1, beta2, eps, weight_decay, t: int, decoupled_wd: bool = True, fp16_grad: bool = False,
-               inv_grad_scale: float = 1.0, v_mode: int = LOG, stats: np.ndarray | None = None) -> None:
+               inv_grad_scale: float = 1.0, v_mode: int = LOG, stats: np.ndarray | None = None, sr_seed: int = 0,
+               tensor_index: int = 0) -> None:
     """The same Algorithm-1 step on the elements [e0, e1) of one tensor, e0 a multiple of the block size (blocks
     are independent given their inputs, so a tensor may be stepped range by range, in any order or in
     parallel).  theta, grad and the buffers of st_in / st_out belong to the whole tensor; theta and st_out are
@@ -237,12 +297,14 @@ def step_range(theta: np.ndarray, grad: np.ndarray, e0: int, e1: int, block: int
     def cut(st: State):
         def codes(c, b):
             return c[e0 * 4:] if b == 32 else c[e0 * b // 8:]          # a block is a whole number of bytes
+        spb = 2 if v_mode == LOG_TS else 1
         return (codes(st.m_codes, st.bits_m), st.m_scales[e0 // block:] if st.bits_m != 32 else st.m_scales,
-                codes(st.v_codes, st.bits_v), st.v_scales[e0 // block:] if st.bits_v != 32 else st.v_scales)
+                codes(st.v_codes, st.bits_v), st.v_scales[spb * (e0 // block):] if st.bits_v != 32 else st.v_scales)
 
     mci, msi, vci, vsi = cut(st_in)
     mco, mso, vco, vso = cut(st_out)
-    hp = HParams(lr, beta1, beta2, eps, weight_decay, t, 1 if decoupled_wd else 0, dt, inv_grad_scale, 0, v_mode)
+    hp = HParams(lr, beta1, beta2, eps, weight_decay, t, 1 if decoupled_wd else 0, dt, inv_grad_scale, 0, v_mode,
+                 sr_seed, tensor_index, e0)
     rc = lib().orc_step(_p(theta[e0:]), _p(grad[e0:]), n, block, _p(mci), _p(msi), st_in.bits_m, _p(vci), _p(vsi),
                         st_in.bits_v, _p(mco), _p(mso), st_out.bits_m, _p(vco), _p(vso), st_out.bits_v,
                         C.byref(hp), _p(stats))
@@ -266,7 +328,7 @@ def widen_f16(bits: np.ndarray) -> np.ndarray:
 
 def repack(codes: np.ndarray, scales: np.ndarray, bits_in: int, bits_out: int, n: int, block: int,
            mode: int):
-    co, so = alloc_state(n, bits_out, block)
+    co, so = alloc_state(n, bits_out, block, mode)
     rc = lib().orc_repack(_p(codes), _p(scales), bits_in, _p(co), _p(so), bits_out, n, block, mode)
     assert rc == 0
     return co, so

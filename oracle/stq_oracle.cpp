@@ -147,6 +147,124 @@ inline int64_t pl_step(int b) {                                                 
   const int64_t K = K_of(b), D = pl_octaves(b);
   return (2 * (D << pl_shift(b)) + K) / (2 * K);
 }
+// Variant "sr" (mode 3; the third reading of "logarithmic": the piecewise-linear logarithm of x/s with
+// STOCHASTIC rounding, so that the stored second moment is an unbiased estimate of the one computed).
+// The level grid has a whole number of levels per octave, L = 1, 1, 1, 8, 2048 at widths 2, 3, 4, 8, 16
+// (g = log2 L = 0, 0, 0, 3, 11), so every power of two below the maximum is a level and the code covers
+// K / L octaves (3, 7, 15, 31.875, 32.0).
+//  * c1 = fl(fl(1/s) * (1 + 2^-21)); y = fl(x * c1): the block maximum lands at or just above 1, never below.
+//  * n = clamp(bits(1.0) - bits(y), 0, K << (23 - g)): distance below the maximum in units of the bit
+//    pattern, i.e. -2^23 times the piecewise-linear log2 of y.
+//  * j = min(((n << (9 + g)) + U) >> 32, K), U the 32-bit random word of the element: j = floor(n * L / 2^23
+//    + U / 2^32), the lower neighbour with probability 1 - frac and the upper one with probability frac.
+//    Code q = K - j.
+//  * decode: y^ = the float with bits(1.0) - (j << (23 - g)); x^ = fl(s * y^).
+// Between two neighbouring levels there is no power of two, so the bit pattern is linear in y there and
+// E[y^] = y EXACTLY, at every width (tests: exact enumeration over all 2^32 words, in rationals).
+// Re-quantizing a decoded state is not the identity under random words (a level re-rounds to itself only
+// when its y lands exactly on it): idempotence is given up for unbiasedness.
+//
+// The random word is a counter-based generator, keyed on (seed, step, tensor, element) and specified to
+// the bit: mix32(h): h ^= h >> 16; h *= 0x85EBCA6B; h ^= h >> 13; h *= 0xC2B2AE35; h ^= h >> 16 (every
+// step is invertible, so mix32 is a bijection of the 32-bit words);
+// key = mix32(seed_lo ^ mix32(seed_hi ^ mix32(step_lo ^ mix32(step_hi ^ mix32(tensor ^ 0x9E3779B9)))));
+// U(element e) = mix32(e_lo ^ mix32(key + e_hi)).  For a fixed key, e_lo -> U is a bijection: over any
+// 2^32 consecutive elements every word occurs exactly once.
+const float kOnePlus = 0x1.000008p+0f;      // 1 + 2^-21
+inline uint32_t mix32(uint32_t h) {
+  h ^= h >> 16; h *= 0x85EBCA6Bu; h ^= h >> 13; h *= 0xC2B2AE35u; h ^= h >> 16;
+  return h;
+}
+inline uint32_t sr_key(uint64_t seed, uint64_t step, uint32_t tensor) {
+  uint32_t k = mix32(tensor ^ 0x9E3779B9u);
+  k = mix32((uint32_t)(step >> 32) ^ k);
+  k = mix32((uint32_t)step ^ k);
+  k = mix32((uint32_t)(seed >> 32) ^ k);
+  k = mix32((uint32_t)seed ^ k);
+  return k;
+}
+inline uint32_t sr_word(uint32_t key, uint64_t e) {
+  return mix32((uint32_t)e ^ mix32(key + (uint32_t)(e >> 32)));
+}
+inline int sr_lg_levels(int b) { return b == 8 ? 3 : b == 16 ? 11 : 0; }      // g
+inline uint32_t sr_code(float x, float s, int b, uint32_t U) {
+  const int64_t K = K_of(b);
+  const int g = sr_lg_levels(b);
+  const float rs = 1.0f / s;
+  const float c1 = rs * kOnePlus;
+  const float y = x * c1;
+  int64_t n = (int64_t)0x3F800000 - (int64_t)f2u(y);
+  if (n < 0) n = 0;
+  if (n > (K << (23 - g))) n = K << (23 - g);
+  int64_t j = ((n << (9 + g)) + (int64_t)U) >> 32;
+  if (j > K) j = K;
+  return (uint32_t)(K - j);
+}
+inline float sr_level(uint32_t code, int b) {      // y^ of a code
+  const int64_t j = (int64_t)K_of(b) - (int64_t)code;
+  return u2f((uint32_t)((int64_t)0x3F800000 - (j << (23 - sr_lg_levels(b)))));
+}
+
+// Variant "ts" (mode 4; two scales per block): the codes are spread evenly, in the logarithm, between the
+// block's own minimum and maximum instead of over a fixed number of octaves below the maximum.
+//  * stored scales (two per block): hi = max x, lo = max(min x, fl(hi * 2^-30)) (at most 30 octaves; a
+//    zero or denormal element is coded at the floor, never as zero).
+//  * d(x) = fl( float(E_x - E_hi) + fl(P(x) - P(hi)) ), the split logarithm of x/hi as in the main code;
+//    W = min(-d(lo), 30); inv = fl(K / W); q = clamp(K + round-half-even(d(x) * inv), 0, K) on the exact
+//    product.  W = 0 (all elements equal): every code is K.
+//  * decode: code 0 is lo exactly; otherwise x^ = fl(hi * ex(fl(float(q - K) * fl(W / K)))), so code K is
+//    hi exactly.  |log2(x^/x)| <= W/(2K) for lo <= x <= hi (plus the ~4e-6 octaves of the polynomials).
+struct TsBlock { float hi, lo, W; int Ehi; float Phi; };
+inline float ts_dist(const TsBlock& t, float x) {
+  float de = (float)(lg_E(x) - t.Ehi);
+  float dp = lg_P(x) - t.Phi;
+  return de + dp;
+}
+inline TsBlock ts_block(float hi, float lo) {
+  TsBlock t;
+  t.hi = hi; t.lo = lo; t.Ehi = lg_E(hi); t.Phi = lg_P(hi);
+  float W = -ts_dist(t, lo);
+  if (W > 30.0f) W = 30.0f;
+  if (!(W > 0.0f)) W = 0.0f;
+  t.W = W;
+  return t;
+}
+void quant_ts_block(const float* x, uint64_t n, int b, uint32_t* code, float* scale2) {
+  float hi = 0.0f;
+  for (uint64_t i = 0; i < n; ++i) if (x[i] > hi) hi = x[i];
+  if (hi < kTinyScale) {
+    scale2[0] = 0.0f; scale2[1] = 0.0f;
+    for (uint64_t i = 0; i < n; ++i) code[i] = 0u;
+    return;
+  }
+  float lo = hi;
+  for (uint64_t i = 0; i < n; ++i) if (x[i] < lo) lo = x[i];
+  const float floor_level = hi * 0x1p-30f;
+  if (lo < floor_level) lo = floor_level;
+  scale2[0] = hi; scale2[1] = lo;
+  const int K = K_of(b);
+  const TsBlock t = ts_block(hi, lo);
+  if (t.W == 0.0f) { for (uint64_t i = 0; i < n; ++i) code[i] = (uint32_t)K; return; }
+  const float inv = (float)K / t.W;
+  for (uint64_t i = 0; i < n; ++i) {
+    float d = ts_dist(t, x[i]);
+    double r = nearbyint((double)d * (double)inv);
+    double q = (double)K + r;
+    if (q < 0) q = 0;
+    if (q > K) q = K;
+    code[i] = (uint32_t)q;
+  }
+}
+inline float dequant_ts(uint32_t code, const TsBlock& t, int b) {
+  if (t.hi == 0.0f) return 0.0f;
+  if (code == 0u) return t.lo;
+  const int K = K_of(b);
+  float step = t.W / (float)K;
+  float e = (float)((int)code - K) * step;
+  float y = ex2(e);
+  return t.hi * y;
+}
+
 void quant_log_block(const float* x, uint64_t n, int b, uint32_t* code, float* scale, bool pl) {
   float s = 0.0f;
   for (uint64_t i = 0; i < n; ++i) if (x[i] > s) s = x[i];
@@ -213,23 +331,48 @@ inline float dequant_log(uint32_t code, float s, int b, bool pl) {
 // ---- state (de)coding over a whole range ------------------------------------------------------
 // mode 0 = linear (m), 1 = log (v), 2 = log with the piecewise-linear logarithm (v, variant "pl").
 // Width 32 stores raw fp32 and no scales.
+// mode 0 = linear (m), 1 = log (v), 2 = log with the piecewise-linear logarithm (v, variant "pl"),
+// 3 = variant "sr" (stochastic rounding; `key` selects the random words), 4 = variant "ts" (two scales per
+// block: scales[2k] = hi, scales[2k+1] = lo).  Width 32 stores raw fp32 and no scales.
+inline uint64_t scales_per_block(int mode) { return mode == 4 ? 2 : 1; }
 void decode_state(const uint8_t* codes, const float* scales, uint64_t n, int b, uint32_t block,
                   int mode, float* out) {
   if (b == 32) { std::memcpy(out, codes, n * 4); return; }
+  TsBlock ts{};
   for (uint64_t i = 0; i < n; ++i) {
     uint32_t c = get_code(codes, i, b);
+    if (mode == 4) {
+      if (i % block == 0) ts = ts_block(scales[2 * (i / block)], scales[2 * (i / block) + 1]);
+      out[i] = dequant_ts(c, ts, b);
+      continue;
+    }
     float s = scales[i / block];
-    out[i] = mode == 0 ? dequant_lin(c, s, b) : dequant_log(c, s, b, mode == 2);
+    if (mode == 0) out[i] = dequant_lin(c, s, b);
+    else if (mode == 3) { float lv = sr_level(c, b); out[i] = s * lv; }
+    else out[i] = dequant_log(c, s, b, mode == 2);
   }
 }
+// key (variant "sr"): selects the random words, which belong to the elements' positions e0 + i in their
+// tensor; without a key (a re-pack has no step to draw from) every word is 2^31, i.e. rounding to nearest.
 void encode_state(const float* x, uint64_t n, int b, uint32_t block, int mode, uint8_t* codes,
-                  float* scales) {
+                  float* scales, const uint32_t* key = nullptr, uint64_t e0 = 0) {
   if (b == 32) { std::memcpy(codes, x, n * 4); return; }
   std::memset(codes, 0, codes_bytes(n, b));
   std::vector<uint32_t> tmp(block);
   for (uint64_t j = 0, k = 0; j < n; j += block, ++k) {
     uint64_t len = n - j < block ? n - j : block;
     if (mode == 0) quant_lin_block(x + j, len, b, tmp.data(), scales + k);
+    else if (mode == 4) quant_ts_block(x + j, len, b, tmp.data(), scales + 2 * k);
+    else if (mode == 3) {
+      float s = 0.0f;
+      for (uint64_t i = 0; i < len; ++i) if (x[j + i] > s) s = x[j + i];
+      if (s < kTinyScale) { scales[k] = 0.0f; for (uint64_t i = 0; i < len; ++i) tmp[i] = 0u; }
+      else {
+        scales[k] = s;
+        for (uint64_t i = 0; i < len; ++i)
+          tmp[i] = sr_code(x[j + i], s, b, key ? sr_word(*key, e0 + j + i) : 0x80000000u);
+      }
+    }
     else quant_log_block(x + j, len, b, tmp.data(), scales + k, mode == 2);
     for (uint64_t i = 0; i < len; ++i) put_code(codes, j + i, b, tmp[i]);
   }
@@ -286,11 +429,33 @@ struct orc_hparams {
   int grad_dtype;      // 0 = fp32, 1 = bf16, 2 = fp16
   float inv_grad_scale;  // loss-scaled training: every gradient is multiplied by this first (1 = off)
   int found_inf;         // non-zero: a non-finite gradient was found, the step is skipped
-  int v_mode;            // quantizer of the second moment: 1 = log, 2 = its "pl" variant
+  int v_mode;            // quantizer of the second moment: 1 = log, 2 = "pl", 3 = "sr", 4 = "ts"
+  uint64_t sr_seed;      // variant "sr": the caller's seed ...
+  uint32_t tensor_index; // ... and the index of this tensor in the caller's list (the step is `step`);
+  uint64_t elem_offset;  // index of the range's first element inside its tensor (the random words are per element)
 };
 
 uint64_t orc_codes_bytes(uint64_t n, int bits) { return codes_bytes(n, bits); }
 uint64_t orc_num_blocks(uint64_t n, uint32_t block) { return (n + block - 1) / block; }
+uint64_t orc_num_scales(uint64_t n, uint32_t block, int mode) { return (n + block - 1) / block * scales_per_block(mode); }
+
+// Test hooks of variant "sr": the generator and the rounding of one element given its random word.
+uint32_t orc_mix32(uint32_t h) { return mix32(h); }
+uint32_t orc_sr_key(uint64_t seed, uint64_t step, uint32_t tensor) { return sr_key(seed, step, tensor); }
+uint32_t orc_sr_word(uint32_t key, uint64_t e) { return sr_word(key, e); }
+uint32_t orc_sr_code(float x, float s, int bits, uint32_t U) { return sr_code(x, s, bits, U); }
+float orc_sr_level(uint32_t code, int bits) { return sr_level(code, bits); }
+// Exact enumeration: over ALL 2^32 random words, how often each code occurs for the element x of a block
+// with maximum s (at most two neighbouring codes occur).  counts[0] goes with codes[0] (the smaller code).
+void orc_sr_enumerate(float x, float s, int bits, uint32_t codes[2], uint64_t counts[2]) {
+  codes[0] = sr_code(x, s, bits, 0xFFFFFFFFu);      // largest word: the lower level (larger j, smaller code)
+  codes[1] = sr_code(x, s, bits, 0u);
+  counts[0] = counts[1] = 0;
+  for (uint64_t U = 0; U < ((uint64_t)1 << 32); ++U) {
+    uint32_t c = sr_code(x, s, bits, (uint32_t)U);
+    if (c == codes[1]) ++counts[1]; else if (c == codes[0]) ++counts[0]; else { counts[0] = counts[1] = ~(uint64_t)0; return; }
+  }
+}
 
 float orc_lg_P(float x) { return lg_P(x); }
 int orc_lg_E(float x) { return lg_E(x); }
@@ -309,6 +474,13 @@ int orc_quantize(const float* x, uint64_t n, int bits, uint32_t block, int mode,
                  float* scales) {
   if (!width_ok(bits) || block == 0) return -1;
   encode_state(x, n, bits, block, mode, codes, scales);
+  return 0;
+}
+// The same with the key of variant "sr" (mode 3) given.
+int orc_quantize_keyed(const float* x, uint64_t n, int bits, uint32_t block, int mode, uint32_t key, uint8_t* codes,
+                       float* scales) {
+  if (!width_ok(bits) || block == 0) return -1;
+  encode_state(x, n, bits, block, mode, codes, scales, &key);
   return 0;
 }
 int orc_dequantize(const uint8_t* codes, const float* scales, uint64_t n, int bits, uint32_t block,
@@ -350,7 +522,8 @@ int orc_step(float* theta, const void* grad, uint64_t n, uint32_t block,
   if (!width_ok(bits_m_in) || !width_ok(bits_v_in) || !width_ok(bits_m_out) || !width_ok(bits_v_out))
     return -1;
   if (block == 0 || hp->step < 1) return -1;
-  if (hp->v_mode != 1 && hp->v_mode != 2) return -1;
+  if (hp->v_mode < 1 || hp->v_mode > 4) return -1;
+  if (hp->v_mode == 3 && hp->elem_offset % block != 0) return -1;
   const int vmode = hp->v_mode;
   if (hp->found_inf) return 0;          // skipped step: nothing is touched
   std::vector<float> m(n), v(n), g(n);
@@ -382,7 +555,14 @@ int orc_step(float* theta, const void* grad, uint64_t n, uint32_t block,
 
   // Quantize(m_t, linear), Quantize(v_t, log) at the widths assigned for this step
   encode_state(m.data(), n, bits_m_out, block, 0, m_codes_out, m_scales_out);
-  encode_state(v.data(), n, bits_v_out, block, vmode, v_codes_out, v_scales_out);
+  if (vmode == 3) {
+    // the random words are those of the elements' positions in their tensor: a range is coded as the
+    // elements [elem_offset, elem_offset + n) of the tensor it belongs to
+    const uint32_t key = sr_key(hp->sr_seed, (uint64_t)hp->step, hp->tensor_index);
+    encode_state(v.data(), n, bits_v_out, block, vmode, v_codes_out, v_scales_out, &key, hp->elem_offset);
+  } else {
+    encode_state(v.data(), n, bits_v_out, block, vmode, v_codes_out, v_scales_out);
+  }
 
   // the update consumes the quantized states
   decode_state(m_codes_out, m_scales_out, n, bits_m_out, block, 0, m.data());

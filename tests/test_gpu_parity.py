@@ -333,7 +333,10 @@ def test_non_finite_gradients_do_not_fault_or_leak_into_other_blocks(H, O):
 def test_element_ranges_of_a_tensor_step_like_the_whole_tensor(H, O, bits):
     """A sharded optimizer hands each rank ranges of a tensor cut on tile boundaries: stepping the
     ranges as rows of their own (here: two handles, one after the other) writes the same bits as
-    stepping the whole tensor, and the per-layer sums of the ranges add up to the tensor's."""
+    stepping the whole tensor, and the per-layer sums of the ranges add up to the tensor's.  Each
+    rank's range is also held against the oracle's run of exactly that range (its own parameters,
+    gradients and zero-initialised state), codes and scales bit for bit."""
+    import oracle
     from paper_2604_06836_b200 import multi, stq
     bm, bv = bits
     n, block, dev = 5 * 4096 + 777, 128, "cuda"
@@ -353,6 +356,8 @@ def test_element_ranges_of_a_tensor_step_like_the_whole_tensor(H, O, bits):
     h_whole.init_state(stq.table([stq.make_row(n, block, None, whole_s)]))
     for h, (_, lo, hi) in zip((h_a, h_b), cuts):
         h.init_state(stq.table([stq.make_row(hi - lo, block, None, view(split_s, lo, hi))]))
+    o_theta = [H.to_np(theta[lo:hi]) for _, lo, hi in cuts]                     # the oracle's ranks
+    o_state = [oracle.new_state(hi - lo, block, bm, bv) for _, lo, hi in cuts]
     for t in (1, 2, 3):
         g = (torch.empty(n, device=dev).normal_(0, 1e-3, generator=g0)).to(torch.bfloat16)
         h_whole.step(stq.table([stq.make_row(n, block, whole_s, whole_s, whole_p, g, 0.01)]), t=t,
@@ -362,7 +367,17 @@ def test_element_ranges_of_a_tensor_step_like_the_whole_tensor(H, O, bits):
             v = view(split_s, lo, hi)
             h.step(stq.table([stq.make_row(hi - lo, block, v, v, split_p[lo:hi], g[lo:hi], 0.01)]), t=t,
                    flags=stq.WITH_STATS, **hp)
-            total += h.layer_stats(1)[0]
+            got = h.layer_stats(1)
+            total += got[0]
+            k = 0 if lo == 0 else 1
+            o_state[k], st_o = oracle.step(o_theta[k], H.to_np(g[lo:hi]), o_state[k], block, lr=1e-3, beta1=0.9,
+                                           beta2=0.999, eps=1e-8, weight_decay=0.01, t=t, want_stats=True)
+            mine = stq.QState(v.m_codes[:o_state[k].m_codes.size], v.m_scales[:o_state[k].m_scales.size], bm,
+                              v.v_codes[:o_state[k].v_codes.size], v.v_scales[:o_state[k].v_scales.size], bv)
+            H.assert_states_equal(mine, o_state[k], f"rank {k} t={t}")
+            H.assert_theta_close(split_p[lo:hi], o_theta[k], REL_1STEP * t, f"rank {k} t={t}",
+                                 upd=np.abs(o_theta[k]) + 2e-3)
+            H.assert_stats_close(got, st_o[None, :], f"rank {k} t={t}")
         want = h_whole.layer_stats(1)[0]
         assert torch.equal(whole_p, split_p)
         for a, b in ((whole_s.m_codes, split_s.m_codes), (whole_s.v_codes, split_s.v_codes),

@@ -232,22 +232,23 @@ def test_loss_scale_and_skipped_step(O):
     assert (th1 == before).all() and st3 is st1
 
 
-@pytest.mark.parametrize("bits_m,bits_v,v_mode", [(4, 8, "log"), (3, 16, "pl"), (32, 4, "log"), (8, 32, "log"), (2, 2, "log")])
+@pytest.mark.parametrize("bits_m,bits_v,v_mode", [(4, 8, "log"), (3, 16, "pl"), (32, 4, "log"), (8, 32, "log"), (2, 2, "log"),
+                                                  (4, 4, "sr"), (8, 16, "sr"), (4, 3, "ts"), (16, 8, "ts")])
 def test_a_tensor_stepped_range_by_range_equals_the_tensor_stepped_whole(O, bits_m, bits_v, v_mode):
     """Blocks are independent given their inputs: stepping block-aligned ranges one by one (as the full-size
     GPU tests do, over a thread pool) writes the same bytes as one call over the tensor, ragged tail included."""
     rng = np.random.RandomState(7)
     n, block = 128 * 37 + 55, 128
-    vm = O.LOG_PL if v_mode == "pl" else O.LOG
+    vm = {"pl": O.LOG_PL, "sr": O.LOG_SR, "ts": O.LOG_TS}.get(v_mode, O.LOG)
     th = (rng.randn(n) * 0.02).astype(np.float32)
-    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01, sr_seed=0xABCDEF0123, tensor_index=7)
     whole_t, parts_t = th.copy(), th.copy()
-    whole = parts = O.new_state(n, block, bits_m, bits_v)
+    whole = parts = O.new_state(n, block, bits_m, bits_v, vm)
     for t in (1, 2, 3):
         g = (rng.standard_t(4, n) * 1e-3).astype(np.float32)
         whole, stats = O.step(whole_t, g, whole, block, t=t, want_stats=True, v_mode=vm, **hp)
         mc, ms = O.alloc_state(n, bits_m, block)
-        vc, vs = O.alloc_state(n, bits_v, block)
+        vc, vs = O.alloc_state(n, bits_v, block, vm)
         nxt = O.State(mc, ms, bits_m, vc, vs, bits_v)
         total = np.zeros(4)
         for e0 in reversed(range(0, n, block * 10)):          # any order

@@ -69,6 +69,29 @@ MUTANTS = [
 ]
 
 
+# the two further readings of the logarithmic mode have their own pins (the 2^32-word enumerations are left
+# out of the mutant runs: the closed-form threshold test covers the same ground in a fraction of the time)
+VARIANT_PINS = ["tests/test_oracle_quantizer_variants.py", "tests/test_oracle_adamw.py", "-k", "not exact_enumeration"]
+VARIANT_MUTANTS = [
+    ("sr: scale nudge dropped, the maximum can fall below the top level", "const float c1 = rs * kOnePlus;", "const float c1 = rs;"),
+    ("sr: the random word is ignored (round to nearest)", "int64_t j = ((n << (9 + g)) + (int64_t)U) >> 32;",
+     "int64_t j = ((n << (9 + g)) + ((int64_t)1 << 31)) >> 32;"),
+    ("sr: level spacing off by a factor of two", "int64_t j = ((n << (9 + g)) + (int64_t)U) >> 32;",
+     "int64_t j = ((n << (8 + g)) + (int64_t)U) >> 32;"),
+    ("sr: decode with the wrong level spacing", "(j << (23 - sr_lg_levels(b)))", "(j << (22 - sr_lg_levels(b)))"),
+    ("sr: key ignores the tensor", "uint32_t k = mix32(tensor ^ 0x9E3779B9u);", "uint32_t k = mix32(0x9E3779B9u);"),
+    ("sr: words taken from the position in the block, not in the tensor", "sr_word(*key, e0 + j + i)", "sr_word(*key, i)"),
+    ("sr: a range forgets where it starts in its tensor", "sr_word(*key, e0 + j + i)", "sr_word(*key, j + i)"),
+    ("sr: a shift of the mixing function changed", "h ^= h >> 13;", "h ^= h >> 12;"),
+    ("ts: minimum not raised to the floor", "if (lo < floor_level) lo = floor_level;", ""),
+    ("ts: code 0 not the stored minimum", "if (code == 0u) return t.lo;", ""),
+    ("ts: K + 1 steps instead of K", "const float inv = (float)K / t.W;", "const float inv = (float)(K + 1) / t.W;"),
+    ("ts: both scales read from the first slot", "scales[2 * (i / block) + 1]", "scales[2 * (i / block)]"),
+    ("ts: distance taken without the exponent difference", "float de = (float)(lg_E(x) - t.Ehi);\n  float dp = lg_P(x) - t.Phi;\n  return de + dp;",
+     "float dp = lg_P(x) - t.Phi;\n  return dp;"),
+]
+
+
 def _build(tmp, idx, edits):
     import oracle
     src = open(SRC).read()
@@ -83,9 +106,9 @@ def _build(tmp, idx, edits):
     return so
 
 
-def _pins_fail(so):
+def _pins_fail(so, pins=None):
     env = dict(os.environ, STQ_ORACLE_LIB=so)
-    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider", *PIN_FILES],
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider", *(pins or PIN_FILES)],
                        cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
     return r.returncode != 0, r.stdout[-400:]
 
@@ -100,5 +123,16 @@ def test_every_planted_mistake_is_caught(tmp_path):
     libs = [(m[0], _build(str(tmp_path), i, m[1:])) for i, m in enumerate(MUTANTS)]
     with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
         results = list(ex.map(lambda nl: (nl[0], _pins_fail(nl[1])), libs))
+    survivors = [name for name, (failed, _) in results if not failed]
+    assert not survivors, "the pins do not notice: " + "; ".join(survivors)
+
+
+def test_every_planted_mistake_in_the_variants_is_caught(tmp_path):
+    ok = _build(str(tmp_path), "ok2", ())
+    failed, tail = _pins_fail(ok, VARIANT_PINS)
+    assert not failed, tail
+    libs = [(m[0], _build(str(tmp_path), f"v{i}", m[1:])) for i, m in enumerate(VARIANT_MUTANTS)]
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+        results = list(ex.map(lambda nl: (nl[0], _pins_fail(nl[1], VARIANT_PINS)), libs))
     survivors = [name for name, (failed, _) in results if not failed]
     assert not survivors, "the pins do not notice: " + "; ".join(survivors)

@@ -20,6 +20,8 @@ def _rows(name):
 def test_worked_examples(O):
     n_seen = 0
     for head, xs, codes, decoded in _rows("quant_worked_examples.txt"):
+        if head[0] == "ts":          # the two-scale lines are read by the pins of that variant
+            continue
         mode = O.LINEAR if head[0] == "lin" else O.LOG
         bits, scale = int(head[1]), float(head[2])
         x = np.array([float(v) for v in xs], dtype=np.float32)
