@@ -38,6 +38,23 @@
  *    B = round(D*2^S/K), S = 12 (8 bits) or 20 (16 bits).  Exact at whole octaves below the
  *    maximum; relative error at most 0.7214*30/K octaves.  A state must be read with the variant
  *    it was written with.
+ *  - second moment, variant STQ_VLOG_SR (a third reading: stochastic rounding, so that the stored
+ *    second moment is an unbiased estimate of the computed one).  Levels: a whole number L = 1, 1, 1,
+ *    8, 2048 per octave at widths 2, 3, 4, 8, 16 (g = log2 L), evenly spaced in the mantissa.  With
+ *    y = fl(x * fl(fl(1/s) * (1 + 2^-21))) and n = clamp(bits(1.0f) - bits(y), 0, K << (23-g)):
+ *    j = min(((n << (9+g)) + U) >> 32, K), code u = K - j, U the element's 32-bit random word;
+ *    code u decodes to fl(s * y^), y^ the float with bits(1.0f) - ((K-u) << (23-g)).  Over the random
+ *    words E[y^] = y exactly.  mix32(h): h ^= h>>16; h *= 0x85EBCA6B; h ^= h>>13; h *= 0xC2B2AE35;
+ *    h ^= h>>16.  h0 = mix32(seed_lo ^ mix32(seed_hi ^ mix32(step_lo ^ mix32(step_hi ^ 0x9E3779B9))))
+ *    with seed = stq_hparams.sr_seed and step = stq_hparams.step; key = mix32(stq_tensor.sr_id ^ h0);
+ *    U of element e of the row = mix32(e_lo ^ mix32(key + e_hi)).  stq_repack has no step to draw
+ *    from and rounds to nearest (U = 2^31).  Re-quantization is not idempotent in this variant.
+ *  - second moment, variant STQ_VLOG_TS (a fourth reading: two scales per block).  The scale buffer
+ *    holds two floats per block, {hi, lo}: hi = max x, lo = max(min x, hi * 2^-30); size
+ *    stq_v_scales_bytes().  With d(x) the split logarithm of x/hi as in the main code and
+ *    W = min(-d(lo), 30): u = clamp(K + rne(clamp(d(x), -W, 0) * fl(K/W)), 0, K); u = 0 decodes to
+ *    lo, otherwise fl(hi * ex(fl((u-K) * fl(W/K)))): both end points exact, error at most W/(2K)
+ *    octaves.  W = 0 (all elements equal): every code is K.
  */
 #ifndef STQ_H_
 #define STQ_H_
@@ -74,8 +91,9 @@ enum { STQ_GRAD_F32 = 0, STQ_GRAD_BF16 = 1, STQ_GRAD_F16 = 2 };
 /* type of the optional low-precision copy of the updated parameters (stq_tensor.param_lp) */
 enum { STQ_LP_NONE = 0, STQ_LP_BF16 = 1, STQ_LP_F16 = 2 };
 
-/* quantizer of the second moment at widths 8 and 16 (stq_tensor.v_log); see "Stored layout" */
-enum { STQ_VLOG_POLY = 0, STQ_VLOG_PL = 1 };
+/* quantizer of the second moment (stq_tensor.v_log); see "Stored layout".  POLY and PL differ at widths 8 and
+ * 16 only; SR and TS are codes of their own at every width and run in the generic kernel. */
+enum { STQ_VLOG_POLY = 0, STQ_VLOG_PL = 1, STQ_VLOG_SR = 2, STQ_VLOG_TS = 3 };
 
 /* flags of stq_step */
 enum { STQ_WITH_STATS = 1u };
@@ -103,9 +121,10 @@ typedef struct stq_tensor {
                              /* rounded (nearest-even) to lp_dtype, the model's working copy   */
                              /* in mixed-precision training; 8-byte aligned; written by         */
                              /* stq_step only                                                  */
-  uint32_t v_log;            /* STQ_VLOG_*: how the second moment is coded at widths 8 and 16,  */
-                             /* on the way in and on the way out (ignored at other widths)     */
-  uint32_t reserved;         /* must be 0                                                      */
+  uint32_t v_log;            /* STQ_VLOG_*: how the second moment is coded, on the way in and  */
+                             /* on the way out                                                 */
+  uint32_t sr_id;            /* STQ_VLOG_SR: identifies this tensor in the random stream (use   */
+                             /* its index in the model); 0 otherwise                           */
 } stq_tensor;
 
 typedef struct stq_hparams {
@@ -125,6 +144,8 @@ typedef struct stq_hparams {
   /* the captured t.  The bias corrections 1 - beta^t are formed on the device in double precision.     */
   const int64_t* step_dev;     /* device pointer to t >= 1 (values below 1 are read as 1)              */
   const float* lr_dev;         /* device pointer to the learning rate                                  */
+  uint64_t sr_seed;            /* seed of the random words of STQ_VLOG_SR tensors (with `step`; not     */
+                               /* available together with step_dev)                                    */
 } stq_hparams;
 
 /* Handle: device copy of the tensor table, tile map and statistics workspace.
@@ -136,6 +157,8 @@ int stq_destroy(stq_handle* h);
 /* Buffer sizes of the stored layout described above. */
 size_t stq_codes_bytes(uint64_t numel, int bits);
 size_t stq_scales_bytes(uint64_t numel, uint32_t block);
+/* Scale buffer of a second moment coded with variant v_log: two floats per block for STQ_VLOG_TS. */
+size_t stq_v_scales_bytes(uint64_t numel, uint32_t block, uint32_t v_log);
 
 /* Algorithm 1, initialisation: m = v = 0.  Writes the canonical zero state (first-moment codes
  * 2^(b-1), second-moment codes 0, all scales 0) into the *_out buffers at bits_m_out/bits_v_out.

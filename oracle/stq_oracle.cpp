@@ -167,8 +167,8 @@ inline int64_t pl_step(int b) {                                                 
 // The random word is a counter-based generator, keyed on (seed, step, tensor, element) and specified to
 // the bit: mix32(h): h ^= h >> 16; h *= 0x85EBCA6B; h ^= h >> 13; h *= 0xC2B2AE35; h ^= h >> 16 (every
 // step is invertible, so mix32 is a bijection of the 32-bit words);
-// key = mix32(seed_lo ^ mix32(seed_hi ^ mix32(step_lo ^ mix32(step_hi ^ mix32(tensor ^ 0x9E3779B9)))));
-// U(element e) = mix32(e_lo ^ mix32(key + e_hi)).  For a fixed key, e_lo -> U is a bijection: over any
+// h = mix32(seed_lo ^ mix32(seed_hi ^ mix32(step_lo ^ mix32(step_hi ^ 0x9E3779B9)))) (one word per step);
+// key = mix32(tensor ^ h); U(element e) = mix32(e_lo ^ mix32(key + e_hi)).  For a fixed key, e_lo -> U is a bijection: over any
 // 2^32 consecutive elements every word occurs exactly once.
 const float kOnePlus = 0x1.000008p+0f;      // 1 + 2^-21
 inline uint32_t mix32(uint32_t h) {
@@ -176,12 +176,11 @@ inline uint32_t mix32(uint32_t h) {
   return h;
 }
 inline uint32_t sr_key(uint64_t seed, uint64_t step, uint32_t tensor) {
-  uint32_t k = mix32(tensor ^ 0x9E3779B9u);
-  k = mix32((uint32_t)(step >> 32) ^ k);
-  k = mix32((uint32_t)step ^ k);
-  k = mix32((uint32_t)(seed >> 32) ^ k);
-  k = mix32((uint32_t)seed ^ k);
-  return k;
+  uint32_t h = mix32((uint32_t)(step >> 32) ^ 0x9E3779B9u);
+  h = mix32((uint32_t)step ^ h);
+  h = mix32((uint32_t)(seed >> 32) ^ h);
+  h = mix32((uint32_t)seed ^ h);
+  return mix32(tensor ^ h);
 }
 inline uint32_t sr_word(uint32_t key, uint64_t e) {
   return mix32((uint32_t)e ^ mix32(key + (uint32_t)(e >> 32)));

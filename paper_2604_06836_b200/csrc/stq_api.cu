@@ -36,6 +36,7 @@ struct stq_handle {
   uint32_t n_main = 0;                              // fast tiles of the fused bodies; [n_main, n_fast) change width
   int fast_grid = 0;
   bool any_lp = false;              // some tensor of the current table wants a low-precision copy
+  bool any_variant = false;         // some tensor's second moment uses a code only the generic kernel serves
   int* d_err = nullptr;         // [0] raised by a kernel whose bounded wait ran out; [1] non-zero if the last call
                                 // that carried statistics really produced them (a skipped step does not)
   float* d_scalars = nullptr;   // {step_size, rsqrt_bc2, lr} when the step count lives on the device
@@ -146,7 +147,8 @@ bool overlap(const void* a, size_t na, const void* b, size_t nb) {
 int validate_row(const stq_tensor& t, int kind) {
   if (t.numel == 0 || t.numel > (1ull << 40)) return STQ_E_NUMEL;
   if (t.lp_dtype > STQ_LP_F16) return STQ_E_ARG;
-  if (t.v_log > STQ_VLOG_PL || t.reserved != 0) return STQ_E_ARG;
+  if (t.v_log > STQ_VLOG_TS) return STQ_E_ARG;
+  if (t.v_log != STQ_VLOG_SR && t.sr_id != 0) return STQ_E_ARG;
   if (kind == kKindStep && t.lp_dtype != STQ_LP_NONE) {
     if (!t.param_lp) return STQ_E_NULL;
     if (!aligned(t.param_lp, 8)) return STQ_E_ALIGN;
@@ -187,12 +189,12 @@ int validate_row(const stq_tensor& t, int kind) {
   if (overlap(t.m_codes_out, mo, t.v_codes_out, vo) || overlap(t.m_codes_in, mi, t.v_codes_out, vo) ||
       overlap(t.v_codes_in, vi, t.m_codes_out, mo))
     return STQ_E_ALIAS;
-  const size_t sb = stq_scales_bytes(t.numel, t.block);
+  const size_t sb = stq_scales_bytes(t.numel, t.block), sbv = stq_v_scales_bytes(t.numel, t.block, t.v_log);
   if (t.bits_m != 32 && t.bits_m_out != 32 && t.m_scales_in != t.m_scales_out &&
       overlap(t.m_scales_in, sb, t.m_scales_out, sb))
     return STQ_E_ALIAS;
   if (t.bits_v != 32 && t.bits_v_out != 32 && t.v_scales_in != t.v_scales_out &&
-      overlap(t.v_scales_in, sb, t.v_scales_out, sb))
+      overlap(t.v_scales_in, sbv, t.v_scales_out, sbv))
     return STQ_E_ALIAS;
   return STQ_OK;
 }
@@ -260,7 +262,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     const bool wide = row_is_wide(t, kind);
     // (the main kernel moves the scales with 16-byte bulk copies as well)
     // (a tensor whose widths change inside the step takes the main kernel's runtime-width body)
-    const bool fast_ok = kind == kKindStep && !wide &&
+    const bool fast_ok = kind == kKindStep && !wide && t.v_log <= STQ_VLOG_PL &&
                          t.numel < (1ull << 32) && aligned(t.m_scales_in, 16) && aligned(t.v_scales_in, 16) &&
                          t.block >= 128 && t.block <= (uint32_t)stq::kFastMaxBlock;   // (one or two rows of a warp)
     const uint64_t nf = fast_ok ? t.numel / stq::kTile : 0;
@@ -271,7 +273,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     if (!wide) slow_narrow += nt - nf;
     sig[l] = t.numel | (wide ? 1ull << 63 : 0ull) | (fast_ok ? 1ull << 62 : 0ull) |
              ((uint64_t)t.bits_m << 56) | ((uint64_t)t.bits_v << 48) |
-             ((uint64_t)(t.v_log & 1u) << 47) |
+             ((uint64_t)(t.v_log & 1u) << 47) | ((uint64_t)(t.v_log >> 1) << 45) |
              ((uint64_t)(t.bits_m != t.bits_m_out || t.bits_v != t.bits_v_out) << 46);   // numel <= 2^40
   }
   if (total > 0xFFFFFFF0ull) return STQ_E_NUMEL;
@@ -413,7 +415,8 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     d.bm_in = t.bits_m; d.bv_in = t.bits_v; d.bm_out = t.bits_m_out; d.bv_out = t.bits_v_out;
     d.wd = t.weight_decay;
     d.lp_dtype = kind == kKindStep ? t.lp_dtype : 0u;
-    d.v_pl = kind != kKindStats && t.v_log == STQ_VLOG_PL ? 1u : 0u;
+    d.v_mode = kind != kKindStats ? t.v_log : 0u;
+    d.sr_id = t.sr_id;
     d.param_lp = kind == kKindStep && t.lp_dtype != STQ_LP_NONE ? t.param_lp : nullptr;
     ht[l] = d;
   }
@@ -430,6 +433,8 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   h->cached_kind = kind;
   h->cached_sig.swap(sig);
   h->any_lp = false;
+  h->any_variant = false;
+  for (int l = 0; l < L; ++l) h->any_variant = h->any_variant || (kind != kKindStats && tensors[l].v_log >= STQ_VLOG_SR);
   for (int l = 0; l < L; ++l) h->any_lp = h->any_lp || (kind == kKindStep && tensors[l].lp_dtype != STQ_LP_NONE);
   h->n_tiles = (uint32_t)total;
   h->n_fast = (uint32_t)fast;
@@ -457,12 +462,12 @@ int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::St
     gs = h->side;
   }
   if (h->n_narrow > h->n_fast) {
-    STQ_CUDA(h, stq::launch_tiles(mode, false, grad_dtype, stats, h->d_table, h->d_tile_map, h->n_fast,
+    STQ_CUDA(h, stq::launch_tiles(mode, false, h->any_variant, grad_dtype, stats, h->d_table, h->d_tile_map, h->n_fast,
                                   h->n_narrow, sc, partials, h->grid, gs));
     h->launches++;
   }
   if (h->n_tiles > h->n_narrow) {
-    STQ_CUDA(h, stq::launch_tiles(mode, true, grad_dtype, stats, h->d_table, h->d_tile_map, h->n_narrow,
+    STQ_CUDA(h, stq::launch_tiles(mode, true, h->any_variant, grad_dtype, stats, h->d_table, h->d_tile_map, h->n_narrow,
                                   h->n_tiles, sc, partials, h->grid, gs));
     h->launches++;
   }
@@ -506,6 +511,14 @@ stq::StepConsts make_consts(const stq_hparams* hp) {
   sc.rsqrt_bc2 = (float)(1.0 / std::sqrt(bc2));
   sc.eps = (float)hp->eps;
   sc.one = 1.0f;
+  {   // stochastic rounding: the word every tensor's key is mixed from (seed and step; see include/stq.h)
+    auto mix32 = [](uint32_t h) { h ^= h >> 16; h *= 0x85EBCA6Bu; h ^= h >> 13; h *= 0xC2B2AE35u; h ^= h >> 16; return h; };
+    const uint64_t step = (uint64_t)hp->step, seed = hp->sr_seed;
+    uint32_t h = mix32((uint32_t)(step >> 32) ^ 0x9E3779B9u);
+    h = mix32((uint32_t)step ^ h);
+    h = mix32((uint32_t)(seed >> 32) ^ h);
+    sc.sr_h = mix32((uint32_t)seed ^ h);
+  }
   sc.l2_mode = hp->decoupled_wd ? 0 : 1;
   sc.lr = hp->lr;
   sc.inv_scale = hp->inv_grad_scale;
@@ -594,6 +607,10 @@ size_t stq_scales_bytes(uint64_t numel, uint32_t block) {
   return (size_t)((numel + block - 1) / block * 4);
 }
 
+size_t stq_v_scales_bytes(uint64_t numel, uint32_t block, uint32_t v_log) {
+  return stq_scales_bytes(numel, block) * (v_log == STQ_VLOG_TS ? 2 : 1);
+}
+
 int stq_init_state(stq_handle* h, const stq_tensor* tensors, int L, void* stream) {
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int rc = prepare(h, tensors, L, kKindInit, s);
@@ -617,6 +634,8 @@ int stq_step(stq_handle* h, const stq_tensor* tensors, int L, const stq_hparams*
     // step count and / or learning rate on the device: a one-thread kernel derives the step's scalars
     // ahead of the step kernels, which then read them instead of their launch parameters
     if (hp->step_dev == nullptr) return STQ_E_ARG;       // (a device learning rate comes with a device step count)
+    for (int l = 0; l < L; ++l)                          // (the random words are keyed on the host's step count)
+      if (tensors[l].v_log == STQ_VLOG_SR) return STQ_E_ARG;
     STQ_CUDA(h, stq::launch_step_scalars(reinterpret_cast<const long long*>(hp->step_dev), hp->lr_dev, hp->lr,
                                          hp->beta1, hp->beta2, h->d_scalars, s));
     h->launches++;
@@ -718,7 +737,8 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
     const stq_tensor& t = tensors[l];
     const size_t sb = stq_scales_bytes(t.numel, t.block);
     need += up(t.numel * 4) + up(t.numel * gsz);
-    need += up(stq_codes_bytes(t.numel, t.bits_m)) + up(stq_codes_bytes(t.numel, t.bits_v)) + 2 * up(sb);
+    need += up(stq_codes_bytes(t.numel, t.bits_m)) + up(stq_codes_bytes(t.numel, t.bits_v)) + up(sb) +
+            up(stq_v_scales_bytes(t.numel, t.block, t.v_log));
     if (t.bits_m_out != t.bits_m) need += up(stq_codes_bytes(t.numel, t.bits_m_out));
     if (t.bits_v_out != t.bits_v) need += up(stq_codes_bytes(t.numel, t.bits_v_out));
     if (t.lp_dtype != STQ_LP_NONE) need += up(t.numel * 2);
@@ -779,7 +799,7 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
       case kMc: return stq_codes_bytes(t.numel, t.bits_m);
       case kVc: return stq_codes_bytes(t.numel, t.bits_v);
       case kMs: return t.bits_m != 32 ? stq_scales_bytes(t.numel, t.block) : 0;
-      default: return t.bits_v != 32 ? stq_scales_bytes(t.numel, t.block) : 0;
+      default: return t.bits_v != 32 ? stq_v_scales_bytes(t.numel, t.block, t.v_log) : 0;
     }
   };
   // the run of kind `kind` over tensors [a, b), or len 0 if the buffers do not lie back to back
@@ -849,7 +869,7 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
       d.m_codes_in = dev_in(t, kMc, 0);
       d.v_codes_in = dev_in(t, kVc, 0);
       d.m_scales_in = reinterpret_cast<float*>(dev_in(t, kMs, sb));   // placed even at 32 bits: the step may write scales
-      d.v_scales_in = reinterpret_cast<float*>(dev_in(t, kVs, sb));
+      d.v_scales_in = reinterpret_cast<float*>(dev_in(t, kVs, stq_v_scales_bytes(t.numel, t.block, t.v_log)));
       if (!d.param || !d.grad || !d.m_codes_in || !d.v_codes_in || !d.m_scales_in || !d.v_scales_in) {
         cudaDeviceSynchronize();
         return STQ_E_CUDA;
@@ -905,8 +925,9 @@ int stq_step_host(stq_handle* h, const stq_tensor* tensors, int L, const stq_hpa
         d2h += sb;
       }
       if (t.bits_v_out != 32 && !out_run[kVs]) {
-        STQ_CUDA(h, cudaMemcpyAsync(t.v_scales_out, d.v_scales_out, sb, cudaMemcpyDeviceToHost, s_out));
-        d2h += sb;
+        const size_t sbv = stq_v_scales_bytes(t.numel, t.block, t.v_log);
+        STQ_CUDA(h, cudaMemcpyAsync(t.v_scales_out, d.v_scales_out, sbv, cudaMemcpyDeviceToHost, s_out));
+        d2h += sbv;
       }
     }
     a = b;

@@ -38,7 +38,9 @@ struct TensorDesc {
   unsigned char bm_in, bv_in, bm_out, bv_out;
   float wd;                 // fp32(lambda)
   unsigned int lp_dtype;    // 0: none, 1: bf16, 2: fp16
-  unsigned int v_pl;        // 1: the second moment uses the piecewise-linear logarithm at widths 8 and 16
+  unsigned int v_mode;      // code of the second moment: 0 polynomial logarithm, 1 piecewise-linear one (differs at
+                            // widths 8 and 16), 2 stochastic rounding, 3 two scales per block (generic kernel only)
+  unsigned int sr_id;       // identifies the tensor in the random stream of the stochastic-rounding code
   void* param_lp;           // low-precision copy of the updated parameters, or nullptr
 };
 
@@ -48,6 +50,7 @@ struct StepConsts {
   float step_size;          // lr / (1 - beta1^t)
   float rsqrt_bc2;          // 1 / sqrt(1 - beta2^t)
   float eps;
+  unsigned int sr_h;        // stochastic rounding: the word mixed from (seed, step); the key of a tensor is mix32(sr_id ^ sr_h)
   float one;                // 1.0f as a run-time value (see the packed arithmetic of the main step kernel)
   int l2_mode;              // 1: g += wd*theta before the moments, no decoupled decay
   double lr;                // decoupled decay factor is fp32(1 - lr*wd), formed per tile
@@ -69,8 +72,9 @@ cudaError_t launch_stats_valid(const float* found_inf, int* valid, cudaStream_t 
 enum Mode { kStep = 0, kRepack = 1, kInit = 2, kStatsOnly = 3 };
 
 // Launches the tile range [tile_begin, tile_end) of the table.  `wide` selects the variant that
-// can read/write 32-bit (raw fp32) states.  partials: 3 doubles per warp and tile, or nullptr.
-cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const TensorDesc* table,
+// can read/write 32-bit (raw fp32) states, `variants` the one that knows the second-moment codes only the
+// generic kernel serves.  partials: 3 doubles per warp and tile, or nullptr.
+cudaError_t launch_tiles(Mode mode, bool wide, bool variants, int grad_dtype, bool stats, const TensorDesc* table,
                          const uint32_t* tile_map, uint32_t tile_begin, uint32_t tile_end,
                          const StepConsts& sc, double* partials, int grid, cudaStream_t stream);
 

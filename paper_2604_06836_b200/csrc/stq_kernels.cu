@@ -262,6 +262,55 @@ __device__ __forceinline__ unsigned long long padded_code_bytes(unsigned long lo
   return (by + 15) & ~15ull;
 }
 
+// ---- variant "sr": stochastic rounding on a grid with a whole number of levels per octave ------------------
+__device__ __forceinline__ uint32_t mix32(uint32_t h) {
+  h ^= h >> 16; h *= 0x85EBCA6Bu; h ^= h >> 13; h *= 0xC2B2AE35u; h ^= h >> 16;
+  return h;
+}
+__device__ __forceinline__ int sr_lg_levels(int b) { return b == 8 ? 3 : b == 16 ? 11 : 0; }
+constexpr float kOnePlus = 0x1.000008p+0f;     // 1 + 2^-21: lifts the block maximum to or just above 1
+// c1 = fl(fl(1/s) * (1 + 2^-21)); word: the element's random word
+__device__ __forceinline__ uint32_t sr_steps_below(float x, float c1, int b, int K, uint32_t word) {
+  const int g = sr_lg_levels(b);
+  const int yb = (int)__float_as_uint(__fmul_rn(x, c1));
+  int n = 0x3F800000 - yb;
+  n = max(n, 0);
+  n = min(n, K << (23 - g));
+  const unsigned long long j = (((unsigned long long)(uint32_t)n << (9 + g)) + word) >> 32;
+  return min((uint32_t)j, (uint32_t)K);
+}
+__device__ __forceinline__ float sr_level(uint32_t j, int b) {
+  return __uint_as_float(0x3F800000u - (j << (23 - sr_lg_levels(b))));
+}
+
+// ---- variant "ts": two scales per block --------------------------------------------------------------------
+struct TsConst {
+  float hi, lo, W, Phi;
+  int Ehi;
+};
+__device__ __forceinline__ float ts_dist(const TsConst& t, uint32_t xb) {
+  const float de = (float)((int)(xb >> 23) - t.Ehi);
+  const float dp = __fadd_rn(lg_poly(xb), -t.Phi);
+  return __fadd_rn(de, dp);
+}
+__device__ __forceinline__ TsConst ts_consts(float hi, float lo) {
+  TsConst t;
+  t.hi = hi; t.lo = lo;
+  t.Ehi = (int)(__float_as_uint(hi) >> 23);
+  t.Phi = lg_poly(__float_as_uint(hi));
+  float W = -ts_dist(t, __float_as_uint(lo));
+  W = W > 30.0f ? 30.0f : W;
+  t.W = W > 0.0f ? W : 0.0f;
+  return t;
+}
+__device__ __forceinline__ float decode_ts(uint32_t c, const TsConst& t, int K) {
+  if (t.hi == 0.0f) return 0.0f;
+  if (c == 0u) return t.lo;
+  const float step = __fdiv_rn(t.W, (float)K);
+  const float e = __fmul_rn((float)((int)c - K), step);
+  return __fmul_rn(t.hi, ex2_poly(e));
+}
+
 // ---- decode ------------------------------------------------------------------------------------
 __device__ __forceinline__ float decode_lin(uint32_t c, float s, const LinW& w) {
   const float q = __fadd_rn(__uint_as_float(kTwo23Bits | c), -(kTwo23 + w.halff));
@@ -278,11 +327,14 @@ __device__ __forceinline__ float decode_pl(uint32_t j, uint32_t s_bits, int b) {
   return __uint_as_float((uint32_t)max(xb, 0));
 }
 
-__device__ __forceinline__ float decode_log(uint32_t c, float s, int b, const LogW& w, bool pl) {
+// vmode: 0 polynomial logarithm, 1 piecewise-linear (8 and 16 bits), 2 stochastic rounding, 3 two scales (ts)
+__device__ __forceinline__ float decode_log(uint32_t c, float s, int b, const LogW& w, unsigned vmode, const TsConst& ts) {
+  if (vmode == 2u) return __fmul_rn(s, sr_level((uint32_t)w.K - c, b));
+  if (vmode == 3u) return decode_ts(c, ts, w.K);
   if (b <= 4) {   // one octave per code: 2^(c-K)
     return __fmul_rn(s, __uint_as_float((c + (uint32_t)(127 - w.K)) << 23));
   }
-  if (pl) return decode_pl((uint32_t)w.K - c, __float_as_uint(s), b);
+  if (vmode == 1u) return decode_pl((uint32_t)w.K - c, __float_as_uint(s), b);
   const float rf = __fadd_rn(__uint_as_float(kTwo23Bits | c), -(kTwo23 + (float)w.K));
   return __fmul_rn(s, ex2_poly(__fmul_rn(rf, w.c)));
 }
@@ -380,7 +432,9 @@ __device__ __forceinline__ void store_param(float* p, int nvl, const float (&x)[
 }
 
 // ---- the tile kernel ---------------------------------------------------------------------------
-template <int MODE, int GDT, bool STATS, bool WIDE>
+// VAR: the table holds tensors whose second moment uses one of the codes that only this kernel serves
+// (stochastic rounding, two scales); compiled apart so that the common launches carry none of it.
+template <int MODE, int GDT, bool STATS, bool WIDE, bool VAR>
 __global__ void __launch_bounds__(kThreads, 2)
 stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map,
                 uint32_t tile_begin, uint32_t tile_end, const StepConsts sc_in, double* __restrict__ partials) {
@@ -405,7 +459,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
 
   // blocks of 1024 elements: maxima of neighbouring warps meet here (two buffers, used alternately: a warp
   // that runs ahead is held by the next tile's barrier before it can overwrite what a slower one still reads)
-  __shared__ uint32_t xchg[2][2 * (kThreads / 32)];
+  __shared__ uint32_t xchg[2][3 * (kThreads / 32)];      // {max |m|, max v, min v} per warp
   int xchg_parity = 0;
 
   for (uint32_t tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
@@ -417,14 +471,17 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
     const bool wide_block = MODE != kStatsOnly && T->block == 1024u;
 
     if (e_warp >= numel && wide_block) {     // nothing to do here, but the neighbour may wait for this warp
-      if (lane == 0) { xchg[xchg_parity][2 * warp] = 0u; xchg[xchg_parity][2 * warp + 1] = 0u; }
+      if (lane == 0) {
+        xchg[xchg_parity][3 * warp] = 0u; xchg[xchg_parity][3 * warp + 1] = 0u; xchg[xchg_parity][3 * warp + 2] = 0x7F800000u;
+      }
       asm volatile("bar.sync 1, %0;" ::"r"(kThreads) : "memory");
     }
     if (e_warp < numel) {
       const uint32_t B = T->block;              // a power of two, 32 .. 1024
       const int lgB = 31 - __clz((int)B);
       const int bm_in = T->bm_in, bv_in = T->bv_in, bm_out = T->bm_out, bv_out = T->bv_out;
-      const bool pl = T->v_pl != 0u;
+      const unsigned vmode = VAR ? T->v_mode : (T->v_mode & 1u);
+      const bool pl = vmode == 1u;
 
       int nvl[R];
 #pragma unroll
@@ -438,6 +495,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
       GradRow<GDT> graw[R];
       Raw<WIDE> rawm[R], rawv[R];
       float s_m_in[R], s_v_in[R];
+      [[maybe_unused]] float s_v2_in[R];      // two-scale code: the block minimum
       if constexpr (MODE == kStep) {
         float* param = T->param;
 #pragma unroll
@@ -466,7 +524,13 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
           const unsigned long long e_lane = e_warp + r * kRowElems + 4 * lane;
           const bool live = e_lane < numel;
           s_m_in[r] = (live && bm_in != 32) ? ms[e_lane >> lgB] : 0.f;
-          s_v_in[r] = (live && bv_in != 32) ? vs[e_lane >> lgB] : 0.f;
+          if (vmode == 3u) {                  // {hi, lo} per block
+            s_v_in[r] = (live && bv_in != 32) ? vs[2 * (e_lane >> lgB)] : 0.f;
+            s_v2_in[r] = (live && bv_in != 32) ? vs[2 * (e_lane >> lgB) + 1] : 0.f;
+          } else {
+            s_v_in[r] = (live && bv_in != 32) ? vs[e_lane >> lgB] : 0.f;
+            s_v2_in[r] = 0.f;
+          }
         }
       }
 
@@ -516,8 +580,10 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
             } else {
               uint32_t c[4];
               split_codes<WIDE>(rawv[r], bv_in, lane, c);
+              TsConst ts_in;
+              if (vmode == 3u) ts_in = ts_consts(s_v_in[r], s_v2_in[r]);
 #pragma unroll
-              for (int k = 0; k < 4; ++k) vh[k] = decode_log(c[k], s_v_in[r], bv_in, gw_in, pl);
+              for (int k = 0; k < 4; ++k) vh[k] = decode_log(c[k], s_v_in[r], bv_in, gw_in, vmode, ts_in);
             }
             if constexpr (MODE == kStep) {
               th[r][0] = th4[r].x; th[r][1] = th4[r].y; th[r][2] = th4[r].z; th[r][3] = th4[r].w;
@@ -554,6 +620,7 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
 
         // ---- block maxima: lane max of 4, warp REDUX on the bit patterns, rows merged per block ----
         uint32_t mxm[R], mxv[R];
+        [[maybe_unused]] uint32_t mnv[R];     // two-scale code: block minimum of v (elements past the end stay out)
         // lanes that share a block with this one: the whole warp, or 8 / 16 neighbours for blocks of 32 / 64
         const unsigned seg_lanes = B >= 128 ? 32u : B / 4;
         const unsigned seg_mask = B >= 128 ? kFull : ((1u << seg_lanes) - 1u) << (lane & ~(seg_lanes - 1u));
@@ -563,29 +630,38 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
           const float av = fmaxf(fmaxf(vt[r][0], vt[r][1]), fmaxf(vt[r][2], vt[r][3]));
           mxm[r] = __reduce_max_sync(seg_mask, __float_as_uint(am));
           mxv[r] = __reduce_max_sync(seg_mask, __float_as_uint(av));
+          mnv[r] = 0x7F800000u;
+          if (vmode == 3u) {
+            uint32_t lm = 0x7F800000u;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if (k < nvl[r]) lm = min(lm, __float_as_uint(vt[r][k]));
+            mnv[r] = __reduce_min_sync(seg_mask, lm);
+          }
         }
         if (B >= 256) {
 #pragma unroll
           for (int r = 0; r < R; r += 2) {
             mxm[r] = mxm[r + 1] = max(mxm[r], mxm[r + 1]);
             mxv[r] = mxv[r + 1] = max(mxv[r], mxv[r + 1]);
+            mnv[r] = mnv[r + 1] = min(mnv[r], mnv[r + 1]);
           }
         }
         if (R >= 4 && B >= 512) {
-          const uint32_t a = max(mxm[0], mxm[R - 2]), b = max(mxv[0], mxv[R - 2]);
+          const uint32_t a = max(mxm[0], mxm[R - 2]), b = max(mxv[0], mxv[R - 2]), c = min(mnv[0], mnv[R - 2]);
 #pragma unroll
-          for (int r = 0; r < R; ++r) { mxm[r] = a; mxv[r] = b; }
+          for (int r = 0; r < R; ++r) { mxm[r] = a; mxv[r] = b; mnv[r] = c; }
         }
         if (B == 1024) {
           // a block of 1024 spans this warp and its neighbour: the two exchange their maxima through shared
           // memory.  Every warp of the CTA takes part in the barrier (the ones past the end of the tensor from
           // the branch below), which the whole CTA reaches because the block size is a property of the tile.
           uint32_t* slot = xchg[xchg_parity];
-          if (lane == 0) { slot[2 * warp] = mxm[0]; slot[2 * warp + 1] = mxv[0]; }
+          if (lane == 0) { slot[3 * warp] = mxm[0]; slot[3 * warp + 1] = mxv[0]; slot[3 * warp + 2] = mnv[0]; }
           asm volatile("bar.sync 1, %0;" ::"r"(kThreads) : "memory");
-          const uint32_t pm = slot[2 * (warp ^ 1)], pv = slot[2 * (warp ^ 1) + 1];
+          const uint32_t pm = slot[3 * (warp ^ 1)], pv = slot[3 * (warp ^ 1) + 1], pn = slot[3 * (warp ^ 1) + 2];
 #pragma unroll
-          for (int r = 0; r < R; ++r) { mxm[r] = max(mxm[r], pm); mxv[r] = max(mxv[r], pv); }
+          for (int r = 0; r < R; ++r) { mxm[r] = max(mxm[r], pm); mxv[r] = max(mxv[r], pv); mnv[r] = min(mnv[r], pn); }
         }
 
         // ---- quantize, pack, store; decode the new codes; update the parameters -------------------
@@ -644,7 +720,40 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
             const float s = zero ? 0.f : s_raw;
             uint32_t x[4];
             uint32_t sub;
-            if (bv_out <= 4) {
+            if (vmode == 2u) {
+              // stochastic rounding: j = floor(n * L / 2^23 + U / 2^32) level steps below the maximum, U the
+              // element's random word (a re-pack has no step to draw from and rounds to nearest)
+              const float c1 = zero ? 0.f : __fmul_rn(__frcp_rn(s_raw), kOnePlus);
+              uint32_t key_e = 0u;
+              if constexpr (MODE == kStep) key_e = mix32(mix32(T->sr_id ^ sc.sr_h) + (uint32_t)(e_row >> 32));
+              sub = 0u;
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                uint32_t word = 0x80000000u;
+                if constexpr (MODE == kStep) word = mix32(((uint32_t)e_row + 4u * lane + k) ^ key_e);
+                const uint32_t j = zero ? (uint32_t)gw.K : sr_steps_below(vt[r][k], c1, bv_out, gw.K, word);
+                x[k] = (uint32_t)gw.K - j;
+                if constexpr (MODE == kStep) vq[k] = __fmul_rn(s, sr_level(j, bv_out));
+              }
+            } else if (vmode == 3u) {
+              // two scales: codes spread evenly in log2 between the block minimum (raised to hi * 2^-30) and maximum
+              const float lo = zero ? 0.f : fmaxf(__uint_as_float(mnv[r]), __fmul_rn(s_raw, 0x1p-30f));
+              const TsConst ts = ts_consts(zero ? 1.0f : s_raw, zero ? 1.0f : lo);
+              const float inv = ts.W > 0.0f ? __fdiv_rn((float)gw.K, ts.W) : 0.0f;
+              sub = kMagicBits - (uint32_t)gw.K;
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const float d = fminf(fmaxf(ts_dist(ts, __float_as_uint(vt[r][k])), -ts.W), 0.0f);
+                const float t = __fmaf_rn(d, inv, kMagic);        // low bits: code - K, in [-K, 0]
+                x[k] = zero ? sub : __float_as_uint(t);
+                if constexpr (MODE == kStep) {
+                  TsConst td = ts;
+                  td.hi = s;          // (a zero block decodes to zero)
+                  vq[k] = decode_ts(x[k] - sub, td, gw.K);
+                }
+              }
+              if (((e_row + 4 * lane) & (B - 1)) == 0 && e_row + 4 * lane < numel) vso[2 * ((e_row + 4 * lane) >> lgB) + 1] = lo;
+            } else if (bv_out <= 4) {
               // one octave per code: the code is the exponent of x*sqrt2/s, floored at -K
               const float c = zero ? 0.f : __fmul_rn(__frcp_rn(s_raw), kSqrt2);
               const float ymin = __uint_as_float((uint32_t)(127 - gw.K) << 23);
@@ -687,7 +796,8 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
               }
             }
             store_codes(vco, e_row, bv_out, lane, lim_vo, x, sub, nvl[r]);
-            if (((e_row + 4 * lane) & (B - 1)) == 0 && e_row + 4 * lane < numel) vso[(e_row + 4 * lane) >> lgB] = s;
+            if (((e_row + 4 * lane) & (B - 1)) == 0 && e_row + 4 * lane < numel)
+              vso[vmode == 3u ? 2 * ((e_row + 4 * lane) >> lgB) : (e_row + 4 * lane) >> lgB] = s;
           }
 
           if constexpr (MODE == kStep) {
@@ -856,42 +966,45 @@ stq_stats_finish_kernel(const TensorDesc* __restrict__ table, int L, const doubl
   if (threadIdx.x == 3) out[(size_t)l * 4 + 3] = (double)table[l].numel;
 }
 
-template <int MODE, int GDT, bool STATS, bool WIDE>
+template <int MODE, int GDT, bool STATS, bool WIDE, bool VAR>
 cudaError_t launch_one(const TensorDesc* table, const uint32_t* tile_map, uint32_t tb, uint32_t te,
                        const StepConsts& sc, double* partials, int grid, cudaStream_t stream) {
   const uint32_t n = te - tb;
   const int g = (int)(n < (uint32_t)grid ? n : (uint32_t)grid);
-  stq_tile_kernel<MODE, GDT, STATS, WIDE><<<g, kThreads, 0, stream>>>(table, tile_map, tb, te, sc, partials);
+  stq_tile_kernel<MODE, GDT, STATS, WIDE, VAR><<<g, kThreads, 0, stream>>>(table, tile_map, tb, te, sc, partials);
   return cudaGetLastError();
 }
 
 template <int MODE, int GDT, bool STATS>
 cudaError_t launch_w(bool wide, const TensorDesc* table, const uint32_t* tile_map, uint32_t tb, uint32_t te,
-                     const StepConsts& sc, double* partials, int grid, cudaStream_t stream) {
-  return wide ? launch_one<MODE, GDT, STATS, true>(table, tile_map, tb, te, sc, partials, grid, stream)
-              : launch_one<MODE, GDT, STATS, false>(table, tile_map, tb, te, sc, partials, grid, stream);
+                     const StepConsts& sc, double* partials, int grid, cudaStream_t stream, bool variants) {
+  if (variants)
+    return wide ? launch_one<MODE, GDT, STATS, true, true>(table, tile_map, tb, te, sc, partials, grid, stream)
+                : launch_one<MODE, GDT, STATS, false, true>(table, tile_map, tb, te, sc, partials, grid, stream);
+  return wide ? launch_one<MODE, GDT, STATS, true, false>(table, tile_map, tb, te, sc, partials, grid, stream)
+              : launch_one<MODE, GDT, STATS, false, false>(table, tile_map, tb, te, sc, partials, grid, stream);
 }
 
 }  // namespace
 
-cudaError_t launch_tiles(Mode mode, bool wide, int grad_dtype, bool stats, const TensorDesc* table,
+cudaError_t launch_tiles(Mode mode, bool wide, bool variants, int grad_dtype, bool stats, const TensorDesc* table,
                          const uint32_t* tile_map, uint32_t tile_begin, uint32_t tile_end,
                          const StepConsts& sc, double* partials, int grid, cudaStream_t stream) {
   if (tile_end <= tile_begin) return cudaSuccess;
   switch (mode) {
     case kStep:
       if (grad_dtype == 0)
-        return stats ? launch_w<kStep, 0, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream)
-                     : launch_w<kStep, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+        return stats ? launch_w<kStep, 0, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream, variants)
+                     : launch_w<kStep, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream, variants);
       if (grad_dtype == 1)
-        return stats ? launch_w<kStep, 1, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream)
-                     : launch_w<kStep, 1, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
-      return stats ? launch_w<kStep, 2, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream)
-                   : launch_w<kStep, 2, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+        return stats ? launch_w<kStep, 1, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream, variants)
+                     : launch_w<kStep, 1, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream, variants);
+      return stats ? launch_w<kStep, 2, true>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream, variants)
+                   : launch_w<kStep, 2, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream, variants);
     case kRepack:
-      return launch_w<kRepack, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+      return launch_w<kRepack, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream, variants);
     case kInit:
-      return launch_w<kInit, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream);
+      return launch_w<kInit, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream, variants);
     case kStatsOnly: {
       const uint32_t n = tile_end - tile_begin;
       const uint32_t want = (uint32_t)grid * 4u;   // small CTAs, 32 registers: many fit per SM
@@ -946,7 +1059,7 @@ cudaError_t launch_stats_valid(const float* found_inf, int* valid, cudaStream_t 
 
 int step_ctas_per_sm() {
   int n = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, stq_tile_kernel<kStep, 1, false, false>, kThreads, 0) !=
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, stq_tile_kernel<kStep, 1, false, false, false>, kThreads, 0) !=
       cudaSuccess)
     return 1;
   return n > 0 ? n : 1;

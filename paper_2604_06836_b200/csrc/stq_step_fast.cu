@@ -1144,11 +1144,11 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
         ti.mso = T->ms_out + (e0 >> lgB);
         ti.vso = T->vs_out + (e0 >> lgB);
         ti.lp = T->param_lp ? reinterpret_cast<uint16_t*>(T->param_lp) + e0 : nullptr;
-        ti.packed = width_index(bm) | ((width_index(bv) + (T->v_pl != 0u && bv >= 8u ? 2u : 0u)) << 8) | (lgB << 16) |
+        ti.packed = width_index(bm) | ((width_index(bv) + (T->v_mode == 1u && bv >= 8u ? 2u : 0u)) << 8) | (lgB << 16) |
                     (T->lp_dtype << 24);
         ti.wdx = sc.l2_mode ? T->wd : (float)(sc.lr * (double)T->wd);
         ti.tile = tile;
-        ti.out = width_index(bmo) | ((width_index(bvo) + (T->v_pl != 0u && bvo >= 8u ? 2u : 0u)) << 8);
+        ti.out = width_index(bmo) | ((width_index(bvo) + (T->v_mode == 1u && bvo >= 8u ? 2u : 0u)) << 8);
         const uint8_t* src_g = reinterpret_cast<const uint8_t*>(T->grad) + e0 * gsz;
         const uint8_t* src_mc = T->mc_in + (e0 >> 3) * bm;
         const uint8_t* src_vc = T->vc_in + (e0 >> 3) * bv;

@@ -35,7 +35,8 @@ class STQAdamW(torch.optim.Optimizer):
     before the update (Algorithm 1 as printed, one more read of the gradients on decision steps);
     "fused" lets them ride on the update of the step before (no extra pass; the decision then sees
     gradients that are one step old, except at t = 1).
-    v_log: "poly" or "pl", the variant of the second-moment code at 8 and 16 bits.
+    v_log: the code of the second moment: "poly" (default) or "pl" (they differ at 8 and 16 bits), "sr"
+    (stochastic rounding; ``self.sr_seed`` seeds its random words) or "ts" (two scales per block).
     grad_scaler_inv / found_inf: optional one-element float32 CUDA tensors for loss-scaled training.
     With ``found_inf`` set, ``step()`` reads it on the host first (one small synchronising copy): a step
     with a non-finite gradient is left out entirely, so the step count t, the bias corrections and the
@@ -59,7 +60,10 @@ class STQAdamW(torch.optim.Optimizer):
         self.betas, self.eps = (float(betas[0]), float(betas[1])), float(eps)
         self.block, self.policy_kind, self.interval = block, policy, int(interval)
         self.decoupled = bool(decoupled_weight_decay)
-        self.v_log = stq.VLOG_PL if v_log == "pl" else stq.VLOG_POLY
+        if v_log not in stq.VLOG_BY_NAME:
+            raise ValueError("v_log is one of " + ", ".join(stq.VLOG_BY_NAME))
+        self.v_log = stq.VLOG_BY_NAME[v_log]
+        self.sr_seed = 0
         bm, bv = (init_bits, init_bits) if isinstance(init_bits, int) else init_bits
         self._params = [p for g in self.param_groups for p in g["params"]]
         if not self._params:
@@ -101,7 +105,7 @@ class STQAdamW(torch.optim.Optimizer):
                     grad = grad.contiguous()
                     p.grad = grad
                 rows.append(stq.make_row(p.numel(), self.block, self.states[k], states_out[k], p.data, grad,
-                                         g["weight_decay"]))
+                                         g["weight_decay"], sr_id=k))
                 k += 1
         return rows
 
@@ -133,7 +137,7 @@ class STQAdamW(torch.optim.Optimizer):
         t = self.t
         hp = dict(lr=self.param_groups[0]["lr"], beta1=self.betas[0], beta2=self.betas[1], eps=self.eps, t=t,
                   grad_dtype=self._grad_dtype(), decoupled_wd=self.decoupled,
-                  inv_grad_scale=self.grad_scaler_inv, found_inf=self.found_inf)
+                  inv_grad_scale=self.grad_scaler_inv, found_inf=self.found_inf, sr_seed=self.sr_seed)
         new_m = new_v = None
         if self.policy_kind == "paper" and self.policy.is_decision_step(t):
             stats, self._carried_stats = self._carried_stats, None    # fused order: they rode on the previous step
@@ -165,7 +169,7 @@ class STQAdamW(torch.optim.Optimizer):
             mc, ms = (old.m_codes, old.m_scales) if bm == old.bits_m else (
                 stq.alloc_codes(n, bm, self.device), stq.alloc_scales(n, bm, self.block, self.device))
             vc, vs = (old.v_codes, old.v_scales) if bv == old.bits_v else (
-                stq.alloc_codes(n, bv, self.device), stq.alloc_scales(n, bv, self.block, self.device))
+                stq.alloc_codes(n, bv, self.device), stq.alloc_scales(n, bv, self.block, self.device, self.v_log))
             out.append(stq.QState(mc, ms, bm, vc, vs, bv, self.v_log))
         self.handle.step(stq.table(self._rows(out)), flags=flags, **hp)
         self._fetch_carried(flags)

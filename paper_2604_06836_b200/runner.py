@@ -72,7 +72,8 @@ class Job:
                 self.params[i].copy_(draw_param(w, i, self.device))
         self.bits_m = np.asarray(bits_m, dtype=np.uint8).copy()
         self.bits_v = np.asarray(bits_v, dtype=np.uint8).copy()
-        self.v_log = stq.VLOG_PL if w.v_log == "pl" else stq.VLOG_POLY
+        self.v_log = stq.VLOG_BY_NAME[w.v_log]
+        self.sr_seed = 0x5EED0000 + w.seed          # random words of the stochastic-rounding code
         self.states = [stq.alloc_state(n, self.block, int(bm), int(bv), self.device, self.v_log)
                        for n, bm, bv in zip(self.numels, self.bits_m, self.bits_v)]
         self.wd = [w.weight_decay] * self.L
@@ -86,7 +87,7 @@ class Job:
         rows = [stq.make_row(n, self.block, si if with_inputs else None, so,
                              self.params[i] if with_inputs else None,
                              self.grads[i] if with_inputs else None, self.wd[i],
-                             self.params_lp[i] if with_inputs else None)
+                             self.params_lp[i] if with_inputs else None, sr_id=i)
                 for i, (n, si, so) in enumerate(zip(self.numels, st_in, st_out))]
         return stq.table(rows)
 
@@ -105,7 +106,7 @@ class Job:
     def hp(self, t: int) -> dict:
         w = self.w
         return dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, t=t, grad_dtype=self.grad_dtype,
-                    inv_grad_scale=self.inv_scale, found_inf=self.found_inf)
+                    inv_grad_scale=self.inv_scale, found_inf=self.found_inf, sr_seed=self.sr_seed)
 
     def step(self, t: int | None = None, stats: bool = False, new_bits=None, stream=None):
         """One optimizer step.  new_bits = (bits_m, bits_v) arrays switches widths inside the step."""
@@ -134,7 +135,7 @@ class Job:
         rows = []
         for i in idx:
             new_states[i] = self._fresh_state(i, int(bm[i]), int(bv[i]))
-            rows.append(stq.make_row(self.numels[i], self.block, self.states[i], new_states[i]))
+            rows.append(stq.make_row(self.numels[i], self.block, self.states[i], new_states[i], sr_id=i))
         self.handle.repack(stq.table(rows), stream=stream)
         self._adopt(new_states, bm, bv)
 
@@ -148,7 +149,7 @@ class Job:
         mc, ms = (old.m_codes, old.m_scales) if bm == old.bits_m else (
             stq.alloc_codes(n, bm, self.device), stq.alloc_scales(n, bm, self.block, self.device))
         vc, vs = (old.v_codes, old.v_scales) if bv == old.bits_v else (
-            stq.alloc_codes(n, bv, self.device), stq.alloc_scales(n, bv, self.block, self.device))
+            stq.alloc_codes(n, bv, self.device), stq.alloc_scales(n, bv, self.block, self.device, self.v_log))
         return stq.QState(mc, ms, bm, vc, vs, bv, self.v_log)
 
     def _adopt(self, new_states, bm, bv):
@@ -187,7 +188,7 @@ class Job:
         mc, ms = mirror([s.m_codes for s in self.states]), mirror([s.m_scales for s in self.states])
         vc, vs = mirror([s.v_codes for s in self.states]), mirror([s.v_scales for s in self.states])
         states = [stq.QState(mc[i], ms[i], s.bits_m, vc[i], vs[i], s.bits_v, s.v_log) for i, s in enumerate(self.states)]
-        rows = [stq.make_row(n, self.block, states[i], states[i], host_p[o:o + n], host_g[o:o + n], self.wd[i])
+        rows = [stq.make_row(n, self.block, states[i], states[i], host_p[o:o + n], host_g[o:o + n], self.wd[i], sr_id=i)
                 for i, (n, o) in enumerate(zip(self.numels, self.offsets))]
         return stq.table(rows), states, host_p, host_g
 

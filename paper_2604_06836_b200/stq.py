@@ -20,7 +20,8 @@ LIB_PATH = os.path.join(_HERE, "libstq.so")
 GRAD_F32, GRAD_BF16, GRAD_F16 = 0, 1, 2
 LP_NONE, LP_BF16, LP_F16 = 0, 1, 2
 WITH_STATS = 1
-VLOG_POLY, VLOG_PL = 0, 1
+VLOG_POLY, VLOG_PL, VLOG_SR, VLOG_TS = 0, 1, 2, 3      # codes of the second moment (stq_tensor.v_log)
+VLOG_BY_NAME = {"poly": VLOG_POLY, "pl": VLOG_PL, "sr": VLOG_SR, "ts": VLOG_TS}
 WIDTHS = (2, 3, 4, 8, 16, 32)
 E_STATE, E_TIMEOUT, E_TOO_LARGE = -10, -11, -12     # the STQ_E_* codes callers test for
 
@@ -43,7 +44,7 @@ class CTensor(C.Structure):
         ("bits_m", C.c_uint8), ("bits_v", C.c_uint8), ("bits_m_out", C.c_uint8), ("bits_v_out", C.c_uint8),
         ("weight_decay", C.c_float), ("lp_dtype", C.c_uint32),
         ("param_lp", C.c_void_p),
-        ("v_log", C.c_uint32), ("reserved", C.c_uint32),
+        ("v_log", C.c_uint32), ("sr_id", C.c_uint32),
     ]
 
 
@@ -52,7 +53,7 @@ class CHParams(C.Structure):
     _fields_ = [("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
                 ("step", C.c_int64), ("decoupled_wd", C.c_int32), ("grad_dtype", C.c_int32),
                 ("inv_grad_scale", C.c_void_p), ("found_inf", C.c_void_p),
-                ("step_dev", C.c_void_p), ("lr_dev", C.c_void_p)]
+                ("step_dev", C.c_void_p), ("lr_dev", C.c_void_p), ("sr_seed", C.c_uint64)]
 
 
 class CPolicyCfg(C.Structure):
@@ -78,6 +79,8 @@ def lib() -> C.CDLL:
         L.stq_codes_bytes.restype = C.c_size_t
         L.stq_scales_bytes.argtypes = [C.c_uint64, C.c_uint32]
         L.stq_scales_bytes.restype = C.c_size_t
+        L.stq_v_scales_bytes.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32]
+        L.stq_v_scales_bytes.restype = C.c_size_t
         L.stq_init_state.argtypes = [vp, PT, C.c_int, vp]
         L.stq_step.argtypes = [vp, PT, C.c_int, C.POINTER(CHParams), C.c_uint, vp]
         L.stq_grad_stats.argtypes = [vp, PT, C.c_int, C.c_int, vp]
@@ -140,14 +143,16 @@ def alloc_codes(numel: int, bits: int, device) -> torch.Tensor:
     return torch.zeros(codes_bytes(numel, bits), dtype=torch.uint8, device=device)
 
 
-def alloc_scales(numel: int, bits: int, block: int, device) -> torch.Tensor:
-    n = scales_bytes(numel, block) // 4
+def alloc_scales(numel: int, bits: int, block: int, device, v_log: int | None = None) -> torch.Tensor:
+    """Scale buffer of a state; v_log (for a second moment) selects the size of its code: the two-scale code
+    keeps two floats per block."""
+    n = (scales_bytes(numel, block) if v_log is None else int(lib().stq_v_scales_bytes(numel, block, v_log))) // 4
     return torch.zeros(n, dtype=torch.float32, device=device)
 
 
 def alloc_state(numel: int, block: int, bits_m: int, bits_v: int, device, v_log: int = 0) -> QState:
     return QState(alloc_codes(numel, bits_m, device), alloc_scales(numel, bits_m, block, device), bits_m,
-                  alloc_codes(numel, bits_v, device), alloc_scales(numel, bits_v, block, device), bits_v, v_log)
+                  alloc_codes(numel, bits_v, device), alloc_scales(numel, bits_v, block, device, v_log), bits_v, v_log)
 
 
 def _ptr(t: torch.Tensor | None) -> int | None:
@@ -160,9 +165,10 @@ def grad_dtype_of(t: torch.Tensor) -> int:
 
 def make_row(numel: int, block: int, st_in: QState | None, st_out: QState, param: torch.Tensor | None = None,
              grad: torch.Tensor | None = None, weight_decay: float = 0.0,
-             param_lp: torch.Tensor | None = None) -> CTensor:
+             param_lp: torch.Tensor | None = None, sr_id: int = 0) -> CTensor:
     """One table row.  st_out may be st_in (in-place) when the widths are unchanged.  param_lp: an
-    optional bf16/fp16 tensor that receives the rounded copy of the updated parameters."""
+    optional bf16/fp16 tensor that receives the rounded copy of the updated parameters.  sr_id: the
+    tensor's number in the random stream of the stochastic-rounding code (ignored by the other codes)."""
     r = CTensor()
     r.param = _ptr(param)
     r.grad = _ptr(grad)
@@ -177,7 +183,7 @@ def make_row(numel: int, block: int, st_in: QState | None, st_out: QState, param
     r.bits_m_out, r.bits_v_out = st_out.bits_m, st_out.bits_v
     if st_in is not None and st_in.v_log != st_out.v_log:
         raise ValueError("a state is read and written with the same variant of the v quantizer")
-    r.v_log, r.reserved = st_out.v_log, 0
+    r.v_log, r.sr_id = st_out.v_log, (sr_id if st_out.v_log == VLOG_SR else 0)
     r.numel, r.block, r.weight_decay = numel, block, weight_decay
     if param_lp is not None:
         r.lp_dtype = LP_BF16 if param_lp.dtype == torch.bfloat16 else LP_F16
@@ -261,8 +267,9 @@ class Handle:
 
     def step(self, tbl, *, lr, beta1, beta2, eps, t, grad_dtype=GRAD_F32, decoupled_wd=True, flags=0, stream=None,
              inv_grad_scale: torch.Tensor | None = None, found_inf: torch.Tensor | None = None,
-             step_dev: torch.Tensor | None = None, lr_dev: torch.Tensor | None = None):
+             step_dev: torch.Tensor | None = None, lr_dev: torch.Tensor | None = None, sr_seed: int = 0):
         """inv_grad_scale / found_inf: optional one-element float32 device tensors (loss-scaled training).
+        sr_seed: seed of the random words of tensors coded with stochastic rounding.
         step_dev (one int64) / lr_dev (one float32): optional device tensors that replace t and lr, for steps
         replayed from a CUDA graph."""
         if step_dev is not None and step_dev.dtype != torch.int64:
@@ -270,7 +277,7 @@ class Handle:
         if lr_dev is not None and lr_dev.dtype != torch.float32:
             raise ValueError("lr_dev holds one float32")
         hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype,
-                      _ptr(inv_grad_scale), _ptr(found_inf), _ptr(step_dev), _ptr(lr_dev))
+                      _ptr(inv_grad_scale), _ptr(found_inf), _ptr(step_dev), _ptr(lr_dev), sr_seed)
         self._check(lib().stq_step(self._h, tbl, len(tbl), C.byref(hp), flags, _stream_ptr(stream)), "stq_step")
 
     def grad_stats(self, tbl, grad_dtype=GRAD_F32, stream=None):
@@ -286,10 +293,10 @@ class Handle:
         self._check(lib().stq_repack(self._h, tbl, len(tbl), _stream_ptr(stream)), "stq_repack")
 
     def step_host(self, tbl, *, lr, beta1, beta2, eps, t, grad_dtype=GRAD_F32, decoupled_wd=True, flags=0,
-                  inv_grad_scale=None, found_inf=None):
+                  inv_grad_scale=None, found_inf=None, sr_seed: int = 0):
         if inv_grad_scale is not None or found_inf is not None:
             raise ValueError("step_host takes host buffers only: unscale the gradients on the device path")
-        hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype, None, None, None, None)
+        hp = CHParams(lr, beta1, beta2, eps, t, 1 if decoupled_wd else 0, grad_dtype, None, None, None, None, sr_seed)
         h2d, d2h = C.c_uint64(0), C.c_uint64(0)
         self._check(lib().stq_step_host(self._h, tbl, len(tbl), C.byref(hp), flags, C.byref(h2d), C.byref(d2h)),
                     "stq_step_host")

@@ -91,7 +91,8 @@ class Workload:
     weight_decay: float = 0.01
     loss_scale: float = 0.0            # > 0: gradients arrive multiplied by it (fp16 training)
     lp_copy: str = ""                  # "bf16" | "fp16": the step also writes the model's working copy
-    v_log: str = "poly"                # "poly" | "pl": variant of the v quantizer at widths 8 and 16
+    v_log: str = "poly"                # code of the second moment: "poly" | "pl" (differ at widths 8 and 16) | "sr"
+                                       # (stochastic rounding) | "ts" (two scales per block)
 
     @property
     def numels(self) -> list[int]:

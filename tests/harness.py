@@ -10,6 +10,8 @@ import torch
 
 import oracle as O
 from paper_2604_06836_b200 import stq
+
+V_MODE = {"poly": O.LOG, "pl": O.LOG_PL, "sr": O.LOG_SR, "ts": O.LOG_TS}      # workload name -> oracle mode
 from paper_2604_06836_b200.runner import Job
 
 
@@ -34,10 +36,11 @@ class OracleJob:
         self.upd_mag = [np.abs(th) for th in self.theta]
         self.bits_m = job.bits_m.copy()
         self.bits_v = job.bits_v.copy()
-        self.states = [O.new_state(n, self.block, int(bm), int(bv))
+        self.v_mode = V_MODE[job.w.v_log]
+        self.sr_seed = job.sr_seed
+        self.states = [O.new_state(n, self.block, int(bm), int(bv), self.v_mode)
                        for n, bm, bv in zip(self.numels, self.bits_m, self.bits_v)]
         self.wd = list(job.wd)
-        self.v_mode = O.LOG_PL if job.w.v_log == "pl" else O.LOG
 
     def step(self, grads, t: int, want_stats=False, new_bits=None, decoupled_wd=True, fp16_grad=False,
              inv_grad_scale=1.0, found_inf=False):
@@ -50,7 +53,8 @@ class OracleJob:
                                        beta2=w.beta2, eps=w.eps, weight_decay=self.wd[i], t=t,
                                        bits_m_out=int(bm[i]), bits_v_out=int(bv[i]),
                                        decoupled_wd=decoupled_wd, want_stats=want_stats, fp16_grad=fp16_grad,
-                                       inv_grad_scale=inv_grad_scale, found_inf=found_inf, v_mode=self.v_mode)
+                                       inv_grad_scale=inv_grad_scale, found_inf=found_inf, v_mode=self.v_mode,
+                                       sr_seed=self.sr_seed, tensor_index=i)
             self.upd_mag[i] = np.maximum(self.upd_mag[i], np.maximum(np.abs(self.theta[i] - before), np.abs(self.theta[i])))
             if want_stats:
                 stats[i] = s
@@ -153,11 +157,12 @@ class SampledOracle:
             self.sel.append((np.array(blocks, dtype=np.int64), tail, nb_full))
             self.n_mini.append(len(blocks) * self.block + tail)
         self.theta = [self._gather_elems(p, i) for i, p in enumerate(job.params)]
-        self.states = [O.new_state(self.n_mini[i], self.block, int(job.bits_m[i]), int(job.bits_v[i]))
+        self.v_mode = V_MODE[job.w.v_log]
+        assert self.v_mode != O.LOG_SR, "the random words belong to element positions: sample-free checks only"
+        self.states = [O.new_state(self.n_mini[i], self.block, int(job.bits_m[i]), int(job.bits_v[i]), self.v_mode)
                        for i in range(job.L)]
         self.mag = [np.abs(t) for t in self.theta]
         self.stepped = False      # the working copy exists only after the first step
-        self.v_mode = O.LOG_PL if job.w.v_log == "pl" else O.LOG
 
     def _elem_index(self, i: int) -> torch.Tensor:
         blocks, tail, nb_full = self.sel[i]
@@ -257,10 +262,10 @@ class FullOracle:
         self.range_elems = range_elems
         self.pool = ThreadPoolExecutor(max_workers=threads or os.cpu_count() or 4)
         self.theta = [to_np(p) for p in job.params]
-        self.states = [O.new_state(n, self.block, int(bm), int(bv))
+        self.v_mode = V_MODE[job.w.v_log]
+        self.states = [O.new_state(n, self.block, int(bm), int(bv), self.v_mode)
                        for n, bm, bv in zip(job.numels, job.bits_m, job.bits_v)]
         self.mag = [p.abs() for p in job.params]          # device: largest magnitude an element or its step has had
-        self.v_mode = O.LOG_PL if job.w.v_log == "pl" else O.LOG
 
     def _ranges(self):
         for i, n in enumerate(self.job.numels):
@@ -276,7 +281,7 @@ class FullOracle:
             bm = self.states[i].bits_m if new_bits is None else int(new_bits[0][i])
             bv = self.states[i].bits_v if new_bits is None else int(new_bits[1][i])
             mc, ms = O.alloc_state(n, bm, self.block)
-            vc, vs = O.alloc_state(n, bv, self.block)
+            vc, vs = O.alloc_state(n, bv, self.block, self.v_mode)
             out.append(O.State(mc, ms, bm, vc, vs, bv))
         amp = dict(fp16_grad=True, inv_grad_scale=1.0 / w.loss_scale) if w.grad_dtype == "fp16" else {}
         tasks = list(self._ranges())
@@ -286,7 +291,7 @@ class FullOracle:
             i, e0, e1 = tasks[k]
             O.step_range(self.theta[i], grads[i], e0, e1, self.block, self.states[i], out[i], lr=w.lr, beta1=w.beta1,
                          beta2=w.beta2, eps=w.eps, weight_decay=job.wd[i], t=t, v_mode=self.v_mode,
-                         stats=part[k] if want_stats else None, **amp)
+                         stats=part[k] if want_stats else None, sr_seed=job.sr_seed, tensor_index=i, **amp)
 
         before = [torch.from_numpy(th).to(job.device) for th in self.theta]
         list(self.pool.map(run, range(len(tasks))))

@@ -26,8 +26,8 @@ def test_every_declared_symbol_is_exported(stq_lib):
 
 def test_struct_sizes_match_the_header(stq_lib):
     from paper_2604_06836_b200 import stq
-    assert C.sizeof(stq.CTensor) == 120        # 10 pointers, numel, block, 4 widths, weight_decay, lp_dtype, param_lp, v_log, reserved
-    assert C.sizeof(stq.CHParams) == 80        # 4 doubles, step, 2 ints, 4 pointers
+    assert C.sizeof(stq.CTensor) == 120        # 10 pointers, numel, block, 4 widths, weight_decay, lp_dtype, param_lp, v_log, sr_id
+    assert C.sizeof(stq.CHParams) == 88        # 4 doubles, step, 2 ints, 4 pointers, sr_seed
     assert C.sizeof(stq.CPolicyCfg) == 40
 
 

@@ -811,3 +811,88 @@ def test_blocks_of_every_size_in_one_table(H, O):
             H.assert_theta_close(params[i], o_theta[i], REL_1STEP * t, f"B={b} t={t}", upd=np.abs(o_theta[i]) + 1e-3)
             H.assert_stats_close(got[i:i + 1], st[None, :], f"B={b} t={t}")
     h.close()
+
+
+# ---- the stochastic-rounding and the two-scale code of the second moment -------------------------------------
+@pytest.mark.parametrize("v_log", ["sr", "ts"])
+@pytest.mark.parametrize("bv", [2, 3, 4, 8, 16])
+@pytest.mark.parametrize("bm,block,gdt", [(4, 128, "bf16"), (16, 256, "fp32"), (3, 64, "fp32"), (8, 1024, "bf16"), (32, 128, "fp32")])
+def test_sr_and_ts_codes_every_width(H, O, v_log, bv, bm, block, gdt):
+    """Both codes at every width of the second moment, with ragged sizes, fused statistics, a width change
+    inside a step and a re-pack: codes and scales (two per block for "ts") bit for bit, the random words of
+    "sr" included."""
+    from dataclasses import replace
+    for n in (4096 * 2 + 128 * 5 + 52, 999):
+        w = replace(_single(n, block, gdt, seed=bm * 100 + bv), v_log=v_log)
+        job = Job(w, [bm], [bv])
+        oj = H.OracleJob(job)
+        H.compare_job(job, oj, 0.0, "init")
+        for t in (1, 2, 3, 4):
+            job.draw_grads(t)
+            new_bits = ([8], [4 if bv != 4 else 8]) if t == 3 else None
+            st = oj.step([H.to_np(g) for g in job.grads], t, want_stats=True, new_bits=new_bits)
+            job.step(t, stats=True, new_bits=new_bits)
+            H.compare_job(job, oj, REL_1STEP * t, f"{v_log} n={n} t={t}")
+            H.assert_stats_close(job.layer_stats(), st, v_log)
+        job.repack(([bm], [bv]))
+        oj.repack(([bm], [bv]))
+        H.compare_job(job, oj, REL_1STEP * 4, f"{v_log} n={n} repack")
+
+
+def test_all_four_codes_in_one_table_and_extreme_values(H, O):
+    """Tensors coded with each of the four readings side by side in one call; zero blocks, denormal and huge
+    gradients, one outlier per block."""
+    import oracle
+    dev, block, n = "cuda", 128, 4096 * 2 + 128 * 3 + 7
+    modes = [("poly", oracle.LOG), ("pl", oracle.LOG_PL), ("sr", oracle.LOG_SR), ("ts", oracle.LOG_TS)] * 2
+    widths = [(4, 8), (8, 16), (4, 4), (3, 8), (16, 2), (2, 8), (8, 16), (4, 2)]
+    h = stq.Handle()
+    gen = torch.Generator(device=dev).manual_seed(3)
+    params = [torch.randn(n, device=dev, generator=gen) * 0.02 for _ in modes]
+    states = [stq.alloc_state(n, block, bm, bv, dev, stq.VLOG_BY_NAME[name]) for (name, _), (bm, bv) in zip(modes, widths)]
+    h.init_state(stq.table([stq.make_row(n, block, None, s) for s in states]))
+    o_theta = [H.to_np(p) for p in params]
+    o_states = [oracle.new_state(n, block, bm, bv, vm) for (_, vm), (bm, bv) in zip(modes, widths)]
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
+    for t in (1, 2, 3):
+        grads = []
+        for i in range(len(modes)):
+            x = torch.randn(n, generator=gen, device=dev) * 1e-3
+            blk = x[:n // block * block].view(-1, block)
+            blk[0::7] = 0.0
+            blk[1::7] *= 1e-42
+            blk[2::7] *= 1e-25
+            blk[3::7] *= 1e15
+            blk[4::7, 5] = 3e3
+            blk[5::7, ::2] = 0.0                                   # zeros among ordinary values: the floor of "ts"
+            grads.append(x)
+        h.step(stq.table([stq.make_row(n, block, s, s, p, g, 0.01, sr_id=i)
+                          for i, (s, p, g) in enumerate(zip(states, params, grads))]), t=t, sr_seed=77, **hp)
+        for i, (_, vm) in enumerate(modes):
+            o_states[i], _ = oracle.step(o_theta[i], H.to_np(grads[i]), o_states[i], block, weight_decay=0.01, t=t,
+                                         v_mode=vm, sr_seed=77, tensor_index=i, **hp)
+            H.assert_states_equal(states[i], o_states[i], f"{modes[i][0]} t={t}")
+            H.assert_theta_close(params[i], o_theta[i], REL_1STEP * t, f"{modes[i][0]} t={t}", upd=np.abs(o_theta[i]) + 1.0)
+    h.close()
+
+
+def test_stochastic_rounding_seeds_and_call_rules(H, O):
+    from dataclasses import replace
+    w = replace(_single(4096 * 2 + 300, 128, "bf16", seed=4), v_log="sr")
+    codes = []
+    for seed in (1, 1, 2):
+        job = Job(w, [4], [4])
+        job.sr_seed = seed
+        job.draw_grads(1)
+        job.step(1)
+        torch.cuda.synchronize()
+        codes.append(job.states[0].v_codes.clone())
+    assert torch.equal(codes[0], codes[1]) and not torch.equal(codes[0], codes[2])
+    # the random words are keyed on the host's step count: a step count kept on the device is refused
+    step_dev = torch.ones(1, dtype=torch.int64, device="cuda")
+    with pytest.raises(stq.StqError) as err:
+        job.handle.step(job.table(), **{**job.hp(2), "step_dev": step_dev})
+    assert err.value.code == -9
+    # sizes: the two-scale code keeps two floats per block
+    assert stq.lib().stq_v_scales_bytes(1000, 128, stq.VLOG_TS) == 2 * stq.scales_bytes(1000, 128)
+    assert stq.lib().stq_v_scales_bytes(1000, 128, stq.VLOG_SR) == stq.scales_bytes(1000, 128)

@@ -79,7 +79,7 @@ VARIANT_MUTANTS = [
     ("sr: level spacing off by a factor of two", "int64_t j = ((n << (9 + g)) + (int64_t)U) >> 32;",
      "int64_t j = ((n << (8 + g)) + (int64_t)U) >> 32;"),
     ("sr: decode with the wrong level spacing", "(j << (23 - sr_lg_levels(b)))", "(j << (22 - sr_lg_levels(b)))"),
-    ("sr: key ignores the tensor", "uint32_t k = mix32(tensor ^ 0x9E3779B9u);", "uint32_t k = mix32(0x9E3779B9u);"),
+    ("sr: key ignores the tensor", "return mix32(tensor ^ h);", "return mix32(h);"),
     ("sr: words taken from the position in the block, not in the tensor", "sr_word(*key, e0 + j + i)", "sr_word(*key, i)"),
     ("sr: a range forgets where it starts in its tensor", "sr_word(*key, e0 + j + i)", "sr_word(*key, j + i)"),
     ("sr: a shift of the mixing function changed", "h ^= h >> 13;", "h ^= h >> 12;"),
