@@ -14,7 +14,7 @@ HEADERS = [os.path.join(CSRC, "stq_internal.h"), os.path.join(os.path.dirname(HE
 # -fmad=false: the code-deciding arithmetic must not be contracted; fused operations are written
 # explicitly where they are wanted.
 NVCC_FLAGS = [
-    "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
+    "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "--threads", "0",
     "-fmad=false", "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
     "-diag-suppress", "177",     # unused members of the per-width constant tables
 ]

@@ -33,7 +33,8 @@ struct stq_handle {
   uint32_t* d_tile_map = nullptr;
   size_t d_tile_cap = 0;
   uint32_t n_tiles = 0, n_fast = 0, n_narrow = 0;   // n_narrow counts fast + remaining narrow
-  uint32_t n_main = 0;                              // fast tiles of the fused bodies; [n_main, n_fast) change width
+  uint32_t n_main = 0, n_var_end = 0;               // fast tiles: [0, n_main) fused bodies, [n_main, n_var_end) fused bodies
+                                                    // of the "sr" / "ts" codes, [n_var_end, n_fast) change width
   int fast_grid = 0;
   bool any_lp = false;              // some tensor of the current table wants a low-precision copy
   bool any_variant = false;         // some tensor's second moment uses a code only the generic kernel serves
@@ -216,12 +217,14 @@ double body_cost(const stq_tensor& t) {
   auto idx = [](int b) { return b == 2 ? 0 : b == 3 ? 1 : b == 4 ? 2 : b == 8 ? 3 : 4; };
   int iv = idx(t.bits_v);
   if (t.v_log == STQ_VLOG_PL && iv >= 3) iv += 2;
+  if (t.v_log >= STQ_VLOG_SR) return 1.2;      // (their own launch: only the spread among themselves matters)
   return 551.0 / kRate[idx(t.bits_m)][iv];
 }
 
-constexpr int kSplitKey = 1 << 20;
+constexpr int kSplitKey = 1 << 20, kVariantKey = 1 << 19;
 int body_key(const stq_tensor& t) {
   if (t.bits_m != t.bits_m_out || t.bits_v != t.bits_v_out) return kSplitKey;   // one runtime-width body for all of them
+  if (t.v_log >= STQ_VLOG_SR) return kVariantKey + ((int)t.v_log * 32 + t.bits_v) * 64 + t.bits_m;
   const int pl = t.v_log == STQ_VLOG_PL && (t.bits_v == 8 || t.bits_v == 16) ? 1 : 0;
   return (t.bits_v * 2 + (1 - pl)) * 64 + t.bits_m;
 }
@@ -262,7 +265,8 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     const bool wide = row_is_wide(t, kind);
     // (the main kernel moves the scales with 16-byte bulk copies as well)
     // (a tensor whose widths change inside the step takes the main kernel's runtime-width body)
-    const bool fast_ok = kind == kKindStep && !wide && t.v_log <= STQ_VLOG_PL &&
+    const bool changes = t.bits_m != t.bits_m_out || t.bits_v != t.bits_v_out;
+    const bool fast_ok = kind == kKindStep && !wide && !(t.v_log >= STQ_VLOG_SR && changes) &&
                          t.numel < (1ull << 32) && aligned(t.m_scales_in, 16) && aligned(t.v_scales_in, 16) &&
                          t.block >= 128 && t.block <= (uint32_t)stq::kFastMaxBlock;   // (one or two rows of a warp)
     const uint64_t nf = fast_ok ? t.numel / stq::kTile : 0;
@@ -286,7 +290,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   const size_t off_sched = (off_map + bytes_map + 255) & ~size_t(255);
   uint64_t n_seg = 0;
   for (int l = 0; l < L; ++l) n_seg += ((uint64_t)nfast[l] + nslow[l] + stq::kStatSegTiles - 1) / stq::kStatSegTiles;
-  const size_t off_seg = (off_sched + 2 * sizeof(stq::FastSched) + 255) & ~size_t(255);
+  const size_t off_seg = (off_sched + 3 * sizeof(stq::FastSched) + 255) & ~size_t(255);
   int rc;
   if ((rc = grow_stage(h, off_seg + sizeof(uint32_t) * (size_t)n_seg)) != STQ_OK) return rc;
   if ((rc = grow(h, h->d_seg_map, h->d_seg_map_cap, (size_t)n_seg)) != STQ_OK) return rc;
@@ -307,80 +311,82 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
     return body_key(tensors[a]) < body_key(tensors[b]);
   });
   std::vector<uint32_t> fast0(L);
-  // two work lists: hs for the fused bodies, hs2 (one group) for the tensors that change width in this step
+  // three work lists: hs[0] for the fused bodies of the default and "pl" codes, hs[1] for the fused bodies of
+  // the "sr" and "ts" codes (its own launch: its own register allocation), hs[2] (one group) for the tensors
+  // that change width in this step
   stq::FastSched* hs = reinterpret_cast<stq::FastSched*>(st + off_sched);
-  stq::FastSched* hs2 = hs + 1;
-  std::memset(hs, 0, 2 * sizeof(*hs));
-  uint32_t split_begin = 0;
+  std::memset(hs, 0, 3 * sizeof(*hs));
+  uint32_t list_begin[4] = {0, 0, 0, 0};
   {
     // groups of equal body, and an estimate of their cost for the initial spread of the CTAs
     // (relative cost per tile from measurement: 8- and 16-bit log codes and 3-bit packing cost more;
     // the estimate only decides where CTAs start, the balance itself is dynamic)
-    double cost[stq::kFastMaxGroups] = {0.0};
+    double cost[2][stq::kFastMaxGroups] = {{0.0}, {0.0}};
     uint32_t next_fast = 0;
-    int last_key = -1;
-    bool in_split = false;
+    int last_key = -1, cur = 0;
     for (int i = 0; i < L; ++i) {
       const int l = order[i];
       fast0[l] = next_fast;
       if (nfast[l] == 0) continue;
       const stq_tensor& t = tensors[l];
       const int key = body_key(t);
-      if (key == kSplitKey) {           // sorted last: everything from here on belongs to the second work list
-        if (!in_split) { in_split = true; split_begin = next_fast; }
-        if (!same_map)
-          for (uint32_t k = 0; k < nfast[l]; ++k) hm[next_fast + k] = (uint32_t)l;
-        next_fast += nfast[l];
-        continue;
+      const int list = key == kSplitKey ? 2 : key >= kVariantKey ? 1 : 0;     // (keys are sorted: lists follow one another)
+      while (cur < list) list_begin[++cur] = next_fast;
+      if (list < 2) {
+        stq::FastSched* q = hs + list;
+        if (key != last_key && q->ng < (uint32_t)stq::kFastMaxGroups) {
+          q->grp_begin[q->ng++] = next_fast;
+          last_key = key;
+        }
+        cost[list][q->ng - 1] += body_cost(t) * nfast[l];
       }
-      if (key != last_key && hs->ng < (uint32_t)stq::kFastMaxGroups) {
-        hs->grp_begin[hs->ng++] = next_fast;
-        last_key = key;
-      }
-      cost[hs->ng - 1] += body_cost(t) * nfast[l];
       if (!same_map)
         for (uint32_t k = 0; k < nfast[l]; ++k) hm[next_fast + k] = (uint32_t)l;
       next_fast += nfast[l];
     }
-    if (!in_split) split_begin = next_fast;
-    hs->grp_begin[hs->ng] = split_begin;
+    while (cur < 3) list_begin[++cur] = next_fast;
     // chunk size: the usual one when every CTA gets several chunks, down to single tiles for small launches
     auto chunk_for = [&](uint64_t tiles) {
       const uint64_t per_cta = tiles / (uint64_t)std::max(1, h->fast_grid);
       return (uint32_t)std::min<uint64_t>(stq::kFastChunk, std::max<uint64_t>(1, per_cta / 4));
     };
-    hs->chunk = chunk_for(split_begin);
-    hs2->ng = 1;
-    hs2->grp_begin[0] = split_begin;
-    hs2->grp_begin[1] = next_fast;
-    hs2->chunk = chunk_for(next_fast - split_begin);     // (cta_group stays 0: every CTA starts in the one group)
+    for (int list = 0; list < 3; ++list) hs[list].chunk = chunk_for(list_begin[list + 1] - list_begin[list]);
+    hs[0].grp_begin[hs[0].ng] = list_begin[1];
+    hs[1].grp_begin[hs[1].ng] = list_begin[2];
+    hs[2].ng = 1;
+    hs[2].grp_begin[0] = list_begin[2];
+    hs[2].grp_begin[1] = list_begin[3];                   // (cta_group stays 0: every CTA starts in the one group)
     // CTAs per group in proportion to cost (largest remainders), at least one each
     const int G = h->fast_grid;
-    double total_cost = 0.0;
-    for (uint32_t g = 0; g < hs->ng; ++g) total_cost += cost[g];
-    std::vector<int> share(hs->ng, 0);
-    std::vector<std::pair<double, int>> rem;
-    int given = 0;
-    for (uint32_t g = 0; g < hs->ng; ++g) {
-      const double exact = total_cost > 0 ? cost[g] / total_cost * G : 0.0;
-      share[g] = std::max(1, (int)exact);
-      given += share[g];
-      rem.push_back({exact - (int)exact, (int)g});
+    for (int list = 0; list < 2; ++list) {
+      stq::FastSched* q = hs + list;
+      if (q->ng == 0) continue;
+      double total_cost = 0.0;
+      for (uint32_t g = 0; g < q->ng; ++g) total_cost += cost[list][g];
+      std::vector<int> share(q->ng, 0);
+      std::vector<std::pair<double, int>> rem;
+      int given = 0;
+      for (uint32_t g = 0; g < q->ng; ++g) {
+        const double exact = total_cost > 0 ? cost[list][g] / total_cost * G : 0.0;
+        share[g] = std::max(1, (int)exact);
+        given += share[g];
+        rem.push_back({exact - (int)exact, (int)g});
+      }
+      std::sort(rem.begin(), rem.end(), [](const std::pair<double, int>& a, const std::pair<double, int>& b) {
+        return a.first > b.first;
+      });
+      for (size_t k = 0; given < G && !rem.empty(); ++k, ++given) share[rem[k % rem.size()].second]++;
+      // Groups are ordered by v width, i.e. from memory-bound bodies to instruction-bound ones.  CTA c
+      // and CTA c + (number of SMs) tend to share an SM, so the second wave is handed out in reverse:
+      // an SM then hosts one CTA from either end, and the issue slots the memory-bound one leaves idle
+      // serve the other.
+      std::vector<uint16_t> glist;
+      for (uint32_t g = 0; g < q->ng; ++g)
+        for (int k = 0; k < share[g] && (int)glist.size() < G; ++k) glist.push_back((uint16_t)g);
+      while ((int)glist.size() < G) glist.push_back((uint16_t)(glist.size() % q->ng));
+      const int wave = std::min(G, h->sm_count);
+      for (int c = 0; c < G; ++c) q->cta_group[c] = c < wave ? glist[c] : glist[G - 1 - (c - wave)];
     }
-    std::sort(rem.begin(), rem.end(), [](const std::pair<double, int>& a, const std::pair<double, int>& b) {
-      return a.first > b.first;
-    });
-    for (size_t k = 0; given < G && !rem.empty(); ++k, ++given) share[rem[k % rem.size()].second]++;
-    // Groups are ordered by v width, i.e. from memory-bound bodies to instruction-bound ones.  CTA c
-    // and CTA c + (number of SMs) tend to share an SM, so the second wave is handed out in reverse:
-    // an SM then hosts one CTA from either end, and the issue slots the memory-bound one leaves idle
-    // serve the other.
-    std::vector<uint16_t> glist;
-    for (uint32_t g = 0; g < hs->ng; ++g)
-      for (int k = 0; k < share[g] && (int)glist.size() < G; ++k) glist.push_back((uint16_t)g);
-    while ((int)glist.size() < G) glist.push_back((uint16_t)(hs->ng ? glist.size() % hs->ng : 0));
-    const int wave = std::min(G, h->sm_count);
-    for (int c = 0; c < G; ++c) hs->cta_group[c] = c < wave ? glist[c] : glist[G - 1 - (c - wave)];
   }
   uint32_t next_narrow = (uint32_t)fast, next_wide = (uint32_t)(fast + slow_narrow);
   uint32_t* hseg = reinterpret_cast<uint32_t*>(st + off_seg);
@@ -423,7 +429,7 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   STQ_CUDA(h, cudaMemcpyAsync(h->d_table, ht, bytes_table, cudaMemcpyHostToDevice, stream));
   if (!same_map)
     STQ_CUDA(h, cudaMemcpyAsync(h->d_tile_map, hm, bytes_map, cudaMemcpyHostToDevice, stream));
-  STQ_CUDA(h, cudaMemcpyAsync(h->d_sched, hs, 2 * sizeof(stq::FastSched), cudaMemcpyHostToDevice, stream));
+  STQ_CUDA(h, cudaMemcpyAsync(h->d_sched, hs, 3 * sizeof(stq::FastSched), cudaMemcpyHostToDevice, stream));
   if (!same_map)
     STQ_CUDA(h, cudaMemcpyAsync(h->d_seg_map, hseg, sizeof(uint32_t) * (size_t)n_seg, cudaMemcpyHostToDevice, stream));
   h->n_seg = (uint32_t)n_seg;
@@ -438,7 +444,8 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   for (int l = 0; l < L; ++l) h->any_lp = h->any_lp || (kind == kKindStep && tensors[l].lp_dtype != STQ_LP_NONE);
   h->n_tiles = (uint32_t)total;
   h->n_fast = (uint32_t)fast;
-  h->n_main = split_begin;
+  h->n_main = list_begin[1];
+  h->n_var_end = list_begin[2];
   h->n_narrow = (uint32_t)(fast + slow_narrow);
   return STQ_OK;
 }
@@ -474,13 +481,19 @@ int run(stq_handle* h, stq::Mode mode, int grad_dtype, bool stats, const stq::St
   if (both) STQ_CUDA(h, cudaEventRecord(h->ev_join, h->side));
   if (h->n_main > 0) {   // only a step table has fast tiles
     const bool amp = h->any_lp || sc.inv_scale != nullptr || sc.dev_scalars != nullptr;
-    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, amp, false, h->d_table, h->d_tile_map, h->d_sched, sc,
+    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, amp, 0, h->d_table, h->d_tile_map, h->d_sched, sc,
                                       partials, h->d_err, h->fast_grid, stream));
     h->launches++;
   }
-  if (h->n_fast > h->n_main) {   // tensors that change width inside this step
-    const int grid = (int)std::min<uint32_t>((uint32_t)h->fast_grid, h->n_fast - h->n_main);
-    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, true, true, h->d_table, h->d_tile_map, h->d_sched + 1, sc,
+  if (h->n_var_end > h->n_main) {   // tensors whose second moment uses the "sr" or the "ts" code
+    const int grid = (int)std::min<uint32_t>((uint32_t)h->fast_grid, h->n_var_end - h->n_main);
+    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, true, 1, h->d_table, h->d_tile_map, h->d_sched + 1, sc,
+                                      partials, h->d_err, grid, stream));
+    h->launches++;
+  }
+  if (h->n_fast > h->n_var_end) {   // tensors that change width inside this step
+    const int grid = (int)std::min<uint32_t>((uint32_t)h->fast_grid, h->n_fast - h->n_var_end);
+    STQ_CUDA(h, stq::launch_step_fast(grad_dtype, stats, true, 2, h->d_table, h->d_tile_map, h->d_sched + 2, sc,
                                       partials, h->d_err, grid, stream));
     h->launches++;
   }
@@ -553,7 +566,7 @@ int stq_create(stq_handle** out, int device) {
   if (cudaMalloc(reinterpret_cast<void**>(&h->d_err), 2 * sizeof(int)) != cudaSuccess ||
       cudaMemset(h->d_err, 0, 2 * sizeof(int)) != cudaSuccess ||
       cudaMalloc(reinterpret_cast<void**>(&h->d_scalars), 4 * sizeof(float)) != cudaSuccess ||
-      cudaMalloc(reinterpret_cast<void**>(&h->d_sched), 2 * sizeof(stq::FastSched)) != cudaSuccess) {
+      cudaMalloc(reinterpret_cast<void**>(&h->d_sched), 3 * sizeof(stq::FastSched)) != cudaSuccess) {
     cudaEventDestroy(h->stage_ev);
     delete h;
     return STQ_E_WORKSPACE;

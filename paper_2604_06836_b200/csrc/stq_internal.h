@@ -96,8 +96,9 @@ struct FastSched {
 // The main step kernel (stq_step_fast.cu) with `grid` CTAs.  err_flag is set to 1 if a bounded wait
 // inside the kernel ran out.
 // amp: some tensor wants a low-precision copy, or the gradients are loss-scaled.
-// split: the launch over the tiles of tensors whose widths change inside the step (its own work list).
-cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, bool split, const TensorDesc* table,
+// list: 0 the fused bodies of the default and "pl" codes, 1 the fused bodies of the "sr" and "ts" codes, 2 the
+// tiles of tensors whose widths change inside the step (each its own work list and instantiation).
+cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, int list, const TensorDesc* table,
                              const uint32_t* tile_map, FastSched* sched, const StepConsts& sc, double* partials,
                              int* err_flag, int grid, cudaStream_t stream);
 int fast_ctas_per_sm();

@@ -52,8 +52,8 @@ constexpr int kOffMc = 8 * kTile;
 constexpr int kOffVc = 10 * kTile;
 constexpr int kScaleBytes = (kTile / 128) * 4;   // block scales of one state of the tile, at most
 constexpr int kOffMs = 12 * kTile;
-constexpr int kOffVs = kOffMs + kScaleBytes;
-constexpr int kStageBytes = 12 * kTile + 2 * kScaleBytes;
+constexpr int kOffVs = kOffMs + kScaleBytes;       // (the two-scale code of v keeps two floats per block)
+constexpr int kStageBytes = 12 * kTile + 3 * kScaleBytes;
 static_assert(kScaleBytes % 16 == 0 && kStageBytes % 128 == 0, "bulk copies need 16-byte aligned destinations");
 
 // What the consumers need to know about a staged tile; written by the producer.
@@ -70,11 +70,15 @@ struct __align__(16) TileInfo {
   uint32_t tile;       // index of the tile in the launch's tile order; 0xFFFFFFFF closes the stream
   uint32_t out;        // width indices to write, m | v << 8 (same coding); equal to the low half of `packed`
                        // unless the step changes the widths of this tensor
+  uint32_t sr_key;     // stochastic rounding: mix32(key of the tensor + high word of the element index)
+  uint32_t e0;         // low word of the index (inside its tensor) of the tile's first element
+  uint32_t pad[2];
 };
-static_assert(sizeof(TileInfo) == 64, "TileInfo is read with four 128-bit loads");
+constexpr int kInfoBytes = 80;
+static_assert(sizeof(TileInfo) == kInfoBytes, "TileInfo is read with five 128-bit loads");
 
 constexpr int kOffInfo = kStages * kStageBytes;
-constexpr int kOffBars = kOffInfo + kStages * 64;        // full[kStages], empty[kStages]
+constexpr int kOffBars = kOffInfo + kStages * kInfoBytes;        // full[kStages], empty[kStages]
 constexpr int kOffLut = kOffBars + 16 * kStages;         // 256 floats: decode table of the 8-bit log code, then
 constexpr int kSmemBytes = kOffLut + 2048;               // 256 integers: the same for its piecewise-linear variant
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: far beyond any copy; then give up
@@ -115,6 +119,12 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
+}
+
+// the mixing function of the stochastic-rounding code (a bijection of the 32-bit words)
+__device__ __forceinline__ uint32_t mix32(uint32_t h) {
+  h ^= h >> 16; h *= 0x85EBCA6Bu; h ^= h >> 13; h *= 0xC2B2AE35u; h ^= h >> 16;
+  return h;
 }
 
 __device__ __forceinline__ float sqrt_fast(float x) {
@@ -869,6 +879,354 @@ __device__ __forceinline__ void tile_body(const uint8_t* __restrict__ stage, con
   }
 }
 
+// ---- fused bodies of the "sr" and the "ts" code of the second moment ------------------------------------------
+// (their own launch and work list; the first moment, the moments and the update are those of tile_body)
+template <int B>
+__device__ __forceinline__ uint32_t code_of(const uint32_t (&w)[2], int k) {
+  if constexpr (B == 16) return (w[k >> 1] >> (16 * (k & 1))) & 0xFFFFu;
+  else return (w[0] >> (B * k)) & Wd<B>::mask;
+}
+// "sr": levels per octave 2^g, spacing of the levels in units of the bit pattern 2^sh, bit pattern of level 0
+template <int B>
+struct Sr {
+  static constexpr int g = B == 8 ? 3 : B == 16 ? 11 : 0;
+  static constexpr int sh = 23 - g;
+  static constexpr uint32_t floor_bits = 0x3F800000u - ((uint32_t)Wd<B>::K << sh);
+};
+constexpr float kOnePlus = 0x1.000008p+0f;      // 1 + 2^-21: lifts the block maximum to or just above 1
+
+// "ts": what a block's two scales give: everything the decode or the encode of its elements needs
+struct TsRow {
+  float W, inv_or_step, Phi;     // range in octaves; K / W (encode) or W / K (decode); P(hi)
+};
+template <int B>
+__device__ __forceinline__ TsRow ts_row(uint32_t hi_bits, uint32_t lo_bits, bool for_encode) {
+  TsRow t;
+  t.Phi = lg_poly(hi_bits);
+  const float de = (float)((int)(lo_bits >> 23) - (int)(hi_bits >> 23));
+  const float dp = __fadd_rn(lg_poly(lo_bits), -t.Phi);
+  float W = -__fadd_rn(de, dp);
+  W = W > 30.0f ? 30.0f : W;
+  t.W = W > 0.0f ? W : 0.0f;
+  if (for_encode) t.inv_or_step = t.W > 0.0f ? __fdiv_rn((float)Wd<B>::K, t.W) : 0.0f;
+  else t.inv_or_step = __fdiv_rn(t.W, (float)Wd<B>::K);
+  return t;
+}
+
+template <int BM, int BV, int VM, int GDT, bool AMP>
+__device__ __forceinline__ void tile_body_var(const uint8_t* __restrict__ stage, const TileInfo& ti, const StepConsts& sc,
+                                              int lane, int warp, uint32_t empty_bar, double* __restrict__ part,
+                                              float grad_mul) {
+  static_assert(VM == 2 || VM == 3, "2: stochastic rounding, 3: two scales per block");
+  static_assert(RP == 2, "rows are taken two per pass");
+  constexpr int K = Wd<BV>::K;
+  constexpr bool kSr = VM == 2, kTs = VM == 3;
+  const int lgB = (int)((ti.packed >> 16) & 0xFFu);
+  [[maybe_unused]] const uint32_t lp_dtype = ti.packed >> 24;
+  const float nlrwd = sc.l2_mode ? 0.0f : -ti.wdx;
+  f2 a0 = splat(0.f), a1 = splat(0.f), a2 = splat(0.f);
+  const f2 one2 = splat(sc.one);
+  // "sr" at <= 4 bits: the levels are s * 2^(level - K), the update's factor per level comes from a lane table
+  constexpr int LV = BV <= 4 ? BV : 2;
+  [[maybe_unused]] const float lvl = __uint_as_float((((uint32_t)lane & Wd<LV>::mask) + Wd<LV>::emin) << 23);
+
+#pragma unroll 1
+  for (int pass = 0; pass < R / RP; ++pass) {
+    const int row0 = warp * R + pass * RP;
+
+    // ---- "ts": the stored {hi, lo} of the two rows' blocks give range and step; lanes of equal parity work
+    // out the same row, lane r's copy is handed to everyone
+    [[maybe_unused]] float step_in[RP] = {0.f, 0.f};
+    if constexpr (kTs) {
+      const int blk_l = ((row0 + (lane & 1)) * kRowElems) >> lgB;
+      const float2 hl = *reinterpret_cast<const float2*>(stage + kOffVs + 8 * blk_l);
+      const TsRow tr = ts_row<BV>(__float_as_uint(hl.x), __float_as_uint(hl.y), false);
+#pragma unroll
+      for (int r = 0; r < RP; ++r) step_in[r] = __shfl_sync(kFull, tr.inv_or_step, r);
+    }
+
+    // ---- staged rows -> registers, decode -----------------------------------------------------------
+    f2 th[RP][2], g[RP][2], mt[RP][2], vt[RP][2];
+#pragma unroll
+    for (int r = 0; r < RP; ++r) {
+      const int elem = (row0 + r) * kRowElems + 4 * lane;
+      const float4 t4 = *reinterpret_cast<const float4*>(stage + kOffTheta + 4 * elem);
+      th[r][0] = make_float2(t4.x, t4.y);
+      th[r][1] = make_float2(t4.z, t4.w);
+      float gs[4];
+      lds_grad<GDT>(stage, elem, gs);
+      g[r][0] = make_float2(gs[0], gs[1]);
+      g[r][1] = make_float2(gs[2], gs[3]);
+      const int blk = ((row0 + r) * kRowElems) >> lgB;
+      const float sm = *reinterpret_cast<const float*>(stage + kOffMs + 4 * blk);
+      uint32_t w[2];
+      lds_codes<BM>(stage + kOffMc + (row0 + r) * (16 * BM), lane, w);
+      decode_lin_pairs<BM>(w, sm, mt[r]);
+      lds_codes<BV>(stage + kOffVc + (row0 + r) * (16 * BV), lane, w);
+      if constexpr (kSr) {
+        // level of code c: the float with bits(level 0) + (c << spacing), times the scale
+        const f2 s2 = splat(*reinterpret_cast<const float*>(stage + kOffVs + 4 * blk));
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+          vt[r][h] = mul2(s2, bits2(Sr<BV>::floor_bits + (code_of<BV>(w, 2 * h) << Sr<BV>::sh),
+                                    Sr<BV>::floor_bits + (code_of<BV>(w, 2 * h + 1) << Sr<BV>::sh)));
+      } else {
+        const float2 hl = *reinterpret_cast<const float2*>(stage + kOffVs + 8 * blk);
+        constexpr float off = kTwo23 + (float)K;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const f2 rf = add2(bits2(code_of<BV>(w, 2 * h) | kTwo23Bits, code_of<BV>(w, 2 * h + 1) | kTwo23Bits), splat(-off));
+          const f2 val = mul2(splat(hl.x), ex2_poly_pair(mul2(rf, splat(step_in[r])), one2));
+          // code 0 is the stored minimum itself
+          vt[r][h] = make_float2(rf.x == -(float)K ? hl.y : val.x, rf.y == -(float)K ? hl.y : val.y);
+        }
+      }
+    }
+    if (pass == R / RP - 1) {   // the last rows are in registers: this warp is done with the stage
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar);
+    }
+
+    if constexpr (AMP) {
+#pragma unroll
+      for (int r = 0; r < RP; ++r)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) g[r][h] = mul2(g[r][h], splat(grad_mul));
+    }
+    if (part != nullptr) {
+#pragma unroll
+      for (int r = 0; r < RP; ++r)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          a0 = fma2(g[r][h], one2, a0);
+          a1 = add2(a1, make_float2(fabsf(g[r][h].x), fabsf(g[r][h].y)));
+          a2 = fma2(g[r][h], g[r][h], a2);
+        }
+    }
+
+    // ---- moments ----------------------------------------------------------------------------------------
+    if (sc.l2_mode) {
+#pragma unroll
+      for (int r = 0; r < RP; ++r)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) g[r][h] = fma2(g[r][h], one2, mul2(splat(ti.wdx), th[r][h]));
+    }
+#pragma unroll
+    for (int r = 0; r < RP; ++r) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const f2 gk = g[r][h];
+        mt[r][h] = fma2(splat(sc.b1), mt[r][h], mul2(splat(sc.c1), gk));
+        vt[r][h] = fma2(splat(sc.b2), vt[r][h], mul2(mul2(splat(sc.c2), gk), gk));
+      }
+    }
+
+    // ---- block maxima (and, for "ts", minima) ---------------------------------------------------------------
+    uint32_t mxm[RP], mxv[RP];
+    [[maybe_unused]] uint32_t mnv[RP];
+#pragma unroll
+    for (int r = 0; r < RP; ++r) {
+      const float am = fmaxf(fmaxf(fabsf(mt[r][0].x), fabsf(mt[r][0].y)), fmaxf(fabsf(mt[r][1].x), fabsf(mt[r][1].y)));
+      const float av = fmaxf(fmaxf(vt[r][0].x, vt[r][0].y), fmaxf(vt[r][1].x, vt[r][1].y));
+      mxm[r] = __reduce_max_sync(kFull, __float_as_uint(am));
+      mxv[r] = __reduce_max_sync(kFull, __float_as_uint(av));
+      if constexpr (kTs) {
+        const float an = fminf(fminf(vt[r][0].x, vt[r][0].y), fminf(vt[r][1].x, vt[r][1].y));
+        mnv[r] = __reduce_min_sync(kFull, __float_as_uint(an));
+      }
+    }
+    if (lgB >= 8) {
+      mxm[0] = mxm[1] = max(mxm[0], mxm[1]);
+      mxv[0] = mxv[1] = max(mxv[0], mxv[1]);
+      if constexpr (kTs) mnv[0] = mnv[1] = min(mnv[0], mnv[1]);
+    }
+
+    // ---- per-block constants: one lane per (row, state) works them out, then they are broadcast --------
+    // lanes 0, 1: inv = fl(qmax * fl(1/s_m)) of rows 0, 1; "sr": lanes 2, 3: c1 = fl(fl(1/s_v) * (1 + 2^-21));
+    // "ts": lanes of equal parity work out the new range of their row, lane r's copy is handed to everyone.
+    // The same lanes store the new scales, for the rows that open a block (a zero block stores 0).
+    float inv_m[RP];
+    [[maybe_unused]] float c1[RP], tsW[RP], tsInv[RP], tsPhi[RP], tsLo[RP], tsHalf[RP];
+    {
+      uint32_t mine = (lane & 1) ? mxm[1] : mxm[0];
+      if constexpr (kSr) {
+        if (lane & RP) mine = (lane & 1) ? mxv[1] : mxv[0];
+      }
+      const float x = __uint_as_float(mine);
+      const bool zero = x < kTiny;
+      const float mul = (kSr && (lane & RP)) ? kOnePlus : (float)Wd<BM>::qmax;
+      const float val = zero ? 0.f : __fmul_rn(mul, __frcp_rn(x));
+      const int e_mine = (row0 + (lane & (RP - 1))) * kRowElems;
+      const bool opens = (e_mine & ((1 << lgB) - 1)) == 0;
+#pragma unroll
+      for (int r = 0; r < RP; ++r) inv_m[r] = __shfl_sync(kFull, val, r);
+      if constexpr (kSr) {
+        if (lane < 2 * RP && opens) ((lane & RP) ? ti.vso : ti.mso)[e_mine >> lgB] = zero ? 0.f : x;
+#pragma unroll
+        for (int r = 0; r < RP; ++r) c1[r] = __shfl_sync(kFull, val, RP + r);
+      } else {
+        const uint32_t hi_b = (lane & 1) ? mxv[1] : mxv[0];
+        const bool vz = __uint_as_float(hi_b) < kTiny;
+        // the minimum, raised to the floor 2^-30 below the maximum
+        const float lo = fmaxf(__uint_as_float((lane & 1) ? mnv[1] : mnv[0]), __fmul_rn(__uint_as_float(hi_b), 0x1p-30f));
+        TsRow tr = ts_row<BV>(hi_b, __float_as_uint(lo), true);
+        // an all-zero block: every code is 0 (one step over a range of one octave, with every distance clamped to it)
+        const float half_l = vz ? 0.f : __fmul_rn(0.5f, __fdiv_rn(tr.W, (float)K));     // half a code step, for the update
+        if (vz) { tr.W = 1.0f; tr.inv_or_step = (float)K; tr.Phi = 0.0f; }
+        if (lane < RP && opens) {
+          ti.mso[e_mine >> lgB] = zero ? 0.f : x;
+          *reinterpret_cast<float2*>(ti.vso + 2 * (e_mine >> lgB)) = vz ? make_float2(0.f, 0.f) : make_float2(__uint_as_float(hi_b), lo);
+        }
+#pragma unroll
+        for (int r = 0; r < RP; ++r) {
+          tsW[r] = __shfl_sync(kFull, tr.W, r);
+          tsInv[r] = __shfl_sync(kFull, tr.inv_or_step, r);
+          tsPhi[r] = __shfl_sync(kFull, tr.Phi, r);
+          tsLo[r] = __shfl_sync(kFull, vz ? 0.f : lo, r);
+          tsHalf[r] = __shfl_sync(kFull, half_l, r);
+        }
+      }
+    }
+
+    // ---- "sr" at <= 4 bits: what each level of each row contributes to the update, one level per lane -----
+    [[maybe_unused]] float lut_upd = 0.f;
+    if constexpr (kSr && BV <= 4) {
+      constexpr float invq = 1.0f / (float)Wd<BM>::qmax;
+      const bool second = (lane >> LV) & 1;
+      const float svr = __uint_as_float(second ? mxv[1] : mxv[0]);
+      const float smr = __uint_as_float(second ? mxm[1] : mxm[0]);
+      const float vl = __fmul_rn(svr < kTiny ? 0.f : svr, lvl);
+      const float den = __fmaf_rn(sqrt_fast(vl), sc.rsqrt_bc2, sc.eps);
+      lut_upd = __fmul_rn(__fmul_rn(__fmul_rn(smr, sc.step_size), invq), rcp_fast(den));
+    }
+
+    // ---- quantize, pack, store; update the parameters ---------------------------------------------------
+    float* param = ti.param + row0 * kRowElems + 4 * lane;
+#pragma unroll
+    for (int r = 0; r < RP; ++r) {
+      constexpr float invq = 1.0f / (float)Wd<BM>::qmax;
+      const float sm_raw = __uint_as_float(mxm[r]);
+      const float sv_raw = __uint_as_float(mxv[r]);
+      const bool vzero = sv_raw < kTiny;
+      f2 nq[2], out[2];
+      encode_lin_pairs<BM>(ti.mco + (row0 + r) * (16 * BM), lane, mt[r], inv_m[r], nq);
+      [[maybe_unused]] const float unit = __fmul_rn(__fmul_rn(sm_raw, sc.step_size), invq);
+      uint8_t* vrow = ti.vco + (row0 + r) * (16 * BV);
+      if constexpr (kSr) {
+        // y = fl(x * c1) clamped to [level 0, 1]; n = bits(1.0) - bits(y); j = ((n << (9+g)) + word) >> 32 level
+        // steps below the maximum (at most K by the clamp), code K - j.  The element's word is
+        // mix32(index ^ key); index = row's first + 4*lane + k, and the first xor-shift of the chain is shared
+        // by the lane's four elements (k touches the two lowest bits only).
+        const uint32_t base = (ti.e0 + (uint32_t)((row0 + r) * kRowElems + 4 * lane)) ^ ti.sr_key;
+        const uint32_t base1 = base ^ (base >> 16);
+        const float floor_y = __uint_as_float(Sr<BV>::floor_bits);
+        uint32_t code[4];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const f2 y = mul2(vt[r][h], splat(c1[r]));
+          const float yc[2] = {fminf(fmaxf(y.x, floor_y), 1.0f), fminf(fmaxf(y.y, floor_y), 1.0f)};
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            const int k = 2 * h + q;
+            uint32_t wd = (base1 ^ (uint32_t)k) * 0x85EBCA6Bu;
+            wd ^= wd >> 13; wd *= 0xC2B2AE35u; wd ^= wd >> 16;
+            const uint32_t n = 0x3F800000u - __float_as_uint(yc[q]);
+            const uint32_t j = (uint32_t)((((unsigned long long)n << (9 + Sr<BV>::g)) + wd) >> 32);
+            code[k] = (uint32_t)K - j;
+          }
+        }
+        pack_store_row<BV>(vrow, lane, code, 0u);
+        if constexpr (BV <= 4) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const f2 base_t = fma2(th[r][h], splat(nlrwd), th[r][h]);
+            const f2 fac = make_float2(__shfl_sync(kFull, lut_upd, code[2 * h] | (uint32_t)(r << LV)),
+                                       __shfl_sync(kFull, lut_upd, code[2 * h + 1] | (uint32_t)(r << LV)));
+            out[h] = fma2(nq[h], fac, base_t);
+          }
+        } else {
+          const float srt = __fmul_rn(sqrt_fast(vzero ? 0.f : sv_raw), sc.rsqrt_bc2);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const f2 sq = make_float2(sqrt_fast(__uint_as_float(Sr<BV>::floor_bits + (code[2 * h] << Sr<BV>::sh))),
+                                      sqrt_fast(__uint_as_float(Sr<BV>::floor_bits + (code[2 * h + 1] << Sr<BV>::sh))));
+            const f2 den = fma2(sq, splat(srt), splat(sc.eps));
+            const f2 base_t = fma2(th[r][h], splat(nlrwd), th[r][h]);
+            out[h] = fma2(mul2(nq[h], splat(unit)), make_float2(rcp_fast(den.x), rcp_fast(den.y)), base_t);
+          }
+        }
+      } else {
+        // d(x) = split logarithm of x / hi, clamped to [-W, 0]; code - K = round-half-even(d * K / W)
+        const uint32_t ebase = kMagicBits - (vzero ? (uint32_t)kZeroBlockExp : (mxv[r] >> 23));
+        const float half_step = tsHalf[r];
+        const float srt_hi = __fmul_rn(sqrt_fast(vzero ? 0.f : sv_raw), sc.rsqrt_bc2);
+        const float den_lo = __fmaf_rn(sqrt_fast(tsLo[r]), sc.rsqrt_bc2, sc.eps);
+        uint32_t x[4];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t b0 = __float_as_uint(vt[r][h].x), b1 = __float_as_uint(vt[r][h].y);
+          const f2 de = add2(bits2(ebase + (b0 >> 23), ebase + (b1 >> 23)), splat(-kMagic));
+          const f2 dp = fma2(lg_poly_pair(b0, b1), one2, splat(-tsPhi[r]));
+          f2 d = add2(de, dp);
+          d = make_float2(fminf(fmaxf(d.x, -tsW[r]), 0.0f), fminf(fmaxf(d.y, -tsW[r]), 0.0f));
+          const f2 t = fma2(d, splat(tsInv[r]), splat(kMagic));
+          x[2 * h] = __float_as_uint(t.x);
+          x[2 * h + 1] = __float_as_uint(t.y);
+          // sqrt of the decoded level: sqrt(hi) * 2^((code-K) * W/K / 2), or sqrt(lo) for code 0
+          const f2 rr = add2(t, splat(-kMagic));
+          const f2 arg = mul2(rr, splat(half_step));
+          f2 den = fma2(make_float2(ex2_fast(arg.x), ex2_fast(arg.y)), splat(srt_hi), splat(sc.eps));
+          den = make_float2(rr.x == -(float)K ? den_lo : den.x, rr.y == -(float)K ? den_lo : den.y);
+          const f2 base_t = fma2(th[r][h], splat(nlrwd), th[r][h]);
+          out[h] = fma2(mul2(nq[h], splat(unit)), make_float2(rcp_fast(den.x), rcp_fast(den.y)), base_t);
+        }
+        pack_store_row<BV>(vrow, lane, x, kMagicBits - (uint32_t)K);
+      }
+      *reinterpret_cast<float4*>(param + r * kRowElems) = make_float4(out[0].x, out[0].y, out[1].x, out[1].y);
+      if constexpr (AMP) {
+        if (ti.lp != nullptr) {
+          const float o4[4] = {out[0].x, out[0].y, out[1].x, out[1].y};
+          *reinterpret_cast<uint2*>(ti.lp + (row0 + r) * kRowElems + 4 * lane) = pack_lp(o4, lp_dtype);
+        }
+      }
+    }
+  }
+
+  if (part != nullptr) {
+    const float s0 = a0.x + a0.y, s1 = a1.x + a1.y, s2 = a2.x + a2.y;
+    const bool hi = lane & 16;
+    float x = (hi ? s2 : s0) + __shfl_xor_sync(kFull, hi ? s0 : s2, 16);
+    float y = (hi ? 0.f : s1) + __shfl_xor_sync(kFull, hi ? s1 : 0.f, 16);
+    const bool q = lane & 8;
+    float z = (q ? y : x) + __shfl_xor_sync(kFull, q ? x : y, 8);
+    z += __shfl_xor_sync(kFull, z, 4);
+    z += __shfl_xor_sync(kFull, z, 2);
+    z += __shfl_xor_sync(kFull, z, 1);
+    if ((lane & 7) == 0 && lane < 24) part[lane >> 3] = (double)z;
+  }
+}
+
+template <int GDT, bool AMP>
+__device__ __forceinline__ void dispatch_variant(const uint8_t* __restrict__ stage, const TileInfo& ti, const StepConsts& sc,
+                                                 int lane, int warp, uint32_t ebar, double* __restrict__ part, float grad_mul) {
+#define STQ_VCASE(IM, IV, BM, BV, VM) \
+  case IM * 10 + IV: tile_body_var<BM, BV, VM, GDT, AMP>(stage, ti, sc, lane, warp, ebar, part, grad_mul); break;
+#define STQ_VCASES_M(IM, BM)                                                                              \
+  STQ_VCASE(IM, 0, BM, 2, 2) STQ_VCASE(IM, 1, BM, 3, 2) STQ_VCASE(IM, 2, BM, 4, 2) STQ_VCASE(IM, 3, BM, 8, 2) \
+  STQ_VCASE(IM, 4, BM, 16, 2) STQ_VCASE(IM, 5, BM, 2, 3) STQ_VCASE(IM, 6, BM, 3, 3) STQ_VCASE(IM, 7, BM, 4, 3) \
+  STQ_VCASE(IM, 8, BM, 8, 3) STQ_VCASE(IM, 9, BM, 16, 3)
+  switch ((ti.packed & 0xFFu) * 10 + (((ti.packed >> 8) & 0xFFu) - 7u)) {
+    STQ_VCASES_M(0, 2)
+    STQ_VCASES_M(1, 3)
+    STQ_VCASES_M(2, 4)
+    STQ_VCASES_M(3, 8)
+    STQ_VCASES_M(4, 16)
+    default: break;
+  }
+#undef STQ_VCASES_M
+#undef STQ_VCASE
+}
+
 // Calls f with the width behind a width index as a compile-time constant (warp-uniform switch).
 template <class F>
 __device__ __forceinline__ void with_m_width(uint32_t idx, F&& f) {
@@ -1056,9 +1414,10 @@ __device__ __forceinline__ uint32_t width_index(uint32_t b) { return b == 2 ? 0u
 
 // AMP: the mixed-precision extras (gradient unscaling, low-precision parameter copy) are compiled
 // in only for launches that use them, so the plain step pays nothing for them.
-// SPLIT: the launch over the tiles of tensors that change width inside the step (one runtime-width
-// body); compiled apart from the fused bodies so that it cannot disturb their register allocation.
-template <int GDT, bool AMP, bool SPLIT>
+// LIST: which work list the launch serves, each compiled apart so that none disturbs the register allocation
+// of another: 0 the fused bodies of the default and "pl" codes, 1 the fused bodies of the "sr" and "ts" codes
+// of the second moment, 2 the tiles of tensors that change width inside the step (one runtime-width body).
+template <int GDT, bool AMP, int LIST>
 __global__ void __launch_bounds__(kFastThreads, kFastCtasPerSm)
 stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map,
                      FastSched* __restrict__ sched, const StepConsts sc_in, double* __restrict__ partials,
@@ -1137,34 +1496,42 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
         const uint32_t bm = T->bm_in, bv = T->bv_in, bmo = T->bm_out, bvo = T->bv_out;
         const uint32_t lgB = T->block == 128 ? 7u : T->block == 256 ? 8u : 9u;
         const uint32_t nb_m = (kTile / 8) * bm, nb_v = (kTile / 8) * bv, nb_s = (uint32_t)(kTile * 4) >> lgB;
+        const uint32_t vmode = LIST == 1 ? T->v_mode : (T->v_mode & 1u);
+        const uint32_t spb = vmode == 3u ? 2u : 1u;          // scales per block of v: two in the two-scale code
         TileInfo ti;
         ti.param = T->param + e0;
         ti.mco = T->mc_out + (e0 >> 3) * bmo;
         ti.vco = T->vc_out + (e0 >> 3) * bvo;
         ti.mso = T->ms_out + (e0 >> lgB);
-        ti.vso = T->vs_out + (e0 >> lgB);
+        ti.vso = T->vs_out + spb * (e0 >> lgB);
         ti.lp = T->param_lp ? reinterpret_cast<uint16_t*>(T->param_lp) + e0 : nullptr;
-        ti.packed = width_index(bm) | ((width_index(bv) + (T->v_mode == 1u && bv >= 8u ? 2u : 0u)) << 8) | (lgB << 16) |
-                    (T->lp_dtype << 24);
+        // v index: 0..4 the widths in the default code, 5, 6: 8 and 16 bits in the "pl" code, 7..11 the widths in the
+        // "sr" code, 12..16 in the "ts" code
+        const uint32_t iv = vmode >= 2u ? width_index(bv) + (vmode == 2u ? 7u : 12u)
+                                        : width_index(bv) + (vmode == 1u && bv >= 8u ? 2u : 0u);
+        ti.packed = width_index(bm) | (iv << 8) | (lgB << 16) | (T->lp_dtype << 24);
         ti.wdx = sc.l2_mode ? T->wd : (float)(sc.lr * (double)T->wd);
         ti.tile = tile;
-        ti.out = width_index(bmo) | ((width_index(bvo) + (T->v_mode == 1u && bvo >= 8u ? 2u : 0u)) << 8);
+        ti.out = width_index(bmo) | ((width_index(bvo) + (vmode == 1u && bvo >= 8u ? 2u : 0u)) << 8);
+        ti.sr_key = LIST == 1 ? mix32(mix32(T->sr_id ^ sc.sr_h) + (uint32_t)(e0 >> 32)) : 0u;
+        ti.e0 = (uint32_t)e0;
+        ti.pad[0] = ti.pad[1] = 0u;
         const uint8_t* src_g = reinterpret_cast<const uint8_t*>(T->grad) + e0 * gsz;
         const uint8_t* src_mc = T->mc_in + (e0 >> 3) * bm;
         const uint8_t* src_vc = T->vc_in + (e0 >> 3) * bv;
         const float* src_ms = T->ms_in + (e0 >> lgB);
-        const float* src_vs = T->vs_in + (e0 >> lgB);
+        const float* src_vs = T->vs_in + spb * (e0 >> lgB);
         if (issued >= (uint32_t)kStages && !mbar_wait(empty0 + 8 * s, phase ^ 1u)) { ok = false; break; }
-        *reinterpret_cast<TileInfo*>(smem + kOffInfo + 64 * s) = ti;
+        *reinterpret_cast<TileInfo*>(smem + kOffInfo + kInfoBytes * s) = ti;
         const uint32_t bar = full0 + 8 * s;
         const uint32_t dst = smem_u32(smem + s * kStageBytes);
-        mbar_expect_tx(bar, kTile * 4 + kTile * gsz + nb_m + nb_v + 2 * nb_s);
+        mbar_expect_tx(bar, kTile * 4 + kTile * gsz + nb_m + nb_v + (1u + spb) * nb_s);
         bulk_g2s(dst + kOffTheta, ti.param, kTile * 4, bar);
         bulk_g2s(dst + kOffGrad, src_g, kTile * gsz, bar);
         bulk_g2s(dst + kOffMc, src_mc, nb_m, bar);
         bulk_g2s(dst + kOffVc, src_vc, nb_v, bar);
         bulk_g2s(dst + kOffMs, src_ms, nb_s, bar);
-        bulk_g2s(dst + kOffVs, src_vs, nb_s, bar);
+        bulk_g2s(dst + kOffVs, src_vs, spb * nb_s, bar);
         ++issued;
 #pragma unroll
         for (int k = 0; k < kStages; ++k)
@@ -1178,7 +1545,7 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
     // none lands in shared memory that no longer belongs to this CTA.
     if (ok && issued >= (uint32_t)kStages) ok = mbar_wait(empty0 + 8 * s, phase ^ 1u);
     if (ok) {
-      reinterpret_cast<TileInfo*>(smem + kOffInfo + 64 * s)->tile = kEnd;
+      reinterpret_cast<TileInfo*>(smem + kOffInfo + kInfoBytes * s)->tile = kEnd;
       mbar_arrive(full0 + 8 * s);
     } else {
       atomicExch(err_flag, 1);
@@ -1198,7 +1565,7 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
       break;
     }
     const uint8_t* stage = smem + s * kStageBytes;
-    const TileInfo ti = *reinterpret_cast<const TileInfo*>(smem + kOffInfo + 64 * s);
+    const TileInfo ti = *reinterpret_cast<const TileInfo*>(smem + kOffInfo + kInfoBytes * s);
     if (ti.tile == kEnd) break;
     const uint32_t ebar = empty0 + 8 * s;
     double* part = partials ? partials + ((size_t)ti.tile * kConsumerWarps + warp) * 3 : nullptr;
@@ -1208,8 +1575,10 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
 #define STQ_CASES_M(IM, BM)                                                                                   \
   STQ_CASE(IM, 0, BM, 2, false) STQ_CASE(IM, 1, BM, 3, false) STQ_CASE(IM, 2, BM, 4, false) STQ_CASE(IM, 3, BM, 8, false) \
   STQ_CASE(IM, 4, BM, 16, false) STQ_CASE(IM, 5, BM, 8, true) STQ_CASE(IM, 6, BM, 16, true)
-    if constexpr (SPLIT) {
+    if constexpr (LIST == 2) {
       tile_body_split<GDT, AMP>(stage, ti, sc, lut8, lane, warp, ebar, part, grad_mul);
+    } else if constexpr (LIST == 1) {
+      dispatch_variant<GDT, AMP>(stage, ti, sc, lane, warp, ebar, part, grad_mul);
     } else {
       switch ((ti.packed & 0xFFu) * 7 + ((ti.packed >> 8) & 0xFFu)) {
         STQ_CASES_M(0, 2)
@@ -1239,10 +1608,10 @@ __global__ void stq_wait_timeout_selftest_kernel(int* __restrict__ err_flag, lon
   if (!done && threadIdx.x == 0) atomicExch(err_flag, 1);
 }
 
-template <int GDT, bool AMP, bool SPLIT>
+template <int GDT, bool AMP, int LIST>
 cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, FastSched* sched, const StepConsts& sc,
                           double* partials, int* err_flag, int grid, cudaStream_t stream) {
-  auto kern = stq_step_fast_kernel<GDT, AMP, SPLIT>;
+  auto kern = stq_step_fast_kernel<GDT, AMP, LIST>;
   // per device and cheap, so simply repeated: the kernel needs more than the default 48 KB
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
@@ -1255,7 +1624,7 @@ cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, Fas
 
 }  // namespace
 
-cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, bool split, const TensorDesc* table,
+cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, int list, const TensorDesc* table,
                              const uint32_t* tile_map, FastSched* sched, const StepConsts& sc, double* partials,
                              int* err_flag, int grid, cudaStream_t stream) {
   double* p = stats ? partials : nullptr;
@@ -1266,14 +1635,17 @@ cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, bool split, c
     case 1: STQ_LAUNCH(1, A, S);        \
     default: STQ_LAUNCH(2, A, S);       \
   }
-  if (split) {
+  if (list == 2) {
     // the mixed-precision extras cost this body nothing measurable: one variant serves both
-    STQ_LAUNCH_G(true, true)
+    STQ_LAUNCH_G(true, 2)
+  }
+  if (list == 1) {
+    STQ_LAUNCH_G(true, 1)
   }
   if (amp) {
-    STQ_LAUNCH_G(true, false)
+    STQ_LAUNCH_G(true, 0)
   }
-  STQ_LAUNCH_G(false, false)
+  STQ_LAUNCH_G(false, 0)
 #undef STQ_LAUNCH_G
 #undef STQ_LAUNCH
 }
@@ -1285,7 +1657,7 @@ cudaError_t launch_wait_timeout_selftest(int* err_flag, cudaStream_t stream) {
 
 int fast_ctas_per_sm() {
   int n = 0;
-  auto kern = stq_step_fast_kernel<1, false, false>;
+  auto kern = stq_step_fast_kernel<1, false, 0>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return 1;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kFastThreads, kSmemBytes) != cudaSuccess) return 1;
   return n > 0 ? n : 1;

@@ -77,15 +77,20 @@ def test_full_size_sampled_blocks(name, gib):
     assert job.state_bytes() < 0.25 * 8 * w.total_params     # far below the fp32 states
 
 
-@pytest.mark.parametrize("name,gib,full_steps", [("cfg2", 8, None), ("cfg3", 6, None), ("cfg4", 30, 3), ("cfg5", 60, 3)])
+@pytest.mark.parametrize("name,gib,full_steps", [("cfg2", 8, None), ("cfg3", 6, None), ("cfg4", 30, 3), ("cfg5", 60, 3),
+                                                 ("cfg2:sr", 8, 6), ("cfg3:ts", 6, 6), ("cfg2:ts", 8, 3), ("cfg3:sr", 6, 3)])
 def test_full_size_every_element(name, gib, full_steps):
     """Whole buffers against the oracle: every code byte, every scale, every parameter, on every step
     run (all of them for cfg2 and cfg3; steps 1-3 for cfg4 and cfg5, which are decision steps with fused
     statistics).  cfg3 changes the widths of 10 % of its tensors on every decision step from t = 5 on,
-    alternately by stq_repack and inside the step."""
+    alternately by stq_repack and inside the step.  The ":sr" and ":ts" cases run the first steps of a
+    configuration with the stochastic-rounding or the two-scale code of the second moment."""
     import harness as H
     _need(gib)
-    w = W.config(name)
+    w = W.config(name.split(":")[0])
+    if ":" in name:               # the same configuration with another code of the second moment (its fused bodies)
+        from dataclasses import replace
+        w = replace(w, v_log=name.split(":")[1])
     bm, bv, _ = W.draw_bits(w)
     job = Job(w, bm, bv)
     fo = H.FullOracle(job)
