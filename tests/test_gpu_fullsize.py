@@ -78,7 +78,7 @@ def test_full_size_sampled_blocks(name, gib):
 
 
 @pytest.mark.parametrize("name,gib,full_steps", [("cfg2", 8, None), ("cfg3", 6, None), ("cfg4", 30, 3), ("cfg5", 60, 3),
-                                                 ("cfg2:sr", 8, 6), ("cfg3:ts", 6, 6), ("cfg2:ts", 8, 3), ("cfg3:sr", 6, 3)])
+                                                 ("cfg2:sr", 8, 3), ("cfg3:ts", 6, 3)])
 def test_full_size_every_element(name, gib, full_steps):
     """Whole buffers against the oracle: every code byte, every scale, every parameter, on every step
     run (all of them for cfg2 and cfg3; steps 1-3 for cfg4 and cfg5, which are decision steps with fused
