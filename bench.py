@@ -490,7 +490,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the extra run with the integer-only v code")
-    ap.add_argument("--v-log", default="poly", choices=["poly", "pl"],
+    ap.add_argument("--v-log", default="poly", choices=["poly", "pl", "sr", "ts"],
                     help="variant of the v quantizer at widths 8 and 16 (default: the polynomial logarithm)")
     ap.add_argument("--shard", action="store_true",
                     help="strong scaling: each rank owns a block-aligned slice of the parameter list "

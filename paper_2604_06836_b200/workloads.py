@@ -137,6 +137,14 @@ def config(name: str) -> Workload:
         return Workload("roberta-large-356M-fp16", tuple(roberta_shapes()), seed=7, **amp)
     if name == "vit_b32":
         return Workload("vit-b32-88M-fp16", tuple(vit_shapes(patch=32, tokens=50)), seed=8, **amp)
+    if name.startswith("pair-"):
+        # one width pair on one large tensor ("pair-4-8": m at 4 bits, v at 8 bits; "pair-4-8-25": 2^25 elements):
+        # isolates one fused body of the step kernel for per-body throughput and profiler counters
+        parts = name.split("-")
+        bm, bv = int(parts[1]), int(parts[2])
+        lg = int(parts[3]) if len(parts) > 3 else 27
+        return Workload(name, (("w", (1 << lg,)),), 128, "bf16", "student_t", nu=3, scale_log10=(-3.0, -3.0),
+                        bits_kind="fixed", bits_fixed=(bm, bv), steps=20, decision_interval=1 << 30, seed=1)
     raise KeyError(name)
 
 
