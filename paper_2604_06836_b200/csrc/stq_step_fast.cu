@@ -1407,7 +1407,7 @@ __device__ __forceinline__ void tile_body_split(const uint8_t* __restrict__ stag
 // Scheduling: the fast tiles are grouped by body (width pair and variant of the v code).  A CTA starts in the group
 // the host assigned to it and takes chunks of consecutive tiles (kFastChunk of them, single tiles when the
 // launch is small) from that group's
-// counter; when its group runs dry it moves on to the next one that still has work.  So a CTA runs
+// counter; when its group runs dry it moves on to the one with the most tiles left.  So a CTA runs
 // few different bodies (a change of body is an instruction-cache refill), the tiles of a group are
 // streamed together, and the balance is dynamic.
 __device__ __forceinline__ uint32_t width_index(uint32_t b) { return b == 2 ? 0u : b == 3 ? 1u : b == 4 ? 2u : b == 8 ? 3u : 4u; }
@@ -1468,7 +1468,6 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
     if (lane != 0) return;
     const uint32_t ng = sched->ng, chunk = sched->chunk;
     uint32_t grp = sched->cta_group[blockIdx.x];
-    uint32_t dry = 0;          // consecutive groups found empty
     uint32_t issued = 0;
     int s = 0;
     uint32_t phase = 0;        // parity of the use of stage s that is being filled
@@ -1476,16 +1475,25 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
 #pragma unroll
     for (int k = 0; k < kStages; ++k) last_use[k] = 2u;
     bool ok = true;
-    while (ok && dry < ng) {
+    while (ok) {
       const uint32_t gbeg = sched->grp_begin[grp], gend = sched->grp_begin[grp + 1];
       const uint32_t c = atomicAdd(&sched->ctr[grp], 1u);
       const unsigned long long t0 = (unsigned long long)gbeg + (unsigned long long)c * chunk;
-      if (t0 >= gend) {        // this group has been handed out completely
-        ++dry;
-        grp = grp + 1 == ng ? 0u : grp + 1;
+      if (t0 >= gend) {
+        // This group has been handed out completely.  Move to the group with the most tiles left (a change
+        // of body is an instruction-cache refill: better paid once, for a long stay); none left: done.
+        // The counters only grow, so a group seen empty stays empty and no tile is missed.
+        uint32_t best = 0u, best_left = 0u;
+        for (uint32_t k = 0; k < ng; ++k) {
+          const unsigned long long size = sched->grp_begin[k + 1] - sched->grp_begin[k];
+          const unsigned long long taken = (unsigned long long)*reinterpret_cast<volatile uint32_t*>(&sched->ctr[k]) * chunk;
+          const uint32_t left = taken < size ? (uint32_t)(size - taken) : 0u;
+          if (left > best_left) { best_left = left; best = k; }
+        }
+        if (best_left == 0u) break;
+        grp = best;
         continue;
       }
-      dry = 0;
       const uint32_t t1 = (uint32_t)(t0 + chunk < gend ? t0 + chunk : gend);
       for (uint32_t tile = (uint32_t)t0; tile < t1; ++tile) {
         // Everything that can be prepared without the stage (table look-ups, addresses) comes before the
