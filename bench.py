@@ -31,7 +31,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter of the step kernel from the ncu captures
 # summarised in profiles/ (cfg5s is the cfg5 recipe on 6 layers), scaled by the parameters per launch.
-NCU_TRAFFIC_BYTES_PER_PARAM = {"cfg5": 12.367, "cfg5s": 12.367, "cfg2": 14.279}
+NCU_TRAFFIC_BYTES_PER_PARAM = {"cfg5": 12.376, "cfg5s": 12.376, "cfg2": 14.237}
 
 
 def dist_env():
