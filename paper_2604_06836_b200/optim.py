@@ -197,7 +197,7 @@ class STQAdamW(torch.optim.Optimizer):
     def state_dict(self):
         d = super().state_dict()
         d["stq"] = dict(t=self.t, bits_m=self.bits_m.copy(), bits_v=self.bits_v.copy(), v_log=self.v_log,
-                        block=self.block, policy=self.policy.state.copy(),
+                        block=self.block, policy=self.policy.state.copy(), sr_seed=self.sr_seed,
                         carried_stats=None if self._carried_stats is None else self._carried_stats.copy(),
                         states=[dict(m_codes=s.m_codes.clone(), m_scales=s.m_scales.clone(),
                                      v_codes=s.v_codes.clone(), v_scales=s.v_scales.clone()) for s in self.states])
@@ -212,6 +212,7 @@ class STQAdamW(torch.optim.Optimizer):
         self.t = int(q["t"])
         self.bits_m, self.bits_v = np.array(q["bits_m"], np.uint8), np.array(q["bits_v"], np.uint8)
         self.policy.state = q["policy"]
+        self.sr_seed = int(q.get("sr_seed", self.sr_seed))
         carried = q.get("carried_stats")
         self._carried_stats = None if carried is None else np.array(carried, dtype=np.float64)
         self.states = [stq.QState(s["m_codes"].to(self.device).clone(), s["m_scales"].to(self.device).clone(), int(bm),

@@ -232,6 +232,31 @@ def test_host_buffer_step_matches_device_step(flat, stats):
             assert (wh[~covered] == 0xA5).all()
 
 
+@pytest.mark.parametrize("v_log", ["sr", "ts"])
+def test_host_buffer_step_with_the_other_codes_of_v(v_log):
+    """The host-buffer call with the stochastic-rounding code (same random words: they are keyed on the row's
+    sr_id and the element's place in its row, not on the chunk a row travels in) and with the two-scale code
+    (twice the scale bytes)."""
+    from dataclasses import replace
+    w = replace(W.scaled(W.config("cfg4"), W.small_gpt2(d=136, n_layer=2), steps=2), v_log=v_log)
+    bm, bv, _ = W.draw_bits(w)
+    job = Job(w, bm, bv)
+    job.draw_grads(1)
+    job.step(1)
+    job.draw_grads(2)
+    tbl, hstates, hp_, hg = job.host_table(flat=True)
+    h2d, d2h = job.handle.step_host(tbl, **job.hp(2))
+    job._tbl = None
+    job.step(2)
+    torch.cuda.synchronize()
+    assert torch.equal(hp_, job.param_flat.cpu())
+    for hs, s in zip(hstates, job.states):
+        assert torch.equal(hs.m_codes, s.m_codes.cpu()) and torch.equal(hs.v_codes, s.v_codes.cpu())
+        assert torch.equal(hs.m_scales, s.m_scales.cpu()) and torch.equal(hs.v_scales, s.v_scales.cpu())
+        if v_log == "ts":
+            assert hs.v_scales.numel() == 2 * hs.m_scales.numel()
+
+
 def test_host_buffer_step_with_a_width_change_and_mixed_layouts():
     """Flat parameters and gradients, states allocated one by one, and new widths written to separate
     host buffers: the run path and the one-by-one path serve the same call."""
