@@ -8,8 +8,9 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libstq.so")
-SOURCES = ["stq_step_fast.cu", "stq_kernels.cu", "stq_static_stats.cu", "stq_api.cu", "stq_policy.cpp"]
-HEADERS = [os.path.join(CSRC, "stq_internal.h"), os.path.join(os.path.dirname(HERE), "include", "stq.h")]
+SOURCES = ["stq_step_fast.cu", "stq_step_variants.cu", "stq_step_split.cu", "stq_kernels.cu", "stq_static_stats.cu",
+           "stq_api.cu", "stq_policy.cpp"]
+HEADERS = [os.path.join(CSRC, "stq_internal.h"), os.path.join(CSRC, "stq_step_fast.cuh"), os.path.join(os.path.dirname(HERE), "include", "stq.h")]
 
 # -fmad=false: the code-deciding arithmetic must not be contracted; fused operations are written
 # explicitly where they are wanted.

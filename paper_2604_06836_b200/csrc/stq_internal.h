@@ -101,6 +101,11 @@ struct FastSched {
 cudaError_t launch_step_fast(int grad_dtype, bool stats, bool amp, int list, const TensorDesc* table,
                              const uint32_t* tile_map, FastSched* sched, const StepConsts& sc, double* partials,
                              int* err_flag, int grid, cudaStream_t stream);
+// (the launches of work lists 1 and 2, each instantiated in a translation unit of its own)
+cudaError_t launch_step_fast_variants(int grad_dtype, const TensorDesc* table, const uint32_t* tile_map, FastSched* sched,
+                                      const StepConsts& sc, double* partials, int* err_flag, int grid, cudaStream_t stream);
+cudaError_t launch_step_fast_split(int grad_dtype, const TensorDesc* table, const uint32_t* tile_map, FastSched* sched,
+                                   const StepConsts& sc, double* partials, int* err_flag, int grid, cudaStream_t stream);
 int fast_ctas_per_sm();
 // Launches the time-out self-test (see stq_step_fast.cu): sets *err_flag after a ~0.1 ms bounded wait.
 cudaError_t launch_wait_timeout_selftest(int* err_flag, cudaStream_t stream);
