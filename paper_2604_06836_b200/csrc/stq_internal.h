@@ -93,7 +93,7 @@ struct FastSched {
   uint16_t cta_group[kFastMaxGrid];        // group a CTA starts in
 };
 
-// The main step kernel (stq_step_fast.cu) with `grid` CTAs.  err_flag is set to 1 if a bounded wait
+// The main step kernel (stq_step_fast.cuh) with `grid` CTAs.  err_flag is set to 1 if a bounded wait
 // inside the kernel ran out.
 // amp: some tensor wants a low-precision copy, or the gradients are loss-scaled.
 // list: 0 the fused bodies of the default and "pl" codes, 1 the fused bodies of the "sr" and "ts" codes, 2 the

@@ -1,7 +1,7 @@
 // Kernels of the mixed-bit quantized AdamW step for sm_100a.
 //
 // Generic path (ragged tails, 32-bit states, width changes, init, repack, statistics alone); the
-// main step kernel is in stq_step_fast.cu.
+// main step kernel is in stq_step_fast.cuh.
 //
 // Work decomposition: the concatenated tensor list is cut into tiles of kTile elements that never
 // cross a tensor; persistent CTAs of 8 warps stride over the tile list.  Inside a tile a warp owns
