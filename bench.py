@@ -420,32 +420,35 @@ def run_ours(args, w, bits_m, bits_v):
         line["e2e"] = {"value": job_params * e2e["steps"] / (e2e_ms * 1e-3), "unit": UNIT,
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"],
                        "ms_per_step": e2e_ms / e2e["steps"]}
-    # ---- the same workload with the integer-only variant of the v code (device time only, 20 steps) ------
-    # An extra, not the headline: the default line above is the polynomial log code of the specification.
+    # ---- the same workload with the other codes of the second moment (device time only, 20 steps each) ---------
+    # Extras, not the headline: the default line above is the polynomial log code of the specification.
     if rank == 0 and world == 1 and w.v_log == "poly" and not args.no_variants and not args.shard:
-        try:
-            from dataclasses import replace
-            del job
-            torch.cuda.empty_cache()
-            wv = replace(w, v_log="pl")
-            jv = Job(wv, bits_m, bits_v, device=dev)
-            jv.draw_grads(1)
-            for tt in (1, 2, 3):
-                jv.step(tt)
-            v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            v0.record(stream)
-            for tt in range(4, 24):
-                jv.step(tt)
-            v1.record(stream)
-            torch.cuda.synchronize()
-            vms = v0.elapsed_time(v1) / 20
-            line["variants"] = {"v_log=pl": {"ms_per_step": vms, "value": params / (vms * 1e-3), "unit": UNIT,
-                                             "steps": 20, "frac": jv.algorithmic_bytes() / (vms * 1e-3) / 1e9 / peak,
-                                             "note": "plain steps, no decision steps, first 20 after warm-up"}}
-            del jv
-        except Exception as exc:          # an extra must never cost the line
-            line["variants"] = {"error": f"{type(exc).__name__}: {exc}"[:200]}
+        from dataclasses import replace
+        del job
+        line["variants"] = {}
+        for code in ("pl", "sr", "ts"):
+            try:
+                torch.cuda.empty_cache()
+                wv = replace(w, v_log=code)
+                jv = Job(wv, bits_m, bits_v, device=dev)
+                jv.draw_grads(1)
+                for tt in (1, 2, 3):
+                    jv.step(tt)
+                v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                v0.record(stream)
+                for tt in range(4, 24):
+                    jv.step(tt)
+                v1.record(stream)
+                torch.cuda.synchronize()
+                vms = v0.elapsed_time(v1) / 20
+                line["variants"]["v_log=" + code] = {
+                    "ms_per_step": vms, "value": params / (vms * 1e-3), "unit": UNIT, "steps": 20,
+                    "frac": jv.algorithmic_bytes() / (vms * 1e-3) / 1e9 / peak,
+                    "note": "plain steps, no decision steps, first 20 after warm-up"}
+                del jv
+            except Exception as exc:          # an extra must never cost the line
+                line["variants"]["v_log=" + code] = {"error": f"{type(exc).__name__}: {exc}"[:200]}
     if rank == 0 and not args.no_cpu_baseline and world == 1:
         res = oracle_run(w, bits_m, bits_v, budget_s=8.0, repeats=1)
         line["cpu_baseline"] = {"value": res["params"] / res["seconds"][0], "unit": UNIT, "cores": res["cores"],
@@ -489,9 +492,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-variants", action="store_true", help="skip the extra run with the integer-only v code")
+    ap.add_argument("--no-variants", action="store_true", help="skip the extra runs with the other codes of the second moment")
     ap.add_argument("--v-log", default="poly", choices=["poly", "pl", "sr", "ts"],
-                    help="variant of the v quantizer at widths 8 and 16 (default: the polynomial logarithm)")
+                    help="code of the second moment (default: the polynomial logarithm)")
     ap.add_argument("--shard", action="store_true",
                     help="strong scaling: each rank owns a block-aligned slice of the parameter list "
                          "(default: every rank steps a full replica)")

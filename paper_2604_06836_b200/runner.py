@@ -18,11 +18,12 @@ def _round_up(x: int, a: int) -> int:
     return (x + a - 1) // a * a
 
 
-def algorithmic_bytes(numels, bits_m, bits_v, block: int, grad_dtype: str, lp_copy: bool = False) -> int:
+def algorithmic_bytes(numels, bits_m, bits_v, block: int, grad_dtype: str, lp_copy: bool = False,
+                      v_scales_per_block: int = 1) -> int:
     """Bytes one step must move over a parameter list: per element the parameter read and written (8),
     the gradient (4 for fp32, 2 for bf16 / fp16), the codes of both states read and written
     (2 * (b_m + b_v) / 8), the working copy if any (2); per block the fp32 scales of both states read and
-    written (16; a 32-bit state has none).  Code bytes are whole bytes per tensor, blocks include a short
+    written (16; a 32-bit state has none; the two-scale code of v keeps two per block).  Code bytes are whole bytes per tensor, blocks include a short
     last one.  This is the numerator of the HBM roofline the benchmark reports."""
     gb = 4 if grad_dtype == "fp32" else 2
     gb += 2 if lp_copy else 0
@@ -31,7 +32,7 @@ def algorithmic_bytes(numels, bits_m, bits_v, block: int, grad_dtype: str, lp_co
         n, bm, bv = int(n), int(bm), int(bv)
         nb = (n + block - 1) // block
         total += n * (8 + gb) + 2 * ((n * bm + 7) // 8 + (n * bv + 7) // 8)
-        total += 4 * nb * (int(bm != 32) + int(bv != 32)) * 2
+        total += 4 * nb * (int(bm != 32) + v_scales_per_block * int(bv != 32)) * 2
     return int(total)
 
 
@@ -196,7 +197,7 @@ class Job:
     def algorithmic_bytes(self) -> int:
         """Bytes one step must move (see the module-level function)."""
         return algorithmic_bytes(self.numels, self.bits_m, self.bits_v, self.block, self.w.grad_dtype,
-                                 bool(self.w.lp_copy))
+                                 bool(self.w.lp_copy), 2 if self.w.v_log == "ts" else 1)
 
     def state_bytes(self) -> int:
         return int(sum(s.m_codes.numel() + s.v_codes.numel() + 4 * (s.m_scales.numel() + s.v_scales.numel())

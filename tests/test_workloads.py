@@ -80,3 +80,4 @@ def test_algorithmic_bytes_count_both_scale_vectors_and_none_at_32_bits():
     assert algorithmic_bytes([n], np.array([8], np.uint8), np.array([8], np.uint8), 256, "bf16", True) == \
         n * (8 + 2 + 2) + 2 * (2 * n) + 16 * (n // 256)
     assert algorithmic_bytes([130], [3], [2], 128, "bf16") == 130 * 10 + 2 * (49 + 33) + 16 * 2
+    assert algorithmic_bytes([n], [4], [4], 128, "fp32", False, 2) == base + 2 * (n // 2 + n // 2) + 24 * (n // 128)
