@@ -35,6 +35,10 @@ def test_our_arm_on_a_small_configuration():
     assert e["value"] < d["value"]                       # the host path pays for the copies
     assert d["gpu_launches"] >= 12
     assert d["clocks"]["sm_max_mhz"] and isinstance(d["clocks"]["reasons"], list)
+    assert "full oracle step" in d["cpu_baseline"]["sample"] and d["cpu_baseline"]["single_thread_value"] > 0
+    for code in ("pl", "sr", "ts"):                      # the extras: the other codes of the second moment
+        v = d["variants"]["v_log=" + code]
+        assert "error" not in v and v["value"] > 0
 
 
 def test_reference_arm_times_the_oracle():
