@@ -86,7 +86,8 @@ constexpr uint32_t kFastChunk = 2;     // tiles handed out per counter increment
                                        // 2-3 beat 1 and 8 by 1-4 % on the small and medium configurations (shorter tail
                                        // when a group runs dry), no difference on the largest
 struct FastSched {
-  uint32_t ctr[kFastMaxGroups];            // chunks handed out so far, per group
+  uint32_t ctr[kFastMaxGroups];            // chunks handed out so far, per group (zero between launches: see `done`)
+  uint32_t done;                           // CTAs that have left their hand-out loop; the last one zeroes the counters
   uint32_t ng;                             // number of groups
   uint32_t chunk;                          // tiles per counter increment for this launch
   uint32_t grp_begin[kFastMaxGroups + 1];  // tile range of group g: [grp_begin[g], grp_begin[g+1])

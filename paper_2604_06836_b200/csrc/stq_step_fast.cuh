@@ -1555,6 +1555,12 @@ stq_step_fast_kernel(const TensorDesc* __restrict__ table, const uint32_t* __res
     // read.  After a time-out the copies still in flight get one more bounded wait instead, so that
     // none lands in shared memory that no longer belongs to this CTA.
     if (ok && issued >= (uint32_t)kStages) ok = mbar_wait(empty0 + 8 * s, phase ^ 1u);
+    // The last producer to get here leaves the work list as the next launch wants to find it.
+    __threadfence();
+    if (atomicAdd(&sched->done, 1u) == gridDim.x - 1u) {
+      for (uint32_t k = 0; k < ng; ++k) sched->ctr[k] = 0u;
+      sched->done = 0u;
+    }
     if (ok) {
       reinterpret_cast<TileInfo*>(smem + kOffInfo + kInfoBytes * s)->tile = kEnd;
       mbar_arrive(full0 + 8 * s);
@@ -1611,9 +1617,7 @@ cudaError_t launch_fast_t(const TensorDesc* table, const uint32_t* tile_map, Fas
   // per device and cheap, so simply repeated: the kernel needs more than the default 48 KB
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
-  // the group counters start every launch at zero
-  e = cudaMemsetAsync(sched, 0, sizeof(uint32_t) * kFastMaxGroups, stream);
-  if (e != cudaSuccess) return e;
+  // (the group counters are zero: uploaded so, and every launch resets them on its way out)
   kern<<<grid, kFastThreads, kSmemBytes, stream>>>(table, tile_map, sched, sc, partials, err_flag);
   return cudaGetLastError();
 }
