@@ -896,3 +896,60 @@ def test_stochastic_rounding_seeds_and_call_rules(H, O):
     # sizes: the two-scale code keeps two floats per block
     assert stq.lib().stq_v_scales_bytes(1000, 128, stq.VLOG_TS) == 2 * stq.scales_bytes(1000, 128)
     assert stq.lib().stq_v_scales_bytes(1000, 128, stq.VLOG_SR) == stq.scales_bytes(1000, 128)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_tables_with_every_code_and_block_size(H, O, seed):
+    """Randomised tables in which every row draws its own block size (32..1024) and its own code of the second
+    moment (default, "pl", "sr", "ts"), next to random sizes, widths 2..32 with width changes, gradient types,
+    weight decay and statistics.  Three steps each, codes and scales (and random words) bit for bit."""
+    import oracle
+    rng = np.random.RandomState(5000 + seed)
+    widths = [2, 3, 4, 8, 16, 32]
+    modes = [oracle.LOG, oracle.LOG_PL, oracle.LOG_SR, oracle.LOG_TS]
+    for case in range(5):
+        L = int(rng.randint(1, 8))
+        gdt = [torch.float32, torch.bfloat16, torch.float16][int(rng.randint(0, 3))]
+        sizes = [int(rng.choice([1, 31, 33, 127, 129, 1000, 1024, 4095, 4096, 4097, 4096 * 2 + 333, 4096 * 4])) if rng.rand() < 0.6
+                 else int(rng.randint(1, 30000)) for _ in range(L)]
+        blocks = [int(rng.choice([32, 64, 128, 128, 256, 256, 512, 1024])) for _ in range(L)]
+        vlog = [int(rng.randint(0, 4)) for _ in range(L)]
+        wds = [float(rng.choice([0.0, 0.01, 0.1])) for _ in range(L)]
+        bits = [(int(rng.choice(widths)), int(rng.choice(widths))) for _ in range(L)]
+        sr_seed = int(rng.randint(0, 2 ** 31)) * 977 + 5
+        gen = torch.Generator(device="cuda").manual_seed(int(rng.randint(0, 2 ** 31)))
+        params = [torch.empty(n, device="cuda").normal_(0, 0.02, generator=gen) for n in sizes]
+        states = [stq.alloc_state(n, b, bm, bv, "cuda", vl) for n, b, (bm, bv), vl in zip(sizes, blocks, bits, vlog)]
+        h = stq.Handle()
+        h.init_state(stq.table([stq.make_row(n, b, None, s) for n, b, s in zip(sizes, blocks, states)]))
+        theta = [H.to_np(p) for p in params]
+        ostates = [oracle.new_state(n, b, bm, bv, modes[vl]) for n, b, (bm, bv), vl in zip(sizes, blocks, bits, vlog)]
+        upd = [np.abs(t) for t in theta]
+        for t in (1, 2, 3):
+            scale = 10.0 ** rng.uniform(-5, -2)
+            grads = [(torch.empty(n, device="cuda").normal_(0, 1.0, generator=gen) * scale).to(gdt) for n in sizes]
+            new_bits = [(int(rng.choice(widths)), int(rng.choice(widths))) if rng.rand() < 0.25 else b for b in bits]
+            out = [s if nb == b else stq.alloc_state(n, blk, nb[0], nb[1], "cuda", vl)
+                   for s, nb, b, n, blk, vl in zip(states, new_bits, bits, sizes, blocks, vlog)]
+            want_stats = bool(rng.randint(0, 2))
+            rows = [stq.make_row(n, blk, s, o, p, g, wd, sr_id=i + 3)
+                    for i, (n, blk, s, o, p, g, wd) in enumerate(zip(sizes, blocks, states, out, params, grads, wds))]
+            h.step(stq.table(rows), lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, t=t, grad_dtype=stq.grad_dtype_of(grads[0]),
+                   flags=stq.WITH_STATS if want_stats else 0, sr_seed=sr_seed)
+            got_stats = h.layer_stats(L) if want_stats else None
+            h.device_status()
+            states, bits = out, new_bits
+            for i in range(L):
+                before = theta[i].copy()
+                ostates[i], st = oracle.step(theta[i], H.to_np(grads[i]), ostates[i], blocks[i], lr=1e-3, beta1=0.9,
+                                             beta2=0.999, eps=1e-8, weight_decay=wds[i], t=t, bits_m_out=bits[i][0],
+                                             bits_v_out=bits[i][1], want_stats=want_stats, fp16_grad=(gdt == torch.float16),
+                                             v_mode=modes[vlog[i]], sr_seed=sr_seed, tensor_index=i + 3)
+                upd[i] = np.maximum(upd[i], np.maximum(np.abs(theta[i]), np.abs(theta[i] - before)))
+                tag = (f"seed {seed} case {case} t={t} tensor {i} n={sizes[i]} B={blocks[i]} bits {bits[i]} "
+                       f"code {vlog[i]} {gdt}")
+                H.assert_states_equal(states[i], ostates[i], tag)
+                H.assert_theta_close(params[i], theta[i], REL_1STEP * t, tag, upd=upd[i])
+                if want_stats:
+                    H.assert_stats_close(got_stats[i:i + 1], st[None, :], tag)
+        h.close()
