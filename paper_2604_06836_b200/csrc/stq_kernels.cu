@@ -837,71 +837,83 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
 // gradients.  Same tile order and the same per-(tile, warp) partials as the fused path, so the
 // second stage is shared.  A warp owns 512 consecutive elements of the tile; a lane reads them as
 // 128-bit loads at a 512-byte warp stride.
+constexpr uint32_t kGradStatsUnroll = 2;
+
 template <int GDT>
 __global__ void __launch_bounds__(kThreads)
 stq_grad_stats_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map,
                       uint32_t tile_begin, uint32_t tile_end, double* __restrict__ partials) {
   constexpr int kPerLoad = GDT == 0 ? 4 : 8;                 // elements per 128-bit load
   constexpr int kLoads = (kTile / (kThreads / 32)) / (32 * kPerLoad);
+  constexpr int kUnroll = kGradStatsUnroll;                  // tiles in flight per CTA: their loads are issued together
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (uint32_t tile = tile_begin + blockIdx.x; tile < tile_end; tile += gridDim.x) {
-    const TensorDesc* __restrict__ T = table + __ldg(tile_map + tile);
-    const unsigned long long numel = T->numel;
-    const unsigned long long e_warp = (unsigned long long)(T->nfast + (tile - T->tile0s)) * kTile +
-                                      (unsigned)warp * (kTile / (kThreads / 32));
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f;
-    uint4 raw[kLoads];
-    bool whole[kLoads];
+  for (uint32_t tile0 = tile_begin + kUnroll * blockIdx.x; tile0 < tile_end; tile0 += kUnroll * gridDim.x) {
+    uint4 raw[kUnroll][kLoads];
 #pragma unroll
-    for (int j = 0; j < kLoads; ++j) {
-      const unsigned long long e = e_warp + (unsigned long long)(j * 32 + lane) * kPerLoad;
-      whole[j] = e + kPerLoad <= numel;
-      raw[j] = make_uint4(0u, 0u, 0u, 0u);
-      if (whole[j]) {
-        raw[j] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(T->grad) + e * (GDT == 0 ? 4 : 2)));
-      } else if (e < numel) {     // ragged end of the tensor: element by element
-        uint32_t w[4] = {0u, 0u, 0u, 0u};
-        for (int k = 0; k < kPerLoad && e + k < numel; ++k) {
-          if constexpr (GDT == 0) w[k] = __float_as_uint(__ldg(reinterpret_cast<const float*>(T->grad) + e + k));
-          else w[k >> 1] |= (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(T->grad) + e + k) << (16 * (k & 1));
-        }
-        raw[j] = make_uint4(w[0], w[1], w[2], w[3]);
-      }
-    }
+    for (int u = 0; u < kUnroll; ++u) {
+      const uint32_t tile = tile0 + u;
 #pragma unroll
-    for (int j = 0; j < kLoads; ++j) {
-      const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+      for (int j = 0; j < kLoads; ++j) raw[u][j] = make_uint4(0u, 0u, 0u, 0u);
+      if (tile >= tile_end) continue;
+      const TensorDesc* __restrict__ T = table + __ldg(tile_map + tile);
+      const unsigned long long numel = T->numel;
+      const unsigned long long e_warp = (unsigned long long)(T->nfast + (tile - T->tile0s)) * kTile +
+                                        (unsigned)warp * (kTile / (kThreads / 32));
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        if constexpr (GDT == 0) {
-          const float g = __uint_as_float(w[k]);
-          a0 += g; a1 += fabsf(g); a2 = __fmaf_rn(g, g, a2);
-        } else {
-          float g0, g1;
-          if constexpr (GDT == 1) {
-            g0 = __uint_as_float(w[k] << 16);
-            g1 = __uint_as_float(w[k] & 0xFFFF0000u);
-          } else {
-            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[k]));
-            g0 = f.x;
-            g1 = f.y;
+      for (int j = 0; j < kLoads; ++j) {
+        const unsigned long long e = e_warp + (unsigned long long)(j * 32 + lane) * kPerLoad;
+        if (e + kPerLoad <= numel) {
+          raw[u][j] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(T->grad) + e * (GDT == 0 ? 4 : 2)));
+        } else if (e < numel) {     // ragged end of the tensor: element by element
+          uint32_t w[4] = {0u, 0u, 0u, 0u};
+          for (int k = 0; k < kPerLoad && e + k < numel; ++k) {
+            if constexpr (GDT == 0) w[k] = __float_as_uint(__ldg(reinterpret_cast<const float*>(T->grad) + e + k));
+            else w[k >> 1] |= (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(T->grad) + e + k) << (16 * (k & 1));
           }
-          a0 += g0; a1 += fabsf(g0); a2 = __fmaf_rn(g0, g0, a2);
-          a0 += g1; a1 += fabsf(g1); a2 = __fmaf_rn(g1, g1, a2);
+          raw[u][j] = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
     }
-    // pairwise butterfly that spreads the three sums over the lanes on the way down
-    const bool hi = lane & 16;
-    float x = (hi ? a2 : a0) + __shfl_xor_sync(kFull, hi ? a0 : a2, 16);
-    float y = (hi ? 0.f : a1) + __shfl_xor_sync(kFull, hi ? a1 : 0.f, 16);
-    const bool q = lane & 8;
-    float z = (q ? y : x) + __shfl_xor_sync(kFull, q ? x : y, 8);
-    z += __shfl_xor_sync(kFull, z, 4);
-    z += __shfl_xor_sync(kFull, z, 2);
-    z += __shfl_xor_sync(kFull, z, 1);
-    if ((lane & 7) == 0 && lane < 24)
-      partials[((size_t)tile * (kThreads / 32) + warp) * 3 + (lane >> 3)] = (double)z;
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const uint32_t tile = tile0 + u;
+      if (tile >= tile_end) continue;
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f;
+#pragma unroll
+      for (int j = 0; j < kLoads; ++j) {
+        const uint32_t w[4] = {raw[u][j].x, raw[u][j].y, raw[u][j].z, raw[u][j].w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if constexpr (GDT == 0) {
+            const float g = __uint_as_float(w[k]);
+            a0 += g; a1 += fabsf(g); a2 = __fmaf_rn(g, g, a2);
+          } else {
+            float g0, g1;
+            if constexpr (GDT == 1) {
+              g0 = __uint_as_float(w[k] << 16);
+              g1 = __uint_as_float(w[k] & 0xFFFF0000u);
+            } else {
+              const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[k]));
+              g0 = f.x;
+              g1 = f.y;
+            }
+            a0 += g0; a1 += fabsf(g0); a2 = __fmaf_rn(g0, g0, a2);
+            a0 += g1; a1 += fabsf(g1); a2 = __fmaf_rn(g1, g1, a2);
+          }
+        }
+      }
+      // pairwise butterfly that spreads the three sums over the lanes on the way down
+      const bool hi = lane & 16;
+      float x = (hi ? a2 : a0) + __shfl_xor_sync(kFull, hi ? a0 : a2, 16);
+      float y = (hi ? 0.f : a1) + __shfl_xor_sync(kFull, hi ? a1 : 0.f, 16);
+      const bool q = lane & 8;
+      float z = (q ? y : x) + __shfl_xor_sync(kFull, q ? x : y, 8);
+      z += __shfl_xor_sync(kFull, z, 4);
+      z += __shfl_xor_sync(kFull, z, 2);
+      z += __shfl_xor_sync(kFull, z, 1);
+      if ((lane & 7) == 0 && lane < 24)
+        partials[((size_t)tile * (kThreads / 32) + warp) * 3 + (lane >> 3)] = (double)z;
+    }
   }
 }
 
@@ -1008,7 +1020,8 @@ cudaError_t launch_tiles(Mode mode, bool wide, bool variants, int grad_dtype, bo
     case kStatsOnly: {
       const uint32_t n = tile_end - tile_begin;
       const uint32_t want = (uint32_t)grid * 4u;   // small CTAs, 32 registers: many fit per SM
-      const int g = (int)(n < want ? n : want);
+      const uint32_t need = (n + kGradStatsUnroll - 1u) / kGradStatsUnroll;   // tiles a CTA takes per turn
+      const int g = (int)(need < want ? need : want);
       if (grad_dtype == 0)
         stq_grad_stats_kernel<0><<<g, kThreads, 0, stream>>>(table, tile_map, tile_begin, tile_end, partials);
       else if (grad_dtype == 1)
