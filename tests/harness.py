@@ -266,6 +266,7 @@ class FullOracle:
         self.states = [O.new_state(n, self.block, int(bm), int(bv), self.v_mode)
                        for n, bm, bv in zip(job.numels, job.bits_m, job.bits_v)]
         self.mag = [p.abs() for p in job.params]          # device: largest magnitude an element or its step has had
+        self.theta_dev = [p.clone() for p in job.params]  # device copy of the oracle's parameters (same bits at the start)
 
     def _ranges(self):
         for i, n in enumerate(self.job.numels):
@@ -275,7 +276,11 @@ class FullOracle:
     def step(self, t: int, new_bits=None, want_stats: bool = False) -> np.ndarray:
         """One oracle step on the gradients the job currently holds.  Returns [L, 4] sums (zeros unless asked)."""
         job, w = self.job, self.w
-        grads = [to_np(g) for g in job.grads]
+
+        def host(t):        # one copy to the host; the array keeps the host tensor alive
+            t = t.detach().cpu()
+            return t.view(torch.int16).numpy().view(np.uint16) if t.dtype in (torch.bfloat16, torch.float16) else t.numpy()
+        grads = [host(g) for g in job.grads]
         out = []
         for i, n in enumerate(job.numels):
             bm = self.states[i].bits_m if new_bits is None else int(new_bits[0][i])
@@ -293,12 +298,12 @@ class FullOracle:
                          beta2=w.beta2, eps=w.eps, weight_decay=job.wd[i], t=t, v_mode=self.v_mode,
                          stats=part[k] if want_stats else None, sr_seed=job.sr_seed, tensor_index=i, **amp)
 
-        before = [torch.from_numpy(th).to(job.device) for th in self.theta]
         list(self.pool.map(run, range(len(tasks))))
         self.states = out
         for i in range(job.L):
             now = torch.from_numpy(self.theta[i]).to(job.device)
-            self.mag[i] = torch.maximum(self.mag[i], torch.maximum(now.abs(), (now - before[i]).abs()))
+            self.mag[i] = torch.maximum(self.mag[i], torch.maximum(now.abs(), (now - self.theta_dev[i]).abs()))
+            self.theta_dev[i] = now
         stats = np.zeros((job.L, 4))
         for k, (i, _, _) in enumerate(tasks):
             stats[i] += part[k]
@@ -339,7 +344,7 @@ class FullOracle:
                 if not torch.equal(g.view(torch.int32), o_d.view(torch.int32)):
                     bad = torch.nonzero(g.view(torch.int32) != o_d.view(torch.int32)).flatten()[:8].tolist()
                     raise AssertionError(f"{name}: {what} differ at blocks {bad}")
-            o = torch.from_numpy(self.theta[i]).to(dev).double()
+            o = self.theta_dev[i].double()
             g = job.params[i].double()
             lim = rel * torch.maximum(self.mag[i].double(), 1e-3 * o.abs().max())
             err = (g - o).abs()
