@@ -283,6 +283,8 @@ int prepare(stq_handle* h, const stq_tensor* tensors, int L, int kind, cudaStrea
   if (total > 0xFFFFFFF0ull) return STQ_E_NUMEL;
   // the tile map depends only on sizes and classes: skip it when unchanged
   const bool same_map = h->cached_kind >= 0 && sig == h->cached_sig && h->n_tiles == (uint32_t)total;
+  // from here on the device image is being rewritten: a failure below must not leave the old table looking current
+  h->cached_kind = -1;
 
   const size_t bytes_table = sizeof(TensorDesc) * (size_t)L;
   const size_t bytes_map = sizeof(uint32_t) * (size_t)total;

@@ -953,3 +953,65 @@ def test_random_tables_with_every_code_and_block_size(H, O, seed):
                 if want_stats:
                     H.assert_stats_close(got_stats[i:i + 1], st[None, :], tag)
         h.close()
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_medium_tables_every_code_in_one_launch(H, O, seed):
+    """Thirty-six tensors of tens to hundreds of tiles, each with its own code of the second moment (default,
+    "pl", "sr", "ts"), its own block size (mostly 128 and 256, some 64 and 512) and random widths, a quarter of
+    them changing width every step: one step runs the three work lists of the main kernel and the generic
+    kernel side by side.  Some tables carry the mixed-precision extras (loss scale, working copy).  Four
+    steps, statistics on every other one; codes, scales and random words bit for bit."""
+    import oracle
+    rng = np.random.RandomState(7000 + seed)
+    widths = [2, 3, 4, 8, 16]
+    modes = [oracle.LOG, oracle.LOG_PL, oracle.LOG_SR, oracle.LOG_TS]
+    L = 36
+    gdt = [torch.bfloat16, torch.float32, torch.float16][seed % 3]
+    sizes = [int(rng.randint(20000, 160000)) for _ in range(L)]
+    blocks = [int(rng.choice([128, 128, 128, 256, 256, 256, 64, 512])) for _ in range(L)]
+    vlog = [int(rng.randint(0, 4)) for _ in range(L)]
+    bits = [(int(rng.choice(widths)), int(rng.choice(widths))) for _ in range(L)]
+    sr_seed = int(rng.randint(0, 2 ** 31)) * 1013 + 7
+    gen = torch.Generator(device="cuda").manual_seed(100 + seed)
+    params = [torch.empty(n, device="cuda").normal_(0, 0.02, generator=gen) for n in sizes]
+    states = [stq.alloc_state(n, b, bm, bv, "cuda", vl) for n, b, (bm, bv), vl in zip(sizes, blocks, bits, vlog)]
+    h = stq.Handle()
+    h.init_state(stq.table([stq.make_row(n, b, None, s) for n, b, s in zip(sizes, blocks, states)]))
+    theta = [H.to_np(p) for p in params]
+    ostates = [oracle.new_state(n, b, bm, bv, modes[vl]) for n, b, (bm, bv), vl in zip(sizes, blocks, bits, vlog)]
+    upd = [np.abs(t) for t in theta]
+    amp = seed % 2 == 1
+    S = 1024.0 if amp else 1.0
+    inv = torch.tensor([np.float32(1.0 / S)], dtype=torch.float32, device="cuda") if amp else None
+    lp_dt = torch.bfloat16 if amp else None
+    lps = [torch.zeros(n, dtype=lp_dt, device="cuda") if amp else None for n in sizes]
+    for t in range(1, 5):
+        scale = 10.0 ** rng.uniform(-4, -2) * S
+        grads = [(torch.empty(n, device="cuda").normal_(0, 1.0, generator=gen) * scale).to(gdt) for n in sizes]
+        new_bits = [(int(rng.choice(widths)), int(rng.choice(widths))) if rng.rand() < 0.25 else b for b in bits]
+        out = [s if nb == b else stq.alloc_state(n, blk, nb[0], nb[1], "cuda", vl)
+               for s, nb, b, n, blk, vl in zip(states, new_bits, bits, sizes, blocks, vlog)]
+        want_stats = t % 2 == 0
+        rows = [stq.make_row(n, blk, s, o, p, g, 0.01, lp, sr_id=i)
+                for i, (n, blk, s, o, p, g, lp) in enumerate(zip(sizes, blocks, states, out, params, grads, lps))]
+        h.step(stq.table(rows), lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, t=t, grad_dtype=stq.grad_dtype_of(grads[0]),
+               flags=stq.WITH_STATS if want_stats else 0, sr_seed=sr_seed, inv_grad_scale=inv)
+        got = h.layer_stats(L) if want_stats else None
+        h.device_status()
+        states, bits = out, new_bits
+        for i in range(L):
+            before = theta[i].copy()
+            ostates[i], st = oracle.step(theta[i], H.to_np(grads[i]), ostates[i], blocks[i], lr=1e-3, beta1=0.9, beta2=0.999,
+                                         eps=1e-8, weight_decay=0.01, t=t, bits_m_out=bits[i][0], bits_v_out=bits[i][1],
+                                         want_stats=want_stats, fp16_grad=(gdt == torch.float16), v_mode=modes[vlog[i]],
+                                         sr_seed=sr_seed, tensor_index=i, inv_grad_scale=float(np.float32(1.0 / S)))
+            upd[i] = np.maximum(upd[i], np.maximum(np.abs(theta[i]), np.abs(theta[i] - before)))
+            tag = f"seed {seed} t={t} tensor {i} n={sizes[i]} B={blocks[i]} bits {bits[i]} code {vlog[i]} {gdt}"
+            H.assert_states_equal(states[i], ostates[i], tag)
+            H.assert_theta_close(params[i], theta[i], REL_1STEP * t, tag, upd=upd[i])
+            if want_stats:
+                H.assert_stats_close(got[i:i + 1], st[None, :], tag)
+            if amp:
+                assert torch.equal(lps[i], params[i].to(lp_dt)), tag + " working copy"
+    h.close()
