@@ -834,86 +834,107 @@ stq_tile_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict
 }
 
 // Statistics alone (Algorithm 1 takes them before the update): a streaming reduction over the
-// gradients.  Same tile order and the same per-(tile, warp) partials as the fused path, so the
-// second stage is shared.  A warp owns 512 consecutive elements of the tile; a lane reads them as
-// 128-bit loads at a 512-byte warp stride.
-constexpr uint32_t kGradStatsUnroll = 2;
+// gradients.  Same tile order and the same slots of partial sums as the fused path (eight per tile, one per
+// warp there), so the second stage is shared; here ONE warp takes 8 KB of a tile (all of it with 16-bit
+// gradients, half with fp32), fills the first of its slots and zeroes the rest: the work that is not arithmetic
+// on the elements (finding the tile, the butterfly, the store) is then paid once per 8 KB and not once per
+// 1 KB, which keeps the pass bound by memory and not by instruction issue.  A lane reads 128-bit words at a
+// 512-byte warp stride.
+constexpr uint32_t kGradStatsTilesPerCta = kThreads / 32;     // shares a CTA takes per turn: one per warp
+
+template <int GDT>
+__device__ __forceinline__ void grad_stats_accumulate(const uint4& raw, float2& a0, float& a1x, float& a1y, float2& a2) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+  if constexpr (GDT == 0) {
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const float2 g = make_float2(__uint_as_float(w[2 * k]), __uint_as_float(w[2 * k + 1]));
+      a0 = __fadd2_rn(a0, g);
+      a1x += fabsf(g.x);
+      a1y += fabsf(g.y);
+      a2 = __ffma2_rn(g, g, a2);
+    }
+  } else {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      float2 g;
+      if constexpr (GDT == 1) g = make_float2(__uint_as_float(w[k] << 16), __uint_as_float(w[k] & 0xFFFF0000u));
+      else g = __half22float2(*reinterpret_cast<const __half2*>(&w[k]));
+      a0 = __fadd2_rn(a0, g);
+      a1x += fabsf(g.x);
+      a1y += fabsf(g.y);
+      a2 = __ffma2_rn(g, g, a2);
+    }
+  }
+}
+
+// warps per tile: a warp's share is 8 KB of gradients whatever their type
+__host__ __device__ constexpr uint32_t grad_stats_split(int gdt) { return gdt == 0 ? 2u : 1u; }
 
 template <int GDT>
 __global__ void __launch_bounds__(kThreads)
 stq_grad_stats_kernel(const TensorDesc* __restrict__ table, const uint32_t* __restrict__ tile_map,
                       uint32_t tile_begin, uint32_t tile_end, double* __restrict__ partials) {
   constexpr int kPerLoad = GDT == 0 ? 4 : 8;                 // elements per 128-bit load
-  constexpr int kLoads = (kTile / (kThreads / 32)) / (32 * kPerLoad);
-  constexpr int kUnroll = kGradStatsUnroll;                  // tiles in flight per CTA: their loads are issued together
+  constexpr uint32_t kSplit = grad_stats_split(GDT);
+  constexpr uint32_t kShare = kTile / kSplit;                // elements a warp takes
+  constexpr int kLoads = kShare / (32 * kPerLoad);           // loads per lane and share
+  constexpr int kBatch = 8;                                  // of which in flight together
+  constexpr uint32_t kSlots = (kThreads / 32) * 3;           // doubles per tile in `partials`
+  constexpr uint32_t kMine = kSlots / kSplit;                // of which this warp writes
+  static_assert(kLoads % kBatch == 0, "whole batches");
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (uint32_t tile0 = tile_begin + kUnroll * blockIdx.x; tile0 < tile_end; tile0 += kUnroll * gridDim.x) {
-    uint4 raw[kUnroll][kLoads];
+  const unsigned long long n_shares = (unsigned long long)(tile_end - tile_begin) * kSplit;
+  const unsigned long long stride = (unsigned long long)gridDim.x * kGradStatsTilesPerCta;
+  for (unsigned long long u = (unsigned long long)blockIdx.x * kGradStatsTilesPerCta + (unsigned)warp; u < n_shares; u += stride) {
+    const uint32_t tile = tile_begin + (uint32_t)(u / kSplit), part = (uint32_t)(u % kSplit);
+    const TensorDesc* __restrict__ T = table + __ldg(tile_map + tile);
+    const unsigned long long numel = T->numel;
+    const unsigned long long e0 = (unsigned long long)(T->nfast + (tile - T->tile0s)) * kTile + part * kShare;
+    const uint8_t* __restrict__ base = reinterpret_cast<const uint8_t*>(T->grad) + e0 * (GDT == 0 ? 4 : 2);
+    float2 a0 = make_float2(0.f, 0.f), a2 = make_float2(0.f, 0.f);
+    float a1x = 0.f, a1y = 0.f;
+    if (e0 + kShare <= numel) {
+      const uint4* __restrict__ src = reinterpret_cast<const uint4*>(base) + lane;
+#pragma unroll 1
+      for (int b = 0; b < kLoads / kBatch; ++b) {
+        uint4 raw[kBatch];
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const uint32_t tile = tile0 + u;
+        for (int j = 0; j < kBatch; ++j) raw[j] = __ldg(src + (b * kBatch + j) * 32);
 #pragma unroll
-      for (int j = 0; j < kLoads; ++j) raw[u][j] = make_uint4(0u, 0u, 0u, 0u);
-      if (tile >= tile_end) continue;
-      const TensorDesc* __restrict__ T = table + __ldg(tile_map + tile);
-      const unsigned long long numel = T->numel;
-      const unsigned long long e_warp = (unsigned long long)(T->nfast + (tile - T->tile0s)) * kTile +
-                                        (unsigned)warp * (kTile / (kThreads / 32));
-#pragma unroll
+        for (int j = 0; j < kBatch; ++j) grad_stats_accumulate<GDT>(raw[j], a0, a1x, a1y, a2);
+      }
+    } else if (e0 < numel) {   // the ragged end of a tensor: whole words while they last, then element by element
+#pragma unroll 1
       for (int j = 0; j < kLoads; ++j) {
-        const unsigned long long e = e_warp + (unsigned long long)(j * 32 + lane) * kPerLoad;
+        const unsigned long long e = e0 + (unsigned long long)(j * 32 + lane) * kPerLoad;
+        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
         if (e + kPerLoad <= numel) {
-          raw[u][j] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(T->grad) + e * (GDT == 0 ? 4 : 2)));
-        } else if (e < numel) {     // ragged end of the tensor: element by element
+          raw = __ldg(reinterpret_cast<const uint4*>(base) + j * 32 + lane);
+        } else if (e < numel) {
           uint32_t w[4] = {0u, 0u, 0u, 0u};
           for (int k = 0; k < kPerLoad && e + k < numel; ++k) {
             if constexpr (GDT == 0) w[k] = __float_as_uint(__ldg(reinterpret_cast<const float*>(T->grad) + e + k));
             else w[k >> 1] |= (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(T->grad) + e + k) << (16 * (k & 1));
           }
-          raw[u][j] = make_uint4(w[0], w[1], w[2], w[3]);
+          raw = make_uint4(w[0], w[1], w[2], w[3]);
         }
+        grad_stats_accumulate<GDT>(raw, a0, a1x, a1y, a2);
       }
     }
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const uint32_t tile = tile0 + u;
-      if (tile >= tile_end) continue;
-      float a0 = 0.f, a1 = 0.f, a2 = 0.f;
-#pragma unroll
-      for (int j = 0; j < kLoads; ++j) {
-        const uint32_t w[4] = {raw[u][j].x, raw[u][j].y, raw[u][j].z, raw[u][j].w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if constexpr (GDT == 0) {
-            const float g = __uint_as_float(w[k]);
-            a0 += g; a1 += fabsf(g); a2 = __fmaf_rn(g, g, a2);
-          } else {
-            float g0, g1;
-            if constexpr (GDT == 1) {
-              g0 = __uint_as_float(w[k] << 16);
-              g1 = __uint_as_float(w[k] & 0xFFFF0000u);
-            } else {
-              const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[k]));
-              g0 = f.x;
-              g1 = f.y;
-            }
-            a0 += g0; a1 += fabsf(g0); a2 = __fmaf_rn(g0, g0, a2);
-            a0 += g1; a1 += fabsf(g1); a2 = __fmaf_rn(g1, g1, a2);
-          }
-        }
-      }
-      // pairwise butterfly that spreads the three sums over the lanes on the way down
-      const bool hi = lane & 16;
-      float x = (hi ? a2 : a0) + __shfl_xor_sync(kFull, hi ? a0 : a2, 16);
-      float y = (hi ? 0.f : a1) + __shfl_xor_sync(kFull, hi ? a1 : 0.f, 16);
-      const bool q = lane & 8;
-      float z = (q ? y : x) + __shfl_xor_sync(kFull, q ? x : y, 8);
-      z += __shfl_xor_sync(kFull, z, 4);
-      z += __shfl_xor_sync(kFull, z, 2);
-      z += __shfl_xor_sync(kFull, z, 1);
-      if ((lane & 7) == 0 && lane < 24)
-        partials[((size_t)tile * (kThreads / 32) + warp) * 3 + (lane >> 3)] = (double)z;
-    }
+    // pairwise butterfly that spreads the three sums over the lanes on the way down: they end in lanes 0, 8, 16
+    const float s0 = a0.x + a0.y, s1 = a1x + a1y, s2 = a2.x + a2.y;
+    const bool hi = lane & 16;
+    float x = (hi ? s2 : s0) + __shfl_xor_sync(kFull, hi ? s0 : s2, 16);
+    float y = (hi ? 0.f : s1) + __shfl_xor_sync(kFull, hi ? s1 : 0.f, 16);
+    const bool q = lane & 8;
+    float z = (q ? y : x) + __shfl_xor_sync(kFull, q ? x : y, 8);
+    z += __shfl_xor_sync(kFull, z, 4);
+    z += __shfl_xor_sync(kFull, z, 2);
+    z += __shfl_xor_sync(kFull, z, 1);
+    const float mine = __shfl_sync(kFull, z, (lane & 3) * 8);
+    // this warp's slots of the tile: its three sums, then zeros
+    if (lane < (int)kMine) partials[(size_t)tile * kSlots + part * kMine + lane] = lane < 3 ? (double)mine : 0.0;
   }
 }
 
@@ -1019,9 +1040,12 @@ cudaError_t launch_tiles(Mode mode, bool wide, bool variants, int grad_dtype, bo
       return launch_w<kInit, 0, false>(wide, table, tile_map, tile_begin, tile_end, sc, partials, grid, stream, variants);
     case kStatsOnly: {
       const uint32_t n = tile_end - tile_begin;
-      const uint32_t want = (uint32_t)grid * 4u;   // small CTAs, 32 registers: many fit per SM
-      const uint32_t need = (n + kGradStatsUnroll - 1u) / kGradStatsUnroll;   // tiles a CTA takes per turn
-      const int g = (int)(need < want ? need : want);
+      const uint32_t want = (uint32_t)grid * 4u;   // small CTAs of few registers: many fit per SM
+      // a warp takes 8 KB of gradients per turn
+      const uint32_t need = (uint32_t)(((unsigned long long)n * grad_stats_split(grad_dtype) + kGradStatsTilesPerCta - 1u) / kGradStatsTilesPerCta);
+      // every CTA gets the same number of turns (a short launch of uneven turns would end on a few stragglers)
+      const uint32_t turns = (need + want - 1u) / want;
+      const int g = (int)((need + turns - 1u) / turns);
       if (grad_dtype == 0)
         stq_grad_stats_kernel<0><<<g, kThreads, 0, stream>>>(table, tile_map, tile_begin, tile_end, partials);
       else if (grad_dtype == 1)
