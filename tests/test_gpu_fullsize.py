@@ -374,6 +374,9 @@ def test_one_tensor_beyond_two_to_the_31_elements():
             x = g[lo:lo + (1 << 28)].double()
             want += np.array([x.sum().item(), x.abs().sum().item(), (x * x).sum().item(), x.numel()])
         H.assert_stats_close(got, want[None, :], f"2^31 t={t}")
+    # the gradient-only pass over the same gradients
+    job.handle.grad_stats(job.table(), job.grad_dtype)
+    H.assert_stats_close(job.layer_stats(), want[None, :], "2^31 statistics alone")
 
 
 def test_one_tensor_beyond_two_to_the_32_elements():
@@ -398,6 +401,8 @@ def test_one_tensor_beyond_two_to_the_32_elements():
         x = g[lo:lo + (1 << 28)].double()
         want += np.array([x.sum().item(), x.abs().sum().item(), (x * x).sum().item(), x.numel()])
     H.assert_stats_close(got, want[None, :], "2^32")
+    job.handle.grad_stats(job.table(), job.grad_dtype)
+    H.assert_stats_close(job.layer_stats(), want[None, :], "2^32 statistics alone")
 
 
 def test_full_size_runs_are_identical_bit_for_bit():
