@@ -940,7 +940,17 @@ __device__ __forceinline__ void tile_body_var(const uint8_t* __restrict__ stage,
     // ---- "ts": the stored {hi, lo} of the two rows' blocks give range and step; lanes of equal parity work
     // out the same row, lane r's copy is handed to everyone
     [[maybe_unused]] float step_in[RP] = {0.f, 0.f};
-    if constexpr (kTs) {
+    // at <= 4 bits a block has at most 16 levels: lane (r << LV | q) works out level q of row r once, the elements
+    // fetch theirs by shuffle (the same arithmetic as the per-element decode of the wider codes, hence the same bits)
+    [[maybe_unused]] float lut_dec = 0.f;
+    if constexpr (kTs && BV <= 4) {
+      const int blk_l = ((row0 + ((lane >> LV) & 1)) * kRowElems) >> lgB;
+      const float2 hl = *reinterpret_cast<const float2*>(stage + kOffVs + 8 * blk_l);
+      const TsRow tr = ts_row<BV>(__float_as_uint(hl.x), __float_as_uint(hl.y), false);
+      const int q = lane & (int)Wd<LV>::mask;
+      const float val = __fmul_rn(hl.x, ex2_poly(__fmul_rn((float)(q - K), tr.inv_or_step)));
+      lut_dec = q == 0 ? hl.y : val;          // code 0 is the stored minimum itself
+    } else if constexpr (kTs) {
       const int blk_l = ((row0 + (lane & 1)) * kRowElems) >> lgB;
       const float2 hl = *reinterpret_cast<const float2*>(stage + kOffVs + 8 * blk_l);
       const TsRow tr = ts_row<BV>(__float_as_uint(hl.x), __float_as_uint(hl.y), false);
@@ -973,6 +983,11 @@ __device__ __forceinline__ void tile_body_var(const uint8_t* __restrict__ stage,
         for (int h = 0; h < 2; ++h)
           vt[r][h] = mul2(s2, bits2(Sr<BV>::floor_bits + (code_of<BV>(w, 2 * h) << Sr<BV>::sh),
                                     Sr<BV>::floor_bits + (code_of<BV>(w, 2 * h + 1) << Sr<BV>::sh)));
+      } else if constexpr (BV <= 4) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+          vt[r][h] = make_float2(__shfl_sync(kFull, lut_dec, (int)(code_of<BV>(w, 2 * h) | (uint32_t)(r << LV))),
+                                 __shfl_sync(kFull, lut_dec, (int)(code_of<BV>(w, 2 * h + 1) | (uint32_t)(r << LV))));
       } else {
         const float2 hl = *reinterpret_cast<const float2*>(stage + kOffVs + 8 * blk);
         constexpr float off = kTwo23 + (float)K;
@@ -1091,8 +1106,21 @@ __device__ __forceinline__ void tile_body_var(const uint8_t* __restrict__ stage,
       }
     }
 
-    // ---- "sr" at <= 4 bits: what each level of each row contributes to the update, one level per lane -----
+    // ---- <= 4 bits: what each level of each row contributes to the update, one level per lane -------------
     [[maybe_unused]] float lut_upd = 0.f;
+    if constexpr (kTs && BV <= 4) {
+      // sqrt of level q of the new code: sqrt(hi) * 2^((q-K) * W/K / 2), or sqrt(lo) for q = 0
+      constexpr float invq = 1.0f / (float)Wd<BM>::qmax;
+      const bool second = (lane >> LV) & 1;
+      const float svr = __uint_as_float(second ? mxv[1] : mxv[0]);
+      const float smr = __uint_as_float(second ? mxm[1] : mxm[0]);
+      const int q = lane & (int)Wd<LV>::mask;
+      const float srt_hi = __fmul_rn(sqrt_fast(svr < kTiny ? 0.f : svr), sc.rsqrt_bc2);
+      const float arg = __fmul_rn((float)(q - K), second ? tsHalf[1] : tsHalf[0]);
+      float den = __fmaf_rn(ex2_fast(arg), srt_hi, sc.eps);
+      if (q == 0) den = __fmaf_rn(sqrt_fast(second ? tsLo[1] : tsLo[0]), sc.rsqrt_bc2, sc.eps);
+      lut_upd = __fmul_rn(__fmul_rn(__fmul_rn(smr, sc.step_size), invq), rcp_fast(den));
+    }
     if constexpr (kSr && BV <= 4) {
       constexpr float invq = 1.0f / (float)Wd<BM>::qmax;
       const bool second = (lane >> LV) & 1;
@@ -1161,9 +1189,9 @@ __device__ __forceinline__ void tile_body_var(const uint8_t* __restrict__ stage,
       } else {
         // d(x) = split logarithm of x / hi, clamped to [-W, 0]; code - K = round-half-even(d * K / W)
         const uint32_t ebase = kMagicBits - (vzero ? (uint32_t)kZeroBlockExp : (mxv[r] >> 23));
-        const float half_step = tsHalf[r];
-        const float srt_hi = __fmul_rn(sqrt_fast(vzero ? 0.f : sv_raw), sc.rsqrt_bc2);
-        const float den_lo = __fmaf_rn(sqrt_fast(tsLo[r]), sc.rsqrt_bc2, sc.eps);
+        [[maybe_unused]] const float half_step = tsHalf[r];
+        [[maybe_unused]] const float srt_hi = __fmul_rn(sqrt_fast(vzero ? 0.f : sv_raw), sc.rsqrt_bc2);
+        [[maybe_unused]] const float den_lo = __fmaf_rn(sqrt_fast(tsLo[r]), sc.rsqrt_bc2, sc.eps);
         uint32_t x[4];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -1175,6 +1203,14 @@ __device__ __forceinline__ void tile_body_var(const uint8_t* __restrict__ stage,
           const f2 t = fma2(d, splat(tsInv[r]), splat(kMagic));
           x[2 * h] = __float_as_uint(t.x);
           x[2 * h + 1] = __float_as_uint(t.y);
+          if constexpr (BV <= 4) {
+            // the new code picks its level's factor from the lane table
+            constexpr uint32_t bias = kMagicBits - (uint32_t)K;
+            const f2 fac = make_float2(__shfl_sync(kFull, lut_upd, (int)((x[2 * h] - bias) | (uint32_t)(r << LV))),
+                                       __shfl_sync(kFull, lut_upd, (int)((x[2 * h + 1] - bias) | (uint32_t)(r << LV))));
+            out[h] = fma2(nq[h], fac, fma2(th[r][h], splat(nlrwd), th[r][h]));
+            continue;
+          }
           // sqrt of the decoded level: sqrt(hi) * 2^((code-K) * W/K / 2), or sqrt(lo) for code 0
           const f2 rr = add2(t, splat(-kMagic));
           const f2 arg = mul2(rr, splat(half_step));
