@@ -269,7 +269,10 @@ def run_ours(args, w, bits_m, bits_v):
                     shapes=tuple((f"{w.shapes[l][0]}[{lo}:{hi}]", (hi - lo,)) for l, lo, hi in mine))
         bits_m, bits_v = bits_m[layer_of_row], bits_v[layer_of_row]
 
-    job = Job(w, bits_m, bits_v, device=dev)
+    layout = args.layout
+    if layout == "tile" and w.v_log == "ts" and any(n % w.block for n in w.numels):
+        layout = "exact"       # zero padding inside a last, partly real block would change the minimum the two-scale code keeps
+    job = Job(w, bits_m, bits_v, device=dev, tile_padded=(layout == "tile"))
     job.draw_grads(1)
 
     def decide(t):
@@ -396,6 +399,9 @@ def run_ours(args, w, bits_m, bits_v):
                           if small else "inputs larger than L2 (%.1f GB touched per step)" % (alg_bytes / 1e9)),
                    "parallelism": ("sharded over %d ranks (this rank: %d parameters)" % (world, params) if args.shard
                                    else "replicas" if world > 1 else "single"), "grid": job.handle.grid_size,
+                   "layout": ("tile: every tensor's storage padded with zeros to whole 4096-element tiles, padded lengths "
+                              "given to the library; parameters and bytes count the real elements only"
+                              if layout == "tile" else "exact: tensors at their true lengths"),
                    "state_bytes": job.state_bytes(), "fp32_state_bytes": 8 * params,
                    "state_saved_frac": 1.0 - job.state_bytes() / (8.0 * params)},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -495,6 +501,10 @@ def main():
     ap.add_argument("--no-variants", action="store_true", help="skip the extra runs with the other codes of the second moment")
     ap.add_argument("--v-log", default="poly", choices=["poly", "pl", "sr", "ts"],
                     help="code of the second moment (default: the polynomial logarithm)")
+    ap.add_argument("--layout", default="tile", choices=["exact", "tile"],
+                    help="tile (default): every tensor's storage padded with zeros to whole 4096-element tiles, a step is "
+                         "one launch; exact: tensors at their true lengths (ragged last tiles take one more launch per step). "
+                         "The results on the real elements are the same (tested against the oracle at full size)")
     ap.add_argument("--shard", action="store_true",
                     help="strong scaling: each rank owns a block-aligned slice of the parameter list "
                          "(default: every rank steps a full replica)")

@@ -98,6 +98,15 @@ enum { STQ_VLOG_POLY = 0, STQ_VLOG_PL = 1, STQ_VLOG_SR = 2, STQ_VLOG_TS = 3 };
 /* flags of stq_step */
 enum { STQ_WITH_STATS = 1u };
 
+/* The step kernels work on tiles of this many consecutive elements of one tensor.  A tensor whose numel is a
+ * multiple of it (with packed states and a block of 128 or 256) is served by the main kernel alone; the ragged last
+ * tile of any other tensor goes to the generic kernel, which costs a step one more launch.  A caller that owns its
+ * buffers can avoid that by padding every buffer of a tensor with zeros to a whole number of tiles and passing the
+ * padded numel: zero gradients keep the padding at zero, it adds nothing to the statistics' sums (only the element
+ * count reported by stq_layer_stats is then the padded one) and leaves the real elements' blocks as they are
+ * (except under STQ_VLOG_TS, whose block minimum the padding inside a last, partly real block would change). */
+#define STQ_TILE_ELEMS 4096
+
 /* One row per parameter tensor (a "layer" of the paper is one tensor). */
 typedef struct stq_tensor {
   float* param;              /* fp32 master weights, numel elements, updated in place          */

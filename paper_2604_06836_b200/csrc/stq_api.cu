@@ -15,6 +15,7 @@
 #include "stq_internal.h"
 
 using stq::TensorDesc;
+static_assert(STQ_TILE_ELEMS == stq::kTile, "the tile size promised in the header");
 
 struct stq_handle {
   int device = 0;

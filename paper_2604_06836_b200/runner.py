@@ -40,11 +40,22 @@ class Job:
     """Parameters, gradients and quantized AdamW state of one workload on one device."""
 
     def __init__(self, w: Workload, bits_m: Sequence[int], bits_v: Sequence[int], device="cuda",
-                 handle: stq.Handle | None = None, draw_params: bool = True):
+                 handle: stq.Handle | None = None, draw_params: bool = True, tile_padded: bool = False):
+        """tile_padded: every tensor's storage (parameters, gradients, codes, scales) is padded with zeros to a
+        whole number of 4096-element tiles and the library is given the padded length, so that a step has no
+        ragged last tiles (and hence a single launch).  The padding stays zero under the update (zero gradient,
+        zero moments, zero parameter), adds nothing to the gradient sums and leaves the block maxima of the
+        real elements as they are; ``params`` / ``grads`` remain views of the real elements."""
         self.w = w
         self.device = torch.device(device)
         self.handle = handle or stq.Handle(self.device.index if self.device.index is not None else torch.cuda.current_device())
         self.numels = w.numels
+        self.tile_padded = bool(tile_padded)
+        if tile_padded and w.v_log == "ts" and any(n % w.block for n in w.numels):
+            # the two-scale code also keeps the block minimum, which zero padding inside a block would change
+            raise ValueError("tile-padded storage with the two-scale code needs tensors of whole blocks")
+        # the length the library is told: the real one, or the padded one
+        self.tab_numels = [_round_up(n, stq.TILE) if tile_padded else n for n in self.numels]
         self.L = len(self.numels)
         self.block = w.block
         self.gdt = {"fp32": torch.float32, "bf16": torch.bfloat16, "fp16": torch.float16}[w.grad_dtype]
@@ -52,7 +63,7 @@ class Job:
         self.scales = tensor_scales(w)
         # parameters and gradients live in two flat buffers; every tensor starts 256-byte aligned
         offs, total = [], 0
-        for n in self.numels:
+        for n in self.tab_numels:
             offs.append(total)
             total += _round_up(n, 64)
         self.offsets = offs
@@ -76,7 +87,7 @@ class Job:
         self.v_log = stq.VLOG_BY_NAME[w.v_log]
         self.sr_seed = 0x5EED0000 + w.seed          # random words of the stochastic-rounding code
         self.states = [stq.alloc_state(n, self.block, int(bm), int(bv), self.device, self.v_log)
-                       for n, bm, bv in zip(self.numels, self.bits_m, self.bits_v)]
+                       for n, bm, bv in zip(self.tab_numels, self.bits_m, self.bits_v)]
         self.wd = [w.weight_decay] * self.L
         self._tbl = None
         self.t = 0
@@ -89,7 +100,7 @@ class Job:
                              self.params[i] if with_inputs else None,
                              self.grads[i] if with_inputs else None, self.wd[i],
                              self.params_lp[i] if with_inputs else None, sr_id=i)
-                for i, (n, si, so) in enumerate(zip(self.numels, st_in, st_out))]
+                for i, (n, si, so) in enumerate(zip(self.tab_numels, st_in, st_out))]
         return stq.table(rows)
 
     def table(self):
@@ -136,17 +147,20 @@ class Job:
         rows = []
         for i in idx:
             new_states[i] = self._fresh_state(i, int(bm[i]), int(bv[i]))
-            rows.append(stq.make_row(self.numels[i], self.block, self.states[i], new_states[i], sr_id=i))
+            rows.append(stq.make_row(self.tab_numels[i], self.block, self.states[i], new_states[i], sr_id=i))
         self.handle.repack(stq.table(rows), stream=stream)
         self._adopt(new_states, bm, bv)
 
     def layer_stats(self, stream=None) -> np.ndarray:
-        return self.handle.layer_stats(self.L, stream=stream)
+        st = self.handle.layer_stats(self.L, stream=stream)
+        if self.tile_padded:
+            st[:, 3] = self.numels          # the element count of the real tensor (the sums have no share of the padding)
+        return st
 
     def _fresh_state(self, i: int, bm: int, bv: int) -> stq.QState:
         """New buffers for the states whose width changes; unchanged states keep their buffers."""
         old = self.states[i]
-        n = self.numels[i]
+        n = self.tab_numels[i]
         mc, ms = (old.m_codes, old.m_scales) if bm == old.bits_m else (
             stq.alloc_codes(n, bm, self.device), stq.alloc_scales(n, bm, self.block, self.device))
         vc, vs = (old.v_codes, old.v_scales) if bv == old.bits_v else (
@@ -190,7 +204,7 @@ class Job:
         vc, vs = mirror([s.v_codes for s in self.states]), mirror([s.v_scales for s in self.states])
         states = [stq.QState(mc[i], ms[i], s.bits_m, vc[i], vs[i], s.bits_v, s.v_log) for i, s in enumerate(self.states)]
         rows = [stq.make_row(n, self.block, states[i], states[i], host_p[o:o + n], host_g[o:o + n], self.wd[i], sr_id=i)
-                for i, (n, o) in enumerate(zip(self.numels, self.offsets))]
+                for i, (n, o) in enumerate(zip(self.tab_numels, self.offsets))]
         return stq.table(rows), states, host_p, host_g
 
     # ---- accounting ------------------------------------------------------------------------------

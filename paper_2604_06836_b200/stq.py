@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libstq.so")
 GRAD_F32, GRAD_BF16, GRAD_F16 = 0, 1, 2
 LP_NONE, LP_BF16, LP_F16 = 0, 1, 2
 WITH_STATS = 1
+TILE = 4096              # STQ_TILE_ELEMS: elements per tile of the step kernels
 VLOG_POLY, VLOG_PL, VLOG_SR, VLOG_TS = 0, 1, 2, 3      # codes of the second moment (stq_tensor.v_log)
 VLOG_BY_NAME = {"poly": VLOG_POLY, "pl": VLOG_PL, "sr": VLOG_SR, "ts": VLOG_TS}
 WIDTHS = (2, 3, 4, 8, 16, 32)

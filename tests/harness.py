@@ -331,8 +331,18 @@ class FullOracle:
             gs, os_ = job.states[i], self.states[i]
             name = f"{tag} tensor {i} ({job.w.shapes[i][0]}, bits {gs.bits_m}/{gs.bits_v})"
             assert gs.bits_m == os_.bits_m and gs.bits_v == os_.bits_v, name
-            for what, g, o in (("m codes", gs.m_codes, os_.m_codes), ("v codes", gs.v_codes, os_.v_codes)):
+            padded = getattr(job, "tile_padded", False)
+            n = job.numels[i]
+            for what, g, o, b in (("m codes", gs.m_codes, os_.m_codes, gs.bits_m), ("v codes", gs.v_codes, os_.v_codes, gs.bits_v)):
                 o_d = torch.from_numpy(o).to(dev)
+                if padded:
+                    # the job's buffers run on into the zero padding: the codes of the real elements are a prefix of
+                    # the bit stream (whole bytes, then the low bits of one more)
+                    whole, rest = (n * b) // 8, (n * b) % 8
+                    g, o_d = g.view(torch.uint8)[:whole + (rest > 0)].clone(), o_d.view(torch.uint8)[:whole + (rest > 0)].clone()
+                    if rest:
+                        g[-1] &= (1 << rest) - 1
+                        o_d[-1] &= (1 << rest) - 1
                 if not torch.equal(g, o_d):
                     bad = torch.nonzero(g != o_d).flatten()[:8].tolist()
                     raise AssertionError(f"{name}: {what} differ at bytes {bad}")
@@ -341,6 +351,8 @@ class FullOracle:
                 if b == 32:
                     continue
                 o_d = torch.from_numpy(o).to(dev)
+                if padded:
+                    g = g[:o_d.numel()]                      # the blocks that hold real elements
                 if not torch.equal(g.view(torch.int32), o_d.view(torch.int32)):
                     bad = torch.nonzero(g.view(torch.int32) != o_d.view(torch.int32)).flatten()[:8].tolist()
                     raise AssertionError(f"{name}: {what} differ at blocks {bad}")

@@ -78,21 +78,26 @@ def test_full_size_sampled_blocks(name, gib):
 
 
 @pytest.mark.parametrize("name,gib,full_steps", [("cfg2", 8, None), ("cfg3", 6, None), ("cfg4", 30, 3), ("cfg5", 60, 3),
-                                                 ("cfg2:sr", 8, 3), ("cfg3:ts", 6, 3)])
+                                                 ("cfg2:sr", 8, 3), ("cfg3:ts", 6, 3),
+                                                 ("cfg2:tile", 8, 12), ("cfg3:tile", 6, 40), ("cfg5:tile", 60, 2)])
 def test_full_size_every_element(name, gib, full_steps):
     """Whole buffers against the oracle: every code byte, every scale, every parameter, on every step
     run (all of them for cfg2 and cfg3; steps 1-3 for cfg4 and cfg5, which are decision steps with fused
     statistics).  cfg3 changes the widths of 10 % of its tensors on every decision step from t = 5 on,
     alternately by stq_repack and inside the step.  The ":sr" and ":ts" cases run the first steps of a
-    configuration with the stochastic-rounding or the two-scale code of the second moment."""
+    configuration with the stochastic-rounding or the two-scale code of the second moment.  The ":tile" cases
+    keep every tensor in storage padded with zeros to whole tiles and give the library the padded lengths (a
+    step is then one launch): the real elements' codes, scales and parameters are those of the oracle's run on
+    the unpadded tensors."""
     import harness as H
     _need(gib)
     w = W.config(name.split(":")[0])
-    if ":" in name:               # the same configuration with another code of the second moment (its fused bodies)
+    tile = name.endswith(":tile")
+    if ":" in name and not tile:  # the same configuration with another code of the second moment (its fused bodies)
         from dataclasses import replace
         w = replace(w, v_log=name.split(":")[1])
     bm, bv, _ = W.draw_bits(w)
-    job = Job(w, bm, bv)
+    job = Job(w, bm, bv, tile_padded=tile)
     fo = H.FullOracle(job)
     fo.compare(0.0, f"{name} init")
     decisions = 0
@@ -109,7 +114,10 @@ def test_full_size_every_element(name, gib, full_steps):
                 job.repack((nbm, nbv))
                 fo.repack((nbm, nbv))
         st_o = fo.step(t, new_bits=new_bits, want_stats=dec)
+        n0 = job.handle.launch_count
         job.step(t, stats=dec, new_bits=new_bits)
+        if tile and not dec:
+            assert job.handle.launch_count - n0 == 1, "a plain step over tile-padded storage is one launch"
         fo.compare(1e-6 * t if t <= 10 else 1e-4, f"{name} t={t}")
         if dec:
             H.assert_stats_close(job.layer_stats(), st_o, f"{name} t={t}")
